@@ -1,0 +1,363 @@
+#!/usr/bin/env python
+"""Benchmark of the segment-KV decode attention path on B200.
+
+One *step* is one decode step of an L-layer stack of attention layers of the
+chosen shape: per layer, append the step's K/V rows (which also updates the
+beam-index table) and run the fused decode attention.  All layers are distinct
+cache handles, so a step touches L x (unique KV bytes) of HBM, far more than
+the L2 holds, and every timed kernel reads cold data.
+
+Printed: ONE JSON line (see README / DESIGN).  `value` is the whole-job
+unique-KV bandwidth in GB/s: the K/V bytes the method has to read (prompt rows
+once per request, every DISTINCT response row once) divided by the step time.
+
+`--impl reference` times the CPU float64 oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "decode_sdpa_unique_kv_bandwidth"
+UNIT = "GB/s"
+DEFAULT_LAYERS = {"tiny": 32, "llama2-7b": 32, "llama2-13b": 32, "gptj-6b": 4, "opt-30b": 1, "bloom-176b": 1}
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2-7b")
+    ap.add_argument("--layers", type=int, default=0, help="distinct cache handles per step (0 = per-workload default)")
+    ap.add_argument("--at-step", type=int, default=0, help="decode step to time, 1-based (0 = the workload's last)")
+    ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def unique_bytes(w, prompt_len, unique_rows_total):
+    """K and V bytes the method must read for one layer at one step."""
+    row = 2 * w.kv_heads * w.head_dim * 2
+    return (w.batch * prompt_len + int(unique_rows_total)) * row
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) != 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(w, t, budget_s=12.0, max_pairs=None):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload at step t.
+    Returns (GB/s of unique KV over the sample, seconds, description, threads)."""
+    import torch
+    import oracle
+    from paper_2401_05391_b200 import workloads as wl
+
+    # one request, all of its heads (every request is an independent unit of the path)
+    w1 = w.scaled(batch=1)
+    par = wl.make_parents(w1)
+    kp, vp = wl.make_prompt(w1, "cpu")
+    steps = [wl.make_step(w1, s, "cpu") for s in range(t + 1)]
+    q = steps[t][0]
+    kr = np.stack([wl.to_bits(s[1]) for s in steps]); vr = np.stack([wl.to_bits(s[2]) for s in steps])
+    slopes = wl.alibi_slopes(w.heads).numpy() if w.alibi else None
+    heads = list(range(w.heads))
+    if max_pairs:
+        heads = heads[:max(1, max_pairs // w.beams)]
+    pairs = [(g, h) for g in range(w1.rows) for h in heads]
+    args = (w.dtype, 1, w.beams, w.heads, w.kv_heads, w.head_dim, wl.to_bits(q), wl.to_bits(kp), wl.to_bits(vp),
+            kr, vr, par, t)
+    anc = oracle.ancestry(par, 1, w.beams, t)
+    uniq = sum(len(set(anc[:, s].tolist())) for s in range(t + 1))
+    kv_heads_used = len({h // (w.heads // w.kv_heads) for h in heads})
+    nbytes = (w.prompt_len + uniq) * 2 * kv_heads_used * w.head_dim * 2
+    oracle.decode_sdpa(*args, slopes=slopes, pairs=pairs[:w.beams])            # load, page in
+    reps, total = 0, 0.0
+    while True:
+        t0 = time.perf_counter()
+        oracle.decode_sdpa(*args, slopes=slopes, pairs=pairs)
+        total += time.perf_counter() - t0
+        reps += 1
+        if total >= budget_s or reps >= 50:
+            break
+    sec = total / reps
+    desc = (f"1 request x {len(heads)} heads x {w.beams} beams of {w.name} at step {t + 1} "
+            f"({len(pairs)} attention rows over {w.prompt_len + t + 1} keys), mean of {reps} runs")
+    return nbytes / sec / 1e9, sec, desc, oracle.threads()
+
+
+def run_reference(args):
+    from paper_2401_05391_b200 import workloads as wl
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = wl.by_name(args.workload)
+    t = (args.at_step or w.steps) - 1
+    vals = []
+    desc = ""
+    threads = 1
+    for i in range(args.warmup + args.steps):
+        gbs, sec, desc, threads = oracle_sample(w, t, budget_s=0.0, max_pairs=256)
+        if i >= args.warmup:
+            vals.append((gbs, sec))
+    gbs = statistics.mean(v[0] for v in vals)
+    sec = statistics.mean(v[1] for v in vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "at_step": t + 1, "sample": desc},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- ours
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2401_05391_b200 import workloads as wl
+    from paper_2401_05391_b200.segkv import SegKV
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = wl.by_name(args.workload)
+    L = args.layers or DEFAULT_LAYERS.get(w.name, 1)
+    T = args.at_step or w.steps
+    t = T - 1
+    # every rank holds its own requests (weak scaling: requests are independent, no exchange)
+    w_rank = w.scaled(index=w.index + 100 * rank) if world > 1 else w
+    parents = torch.from_numpy(wl.make_parents(w_rank)).to(dev)
+    slopes = wl.alibi_slopes(w.heads).to(dev) if w.alibi else None
+
+    handles = []
+    for layer in range(L):
+        wl_layer = w_rank.scaled(index=w_rank.index + 1000 * layer)
+        h = SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, w.steps, w.torch_dtype)
+        if args.splits:
+            h.set_splits(args.splits)
+        kp, vp = wl.make_prompt(wl_layer, dev)
+        h.prefill_write(kp, vp)
+        del kp, vp
+        for s in range(T):
+            q, k, v = wl.make_step(wl_layer, s, dev)
+            h.append(s, parents[s] if s > 0 else None, k, v)
+        handles.append((h, q, k, v, torch.empty_like(q)))
+    torch.cuda.synchronize()
+    uniq_rows = int(handles[0][0].get_unique_rows().sum())
+    ubytes = unique_bytes(w, w.prompt_len, uniq_rows)
+    logical_bytes = w.rows * (w.prompt_len + T) * 2 * w.kv_heads * w.head_dim * 2
+    par_t = parents[t] if t > 0 else None
+    stream = torch.cuda.Stream()
+
+    def layer_pass(append: bool):
+        for h, q, k, v, out in handles:
+            if append:
+                h.truncate_last()
+                h.append(t, par_t, k, v, stream=stream)
+            h.decode_sdpa(q, out, slopes, stream=stream)
+
+    def make_runner(append: bool):
+        with torch.cuda.stream(stream):
+            layer_pass(append)                               # lazy initialisation outside any capture
+        stream.synchronize()
+        if args.no_graph:
+            return lambda: layer_pass(append), False
+        g = torch.cuda.CUDAGraph()
+        try:
+            with torch.cuda.graph(g, stream=stream):
+                layer_pass(append)
+        except Exception as e:                               # report, never hide
+            sys.stderr.write(f"[bench] CUDA graph capture failed ({e}); timing direct launches\n")
+            return lambda: layer_pass(append), False
+
+        def replay():
+            with torch.cuda.stream(stream):
+                g.replay()
+        return replay, True
+
+    def timed(run, steps, warmup):
+        for _ in range(warmup):
+            run()
+        stream.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            run()
+        e1.record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            tt = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            dist.barrier()
+            ms = float(tt.item())
+        return ms
+
+    # ---- the timed region: K whole steps (append + attention, all layers)
+    run_step, graphed = make_runner(True)
+    launches0 = sum(h[0].launch_count for h in handles)
+    sampler = ClockSampler(f"GPU-{torch.cuda.get_device_properties(dev).uuid}") if rank == 0 else None
+    ms_total = timed(run_step, args.steps, args.warmup)
+    # ---- the attention kernel alone, same rotation over cold layers (roofline numerator)
+    run_sdpa, _ = make_runner(False)
+    ms_sdpa = timed(run_sdpa, args.steps, max(3, args.warmup))
+    clocks = sampler.stop() if sampler else None
+    launches_per_step = 2 * L
+    ms_per_step = ms_total / args.steps
+    us_layer = ms_per_step * 1e3 / L
+    us_sdpa = ms_sdpa / args.steps * 1e3 / L
+    value = world * L * ubytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end from host memory through segkv_step_host
+    e2e = None
+    if not args.no_e2e:
+        hq = [tuple(x.cpu().pin_memory() for x in (q, k, v)) + (torch.empty_like(q, device="cpu").pin_memory(),)
+              for _, q, k, v, _ in handles]
+        hp = parents[t].cpu().pin_memory() if t > 0 else None
+        hs = slopes.cpu().pin_memory() if slopes is not None else None
+
+        def host_step():
+            for (h, *_), (q, k, v, o) in zip(handles, hq):
+                h.truncate_last()
+                h.step_host(t, hp, k, v, q, o, hs, stream=stream)
+        n_e2e = max(3, min(args.steps, 20))
+        for _ in range(3):
+            host_step()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            host_step()
+        torch.cuda.synchronize()
+        sec = (time.perf_counter() - t0) / n_e2e
+        if world > 1:
+            tt = torch.tensor([sec], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            sec = float(tt.item())
+        q, k = handles[0][1], handles[0][2]
+        h2d = L * (q.numel() * 2 + 2 * k.numel() * 2 + (w.rows * 4 if t > 0 else 0) + (w.heads * 4 if hs is not None else 0))
+        d2h = L * q.numel() * 2
+        e2e = {"value": world * L * ubytes / sec / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "us_per_step_per_layer": sec * 1e6 / L}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = peaks()
+    achieved = ubytes / (us_sdpa * 1e-6) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f16" if w.dtype == "f16" else "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.batch, "beams": w.beams, "heads": w.heads, "kv_heads": w.kv_heads,
+                   "head_dim": w.head_dim, "prompt_len": w.prompt_len, "at_step": T, "layers_per_step": L,
+                   "l2": f"{L} distinct layer caches per step, {L * ubytes / 1e6:.0f} MB > L2", "cuda_graph": graphed,
+                   "splits": handles[0][0].get_splits(), "parallelism": f"replica x{world}" if world > 1 else "1 gpu"},
+        "us_per_step_per_layer": us_layer,
+        "us_sdpa_per_layer": us_sdpa,
+        "unique_kv_bytes_per_layer": ubytes,
+        "logical_kv_bytes_per_layer": logical_bytes,
+        "pct_of_8000_GBps": 100.0 * achieved / 8000.0,
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "segkv decode attention",
+                     "bytes_per_launch": ubytes, "us_per_launch": us_sdpa},
+        "e2e": e2e,
+        "clocks": clocks,
+    }
+    assert sum(h[0].launch_count for h in handles) > launches0
+    if not args.no_cpu_baseline:
+        gbs, sec, desc, threads = oracle_sample(w, t)
+        line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
+                                "seconds": sec}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,199 @@
+/*
+ * segkv — decode-step attention over a segment KV cache, for NVIDIA B200 (sm_100a).
+ *
+ * One handle is one attention layer's cache.  The cache has two segments
+ * (paper Section 3.2, "Segment KV Cache"):
+ *   - the PROMPT segment: K/V of each request's prompt, stored once per request
+ *     and shared by all of its beams;
+ *   - the RESPONSE segment: K/V of generated tokens, sequence-first
+ *     [step, batch*beams, kv_heads, head_dim] (Section 3.1), written in place,
+ *     one slab per decode step, never concatenated or re-ordered.
+ * Beam search hands over, per step, which earlier beam each beam slot extends.
+ * Instead of re-ordering the past cache with an index select (Section 3.1,
+ * Fig. 1) the library keeps those parent ids, derives the beam-index table
+ * (Section 3.3, "Index select fusion") and lets the attention kernel read the
+ * response rows through it.
+ *
+ * Conventions for every entry point
+ *   - return value: SEGKV_OK (0) or a negative SEGKV_E* code; no exceptions, no
+ *     process exit, no device-side trap;
+ *   - "device pointer" = memory of the device that was current at segkv_create,
+ *     16-byte aligned, contiguous in the stated layout, owned by the caller and
+ *     only read/written by the work the call enqueues;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream); calls that enqueue work are asynchronous on it;
+ *   - the handle is not thread-safe; calls on one handle must be ordered by
+ *     the caller (same stream, or explicit synchronisation);
+ *   - beam slot g = b*beams + j (request b, beam j); query head h reads kv head
+ *     h / (heads/kv_heads).
+ */
+#ifndef SEGKV_H
+#define SEGKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SEGKV_API __attribute__((visibility("default")))
+#else
+#define SEGKV_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct segkv* segkv_t;
+
+enum { SEGKV_F16 = 0, SEGKV_BF16 = 1 };
+
+enum {
+    SEGKV_OK = 0,
+    SEGKV_EINVAL = -1,    /* bad dimension, NULL/unaligned pointer, unknown dtype        */
+    SEGKV_ESTATE = -2,    /* call out of order (append before prefill, wrong step, ...)  */
+    SEGKV_ECAPACITY = -3, /* prompt_len > max_prompt or step >= max_steps                */
+    SEGKV_ENOMEM = -4,    /* host or device allocation failed                            */
+    SEGKV_ECUDA = -5,     /* a CUDA call failed; segkv_last_cuda_error() names it        */
+    SEGKV_EDEVICE = -6    /* a kernel reported a problem; see segkv_get_error()          */
+};
+
+/* bits of the device error word returned by segkv_get_error */
+enum {
+    SEGKV_DEV_BAD_PARENT = 1, /* a beam_parent value outside [0,beams) was clamped       */
+    SEGKV_DEV_WAIT_LIMIT = 2  /* a bounded wait inside a kernel ran out (never expected) */
+};
+
+/*
+ * Allocate one layer's cache on the current device: prompt segment
+ * [batch, kv_heads, max_prompt, head_dim] x {K,V}, response segment
+ * [max_steps, batch*beams, kv_heads, head_dim] x {K,V} (pre-allocated to
+ * max_steps, the fixed-capacity variant Section 3.2 describes), the parent
+ * table [max_steps, batch*beams], the beam-index tables and the split
+ * workspace of the attention kernel.
+ * Requirements: all dims > 0 (max_prompt may be 0), heads % kv_heads == 0,
+ * head_dim in {64,128,256}, beams*(heads/kv_heads) <= 32, dtype SEGKV_F16/BF16.
+ * The softmax scale is 1/sqrt(head_dim).
+ * Errors: EINVAL, ENOMEM, ECUDA.  *out is set only on success.
+ */
+SEGKV_API int segkv_create(segkv_t* out, int batch, int beams, int heads, int kv_heads, int head_dim,
+                 int max_prompt, int max_steps, int dtype);
+
+/* Free everything the handle owns.  Synchronises the device.  NULL is allowed. */
+SEGKV_API int segkv_destroy(segkv_t h);
+
+/*
+ * Store the prompt K/V (Section 3.2: kept once per request at prefill).
+ * k, v: device pointers, token-major [batch, prompt_len, kv_heads, head_dim],
+ * the layout a fused QKV projection produces (Section 3.1 batch-first).  The
+ * library keeps them head-major [batch, kv_heads, prompt_len, head_dim].
+ * Resets the number of appended steps to 0.  prompt_len == 0 is allowed (then
+ * k and v may be NULL).  Errors: EINVAL, ECAPACITY, ECUDA.
+ */
+SEGKV_API int segkv_prefill_write(segkv_t h, const void* k, const void* v, int prompt_len, void* stream);
+
+/*
+ * Decode step `step` (0-based), before its attention call: write the step's
+ * new K/V rows into slab `step` of the response segment (Section 3.1: Key_t,
+ * Value_t kept in place in the pre-allocated buffer), record the beam parents
+ * as row `step` of the parent table, and update the beam-index table
+ * (Section 3.3) so that it resolves every beam slot's row at every step <= step.
+ *   beam_parent: device int32 [batch*beams]; value = LOCAL beam id in [0,beams)
+ *                of the slot (same request) at step-1 that this slot extends.
+ *                Ignored, and may be NULL, when step == 0: all beams descend
+ *                from the shared prompt.  Out-of-range values are clamped into
+ *                range and flagged in the device error word (SEGKV_DEV_BAD_PARENT).
+ *   k_new, v_new: device [batch*beams, kv_heads, head_dim].
+ * `step` must equal the number of steps appended so far.
+ * Errors: EINVAL, ESTATE (no prefill yet, wrong step), ECAPACITY, ECUDA.
+ */
+SEGKV_API int segkv_append(segkv_t h, int step, const int32_t* beam_parent, const void* k_new,
+                 const void* v_new, void* stream);
+
+/*
+ * The fused decode attention (Section 3.3, "Customized SDPA Kernel"): for every
+ * beam slot g and head hd,
+ *     out[g,hd,:] = softmax(q[g,hd,:] . K^T / sqrt(head_dim) + bias) . V
+ * over the request's prompt rows followed by the beam's own response row of
+ * every appended step, selected through the beam-index table inside the kernel.
+ * fp16/bf16 operands, fp32 scores, softmax and accumulation, output rounded to
+ * nearest-even in the cache dtype.
+ *   q, out: device [batch*beams, heads, head_dim] (Section 3.3: [1, BSxBW, H, D]).
+ *   alibi_slopes: device float [heads] or NULL.  When given, bias for the key
+ *       at sequence position p is slope[hd] * (p - qpos), prompt rows at
+ *       p = 0..prompt_len-1, the step-s row at prompt_len + s, qpos the newest
+ *       position.  (ALiBi is not in the paper; the Bloom workload needs it.)
+ * With no step appended the call attends to the prompt only (the paper's
+ * "special case" of the kernel).  The call may be repeated; it changes nothing
+ * but `out` and the library's own workspace.
+ * Errors: EINVAL, ESTATE (nothing to attend to), ECUDA.
+ */
+SEGKV_API int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_slopes, void* stream);
+
+/*
+ * One whole decode step from HOST memory: copies beam_parent, k_new, v_new, q
+ * (and slopes, if given) to the device, runs segkv_append + segkv_decode_sdpa,
+ * copies `out` back and waits for it.  All pointers are host pointers (pinned
+ * memory makes the copies asynchronous); layouts as in the device calls.
+ * Staging buffers are part of the handle.  Errors: as the two calls.
+ */
+SEGKV_API int segkv_step_host(segkv_t h, int step, const int32_t* beam_parent, const void* k_new,
+                    const void* v_new, const void* q, void* out, const float* alibi_slopes,
+                    void* stream);
+
+/* ---- test and benchmark aids ------------------------------------------- */
+
+/* Forget all appended steps; keep_prompt == 0 also forgets the prompt. */
+SEGKV_API int segkv_reset(segkv_t h, int keep_prompt);
+
+/*
+ * Drop the LAST appended step so that it can be appended again (used to time
+ * a step repeatedly).  Only one step back is possible: the beam-index table
+ * is updated incrementally and keeps one earlier generation.  ESTATE if no
+ * step is appended or the previous call was also segkv_truncate_last.
+ */
+SEGKV_API int segkv_truncate_last(segkv_t h);
+
+/* Copy the beam-index table to host_out [batch*beams][steps] (physical row in
+ * [0,batch*beams) per beam slot and step).  Synchronises `stream`. */
+SEGKV_API int segkv_get_ancestry(segkv_t h, int32_t* host_out, void* stream);
+
+/* Per request, how many DISTINCT response rows its beams reference over all
+ * appended steps (host_out [batch]); this is what the kernel reads.  Synchronises. */
+SEGKV_API int segkv_get_unique_rows(segkv_t h, int32_t* host_out, void* stream);
+
+/* Read and clear the device error word (SEGKV_DEV_* bits).  Synchronises the device. */
+SEGKV_API int segkv_get_error(segkv_t h, int* device_flags);
+
+/* Number of appended steps / current prompt length, or a negative error. */
+SEGKV_API int segkv_steps(segkv_t h);
+SEGKV_API int segkv_prompt_len(segkv_t h);
+
+/*
+ * Force the number of KV splits per (request, kv head) of the attention kernel
+ * (0 = choose automatically from the shape, the default).  Re-allocates the
+ * split workspace; synchronises the device.  segkv_get_splits returns the value
+ * the next segkv_decode_sdpa will use.
+ */
+SEGKV_API int segkv_set_splits(segkv_t h, int splits);
+SEGKV_API int segkv_get_splits(segkv_t h);
+
+/* Kernels launched by the handle since creation (each launch counted once). */
+SEGKV_API long long segkv_launch_count(segkv_t h);
+
+/*
+ * K/V bytes one handle holds for the given shape: Eq. 3 of the paper for one
+ * layer with the response capacity fixed at max_steps,
+ *   batch * (max_prompt + beams*max_steps) * 2*kv_heads*head_dim*sizeof(dtype).
+ * Pure host arithmetic; 0 on a bad argument.
+ */
+SEGKV_API size_t segkv_storage_bytes(int batch, int beams, int kv_heads, int head_dim, int max_prompt,
+                           int max_steps, int dtype);
+
+SEGKV_API const char* segkv_strerror(int code);
+/* Text of the last CUDA error seen by this thread inside the library ("" if none). */
+SEGKV_API const char* segkv_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SEGKV_H */

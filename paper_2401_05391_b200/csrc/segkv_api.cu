@@ -1,0 +1,367 @@
+// Host side of the segkv C-ABI: handle life cycle, argument checks, launches.
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "segkv_internal.h"
+
+using namespace segkv_impl;
+
+namespace {
+
+thread_local char g_cuda_err[256] = "";
+
+int cuda_fail(cudaError_t e, const char* what) {
+    snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s (%s)", what, cudaGetErrorName(e), cudaGetErrorString(e));
+    return e == cudaErrorMemoryAllocation ? SEGKV_ENOMEM : SEGKV_ECUDA;
+}
+
+#define SEGKV_CUDA(call)                                   \
+    do {                                                   \
+        cudaError_t e__ = (call);                          \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #call); \
+    } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+size_t elem_bytes(int dtype) { return (dtype == SEGKV_F16 || dtype == SEGKV_BF16) ? 2 : 0; }
+
+bool dims_ok(int batch, int beams, int heads, int kv_heads, int head_dim, int max_prompt, int max_steps,
+             int dtype) {
+    if (batch <= 0 || beams <= 0 || heads <= 0 || kv_heads <= 0 || max_steps <= 0 || max_prompt < 0) return false;
+    if (heads % kv_heads) return false;
+    if (head_dim != 64 && head_dim != 128 && head_dim != 256) return false;
+    if ((long long)beams * (heads / kv_heads) > kMaxCols) return false;
+    if (elem_bytes(dtype) == 0) return false;
+    return true;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// Tensor map over one prompt array seen as [batch*kv_heads][prompt_len][D]:
+// rows >= prompt_len read as zero, a box never crosses a (request, head) slab.
+// Box = 64 elements (128 bytes, one swizzle span) x kTileKeys rows.
+int make_prompt_map(const segkv* h, void* base, int prompt_len, CUtensorMap* out) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled entry point not available");
+        return SEGKV_ECUDA;
+    }
+    const Dims& d = h->d;
+    cuuint64_t dims[3] = {(cuuint64_t)d.head_dim, (cuuint64_t)prompt_len, (cuuint64_t)d.batch * d.kv_heads};
+    cuuint64_t strides[2] = {(cuuint64_t)d.head_dim * 2, (cuuint64_t)d.max_prompt * d.head_dim * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)kTileKeys, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUtensorMapDataType dt = d.dtype == SEGKV_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    CUresult r = fn(out, dt, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        return SEGKV_ECUDA;
+    }
+    return SEGKV_OK;
+}
+
+void free_all(segkv* h) {
+    void* ptrs[] = {h->kp, h->vp, h->kr, h->vr, h->parent, h->anc[0], h->anc[1], h->ulist, h->ucount,
+                    h->err_word, h->ws, h->tickets, h->st_q, h->st_out, h->st_k, h->st_v, h->st_parent,
+                    h->st_slopes};
+    for (void* p : ptrs)
+        if (p) cudaFree(p);
+}
+
+template <typename T>
+cudaError_t dmalloc(T** p, size_t bytes) {
+    return cudaMalloc((void**)p, bytes ? bytes : 16);
+}
+
+int alloc_workspace(segkv* h, int splits) {
+    const Dims& d = h->d;
+    size_t cols = (size_t)d.beams * d.group;
+    size_t bytes = (size_t)d.batch * d.kv_heads * splits * cols * (d.head_dim + 2) * sizeof(float);
+    if (h->ws) {
+        cudaFree(h->ws);
+        h->ws = nullptr;
+    }
+    SEGKV_CUDA(dmalloc(&h->ws, bytes));
+    h->ws_bytes = bytes;
+    h->ws_splits = splits;
+    return SEGKV_OK;
+}
+
+SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes, int splits) {
+    SdpaArgs a;
+    a.q = q;
+    a.out = out;
+    a.slopes = slopes;
+    a.kp = h->kp;
+    a.vp = h->vp;
+    a.kr = h->kr;
+    a.vr = h->vr;
+    a.anc = h->anc[h->steps > 0 ? ((h->steps - 1) & 1) : 0];
+    a.ulist = h->ulist;
+    a.ucount = h->ucount;
+    a.ws = h->ws;
+    a.tickets = h->tickets;
+    a.err_word = h->err_word;
+    a.prompt_len = h->prompt_len > 0 ? h->prompt_len : 0;
+    a.steps = h->steps;
+    a.splits = splits;
+    return a;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t segkv_storage_bytes(int batch, int beams, int kv_heads, int head_dim, int max_prompt, int max_steps,
+                           int dtype) {
+    if (batch <= 0 || beams <= 0 || kv_heads <= 0 || head_dim <= 0 || max_prompt < 0 || max_steps < 0) return 0;
+    size_t eb = elem_bytes(dtype);
+    if (!eb) return 0;
+    size_t token = 2 * (size_t)kv_heads * head_dim * eb;
+    return (size_t)batch * ((size_t)max_prompt + (size_t)beams * max_steps) * token;
+}
+
+const char* segkv_strerror(int code) {
+    switch (code) {
+        case SEGKV_OK: return "ok";
+        case SEGKV_EINVAL: return "invalid argument";
+        case SEGKV_ESTATE: return "call out of order for the handle's state";
+        case SEGKV_ECAPACITY: return "beyond the capacity given at segkv_create";
+        case SEGKV_ENOMEM: return "out of memory";
+        case SEGKV_ECUDA: return "CUDA error (see segkv_last_cuda_error)";
+        case SEGKV_EDEVICE: return "a kernel reported an error (see segkv_get_error)";
+        default: return "unknown segkv error code";
+    }
+}
+
+const char* segkv_last_cuda_error(void) { return g_cuda_err; }
+
+int segkv_create(segkv_t* out, int batch, int beams, int heads, int kv_heads, int head_dim, int max_prompt,
+                 int max_steps, int dtype) {
+    if (!out) return SEGKV_EINVAL;
+    if (!dims_ok(batch, beams, heads, kv_heads, head_dim, max_prompt, max_steps, dtype)) return SEGKV_EINVAL;
+    segkv* h = new (std::nothrow) segkv();
+    if (!h) return SEGKV_ENOMEM;
+    memset(h, 0, sizeof *h);
+    Dims& d = h->d;
+    d.batch = batch; d.beams = beams; d.heads = heads; d.kv_heads = kv_heads; d.head_dim = head_dim;
+    d.group = heads / kv_heads; d.max_prompt = max_prompt; d.max_steps = max_steps;
+    d.rows = batch * beams; d.dtype = dtype;
+    h->prompt_len = -1;
+
+    int rc = SEGKV_OK;
+    auto fail = [&](int code) { free_all(h); delete h; return code; };
+#define SEGKV_TRY(call)                                     \
+    do {                                                    \
+        cudaError_t e__ = (call);                           \
+        if (e__ != cudaSuccess) return fail(cuda_fail(e__, #call)); \
+    } while (0)
+    SEGKV_TRY(cudaGetDevice(&h->device));
+    SEGKV_TRY(cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device));
+    int optin = 0;
+    SEGKV_TRY(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device));
+    h->smem_optin = (size_t)optin;
+
+    const size_t eb = 2;
+    const size_t prompt_bytes = (size_t)batch * kv_heads * max_prompt * head_dim * eb;
+    const size_t resp_bytes = (size_t)max_steps * d.rows * kv_heads * head_dim * eb;
+    SEGKV_TRY(dmalloc(&h->kp, prompt_bytes));
+    SEGKV_TRY(dmalloc(&h->vp, prompt_bytes));
+    SEGKV_TRY(dmalloc(&h->kr, resp_bytes));
+    SEGKV_TRY(dmalloc(&h->vr, resp_bytes));
+    SEGKV_TRY(dmalloc(&h->parent, (size_t)max_steps * d.rows * sizeof(int32_t)));
+    SEGKV_TRY(dmalloc(&h->anc[0], (size_t)max_steps * d.rows * sizeof(int32_t)));
+    SEGKV_TRY(dmalloc(&h->anc[1], (size_t)max_steps * d.rows * sizeof(int32_t)));
+    SEGKV_TRY(dmalloc(&h->ulist, (size_t)max_steps * d.rows * sizeof(URow)));
+    SEGKV_TRY(dmalloc(&h->ucount, (size_t)batch * sizeof(int32_t)));
+    SEGKV_TRY(dmalloc(&h->err_word, sizeof(int)));
+    SEGKV_TRY(dmalloc(&h->tickets, (size_t)batch * kv_heads * sizeof(int)));
+    SEGKV_TRY(cudaMemset(h->ucount, 0, (size_t)batch * sizeof(int32_t)));
+    SEGKV_TRY(cudaMemset(h->err_word, 0, sizeof(int)));
+    SEGKV_TRY(cudaMemset(h->tickets, 0, (size_t)batch * kv_heads * sizeof(int)));
+    const size_t qbytes = (size_t)d.rows * heads * head_dim * eb;
+    const size_t kvbytes = (size_t)d.rows * kv_heads * head_dim * eb;
+    SEGKV_TRY(dmalloc(&h->st_q, qbytes));
+    SEGKV_TRY(dmalloc(&h->st_out, qbytes));
+    SEGKV_TRY(dmalloc(&h->st_k, kvbytes));
+    SEGKV_TRY(dmalloc(&h->st_v, kvbytes));
+    SEGKV_TRY(dmalloc(&h->st_parent, (size_t)d.rows * sizeof(int32_t)));
+    SEGKV_TRY(dmalloc(&h->st_slopes, (size_t)heads * sizeof(float)));
+#undef SEGKV_TRY
+    rc = alloc_workspace(h, 1);
+    if (rc != SEGKV_OK) return fail(rc);
+    *out = h;
+    return SEGKV_OK;
+}
+
+int segkv_destroy(segkv_t h) {
+    if (!h) return SEGKV_OK;
+    cudaDeviceSynchronize();
+    free_all(h);
+    delete h;
+    return SEGKV_OK;
+}
+
+int segkv_prefill_write(segkv_t h, const void* k, const void* v, int prompt_len, void* stream) {
+    if (!h || prompt_len < 0) return SEGKV_EINVAL;
+    if (prompt_len > h->d.max_prompt) return SEGKV_ECAPACITY;
+    if (prompt_len > 0 && (!k || !v || !aligned16(k) || !aligned16(v))) return SEGKV_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    h->tm_valid = false;
+    if (prompt_len > 0) {
+        SEGKV_CUDA(launch_prefill_transpose(h->d, k, v, h->kp, h->vp, prompt_len, st));
+        h->launches++;
+        int rc = make_prompt_map(h, h->kp, prompt_len, &h->tm_kp);
+        if (rc == SEGKV_OK) rc = make_prompt_map(h, h->vp, prompt_len, &h->tm_vp);
+        if (rc != SEGKV_OK) return rc;
+        h->tm_valid = true;
+    }
+    h->prompt_len = prompt_len;
+    h->steps = 0;
+    h->truncated = false;
+    return SEGKV_OK;
+}
+
+int segkv_append(segkv_t h, int step, const int32_t* beam_parent, const void* k_new, const void* v_new,
+                 void* stream) {
+    if (!h || step < 0 || !k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return SEGKV_EINVAL;
+    if (step > 0 && (!beam_parent || (reinterpret_cast<uintptr_t>(beam_parent) & 3u))) return SEGKV_EINVAL;
+    if (h->prompt_len < 0) return SEGKV_ESTATE;
+    if (step != h->steps) return SEGKV_ESTATE;
+    if (step >= h->d.max_steps) return SEGKV_ECAPACITY;
+    SEGKV_CUDA(launch_append(h->d, step, beam_parent, k_new, v_new, h->kr, h->vr, h->parent,
+                             h->anc[(step + 1) & 1], h->anc[step & 1], h->ulist, h->ucount, h->err_word,
+                             h->sm_count, (cudaStream_t)stream));
+    h->launches++;
+    h->steps = step + 1;
+    h->truncated = false;
+    return SEGKV_OK;
+}
+
+int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_slopes, void* stream) {
+    if (!h || !q || !out || !aligned16(q) || !aligned16(out)) return SEGKV_EINVAL;
+    if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SEGKV_EINVAL;
+    if (h->prompt_len < 0) return SEGKV_ESTATE;
+    if (h->prompt_len + h->steps <= 0) return SEGKV_ESTATE;
+    SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, 1);
+    SEGKV_CUDA(launch_sdpa_rowwise(h->d, a, (cudaStream_t)stream));
+    h->launches++;
+    return SEGKV_OK;
+}
+
+int segkv_step_host(segkv_t h, int step, const int32_t* beam_parent, const void* k_new, const void* v_new,
+                    const void* q, void* out, const float* alibi_slopes, void* stream) {
+    if (!h || !k_new || !v_new || !q || !out) return SEGKV_EINVAL;
+    if (step > 0 && !beam_parent) return SEGKV_EINVAL;
+    const Dims& d = h->d;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t qbytes = (size_t)d.rows * d.heads * d.head_dim * 2;
+    const size_t kvbytes = (size_t)d.rows * d.kv_heads * d.head_dim * 2;
+    if (step > 0)
+        SEGKV_CUDA(cudaMemcpyAsync(h->st_parent, beam_parent, (size_t)d.rows * sizeof(int32_t),
+                                   cudaMemcpyHostToDevice, st));
+    SEGKV_CUDA(cudaMemcpyAsync(h->st_k, k_new, kvbytes, cudaMemcpyHostToDevice, st));
+    SEGKV_CUDA(cudaMemcpyAsync(h->st_v, v_new, kvbytes, cudaMemcpyHostToDevice, st));
+    SEGKV_CUDA(cudaMemcpyAsync(h->st_q, q, qbytes, cudaMemcpyHostToDevice, st));
+    if (alibi_slopes)
+        SEGKV_CUDA(cudaMemcpyAsync(h->st_slopes, alibi_slopes, (size_t)d.heads * sizeof(float),
+                                   cudaMemcpyHostToDevice, st));
+    int rc = segkv_append(h, step, step > 0 ? h->st_parent : nullptr, h->st_k, h->st_v, stream);
+    if (rc != SEGKV_OK) return rc;
+    rc = segkv_decode_sdpa(h, h->st_q, h->st_out, alibi_slopes ? h->st_slopes : nullptr, stream);
+    if (rc != SEGKV_OK) return rc;
+    SEGKV_CUDA(cudaMemcpyAsync(out, h->st_out, qbytes, cudaMemcpyDeviceToHost, st));
+    SEGKV_CUDA(cudaStreamSynchronize(st));
+    return SEGKV_OK;
+}
+
+int segkv_reset(segkv_t h, int keep_prompt) {
+    if (!h) return SEGKV_EINVAL;
+    h->steps = 0;
+    h->truncated = false;
+    if (!keep_prompt) {
+        h->prompt_len = -1;
+        h->tm_valid = false;
+    }
+    return SEGKV_OK;
+}
+
+int segkv_truncate_last(segkv_t h) {
+    if (!h) return SEGKV_EINVAL;
+    if (h->steps <= 0 || h->truncated) return SEGKV_ESTATE;
+    h->steps -= 1;
+    h->truncated = true;
+    return SEGKV_OK;
+}
+
+int segkv_get_ancestry(segkv_t h, int32_t* host_out, void* stream) {
+    if (!h || !host_out) return SEGKV_EINVAL;
+    if (h->truncated) return SEGKV_ESTATE;   // the table of the dropped step is what is stored
+    if (h->steps == 0) return SEGKV_OK;
+    const Dims& d = h->d;
+    const int32_t* src = h->anc[(h->steps - 1) & 1];
+    SEGKV_CUDA(cudaMemcpy2DAsync(host_out, (size_t)h->steps * sizeof(int32_t), src,
+                                 (size_t)d.max_steps * sizeof(int32_t), (size_t)h->steps * sizeof(int32_t),
+                                 d.rows, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    SEGKV_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    return SEGKV_OK;
+}
+
+int segkv_get_unique_rows(segkv_t h, int32_t* host_out, void* stream) {
+    if (!h || !host_out) return SEGKV_EINVAL;
+    if (h->truncated) return SEGKV_ESTATE;
+    if (h->steps == 0) {
+        memset(host_out, 0, (size_t)h->d.batch * sizeof(int32_t));
+        return SEGKV_OK;
+    }
+    SEGKV_CUDA(cudaMemcpyAsync(host_out, h->ucount, (size_t)h->d.batch * sizeof(int32_t), cudaMemcpyDeviceToHost,
+                               (cudaStream_t)stream));
+    SEGKV_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    return SEGKV_OK;
+}
+
+int segkv_get_error(segkv_t h, int* device_flags) {
+    if (!h || !device_flags) return SEGKV_EINVAL;
+    SEGKV_CUDA(cudaDeviceSynchronize());
+    SEGKV_CUDA(cudaMemcpy(device_flags, h->err_word, sizeof(int), cudaMemcpyDeviceToHost));
+    SEGKV_CUDA(cudaMemset(h->err_word, 0, sizeof(int)));
+    return SEGKV_OK;
+}
+
+int segkv_steps(segkv_t h) { return h ? h->steps : SEGKV_EINVAL; }
+int segkv_prompt_len(segkv_t h) { return h ? h->prompt_len : SEGKV_EINVAL; }
+
+int segkv_set_splits(segkv_t h, int splits) {
+    if (!h || splits < 0 || splits > 1024) return SEGKV_EINVAL;
+    h->splits_forced = splits;
+    return SEGKV_OK;
+}
+
+int segkv_get_splits(segkv_t h) {
+    if (!h) return SEGKV_EINVAL;
+    return h->splits_forced > 0 ? h->splits_forced : 1;
+}
+
+long long segkv_launch_count(segkv_t h) { return h ? h->launches : (long long)SEGKV_EINVAL; }
+
+}  // extern "C"

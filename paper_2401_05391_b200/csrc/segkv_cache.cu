@@ -1,0 +1,194 @@
+// Cache-maintenance kernels: prompt store at prefill, per-step append and the
+// beam-index (ancestry) update.
+#include "segkv_internal.h"
+
+namespace segkv_impl {
+
+// ---------------------------------------------------------------------------
+// Prompt store (paper Section 3.2: prompt K/V generated at prefill and kept
+// once per request).  Input token-major [B, P, Hkv, D]; stored head-major
+// [B, Hkv, max_prompt, D] so that each (request, kv head) slab is one
+// contiguous [P, D] matrix the attention kernel can fetch with 2-D TMA boxes.
+// One thread moves one 16-byte chunk; consecutive threads read consecutive
+// chunks of the source.
+// ---------------------------------------------------------------------------
+__global__ void prefill_transpose_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v,
+                                         uint4* __restrict__ kp, uint4* __restrict__ vp, int B, int P,
+                                         int Hkv, int chunks /* D*2/16 */, int max_prompt) {
+    const long long total = (long long)B * P * Hkv * chunks;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        int c = (int)(i % chunks);
+        long long r = i / chunks;
+        int h = (int)(r % Hkv);
+        r /= Hkv;
+        int p = (int)(r % P);
+        int b = (int)(r / P);
+        long long dst = (((long long)b * Hkv + h) * max_prompt + p) * chunks + c;
+        kp[dst] = k[i];
+        vp[dst] = v[i];
+    }
+}
+
+cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v, void* kp, void* vp,
+                                     int prompt_len, cudaStream_t st) {
+    const int chunks = d.head_dim * 2 / 16;
+    long long total = (long long)d.batch * prompt_len * d.kv_heads * chunks;
+    if (total == 0) return cudaSuccess;
+    int threads = 256;
+    long long blocks = (total + threads - 1) / threads;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    prefill_transpose_kernel<<<(unsigned)blocks, threads, 0, st>>>(
+        (const uint4*)k, (const uint4*)v, (uint4*)kp, (uint4*)vp, d.batch, prompt_len, d.kv_heads, chunks,
+        d.max_prompt);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// Append + beam-index update, one launch per decode step.
+//
+// Blocks [0, B) update the beam-index table of one request each; the remaining
+// blocks copy the step's new K/V rows into slab `step` of the response segment
+// (Section 3.1: Key_t / Value_t are kept in place, no Cat) and record the
+// parent ids as row `step` of the parent table.
+//
+// Index table (Section 3.3, "Index select fusion"): anc_t[g][s] is the row of
+// slab s that beam slot g reads.  Re-ordering the whole past cache by the beam
+// indices at every step (Section 3.1) is the recurrence
+//     anc_t[g][s] = anc_{t-1}[ b*W + parent_t[g] ][s]   for s < t,
+//     anc_t[g][t] = g,
+// which is independent per s, so one thread takes one step s and the update
+// has no serial chain.  Two generations are kept (t & 1).
+//
+// While the W rows of a step are in registers the same thread also emits the
+// step's DISTINCT rows with the set of beams that read each (a bit mask), and
+// a block-wide prefix sum packs them into the request's list.  The attention
+// kernel walks that list, so a row shared by several beams is fetched once.
+// ---------------------------------------------------------------------------
+constexpr int kBtThreads = 256;
+
+__device__ __forceinline__ int warp_incl_scan(int v) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, v, o);
+        if ((threadIdx.x & 31) >= o) v += n;
+    }
+    return v;
+}
+
+__global__ void __launch_bounds__(kBtThreads)
+append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __restrict__ beam_parent,
+              const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, uint4* __restrict__ kr_slab,
+              uint4* __restrict__ vr_slab, long long slab_chunks, int32_t* __restrict__ parent_row,
+              const int32_t* __restrict__ anc_prev, int32_t* __restrict__ anc_cur, URow* __restrict__ ulist,
+              int32_t* __restrict__ ucount, int* __restrict__ err_word) {
+    if ((int)blockIdx.x >= B) {
+        // ---- copy blocks -------------------------------------------------
+        const long long nb = gridDim.x - B;
+        const long long first = ((long long)blockIdx.x - B) * blockDim.x + threadIdx.x;
+        for (long long i = first; i < slab_chunks; i += nb * blockDim.x) {
+            kr_slab[i] = k_new[i];
+            vr_slab[i] = v_new[i];
+        }
+        if (beam_parent != nullptr)
+            for (long long i = first; i < rows; i += nb * blockDim.x) parent_row[i] = beam_parent[i];
+        else
+            for (long long i = first; i < rows; i += nb * blockDim.x) parent_row[i] = (int)(i % W);
+        return;
+    }
+
+    // ---- index-table block of request b ------------------------------------
+    const int b = blockIdx.x;
+    const int tid = threadIdx.x;
+    __shared__ int s_par[kMaxCols];
+    __shared__ int s_warp[kBtThreads / 32];
+    __shared__ int s_base;
+    if (tid < W) {
+        int p = tid;
+        if (step > 0) {
+            p = beam_parent[b * W + tid];
+            if (p < 0 || p >= W) {
+                atomicOr(err_word, SEGKV_DEV_BAD_PARENT);
+                p = p < 0 ? 0 : W - 1;
+            }
+        }
+        s_par[tid] = p;
+    }
+    if (tid == 0) s_base = 0;
+    __syncthreads();
+
+    URow* list = ulist + (size_t)b * W * max_steps;
+    const int n = step + 1;
+    for (int s0 = 0; s0 < n; s0 += kBtThreads) {
+        const int s = s0 + tid;
+        int r[kMaxCols];
+        int cnt = 0;
+        if (s < n) {
+#pragma unroll 4
+            for (int j = 0; j < W; ++j) {
+                int v = (s == step) ? b * W + j
+                                    : anc_prev[(size_t)(b * W + s_par[j]) * max_steps + s];
+                r[j] = v;
+                anc_cur[(size_t)(b * W + j) * max_steps + s] = v;
+            }
+            for (int j = 0; j < W; ++j) {
+                bool first = true;
+                for (int i = 0; i < j; ++i) first = first && (r[i] != r[j]);
+                cnt += first ? 1 : 0;
+            }
+        }
+        // exclusive prefix of cnt over the block
+        int incl = warp_incl_scan(cnt);
+        if ((tid & 31) == 31) s_warp[tid >> 5] = incl;
+        __syncthreads();
+        int woff = 0, total = 0;
+#pragma unroll
+        for (int w = 0; w < kBtThreads / 32; ++w) {
+            int v = s_warp[w];
+            if (w < (tid >> 5)) woff += v;
+            total += v;
+        }
+        int pos = s_base + woff + incl - cnt;
+        if (s < n) {
+            for (int j = 0; j < W; ++j) {
+                bool first = true;
+                uint32_t mask = 0;
+                for (int i = 0; i < W; ++i) {
+                    bool same = (r[i] == r[j]);
+                    if (same && i < j) first = false;
+                    mask |= same ? (1u << i) : 0u;
+                }
+                if (first) {
+                    URow u;
+                    u.row = s * rows + r[j];
+                    u.mask = mask;
+                    list[pos++] = u;
+                }
+            }
+        }
+        __syncthreads();
+        if (tid == 0) s_base += total;
+        __syncthreads();
+    }
+    if (tid == 0) ucount[b] = s_base;
+}
+
+cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, const void* k_new,
+                          const void* v_new, void* kr, void* vr, int32_t* parent_tab,
+                          const int32_t* anc_prev, int32_t* anc_cur, URow* ulist, int32_t* ucount,
+                          int* err_word, int sm_count, cudaStream_t st) {
+    const long long slab_elems = (long long)d.rows * d.kv_heads * d.head_dim;
+    const long long slab_chunks = slab_elems * 2 / 16;
+    long long copy_blocks = (slab_chunks + kBtThreads * 4 - 1) / (kBtThreads * 4);
+    if (copy_blocks < 1) copy_blocks = 1;
+    if (copy_blocks > (long long)sm_count * 8) copy_blocks = (long long)sm_count * 8;
+    uint4* kr_slab = (uint4*)((char*)kr + (size_t)step * slab_elems * 2);
+    uint4* vr_slab = (uint4*)((char*)vr + (size_t)step * slab_elems * 2);
+    append_kernel<<<(unsigned)(d.batch + copy_blocks), kBtThreads, 0, st>>>(
+        d.batch, d.beams, d.rows, d.max_steps, step, step > 0 ? beam_parent : nullptr, (const uint4*)k_new,
+        (const uint4*)v_new, kr_slab, vr_slab, slab_chunks, parent_tab + (size_t)step * d.rows, anc_prev,
+        anc_cur, ulist, ucount, err_word);
+    return cudaGetLastError();
+}
+
+}  // namespace segkv_impl

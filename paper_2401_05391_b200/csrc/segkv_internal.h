@@ -1,0 +1,98 @@
+// Internal declarations shared by the segkv translation units (host API and kernels).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "segkv.h"
+
+namespace segkv_impl {
+
+constexpr int kMaxCols = 32;       // beams * (heads/kv_heads) handled by one CTA
+constexpr int kTileKeys = 64;      // keys per shared-memory tile of the attention kernel
+
+// One entry of the per-request list of DISTINCT response rows: `row` indexes the
+// response segment's [step*rows + slot] axis, `mask` has bit j set when beam j of
+// the request reads this row.
+struct URow {
+    int32_t row;
+    uint32_t mask;
+};
+
+struct Dims {
+    int batch, beams, heads, kv_heads, head_dim, group;  // group = heads / kv_heads
+    int max_prompt, max_steps;
+    int rows;                                            // batch * beams
+    int dtype;
+};
+
+}  // namespace segkv_impl
+
+struct segkv {
+    segkv_impl::Dims d;
+    int device;
+    int sm_count;
+    size_t smem_optin;
+    // state
+    int prompt_len;      // -1 until segkv_prefill_write
+    int steps;
+    bool truncated;      // last state change was segkv_truncate_last
+    int splits_forced;   // 0 = automatic
+    long long launches;
+    // device storage (owned)
+    void* kp;            // [batch, kv_heads, max_prompt, D]
+    void* vp;
+    void* kr;            // [max_steps, rows, kv_heads, D]
+    void* vr;
+    int32_t* parent;     // [max_steps, rows]
+    int32_t* anc[2];     // [rows, max_steps], generation t lives in anc[t & 1]
+    segkv_impl::URow* ulist;   // [batch, beams*max_steps]
+    int32_t* ucount;     // [batch]
+    int* err_word;       // device error word
+    float* ws;           // split workspace
+    size_t ws_bytes;
+    int* tickets;        // [batch*kv_heads] arrival counters, zero between launches
+    int ws_splits;       // splits the workspace was sized for
+    // staging for segkv_step_host
+    void *st_q, *st_out, *st_k, *st_v;
+    int32_t* st_parent;
+    float* st_slopes;
+    // tensor maps of the prompt segment (valid once prompt_len > 0)
+    CUtensorMap tm_kp, tm_vp;
+    bool tm_valid;
+};
+
+namespace segkv_impl {
+
+// ---- kernels (each returns the cudaError_t of its launch) -----------------
+cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v, void* kp, void* vp,
+                                     int prompt_len, cudaStream_t st);
+
+cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, const void* k_new,
+                          const void* v_new, void* kr, void* vr, int32_t* parent_tab,
+                          const int32_t* anc_prev, int32_t* anc_cur, URow* ulist, int32_t* ucount,
+                          int* err_word, int sm_count, cudaStream_t st);
+
+struct SdpaArgs {
+    const void* q;
+    void* out;
+    const float* slopes;
+    const void* kp;
+    const void* vp;
+    const void* kr;
+    const void* vr;
+    const int32_t* anc;      // generation of the newest step
+    const URow* ulist;
+    const int32_t* ucount;
+    float* ws;
+    int* tickets;
+    int* err_word;
+    int prompt_len, steps, splits;
+};
+
+// Plain gather kernel: one CTA per (beam slot, head), fp32 ALU; kept for shapes
+// the tiled kernel does not cover and as an in-library cross-check.
+cudaError_t launch_sdpa_rowwise(const Dims& d, const SdpaArgs& a, cudaStream_t st);
+
+}  // namespace segkv_impl

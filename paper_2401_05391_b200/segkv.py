@@ -1,0 +1,220 @@
+"""Thin ctypes binding of the segkv C-ABI (``include/segkv.h``).
+
+Argument marshalling only: every step of the decode path runs in the library's
+CUDA kernels.  PyTorch appears only as the owner of device memory and streams.
+The module-level functions carry the C names; :class:`SegKV` wraps a handle.
+There is no fallback: if ``libsegkv.so`` has not been built the import of the
+library fails with an error that says how to build it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libsegkv.so")
+
+SEGKV_F16, SEGKV_BF16 = 0, 1
+SEGKV_OK, SEGKV_EINVAL, SEGKV_ESTATE, SEGKV_ECAPACITY, SEGKV_ENOMEM, SEGKV_ECUDA, SEGKV_EDEVICE = 0, -1, -2, -3, -4, -5, -6
+SEGKV_DEV_BAD_PARENT, SEGKV_DEV_WAIT_LIMIT = 1, 2
+
+_vp, _int, _i32p = ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int32)
+
+# name -> (restype, argtypes); one entry per symbol include/segkv.h declares
+SIGNATURES = {
+    "segkv_create": (_int, [ctypes.POINTER(_vp)] + [_int] * 8),
+    "segkv_destroy": (_int, [_vp]),
+    "segkv_prefill_write": (_int, [_vp, _vp, _vp, _int, _vp]),
+    "segkv_append": (_int, [_vp, _int, _vp, _vp, _vp, _vp]),
+    "segkv_decode_sdpa": (_int, [_vp, _vp, _vp, _vp, _vp]),
+    "segkv_step_host": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "segkv_reset": (_int, [_vp, _int]),
+    "segkv_truncate_last": (_int, [_vp]),
+    "segkv_get_ancestry": (_int, [_vp, _vp, _vp]),
+    "segkv_get_unique_rows": (_int, [_vp, _vp, _vp]),
+    "segkv_get_error": (_int, [_vp, ctypes.POINTER(_int)]),
+    "segkv_steps": (_int, [_vp]),
+    "segkv_prompt_len": (_int, [_vp]),
+    "segkv_set_splits": (_int, [_vp, _int]),
+    "segkv_get_splits": (_int, [_vp]),
+    "segkv_launch_count": (ctypes.c_longlong, [_vp]),
+    "segkv_storage_bytes": (ctypes.c_size_t, [_int] * 7),
+    "segkv_strerror": (ctypes.c_char_p, [_int]),
+    "segkv_last_cuda_error": (ctypes.c_char_p, []),
+}
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load ``libsegkv.so`` (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2401_05391_b200.build` "
+                "(needs nvcc); there is no non-CUDA fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+class SegKVError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().segkv_strerror(code).decode()
+        if code == SEGKV_ECUDA:
+            msg += ": " + lib().segkv_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != SEGKV_OK:
+        raise SegKVError(code, where)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _dev(t: Optional[torch.Tensor], shape, dtype, name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA tensor")
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: expected {tuple(shape)} {dtype}, got {tuple(t.shape)} {t.dtype}")
+    return t.data_ptr()
+
+
+def _host(t: Optional[torch.Tensor], shape, dtype, name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous host tensor")
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: expected {tuple(shape)} {dtype}, got {tuple(t.shape)} {t.dtype}")
+    return t.data_ptr()
+
+
+def segkv_storage_bytes(batch, beams, kv_heads, head_dim, max_prompt, max_steps, dtype) -> int:
+    return int(lib().segkv_storage_bytes(batch, beams, kv_heads, head_dim, max_prompt, max_steps, dtype))
+
+
+def segkv_strerror(code: int) -> str:
+    return lib().segkv_strerror(code).decode()
+
+
+class SegKV:
+    """One attention layer's segment KV cache; methods mirror the C entry points."""
+
+    def __init__(self, batch, beams, heads, kv_heads, head_dim, max_prompt, max_steps, dtype=torch.float16):
+        self.batch, self.beams, self.heads, self.kv_heads = batch, beams, heads, kv_heads
+        self.head_dim, self.max_prompt, self.max_steps = head_dim, max_prompt, max_steps
+        self.dtype = dtype
+        self.rows = batch * beams
+        code = {torch.float16: SEGKV_F16, torch.bfloat16: SEGKV_BF16}.get(dtype, -1)
+        self._h = _vp()
+        _check(lib().segkv_create(ctypes.byref(self._h), batch, beams, heads, kv_heads, head_dim,
+                                  max_prompt, max_steps, code), "segkv_create")
+
+    # ------------------------------------------------------------ life cycle
+    def destroy(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h:
+            lib().segkv_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.destroy()
+
+    # -------------------------------------------------------------- hot path
+    def prefill_write(self, k: Optional[torch.Tensor], v: Optional[torch.Tensor], stream=None) -> None:
+        p = 0 if k is None else int(k.shape[1])
+        shape = (self.batch, p, self.kv_heads, self.head_dim)
+        _check(lib().segkv_prefill_write(self._h, _dev(k, shape, self.dtype, "k"), _dev(v, shape, self.dtype, "v"),
+                                         p, _stream_ptr(stream)), "segkv_prefill_write")
+
+    def append(self, step: int, beam_parent: Optional[torch.Tensor], k_new: torch.Tensor, v_new: torch.Tensor,
+               stream=None) -> None:
+        shape = (self.rows, self.kv_heads, self.head_dim)
+        _check(lib().segkv_append(self._h, step, _dev(beam_parent, (self.rows,), torch.int32, "beam_parent"),
+                                  _dev(k_new, shape, self.dtype, "k_new"), _dev(v_new, shape, self.dtype, "v_new"),
+                                  _stream_ptr(stream)), "segkv_append")
+
+    def decode_sdpa(self, q: torch.Tensor, out: Optional[torch.Tensor] = None,
+                    alibi_slopes: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        shape = (self.rows, self.heads, self.head_dim)
+        if out is None:
+            out = torch.empty(shape, dtype=self.dtype, device=q.device)
+        _check(lib().segkv_decode_sdpa(self._h, _dev(q, shape, self.dtype, "q"), _dev(out, shape, self.dtype, "out"),
+                                       _dev(alibi_slopes, (self.heads,), torch.float32, "alibi_slopes"),
+                                       _stream_ptr(stream)), "segkv_decode_sdpa")
+        return out
+
+    def step_host(self, step: int, beam_parent, k_new, v_new, q, out, alibi_slopes=None, stream=None) -> torch.Tensor:
+        kv = (self.rows, self.kv_heads, self.head_dim)
+        qs = (self.rows, self.heads, self.head_dim)
+        _check(lib().segkv_step_host(self._h, step, _host(beam_parent, (self.rows,), torch.int32, "beam_parent"),
+                                     _host(k_new, kv, self.dtype, "k_new"), _host(v_new, kv, self.dtype, "v_new"),
+                                     _host(q, qs, self.dtype, "q"), _host(out, qs, self.dtype, "out"),
+                                     _host(alibi_slopes, (self.heads,), torch.float32, "alibi_slopes"),
+                                     _stream_ptr(stream)), "segkv_step_host")
+        return out
+
+    # ------------------------------------------------------------------ aids
+    def reset(self, keep_prompt: bool = True) -> None:
+        _check(lib().segkv_reset(self._h, int(keep_prompt)), "segkv_reset")
+
+    def truncate_last(self) -> None:
+        _check(lib().segkv_truncate_last(self._h), "segkv_truncate_last")
+
+    @property
+    def steps(self) -> int:
+        return int(lib().segkv_steps(self._h))
+
+    @property
+    def prompt_len(self) -> int:
+        return int(lib().segkv_prompt_len(self._h))
+
+    def get_ancestry(self, stream=None) -> np.ndarray:
+        out = np.empty((self.rows, self.steps), dtype=np.int32)
+        _check(lib().segkv_get_ancestry(self._h, out.ctypes.data, _stream_ptr(stream)), "segkv_get_ancestry")
+        return out
+
+    def get_unique_rows(self, stream=None) -> np.ndarray:
+        out = np.empty((self.batch,), dtype=np.int32)
+        _check(lib().segkv_get_unique_rows(self._h, out.ctypes.data, _stream_ptr(stream)), "segkv_get_unique_rows")
+        return out
+
+    def get_error(self) -> int:
+        flags = _int(0)
+        _check(lib().segkv_get_error(self._h, ctypes.byref(flags)), "segkv_get_error")
+        return flags.value
+
+    def set_splits(self, splits: int) -> None:
+        _check(lib().segkv_set_splits(self._h, splits), "segkv_set_splits")
+
+    def get_splits(self) -> int:
+        return int(lib().segkv_get_splits(self._h))
+
+    @property
+    def launch_count(self) -> int:
+        return int(lib().segkv_launch_count(self._h))

@@ -24,3 +24,15 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Build the CUDA library (if nvcc is here and it is stale) and the C oracle once per session."""
+    import shutil
+    from paper_2401_05391_b200 import build as b
+    if shutil.which(b.NVCC) or os.path.exists(b.NVCC):
+        b.build()
+    import oracle
+    oracle.build()
+    yield

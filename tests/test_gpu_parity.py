@@ -1,0 +1,176 @@
+"""GPU parity: the CUDA path against the CPU oracle, element by element, through the C-ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2401_05391_b200 import workloads as wl
+from paper_2401_05391_b200 import segkv as sk
+
+from _harness import Run, all_pairs, sampled_pairs, unique_rows_from_ancestry
+
+pytestmark = pytest.mark.gpu
+
+CHECK_STEPS = (0, 1, 2, 3, 7, 15, 16, 17, 31, 63, 127, 255)
+
+
+def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, every_step_ancestry=True):
+    r = Run(w, splits=splits)
+    try:
+        worst = 0.0
+        for t in range(w.steps):
+            r.append_next()
+            if every_step_ancestry or t in check_steps or t == w.steps - 1:
+                anc = r.h.get_ancestry()
+                ref = r.oracle_ancestry(t)
+                assert np.array_equal(anc, ref), f"beam-index table differs at step {t}"
+                assert np.array_equal(r.h.get_unique_rows(), unique_rows_from_ancestry(ref, w.batch, w.beams))
+            if t in check_steps or t == w.steps - 1:
+                out, q = r.decode()
+                worst = max(worst, r.check(out, q, t, pairs_fn(w)))
+        assert r.h.get_error() == 0
+        return worst
+    finally:
+        r.close()
+
+
+def test_tiny_every_step_all_outputs():
+    w = wl.CONFIGS[0]
+    run_workload(w, all_pairs, check_steps=tuple(range(w.steps)))
+
+
+def test_llama2_7b_shape():
+    run_workload(wl.CONFIGS[1], all_pairs)
+
+
+def test_gptj_shape_sampled():
+    run_workload(wl.CONFIGS[2], lambda w: sampled_pairs(w, 64), every_step_ancestry=False)
+
+
+@pytest.mark.parametrize("idx", [3, 4])
+def test_large_shapes_sampled(idx):
+    w = wl.CONFIGS[idx]
+    run_workload(w, lambda w: sampled_pairs(w, 64), check_steps=(0, 17, 127, 255), every_step_ancestry=False)
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("D", [64, 128, 256])
+def test_ragged_small_shapes(dtype, D):
+    # prompt not a multiple of the tile, several tiles, GQA, ALiBi on one variant
+    w = wl.Workload("ragged", 3, 3, 6, 2, D, 150, 21, dtype, "uniform", dtype == "bf16", 10 + D // 64)
+    run_workload(w, all_pairs, check_steps=(0, 1, 5, 20))
+
+
+def test_prompt_only_and_response_only():
+    w = wl.Workload("ponly", 2, 4, 4, 4, 128, 100, 4, "f16", "uniform", False, 20)
+    r = Run(w)
+    try:
+        out, q = r.decode()
+        r.check(out, q, -1, all_pairs(w))
+    finally:
+        r.close()
+    w0 = w.scaled(prompt_len=0, index=21, steps=70)
+    run_workload(w0, all_pairs, check_steps=(0, 1, 33, 69))
+
+
+def test_single_beam_and_wide_beam():
+    run_workload(wl.Workload("w1", 2, 1, 4, 4, 128, 77, 9, "f16", "uniform", False, 22), all_pairs)
+    run_workload(wl.Workload("w8", 2, 8, 2, 2, 64, 77, 40, "f16", "uniform", False, 23), all_pairs,
+                 check_steps=(0, 3, 39))
+
+
+def test_repeat_is_bit_identical_and_every_output_is_written():
+    w = wl.CONFIGS[1].scaled(steps=24)
+    r = Run(w)
+    try:
+        r.advance_to(23)
+        a, q = r.decode()
+        b, _ = r.decode(q)
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+        assert not torch.isnan(a.float()).any()
+    finally:
+        r.close()
+
+
+def test_truncate_and_reappend_gives_same_result():
+    w = wl.CONFIGS[0]
+    r = Run(w)
+    try:
+        r.advance_to(5)
+        a, q = r.decode()
+        anc = r.h.get_ancestry()
+        r.h.truncate_last()
+        with pytest.raises(sk.SegKVError):
+            r.h.truncate_last()
+        r.h.append(5, r.parents_dev[5], r.k_steps[5], r.v_steps[5])
+        b, _ = r.decode(q)
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+        assert np.array_equal(anc, r.h.get_ancestry())
+    finally:
+        r.close()
+
+
+def test_step_host_matches_device_calls():
+    w = wl.CONFIGS[0]
+    r = Run(w)
+    r2 = Run(w)
+    try:
+        for t in range(w.steps):
+            r.append_next()
+            out, q = r.decode()
+            qh, kh, vh = (x.cpu().pin_memory() for x in (q, r.k_steps[t], r.v_steps[t]))
+            oh = torch.empty_like(qh).pin_memory()
+            ph = torch.from_numpy(r.parents[t]).pin_memory() if t > 0 else None
+            r2.h.step_host(t, ph, kh, vh, qh, oh)
+            assert torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16))
+    finally:
+        r.close(); r2.close()
+
+
+def test_argument_and_state_errors():
+    h = sk.SegKV(1, 2, 2, 2, 64, 16, 4, torch.float16)
+    dev = "cuda"
+    k = torch.zeros(2, 2, 64, dtype=torch.float16, device=dev)
+    q = torch.zeros(2, 2, 64, dtype=torch.float16, device=dev)
+    par = torch.zeros(2, dtype=torch.int32, device=dev)
+    with pytest.raises(sk.SegKVError) as e:
+        h.append(0, None, k, k)
+    assert e.value.code == sk.SEGKV_ESTATE                      # no prefill yet
+    with pytest.raises(sk.SegKVError) as e:
+        h.prefill_write(torch.zeros(1, 17, 2, 64, dtype=torch.float16, device=dev),
+                        torch.zeros(1, 17, 2, 64, dtype=torch.float16, device=dev))
+    assert e.value.code == sk.SEGKV_ECAPACITY
+    h.prefill_write(None, None)
+    with pytest.raises(sk.SegKVError) as e:
+        h.decode_sdpa(q)
+    assert e.value.code == sk.SEGKV_ESTATE                      # nothing to attend to
+    with pytest.raises(sk.SegKVError) as e:
+        h.append(1, par, k, k)
+    assert e.value.code == sk.SEGKV_ESTATE                      # wrong step
+    for t in range(4):
+        h.append(t, par if t else None, k, k)
+    with pytest.raises(sk.SegKVError) as e:
+        h.append(4, par, k, k)
+    assert e.value.code == sk.SEGKV_ECAPACITY
+    assert h.get_error() == 0
+    h.destroy()
+    with pytest.raises(sk.SegKVError) as e:
+        sk.SegKV(1, 2, 3, 2, 64, 16, 4, torch.float16)
+    assert e.value.code == sk.SEGKV_EINVAL
+
+
+def test_out_of_range_parent_is_clamped_and_flagged():
+    w = wl.CONFIGS[0]
+    par = wl.make_parents(w)
+    bad = par.copy(); bad[3, 1] = 9; bad[4, 2] = -5
+    clamped = par.copy(); clamped[3, 1] = w.beams - 1; clamped[4, 2] = 0
+    r = Run(w, parents=bad)
+    r.parents = clamped          # what the oracle should see
+    try:
+        r.advance_to(7)
+        assert r.h.get_error() == sk.SEGKV_DEV_BAD_PARENT
+        assert r.h.get_error() == 0                 # read clears
+        assert np.array_equal(r.h.get_ancestry(), r.oracle_ancestry(7))
+        out, q = r.decode()
+        r.check(out, q, 7, all_pairs(w))
+    finally:
+        r.close()
