@@ -43,6 +43,7 @@ def parse():
     ap.add_argument("--layers", type=int, default=0, help="distinct cache handles per step (0 = per-workload default)")
     ap.add_argument("--at-step", type=int, default=0, help="decode step to time, 1-based (0 = the workload's last)")
     ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -202,8 +203,8 @@ def run_ours(args):
     for layer in range(L):
         wl_layer = w_rank.scaled(index=w_rank.index + 1000 * layer)
         h = SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, w.steps, w.torch_dtype)
-        if args.splits:
-            h.set_splits(args.splits)
+        if args.splits or args.stages:
+            h.set_tuning(args.splits, args.stages)
         kp, vp = wl.make_prompt(wl_layer, dev)
         h.prefill_write(kp, vp)
         del kp, vp

@@ -169,13 +169,24 @@ SEGKV_API int segkv_steps(segkv_t h);
 SEGKV_API int segkv_prompt_len(segkv_t h);
 
 /*
- * Force the number of KV splits per (request, kv head) of the attention kernel
- * (0 = choose automatically from the shape, the default).  Re-allocates the
- * split workspace; synchronises the device.  segkv_get_splits returns the value
- * the next segkv_decode_sdpa will use.
+ * Override the launch shape of the attention kernel: `splits` = CTAs that share
+ * the keys of one (request, kv head) work group, `stages` = depth of the
+ * shared-memory ring; 0 = choose automatically from the shape (the default).
+ * EINVAL if the stages do not fit in shared memory.  segkv_get_splits returns
+ * the split count the next segkv_decode_sdpa will use.
  */
-SEGKV_API int segkv_set_splits(segkv_t h, int splits);
+SEGKV_API int segkv_set_tuning(segkv_t h, int splits, int stages);
 SEGKV_API int segkv_get_splits(segkv_t h);
+
+/*
+ * The same attention as segkv_decode_sdpa computed by the plain per-beam kernel
+ * (each beam walks its own rows through the beam-index table, Section 3.3's
+ * formulation taken literally; the prompt is re-read per beam).  Used for
+ * shapes with more than 16 query columns per kv head, and as a cross-check.
+ * Arguments and errors as segkv_decode_sdpa.
+ */
+SEGKV_API int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, const float* alibi_slopes,
+                                        void* stream);
 
 /* Kernels launched by the handle since creation (each launch counted once). */
 SEGKV_API long long segkv_launch_count(segkv_t h);

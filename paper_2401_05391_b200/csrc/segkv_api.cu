@@ -57,7 +57,7 @@ EncodeTiledFn encode_tiled_fn() {
 
 // Tensor map over one prompt array seen as [batch*kv_heads][prompt_len][D]:
 // rows >= prompt_len read as zero, a box never crosses a (request, head) slab.
-// Box = 64 elements (128 bytes, one swizzle span) x kTileKeys rows.
+// Box = 64 elements (128 bytes, one swizzle span) x one tile of rows.
 int make_prompt_map(const segkv* h, void* base, int prompt_len, CUtensorMap* out) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) {
@@ -67,7 +67,7 @@ int make_prompt_map(const segkv* h, void* base, int prompt_len, CUtensorMap* out
     const Dims& d = h->d;
     cuuint64_t dims[3] = {(cuuint64_t)d.head_dim, (cuuint64_t)prompt_len, (cuuint64_t)d.batch * d.kv_heads};
     cuuint64_t strides[2] = {(cuuint64_t)d.head_dim * 2, (cuuint64_t)d.max_prompt * d.head_dim * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)kTileKeys, 1};
+    cuuint32_t box[3] = {64, (cuuint32_t)tiled_tile_keys(d.head_dim), 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUtensorMapDataType dt = d.dtype == SEGKV_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
     CUresult r = fn(out, dt, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -105,6 +105,38 @@ int alloc_workspace(segkv* h, int splits) {
     h->ws_bytes = bytes;
     h->ws_splits = splits;
     return SEGKV_OK;
+}
+
+// Launch shape of the tiled kernel.  Stages: as many as keep two CTAs resident per SM.
+// Splits: none when the work groups alone fill the GPU twice over, else enough to give
+// every CTA slot of one wave a share (never less than one tile each).
+void choose_tiling(const segkv* h, int* splits, int* stages) {
+    const Dims& d = h->d;
+    int st = h->stages_forced;
+    if (st <= 0) {
+        st = 2;
+        const size_t budget = (h->smem_optin + 1024) / 2 - 1024 - 2048;
+        while (st < 8 && tiled_smem_bytes(d, st + 1) <= budget) ++st;
+    }
+    while (st > 1 && tiled_smem_bytes(d, st) > h->smem_optin) --st;
+    int sp = h->splits_forced;
+    if (sp <= 0) {
+        const int tile = tiled_tile_keys(d.head_dim);
+        const int P = h->prompt_len > 0 ? h->prompt_len : 0;
+        const long long tiles = (P + tile - 1) / tile + (h->steps + 2 * d.beams + tile - 1) / tile;
+        const long long slabs = (long long)d.batch * d.kv_heads;
+        const long long slots = (long long)h->sm_count * 2;
+        sp = 1;
+        if (slabs < 2 * slots) {
+            long long want = slots / slabs;
+            if (want > tiles) want = tiles;
+            if (want > 64) want = 64;
+            if (want < 1) want = 1;
+            sp = (int)want;
+        }
+    }
+    *splits = sp;
+    *stages = st;
 }
 
 SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes, int splits) {
@@ -263,8 +295,22 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
     if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SEGKV_EINVAL;
     if (h->prompt_len < 0) return SEGKV_ESTATE;
     if (h->prompt_len + h->steps <= 0) return SEGKV_ESTATE;
-    SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, 1);
-    SEGKV_CUDA(launch_sdpa_rowwise(h->d, a, (cudaStream_t)stream));
+    if (!tiled_supported(h->d)) {
+        SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, 1);
+        SEGKV_CUDA(launch_sdpa_rowwise(h->d, a, (cudaStream_t)stream));
+        h->launches++;
+        return SEGKV_OK;
+    }
+    int splits, stages;
+    choose_tiling(h, &splits, &stages);
+    if (splits > h->ws_splits) {
+        // growing the workspace must not race with work still using the old one
+        SEGKV_CUDA(cudaDeviceSynchronize());
+        int rc = alloc_workspace(h, splits);
+        if (rc != SEGKV_OK) return rc;
+    }
+    SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, splits);
+    SEGKV_CUDA(launch_sdpa_tiled(h->d, a, h->tm_kp, h->tm_vp, stages, (cudaStream_t)stream));
     h->launches++;
     return SEGKV_OK;
 }
@@ -351,15 +397,31 @@ int segkv_get_error(segkv_t h, int* device_flags) {
 int segkv_steps(segkv_t h) { return h ? h->steps : SEGKV_EINVAL; }
 int segkv_prompt_len(segkv_t h) { return h ? h->prompt_len : SEGKV_EINVAL; }
 
-int segkv_set_splits(segkv_t h, int splits) {
-    if (!h || splits < 0 || splits > 1024) return SEGKV_EINVAL;
+int segkv_set_tuning(segkv_t h, int splits, int stages) {
+    if (!h || splits < 0 || splits > 1024 || stages < 0 || stages > 16) return SEGKV_EINVAL;
+    if (stages > 0 && tiled_smem_bytes(h->d, stages) > h->smem_optin) return SEGKV_EINVAL;
     h->splits_forced = splits;
+    h->stages_forced = stages;
     return SEGKV_OK;
 }
 
 int segkv_get_splits(segkv_t h) {
     if (!h) return SEGKV_EINVAL;
-    return h->splits_forced > 0 ? h->splits_forced : 1;
+    if (!tiled_supported(h->d)) return 1;
+    int splits, stages;
+    choose_tiling(h, &splits, &stages);
+    return splits;
+}
+
+int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, const float* alibi_slopes, void* stream) {
+    if (!h || !q || !out || !aligned16(q) || !aligned16(out)) return SEGKV_EINVAL;
+    if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SEGKV_EINVAL;
+    if (h->prompt_len < 0) return SEGKV_ESTATE;
+    if (h->prompt_len + h->steps <= 0) return SEGKV_ESTATE;
+    SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, 1);
+    SEGKV_CUDA(launch_sdpa_rowwise(h->d, a, (cudaStream_t)stream));
+    h->launches++;
+    return SEGKV_OK;
 }
 
 long long segkv_launch_count(segkv_t h) { return h ? h->launches : (long long)SEGKV_EINVAL; }

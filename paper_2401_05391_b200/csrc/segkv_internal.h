@@ -10,7 +10,6 @@
 namespace segkv_impl {
 
 constexpr int kMaxCols = 32;       // beams * (heads/kv_heads) handled by one CTA
-constexpr int kTileKeys = 64;      // keys per shared-memory tile of the attention kernel
 
 // One entry of the per-request list of DISTINCT response rows: `row` indexes the
 // response segment's [step*rows + slot] axis, `mask` has bit j set when beam j of
@@ -39,6 +38,7 @@ struct segkv {
     int steps;
     bool truncated;      // last state change was segkv_truncate_last
     int splits_forced;   // 0 = automatic
+    int stages_forced;   // 0 = automatic
     long long launches;
     // device storage (owned)
     void* kp;            // [batch, kv_heads, max_prompt, D]
@@ -94,5 +94,12 @@ struct SdpaArgs {
 // Plain gather kernel: one CTA per (beam slot, head), fp32 ALU; kept for shapes
 // the tiled kernel does not cover and as an in-library cross-check.
 cudaError_t launch_sdpa_rowwise(const Dims& d, const SdpaArgs& a, cudaStream_t st);
+
+// Tiled split-KV kernel (TMA-staged prompt tiles, gathered response rows, tensor-core tiles).
+bool tiled_supported(const Dims& d);
+int tiled_tile_keys(int head_dim);                       // rows of one shared-memory tile
+size_t tiled_smem_bytes(const Dims& d, int stages);      // dynamic shared memory of one CTA
+cudaError_t launch_sdpa_tiled(const Dims& d, const SdpaArgs& a, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                              int stages, cudaStream_t st);
 
 }  // namespace segkv_impl

@@ -39,7 +39,8 @@ SIGNATURES = {
     "segkv_get_error": (_int, [_vp, ctypes.POINTER(_int)]),
     "segkv_steps": (_int, [_vp]),
     "segkv_prompt_len": (_int, [_vp]),
-    "segkv_set_splits": (_int, [_vp, _int]),
+    "segkv_set_tuning": (_int, [_vp, _int, _int]),
+    "segkv_decode_sdpa_rowwise": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "segkv_get_splits": (_int, [_vp]),
     "segkv_launch_count": (ctypes.c_longlong, [_vp]),
     "segkv_storage_bytes": (ctypes.c_size_t, [_int] * 7),
@@ -209,8 +210,19 @@ class SegKV:
         _check(lib().segkv_get_error(self._h, ctypes.byref(flags)), "segkv_get_error")
         return flags.value
 
-    def set_splits(self, splits: int) -> None:
-        _check(lib().segkv_set_splits(self._h, splits), "segkv_set_splits")
+    def set_tuning(self, splits: int = 0, stages: int = 0) -> None:
+        _check(lib().segkv_set_tuning(self._h, splits, stages), "segkv_set_tuning")
+
+    def decode_sdpa_rowwise(self, q: torch.Tensor, out: Optional[torch.Tensor] = None,
+                            alibi_slopes: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        shape = (self.rows, self.heads, self.head_dim)
+        if out is None:
+            out = torch.empty(shape, dtype=self.dtype, device=q.device)
+        _check(lib().segkv_decode_sdpa_rowwise(self._h, _dev(q, shape, self.dtype, "q"),
+                                               _dev(out, shape, self.dtype, "out"),
+                                               _dev(alibi_slopes, (self.heads,), torch.float32, "alibi_slopes"),
+                                               _stream_ptr(stream)), "segkv_decode_sdpa_rowwise")
+        return out
 
     def get_splits(self) -> int:
         return int(lib().segkv_get_splits(self._h))

@@ -13,8 +13,8 @@ pytestmark = pytest.mark.gpu
 CHECK_STEPS = (0, 1, 2, 3, 7, 15, 16, 17, 31, 63, 127, 255)
 
 
-def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, every_step_ancestry=True):
-    r = Run(w, splits=splits)
+def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, every_step_ancestry=True):
+    r = Run(w, splits=splits, stages=stages)
     try:
         worst = 0.0
         for t in range(w.steps):
@@ -58,6 +58,27 @@ def test_ragged_small_shapes(dtype, D):
     # prompt not a multiple of the tile, several tiles, GQA, ALiBi on one variant
     w = wl.Workload("ragged", 3, 3, 6, 2, D, 150, 21, dtype, "uniform", dtype == "bf16", 10 + D // 64)
     run_workload(w, all_pairs, check_steps=(0, 1, 5, 20))
+
+
+@pytest.mark.parametrize("splits,stages", [(1, 0), (2, 2), (5, 1), (19, 3), (40, 0)])
+def test_forced_splits_and_stages(splits, stages):
+    # more splits than tiles leaves some CTAs without keys; one stage serialises the ring
+    w = wl.CONFIGS[1].scaled(steps=40, index=30)
+    run_workload(w, lambda w: sampled_pairs(w, 12), check_steps=(0, 7, 39), splits=splits, stages=stages,
+                 every_step_ancestry=False)
+
+
+def test_tiled_kernel_agrees_with_rowwise_kernel():
+    w = wl.Workload("cross", 2, 4, 8, 4, 128, 333, 30, "bf16", "uniform", True, 31)
+    r = Run(w)
+    try:
+        r.advance_to(29)
+        a, q = r.decode()
+        b = r.h.decode_sdpa_rowwise(q, None, r.slopes)
+        torch.cuda.synchronize()
+        assert torch.allclose(a.float(), b.float(), atol=4e-3, rtol=2e-2)
+    finally:
+        r.close()
 
 
 def test_prompt_only_and_response_only():
