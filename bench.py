@@ -44,7 +44,9 @@ def parse():
     ap.add_argument("--at-step", type=int, default=0, help="decode step to time, 1-based (0 = the workload's last)")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--combine", type=int, default=0, help="0 auto, 1 workspace+ticket, 2 cluster")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true", help="turn programmatic dependent launch off")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -203,8 +205,10 @@ def run_ours(args):
     for layer in range(L):
         wl_layer = w_rank.scaled(index=w_rank.index + 1000 * layer)
         h = SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, w.steps, w.torch_dtype)
-        if args.splits or args.stages:
-            h.set_tuning(args.splits, args.stages)
+        if args.splits or args.stages or args.combine:
+            h.set_tuning(args.splits, args.stages, args.combine)
+        if args.no_overlap:
+            h.set_overlap(False)
         kp, vp = wl.make_prompt(wl_layer, dev)
         h.prefill_write(kp, vp)
         del kp, vp
@@ -328,7 +332,7 @@ def run_ours(args):
         "dtype": "f16" if w.dtype == "f16" else "bf16", "data": "synthetic",
         "config": {"workload": w.name, "batch": w.batch, "beams": w.beams, "heads": w.heads, "kv_heads": w.kv_heads,
                    "head_dim": w.head_dim, "prompt_len": w.prompt_len, "at_step": T, "layers_per_step": L,
-                   "l2": f"{L} distinct layer caches per step, {L * ubytes / 1e6:.0f} MB > L2", "cuda_graph": graphed,
+                   "l2": f"{L} distinct layer caches per step, {L * ubytes / 1e6:.0f} MB > L2", "cuda_graph": graphed, "dependent_launch": not args.no_overlap,
                    "splits": handles[0][0].get_splits(), "parallelism": f"replica x{world}" if world > 1 else "1 gpu"},
         "us_per_step_per_layer": us_layer,
         "us_sdpa_per_layer": us_sdpa,

@@ -170,12 +170,16 @@ SEGKV_API int segkv_prompt_len(segkv_t h);
 
 /*
  * Override the launch shape of the attention kernel: `splits` = CTAs that share
- * the keys of one (request, kv head) work group, `stages` = depth of the
- * shared-memory ring; 0 = choose automatically from the shape (the default).
- * EINVAL if the stages do not fit in shared memory.  segkv_get_splits returns
- * the split count the next segkv_decode_sdpa will use.
+ * the keys of one (request, kv head) work group (at most 64), `stages` = depth
+ * of the shared-memory ring, `combine` = how the splits are merged: 1 = partials
+ * in a global workspace, merged by the last CTA to arrive; 2 = inside a
+ * thread-block cluster through distributed shared memory (splits must be 2, 4
+ * or 8).  0 = choose automatically from the shape (the default).  EINVAL if the
+ * stages do not fit in shared memory; a forced cluster merge that the split
+ * count does not allow is reported by the next segkv_decode_sdpa.
+ * segkv_get_splits returns the split count the next segkv_decode_sdpa will use.
  */
-SEGKV_API int segkv_set_tuning(segkv_t h, int splits, int stages);
+SEGKV_API int segkv_set_tuning(segkv_t h, int splits, int stages, int combine);
 SEGKV_API int segkv_get_splits(segkv_t h);
 
 /*
@@ -187,6 +191,16 @@ SEGKV_API int segkv_get_splits(segkv_t h);
  */
 SEGKV_API int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, const float* alibi_slopes,
                                         void* stream);
+
+/*
+ * Programmatic dependent launch between the library's consecutive kernels on a
+ * stream (on by default): a kernel may start while the previous one drains, and
+ * the attention kernel requests its prompt tiles, which no decode-time call
+ * modifies, before the previous kernel has finished; everything else is ordered
+ * after it.  The first append after a prefill is always a fully serialised
+ * launch.  enable == 0 turns it off (plain stream order).
+ */
+SEGKV_API int segkv_set_overlap(segkv_t h, int enable);
 
 /* Kernels launched by the handle since creation (each launch counted once). */
 SEGKV_API long long segkv_launch_count(segkv_t h);

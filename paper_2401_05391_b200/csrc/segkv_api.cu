@@ -110,33 +110,45 @@ int alloc_workspace(segkv* h, int splits) {
 // Launch shape of the tiled kernel.  Stages: as many as keep two CTAs resident per SM.
 // Splits: none when the work groups alone fill the GPU twice over, else enough to give
 // every CTA slot of one wave a share (never less than one tile each).
-void choose_tiling(const segkv* h, int* splits, int* stages) {
+void choose_tiling(const segkv* h, int* splits, int* stages, bool* cluster) {
     const Dims& d = h->d;
-    int st = h->stages_forced;
-    if (st <= 0) {
-        st = 2;
-        const size_t budget = (h->smem_optin + 1024) / 2 - 1024 - 2048;
-        while (st < 8 && tiled_smem_bytes(d, st + 1) <= budget) ++st;
-    }
-    while (st > 1 && tiled_smem_bytes(d, st) > h->smem_optin) --st;
+    const int tile = tiled_tile_keys(d.head_dim);
+    const int P = h->prompt_len > 0 ? h->prompt_len : 0;
+    const long long ntp = (P + tile - 1) / tile;
+    const long long ntr = (h->steps + 2 * d.beams + tile - 1) / tile;      // estimate, rows are mostly shared
+    const long long slabs = (long long)d.batch * d.kv_heads;
+    const long long slots = (long long)h->sm_count * 2;
     int sp = h->splits_forced;
     if (sp <= 0) {
-        const int tile = tiled_tile_keys(d.head_dim);
-        const int P = h->prompt_len > 0 ? h->prompt_len : 0;
-        const long long tiles = (P + tile - 1) / tile + (h->steps + 2 * d.beams + tile - 1) / tile;
-        const long long slabs = (long long)d.batch * d.kv_heads;
-        const long long slots = (long long)h->sm_count * 2;
         sp = 1;
         if (slabs < 2 * slots) {
             long long want = slots / slabs;
-            if (want > tiles) want = tiles;
-            if (want > 64) want = 64;
+            if (want > ntp + ntr) want = ntp + ntr;
             if (want < 1) want = 1;
-            sp = (int)want;
+            // the fewest splits that reach the same number of prompt tiles per CTA
+            const long long per = ntp > 0 ? (ntp + want - 1) / want : 1;
+            long long s = ntp > 0 ? (ntp + per - 1) / per : want;
+            if (s > kMaxSplits) s = kMaxSplits;
+            sp = (int)s;
         }
     }
+    if (sp > kMaxSplits) sp = kMaxSplits;
+    int st = h->stages_forced;
+    if (st <= 0) {
+        // as deep a ring as still lets two CTAs share an SM ...
+        st = 2;
+        const size_t budget = (h->smem_optin + 1024) / 2 - 1024 - 2048;
+        while (st < 8 && tiled_smem_bytes(d, st + 1) <= budget) ++st;
+        // ... or, when the whole launch is one wave, deep enough to hold a CTA's whole share
+        const long long per_cta = (ntp + sp - 1) / sp + (ntr + sp - 1) / sp;
+        if (slabs * sp <= h->sm_count && per_cta > st) {
+            while (st < per_cta && st < 8 && tiled_smem_bytes(d, st + 1) <= h->smem_optin) ++st;
+        }
+    }
+    while (st > 1 && tiled_smem_bytes(d, st) > h->smem_optin) --st;
     *splits = sp;
     *stages = st;
+    *cluster = sp > 1 && h->combine_forced != 1 && tiled_cluster_ok(d, sp);
 }
 
 SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes, int splits) {
@@ -157,6 +169,8 @@ SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes
     a.prompt_len = h->prompt_len > 0 ? h->prompt_len : 0;
     a.steps = h->steps;
     a.splits = splits;
+    a.cluster = false;
+    a.pdl = false;
     return a;
 }
 
@@ -200,6 +214,7 @@ int segkv_create(segkv_t* out, int batch, int beams, int heads, int kv_heads, in
     d.group = heads / kv_heads; d.max_prompt = max_prompt; d.max_steps = max_steps;
     d.rows = batch * beams; d.dtype = dtype;
     h->prompt_len = -1;
+    h->overlap = true;
 
     int rc = SEGKV_OK;
     auto fail = [&](int code) { free_all(h); delete h; return code; };
@@ -283,7 +298,7 @@ int segkv_append(segkv_t h, int step, const int32_t* beam_parent, const void* k_
     if (step >= h->d.max_steps) return SEGKV_ECAPACITY;
     SEGKV_CUDA(launch_append(h->d, step, beam_parent, k_new, v_new, h->kr, h->vr, h->parent,
                              h->anc[(step + 1) & 1], h->anc[step & 1], h->ulist, h->ucount, h->err_word,
-                             h->sm_count, (cudaStream_t)stream));
+                             h->sm_count, h->overlap && step > 0, (cudaStream_t)stream));
     h->launches++;
     h->steps = step + 1;
     h->truncated = false;
@@ -302,14 +317,18 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
         return SEGKV_OK;
     }
     int splits, stages;
-    choose_tiling(h, &splits, &stages);
-    if (splits > h->ws_splits) {
+    bool cluster;
+    choose_tiling(h, &splits, &stages, &cluster);
+    if (h->combine_forced == 2 && splits > 1 && !cluster) return SEGKV_EINVAL;
+    if (!cluster && splits > h->ws_splits) {
         // growing the workspace must not race with work still using the old one
         SEGKV_CUDA(cudaDeviceSynchronize());
         int rc = alloc_workspace(h, splits);
         if (rc != SEGKV_OK) return rc;
     }
     SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, splits);
+    a.cluster = cluster;
+    a.pdl = h->overlap;
     SEGKV_CUDA(launch_sdpa_tiled(h->d, a, h->tm_kp, h->tm_vp, stages, (cudaStream_t)stream));
     h->launches++;
     return SEGKV_OK;
@@ -397,11 +416,13 @@ int segkv_get_error(segkv_t h, int* device_flags) {
 int segkv_steps(segkv_t h) { return h ? h->steps : SEGKV_EINVAL; }
 int segkv_prompt_len(segkv_t h) { return h ? h->prompt_len : SEGKV_EINVAL; }
 
-int segkv_set_tuning(segkv_t h, int splits, int stages) {
-    if (!h || splits < 0 || splits > 1024 || stages < 0 || stages > 16) return SEGKV_EINVAL;
+int segkv_set_tuning(segkv_t h, int splits, int stages, int combine) {
+    if (!h || splits < 0 || splits > kMaxSplits || stages < 0 || stages > 16) return SEGKV_EINVAL;
+    if (combine < 0 || combine > 2) return SEGKV_EINVAL;
     if (stages > 0 && tiled_smem_bytes(h->d, stages) > h->smem_optin) return SEGKV_EINVAL;
     h->splits_forced = splits;
     h->stages_forced = stages;
+    h->combine_forced = combine;
     return SEGKV_OK;
 }
 
@@ -409,7 +430,8 @@ int segkv_get_splits(segkv_t h) {
     if (!h) return SEGKV_EINVAL;
     if (!tiled_supported(h->d)) return 1;
     int splits, stages;
-    choose_tiling(h, &splits, &stages);
+    bool cluster;
+    choose_tiling(h, &splits, &stages, &cluster);
     return splits;
 }
 
@@ -421,6 +443,12 @@ int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, const float* 
     SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, 1);
     SEGKV_CUDA(launch_sdpa_rowwise(h->d, a, (cudaStream_t)stream));
     h->launches++;
+    return SEGKV_OK;
+}
+
+int segkv_set_overlap(segkv_t h, int enable) {
+    if (!h) return SEGKV_EINVAL;
+    h->overlap = enable != 0;
     return SEGKV_OK;
 }
 

@@ -82,6 +82,10 @@ append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __
               uint4* __restrict__ vr_slab, long long slab_chunks, int32_t* __restrict__ parent_row,
               const int32_t* __restrict__ anc_prev, int32_t* __restrict__ anc_cur, URow* __restrict__ ulist,
               int32_t* __restrict__ ucount, int* __restrict__ err_word) {
+    // Programmatic dependent launch: the next kernel may start its prologue now; this one
+    // touches nothing until the previous kernel of the stream has completed.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if ((int)blockIdx.x >= B) {
         // ---- copy blocks -------------------------------------------------
         const long long nb = gridDim.x - B;
@@ -176,7 +180,7 @@ append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __
 cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, const void* k_new,
                           const void* v_new, void* kr, void* vr, int32_t* parent_tab,
                           const int32_t* anc_prev, int32_t* anc_cur, URow* ulist, int32_t* ucount,
-                          int* err_word, int sm_count, cudaStream_t st) {
+                          int* err_word, int sm_count, bool pdl, cudaStream_t st) {
     const long long slab_elems = (long long)d.rows * d.kv_heads * d.head_dim;
     const long long slab_chunks = slab_elems * 2 / 16;
     long long copy_blocks = (slab_chunks + kBtThreads * 4 - 1) / (kBtThreads * 4);
@@ -184,11 +188,22 @@ cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, c
     if (copy_blocks > (long long)sm_count * 8) copy_blocks = (long long)sm_count * 8;
     uint4* kr_slab = (uint4*)((char*)kr + (size_t)step * slab_elems * 2);
     uint4* vr_slab = (uint4*)((char*)vr + (size_t)step * slab_elems * 2);
-    append_kernel<<<(unsigned)(d.batch + copy_blocks), kBtThreads, 0, st>>>(
-        d.batch, d.beams, d.rows, d.max_steps, step, step > 0 ? beam_parent : nullptr, (const uint4*)k_new,
-        (const uint4*)v_new, kr_slab, vr_slab, slab_chunks, parent_tab + (size_t)step * d.rows, anc_prev,
-        anc_cur, ulist, ucount, err_word);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(d.batch + copy_blocks), 1, 1);
+    cfg.blockDim = dim3(kBtThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (pdl) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    const int32_t* bp = step > 0 ? beam_parent : nullptr;
+    return cudaLaunchKernelEx(&cfg, append_kernel, d.batch, d.beams, d.rows, d.max_steps, step, bp,
+                              (const uint4*)k_new, (const uint4*)v_new, kr_slab, vr_slab, slab_chunks,
+                              parent_tab + (size_t)step * d.rows, anc_prev, anc_cur, ulist, ucount, err_word);
 }
 
 }  // namespace segkv_impl

@@ -10,6 +10,8 @@
 namespace segkv_impl {
 
 constexpr int kMaxCols = 32;       // beams * (heads/kv_heads) handled by one CTA
+constexpr int kMaxSplits = 64;     // CTAs that may share one (request, kv head) work group
+constexpr int kMaxCluster = 8;     // largest portable thread-block cluster
 
 // One entry of the per-request list of DISTINCT response rows: `row` indexes the
 // response segment's [step*rows + slot] axis, `mask` has bit j set when beam j of
@@ -39,6 +41,8 @@ struct segkv {
     bool truncated;      // last state change was segkv_truncate_last
     int splits_forced;   // 0 = automatic
     int stages_forced;   // 0 = automatic
+    int combine_forced;  // 0 = automatic, 1 = global workspace + ticket, 2 = cluster
+    bool overlap;        // programmatic dependent launch between consecutive kernels
     long long launches;
     // device storage (owned)
     void* kp;            // [batch, kv_heads, max_prompt, D]
@@ -72,7 +76,7 @@ cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v
 cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, const void* k_new,
                           const void* v_new, void* kr, void* vr, int32_t* parent_tab,
                           const int32_t* anc_prev, int32_t* anc_cur, URow* ulist, int32_t* ucount,
-                          int* err_word, int sm_count, cudaStream_t st);
+                          int* err_word, int sm_count, bool pdl, cudaStream_t st);
 
 struct SdpaArgs {
     const void* q;
@@ -89,6 +93,8 @@ struct SdpaArgs {
     int* tickets;
     int* err_word;
     int prompt_len, steps, splits;
+    bool cluster;            // merge the splits inside a thread-block cluster
+    bool pdl;                // launch with programmatic stream serialisation
 };
 
 // Plain gather kernel: one CTA per (beam slot, head), fp32 ALU; kept for shapes
@@ -97,6 +103,7 @@ cudaError_t launch_sdpa_rowwise(const Dims& d, const SdpaArgs& a, cudaStream_t s
 
 // Tiled split-KV kernel (TMA-staged prompt tiles, gathered response rows, tensor-core tiles).
 bool tiled_supported(const Dims& d);
+bool tiled_cluster_ok(const Dims& d, int splits);        // can `splits` CTAs merge as one cluster?
 int tiled_tile_keys(int head_dim);                       // rows of one shared-memory tile
 size_t tiled_smem_bytes(const Dims& d, int stages);      // dynamic shared memory of one CTA
 cudaError_t launch_sdpa_tiled(const Dims& d, const SdpaArgs& a, const CUtensorMap& tm_k, const CUtensorMap& tm_v,

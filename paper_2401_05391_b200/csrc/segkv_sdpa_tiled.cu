@@ -137,6 +137,51 @@ template <> struct Mma<__nv_bfloat16> {
     static __device__ __forceinline__ __nv_bfloat16 down(float f) { return __float2bfloat16_rn(f); }
 };
 
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_arrive_relaxed() {
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_arrive_release() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait_acquire() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float4 v) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_cluster_v2(uint32_t addr, float a, float b) {
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
+}
+// Programmatic dependent launch: let the next kernel of the stream begin, and wait for the
+// previous one to have completed with its writes visible (no-ops without the launch attribute).
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+#ifdef SEGKV_TIMELINE
+}  // namespace
+__device__ unsigned long long g_timeline[1024 * 16];
+#define SEGKV_STAMP(ev)                                                                    \
+    do {                                                                                   \
+        if ((threadIdx.x & 31) == 0 && blockIdx.x < 1024) {                                \
+            g_timeline[blockIdx.x * 16 + (ev)] = (ev) == 0 ? global_ns() : (unsigned long long)clock64(); \
+        }                                                                                  \
+    } while (0)
+namespace {
+#else
+#define SEGKV_STAMP(ev) do {} while (0)
+#endif
+
 struct TiledParams {
     const void* q;
     void* out;
@@ -145,18 +190,22 @@ struct TiledParams {
     const char* vr;
     const URow* ulist;
     const int32_t* ucount;
-    float* ws;
+    float* ws_o;    // [slab][S][ncols][D]   un-normalised partial outputs (ticket combine only)
+    float* ws_ml;   // [slab][S][ncols][2]   running max (base-2 domain) and sum
     int* tickets;
     int* err_word;
     int P, steps, S, W, G, H, Hkv, rows, max_steps, ncols, stages;
-    float scale2;  // log2(e) / sqrt(D)
+    int cluster;    // 1: the S CTAs of a work group form a thread-block cluster
+    int early_prompt;  // 1: prompt tiles may be fetched before the previous kernel has completed
+    float scale2;   // log2(e) / sqrt(D)
 };
 
 // Shared-memory carve-up (after rounding the base up to 1024 bytes):
 //   stages x { K tile, V tile }      each tile = D/64 boxes of [TILE rows][128 B], 128B-swizzled
 //   stages x URow[TILE]              per-key row id and beam mask of response tiles
-//   full[stages], empty[stages]      mbarriers
-// The warp-merge buffer of the epilogue re-uses the stage area.
+//     (the warp-merge buffer and the ticket-combine scratch of the epilogue re-use this area)
+//   full[stages], empty[stages], hand   mbarriers
+//   recv_o, recv_ml                  landing area for the other CTAs' partials (cluster combine)
 template <int D, int CW>
 struct Layout {
     static constexpr int TILE = 16 * CW;
@@ -164,129 +213,202 @@ struct Layout {
     static constexpr int TILE_BYTES = TILE * D * 2;
     static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
     static constexpr int META_BYTES = TILE * (int)sizeof(URow);
-    static __host__ __device__ constexpr size_t bytes(int stages, int nt) {
+    static __host__ __device__ constexpr size_t body(int stages, int nt) {
         size_t ring = (size_t)stages * (STAGE_BYTES + META_BYTES);
         size_t merge = (size_t)CW * 8 * nt * (D + 4 + 2) * 4;
-        size_t body = ring > merge ? ring : merge;
-        return 1024 + body + (size_t)stages * 16 + 64;
+        size_t comb = (size_t)2 * kMaxSplits * 8 * nt * 4;
+        size_t b = ring > merge ? ring : merge;
+        b = b > comb ? b : comb;
+        return (b + 127) & ~(size_t)127;
+    }
+    static __host__ __device__ constexpr size_t bars(int stages) { return ((size_t)stages * 16 + 8 + 127) & ~(size_t)127; }
+    static __host__ __device__ constexpr size_t recv(int nt) {
+        return (size_t)8 * nt * D * 4 + (size_t)kMaxCluster * 8 * nt * 2 * 4;
+    }
+    static __host__ __device__ constexpr size_t bytes(int stages, int nt) {
+        return 1024 + body(stages, nt) + bars(stages) + recv(nt);
     }
 };
 
 template <typename T, int D, int NT, int CW>
-__global__ void __launch_bounds__(32 * (CW + 1), NT > 1 ? 1 : 2)
+__global__ void __launch_bounds__(32 * (CW + 2), NT > 1 ? 1 : 2)
 sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                   const TiledParams p) {
     using L = Layout<D, CW>;
     constexpr int TILE = L::TILE;
     constexpr int KS = D / 16;           // k-steps of Q.K, m-tiles of P.V
-    constexpr int NTHREADS = 32 * (CW + 1);
+    constexpr int NTHREADS = 32 * (CW + 2);
     constexpr int DP = D + 4;            // padded row of the merge buffer (conflict-free)
+    constexpr int UK = (TILE + 31) / 32;
+    constexpr int D4 = D / 4;
+    constexpr int TMA_WARP = CW, GATHER_WARP = CW + 1;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int stages = p.stages;
     uint8_t* ring = smem;
     URow* meta = reinterpret_cast<URow*>(ring + (size_t)stages * L::STAGE_BYTES);
-    size_t ring_bytes = (size_t)stages * (L::STAGE_BYTES + L::META_BYTES);
-    size_t merge_bytes = (size_t)CW * 8 * NT * (DP + 2) * 4;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (ring_bytes > merge_bytes ? ring_bytes : merge_bytes));
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + stages);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::body(stages, NT));
+    float* recv_o = reinterpret_cast<float*>(smem + L::body(stages, NT) + L::bars(stages));   // [S][slice]
+    float* recv_ml = recv_o + 8 * NT * D;                                                     // [S][ncols][2]
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + stages), hand = smem_u32(bars + 2 * stages);
     __shared__ int s_last, s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) { SEGKV_STAMP(0); SEGKV_STAMP(1); }
+    grid_launch_dependents();
     const int split = blockIdx.x % p.S;
     const int slab = blockIdx.x / p.S;           // b * Hkv + kvh
     const int b = slab / p.Hkv, kvh = slab % p.Hkv;
 
-    // this CTA's share: whole prompt tiles, and a range of the request's distinct response rows
+    // This CTA's share of the work group: whole prompt tiles (known from the launch shape
+    // alone, so their loads start at once) and a range of the request's distinct response
+    // rows (known once the row count has been read).
     const int ntp = (p.P + TILE - 1) / TILE;
     const int pt0 = (int)((long long)split * ntp / p.S), pt1 = (int)((long long)(split + 1) * ntp / p.S);
-    const int n_b = p.steps > 0 ? p.ucount[b] : 0;
-    const int e0 = (int)((long long)split * n_b / p.S), e1 = (int)((long long)(split + 1) * n_b / p.S);
     const int npt = pt1 - pt0;
-    const int nrt = (e1 - e0 + TILE - 1) / TILE;
-    const int ntiles = npt + nrt;
     const URow* ulist_b = p.ulist + (size_t)b * p.W * p.max_steps;
 
-    if (tid == 0) {
-        for (int s = 0; s < stages; ++s) {
-            mbar_init(full0 + 8 * s, 32);     // every producer lane arrives once per fill
-            mbar_init(empty0 + 8 * s, CW);    // one arrival per consumer warp
+    auto issue_prompt_tile = [&](int k) {
+        const int st = k % stages;
+        const uint32_t full = full0 + 8 * st;
+        if (lane == 0) {
+            const uint32_t k_dst = smem_u32(ring + (size_t)st * L::STAGE_BYTES);
+            const uint32_t v_dst = k_dst + L::TILE_BYTES;
+            mbar_arrive_expect_tx(full, (uint32_t)L::STAGE_BYTES);
+            const int y = (pt0 + k) * TILE;
+#pragma unroll
+            for (int bx = 0; bx < D / 64; ++bx) {
+                tma_load_3d(k_dst + bx * L::BOX_BYTES, &tm_k, bx * 64, y, slab, full);
+                tma_load_3d(v_dst + bx * L::BOX_BYTES, &tm_v, bx * 64, y, slab, full);
+            }
+        } else {
+            mbar_arrive(full);
         }
-        s_abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        fence_proxy_async();
+    };
+
+    int tma_issued = 0;       // TMA warp: fills started (for the wind-down after an expired wait)
+    if (warp == TMA_WARP) {
+        // The warp that issues the bulk loads sets the barriers up itself and starts the
+        // first round of prompt tiles before the rest of the CTA has even synchronised.
+        if (lane == 0) {
+            for (int s = 0; s < stages; ++s) {
+                mbar_init(full0 + 8 * s, 32);     // every lane of the filling warp arrives once per fill
+                mbar_init(empty0 + 8 * s, CW);    // one arrival per consumer warp
+            }
+            mbar_init(hand, 1);                   // ring handed from the TMA warp to the gather warp
+            s_abort = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            fence_proxy_async();
+            if (npt > 0) {
+                prefetch_tmap(&tm_k);
+                prefetch_tmap(&tm_v);
+            }
+        }
+        __syncwarp();
+        // The prompt segment does not change during decoding, so when the host says so its
+        // tiles are requested before the previous kernel of the stream has finished.
+        if (!p.early_prompt) grid_wait();
+        const int first = min(npt, stages);
+        for (int k = 0; k < first; ++k) issue_prompt_tile(k);
+        tma_issued = first;
+        if (first == npt && lane == 0) mbar_arrive(hand);
+        SEGKV_STAMP(3);
     }
+    if (p.cluster) cluster_arrive_relaxed();     // "this CTA has started" (waited for before any remote store)
     __syncthreads();
+    grid_wait();      // everything else (q, row lists, response rows, outputs) follows the previous kernel
+    if (tid == 0) SEGKV_STAMP(2);
 
     // consumer state (declared here so that the epilogue sees it)
     float o_acc[NT][KS][4];
     float m_run[NT][2], l_run[NT][2];
 
-    if (warp == CW) {
-        // ================================ producer warp ================================
-        if (lane == 0 && npt > 0) {
-            prefetch_tmap(&tm_k);
-            prefetch_tmap(&tm_v);
-        }
+    if (warp == TMA_WARP) {
+        // ============================ prompt tiles beyond the first round ============================
         bool ok = true;
-        for (int k = 0; k < ntiles && ok; ++k) {
+        for (int k = tma_issued; k < npt; ++k) {
+            ok = mbar_wait(empty0 + 8 * (k % stages), (((uint32_t)(k / stages)) & 1) ^ 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            issue_prompt_tile(k);
+            tma_issued = k + 1;
+            if (k + 1 == npt && lane == 0) mbar_arrive(hand);
+        }
+        if (!ok && lane == 0) {
+            atomicOr(p.err_word, SEGKV_DEV_WAIT_LIMIT);
+            s_abort = 1;
+        }
+    } else if (warp == GATHER_WARP) {
+        // ================== response tiles: gather the request's distinct rows ==================
+        // The chain row count -> row list starts at once, beside the TMA warp; the ring itself
+        // is taken over only when the last prompt tile has been issued (a parity wait cannot
+        // tell a far-future round of a stage from the current one).
+        const int n_b = p.steps > 0 ? p.ucount[b] : 0;
+        const int e0 = (int)((long long)split * n_b / p.S), e1 = (int)((long long)(split + 1) * n_b / p.S);
+        const int nrt = (e1 - e0 + TILE - 1) / TILE;
+        SEGKV_STAMP(4);
+        bool ok = true;
+        // row ids of the next tile are fetched while the current one is being issued
+        int urow[UK], urow_next[UK];
+#pragma unroll
+        for (int kk = 0; kk < UK; ++kk) {
+            const int key = lane + 32 * kk;
+            urow_next[kk] = (key < TILE && e0 + key < e1) ? ulist_b[e0 + key].row : 0;
+        }
+        if (nrt > 0) {
+            ok = mbar_wait(hand, 0);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        for (int r = 0; r < nrt && ok; ++r) {
+            const int k = npt + r;
+            const int eb = e0 + r * TILE;
+            const int cnt = min(TILE, e1 - eb);
+#pragma unroll
+            for (int kk = 0; kk < UK; ++kk) {
+                urow[kk] = urow_next[kk];
+                const int key = lane + 32 * kk;
+                urow_next[kk] = (key < TILE && eb + TILE + key < e1) ? ulist_b[eb + TILE + key].row : 0;
+            }
             const int st = k % stages;
-            const uint32_t round = (uint32_t)(k / stages);
-            ok = mbar_wait(empty0 + 8 * st, (round & 1) ^ 1);
+            ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const uint32_t full = full0 + 8 * st;
             const uint32_t k_dst = smem_u32(ring + (size_t)st * L::STAGE_BYTES);
             const uint32_t v_dst = k_dst + L::TILE_BYTES;
-            if (k < npt) {
-                if (lane == 0) {
-                    mbar_arrive_expect_tx(full, (uint32_t)L::STAGE_BYTES);
-                    const int y = (pt0 + k) * TILE;
+            const uint32_t meta_dst = smem_u32(meta + (size_t)st * TILE);
 #pragma unroll
-                    for (int bx = 0; bx < D / 64; ++bx) {
-                        tma_load_3d(k_dst + bx * L::BOX_BYTES, &tm_k, bx * 64, y, slab, full);
-                        tma_load_3d(v_dst + bx * L::BOX_BYTES, &tm_v, bx * 64, y, slab, full);
-                    }
-                } else {
-                    mbar_arrive(full);
-                }
-            } else {
-                const int eb = e0 + (k - npt) * TILE;
-                const int cnt = min(TILE, e1 - eb);
-                const uint32_t meta_dst = smem_u32(meta + (size_t)st * TILE);
-                constexpr int UK = (TILE + 31) / 32;
-                int urow[UK];
-#pragma unroll
-                for (int kk = 0; kk < UK; ++kk) {
-                    const int key = lane + 32 * kk;
-                    urow[kk] = 0;
-                    if (key < TILE) {
-                        const bool valid = key < cnt;
-                        if (valid) urow[kk] = ulist_b[eb + key].row;
-                        cp_async_8(meta_dst + key * 8, valid ? (const void*)(ulist_b + eb + key) : (const void*)p.ulist,
-                                   valid ? 8u : 0u);
-                    }
-                }
-                constexpr int CPR = D / 8;        // 16-byte chunks per row
-                constexpr int RPI = 32 / CPR;     // rows covered by one warp-wide copy
-                const int c = lane % CPR;
-                const uint32_t c_off = (uint32_t)(c / 8) * L::BOX_BYTES;
-#pragma unroll 4
-                for (int i = 0; i < TILE / RPI; ++i) {
-                    const int key = i * RPI + lane / CPR;
-                    int r = urow[0];
-                    if (TILE > 32 && key >= 32) r = urow[UK - 1];
-                    r = __shfl_sync(0xffffffffu, r, key & 31);
+            for (int kk = 0; kk < UK; ++kk) {
+                const int key = lane + 32 * kk;
+                if (key < TILE) {
                     const bool valid = key < cnt;
-                    const size_t src = ((size_t)r * p.Hkv + kvh) * (size_t)(D * 2) + (size_t)c * 16;
-                    const uint32_t off = c_off + (uint32_t)key * 128 + (uint32_t)(((c & 7) ^ (key & 7)) << 4);
-                    cp_async_16(k_dst + off, valid ? p.kr + src : p.kr, valid ? 16u : 0u);
-                    cp_async_16(v_dst + off, valid ? p.vr + src : p.vr, valid ? 16u : 0u);
+                    cp_async_8(meta_dst + key * 8, valid ? (const void*)(ulist_b + eb + key) : (const void*)p.ulist,
+                               valid ? 8u : 0u);
                 }
-                cp_async_mbar_arrive_noinc(full);
             }
+            constexpr int CPR = D / 8;        // 16-byte chunks per row
+            constexpr int RPI = 32 / CPR;     // rows covered by one warp-wide copy
+            const int c = lane % CPR;
+            const uint32_t c_off = (uint32_t)(c / 8) * L::BOX_BYTES;
+            // rows past the last one a consumer warp will look at need no zero fill
+            const int fill = min(TILE, (cnt + 15) & ~15);
+#pragma unroll 4
+            for (int i = 0; i < TILE / RPI; ++i) {
+                const int key = i * RPI + lane / CPR;
+                int rr = urow[0];
+                if (TILE > 32 && key >= 32) rr = urow[UK - 1];
+                rr = __shfl_sync(0xffffffffu, rr, key & 31);
+                if (i * RPI >= fill) continue;            // warp-uniform
+                const bool valid = key < cnt;
+                const size_t src = ((size_t)rr * p.Hkv + kvh) * (size_t)(D * 2) + (size_t)c * 16;
+                const uint32_t off = c_off + (uint32_t)key * 128 + (uint32_t)(((c & 7) ^ (key & 7)) << 4);
+                cp_async_16(k_dst + off, valid ? p.kr + src : p.kr, valid ? 16u : 0u);
+                cp_async_16(v_dst + off, valid ? p.vr + src : p.vr, valid ? 16u : 0u);
+            }
+            cp_async_mbar_arrive_noinc(full);
         }
+        SEGKV_STAMP(5);
         if (!ok && lane == 0) {
             atomicOr(p.err_word, SEGKV_DEV_WAIT_LIMIT);
             s_abort = 1;
@@ -332,116 +454,134 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         const int qpos = p.P + (p.steps > 0 ? p.steps - 1 : -1);
         const int key_lo = warp * 16 + (lane >> 2);       // tile-local key of accumulator rows 0..7
 
-        bool ok = true;
-        for (int k = 0; k < ntiles; ++k) {
-            const int st = k % stages;
-            const uint32_t round = (uint32_t)(k / stages);
-            ok = mbar_wait(full0 + 8 * st, round & 1);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+        // One tile: `nvalid` keys exist; for a response tile the per-key beam masks and row
+        // ids are in the stage's meta array, for a prompt tile key i sits at position pos0 + i.
+        auto consume = [&](int st, bool resp, int nvalid, int pos0) {
+            if (warp * 16 >= nvalid) return;
             const uint32_t k_src = smem_u32(ring + (size_t)st * L::STAGE_BYTES);
             const uint32_t v_src = k_src + L::TILE_BYTES;
-            const bool resp = k >= npt;
-            int nvalid;        // keys of this tile that exist
-            if (!resp) nvalid = min(TILE, p.P - (pt0 + k) * TILE);
-            else nvalid = min(TILE, e1 - (e0 + (k - npt) * TILE));
-
-            if (warp * 16 < nvalid) {
-                // ---- S^T = K . Q^T ----
-                float sc[NT][4];
+            // ---- S^T = K . Q^T ----
+            float sc[NT][4];
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
-                {
-                    const int key = warp * 16 + (lane & 15);
-                    const uint32_t rowaddr = k_src + (uint32_t)key * 128;
-                    const int sw = key & 7;
+            for (int nt = 0; nt < NT; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+            {
+                const int key = warp * 16 + (lane & 15);
+                const uint32_t rowaddr = k_src + (uint32_t)key * 128;
+                const int sw = key & 7;
 #pragma unroll
-                    for (int ks = 0; ks < KS; ++ks) {
-                        const int ch = 2 * ks + (lane >> 4);
-                        uint32_t a[4];
-                        ldmatrix_x4(a, rowaddr + (uint32_t)(ch >> 3) * L::BOX_BYTES + (uint32_t)(((ch & 7) ^ sw) << 4));
+                for (int ks = 0; ks < KS; ++ks) {
+                    const int ch = 2 * ks + (lane >> 4);
+                    uint32_t a[4];
+                    ldmatrix_x4(a, rowaddr + (uint32_t)(ch >> 3) * L::BOX_BYTES + (uint32_t)(((ch & 7) ^ sw) << 4));
 #pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) Mma<T>::run(sc[nt], a, qf[nt][ks][0], qf[nt][ks][1]);
-                    }
-                }
-                // ---- mask, bias, online softmax ----
-                uint32_t kmask[2];
-                float kpos[2];
-#pragma unroll
-                for (int r = 0; r < 2; ++r) {
-                    const int key = key_lo + 8 * r;
-                    if (resp) {
-                        const URow u = meta[(size_t)st * TILE + key];
-                        kmask[r] = u.mask;                      // zero for padding rows
-                        kpos[r] = (float)(p.P + u.row / p.rows - qpos);
-                    } else {
-                        kmask[r] = key < nvalid ? 0xffffffffu : 0u;
-                        kpos[r] = (float)((pt0 + k) * TILE + key - qpos);
-                    }
-                }
-                uint32_t pfrag[NT][2];
-                bool rescale = false;
-                float alpha[NT][2];
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    float s[2][2];
-#pragma unroll
-                    for (int r = 0; r < 2; ++r)
-#pragma unroll
-                        for (int c = 0; c < 2; ++c) {
-                            float v = sc[nt][2 * r + c] * p.scale2 + slope2[nt][c] * kpos[r];
-                            s[r][c] = (kmask[r] & beambit[nt][c]) ? v : -INFINITY;
-                        }
-#pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        float tm = fmaxf(s[0][c], s[1][c]);
-                        tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, 4));
-                        tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, 8));
-                        tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, 16));
-                        const float m_old = m_run[nt][c];
-                        const float m_new = fmaxf(m_old, tm);
-                        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-                        const float a = exp2f(m_old - m_use);
-                        alpha[nt][c] = a;
-                        rescale = rescale || (a != 1.f);
-                        m_run[nt][c] = m_new;
-                        const float p0 = exp2f(s[0][c] - m_use), p1 = exp2f(s[1][c] - m_use);
-                        s[0][c] = p0;
-                        s[1][c] = p1;
-                        l_run[nt][c] = l_run[nt][c] * a + p0 + p1;
-                    }
-                    // P^T as the B operand of O^T += V^T . P^T
-                    pfrag[nt][0] = movmatrix_trans(Mma<T>::pack(s[0][0], s[0][1]));
-                    pfrag[nt][1] = movmatrix_trans(Mma<T>::pack(s[1][0], s[1][1]));
-                }
-                if (__any_sync(0xffffffffu, rescale)) {
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                        for (int mt = 0; mt < KS; ++mt) {
-                            o_acc[nt][mt][0] *= alpha[nt][0];
-                            o_acc[nt][mt][1] *= alpha[nt][1];
-                            o_acc[nt][mt][2] *= alpha[nt][0];
-                            o_acc[nt][mt][3] *= alpha[nt][1];
-                        }
-                }
-                // ---- O^T += V^T . P^T ----
-                {
-                    const int key = warp * 16 + (lane & 7) + 8 * (lane >> 4);
-                    const uint32_t rowaddr = v_src + (uint32_t)key * 128;
-                    const int sw = key & 7;
-#pragma unroll
-                    for (int mt = 0; mt < KS; ++mt) {
-                        const int ch = 2 * mt + ((lane >> 3) & 1);
-                        uint32_t a[4];
-                        ldmatrix_x4_trans(a, rowaddr + (uint32_t)(ch >> 3) * L::BOX_BYTES + (uint32_t)(((ch & 7) ^ sw) << 4));
-#pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) Mma<T>::run(o_acc[nt][mt], a, pfrag[nt][0], pfrag[nt][1]);
-                    }
+                    for (int nt = 0; nt < NT; ++nt) Mma<T>::run(sc[nt], a, qf[nt][ks][0], qf[nt][ks][1]);
                 }
             }
+            // ---- mask, bias, online softmax ----
+            uint32_t kmask[2];
+            float kpos[2];
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int key = key_lo + 8 * r;
+                if (resp) {
+                    const URow u = meta[(size_t)st * TILE + key];
+                    kmask[r] = key < nvalid ? u.mask : 0u;
+                    kpos[r] = (float)(p.P + u.row / p.rows - qpos);
+                } else {
+                    kmask[r] = key < nvalid ? 0xffffffffu : 0u;
+                    kpos[r] = (float)(pos0 + key - qpos);
+                }
+            }
+            uint32_t pfrag[NT][2];
+            bool rescale = false;
+            float alpha[NT][2];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                float s[2][2];
+#pragma unroll
+                for (int r = 0; r < 2; ++r)
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        float v = sc[nt][2 * r + c] * p.scale2 + slope2[nt][c] * kpos[r];
+                        s[r][c] = (kmask[r] & beambit[nt][c]) ? v : -INFINITY;
+                    }
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    float tm = fmaxf(s[0][c], s[1][c]);
+                    tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, 4));
+                    tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, 8));
+                    tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, 16));
+                    const float m_old = m_run[nt][c];
+                    const float m_new = fmaxf(m_old, tm);
+                    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+                    const float a = exp2f(m_old - m_use);
+                    alpha[nt][c] = a;
+                    rescale = rescale || (a != 1.f);
+                    m_run[nt][c] = m_new;
+                    const float p0 = exp2f(s[0][c] - m_use), p1 = exp2f(s[1][c] - m_use);
+                    s[0][c] = p0;
+                    s[1][c] = p1;
+                    l_run[nt][c] = l_run[nt][c] * a + p0 + p1;
+                }
+                // P^T as the B operand of O^T += V^T . P^T
+                pfrag[nt][0] = movmatrix_trans(Mma<T>::pack(s[0][0], s[0][1]));
+                pfrag[nt][1] = movmatrix_trans(Mma<T>::pack(s[1][0], s[1][1]));
+            }
+            if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int mt = 0; mt < KS; ++mt) {
+                        o_acc[nt][mt][0] *= alpha[nt][0];
+                        o_acc[nt][mt][1] *= alpha[nt][1];
+                        o_acc[nt][mt][2] *= alpha[nt][0];
+                        o_acc[nt][mt][3] *= alpha[nt][1];
+                    }
+            }
+            // ---- O^T += V^T . P^T ----
+            {
+                const int key = warp * 16 + (lane & 7) + 8 * (lane >> 4);
+                const uint32_t rowaddr = v_src + (uint32_t)key * 128;
+                const int sw = key & 7;
+#pragma unroll
+                for (int mt = 0; mt < KS; ++mt) {
+                    const int ch = 2 * mt + ((lane >> 3) & 1);
+                    uint32_t a[4];
+                    ldmatrix_x4_trans(a, rowaddr + (uint32_t)(ch >> 3) * L::BOX_BYTES + (uint32_t)(((ch & 7) ^ sw) << 4));
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) Mma<T>::run(o_acc[nt][mt], a, pfrag[nt][0], pfrag[nt][1]);
+                }
+            }
+        };
+
+        bool ok = true;
+        int k = 0;
+        if (warp == 0) SEGKV_STAMP(6);
+        for (; k < npt; ++k) {
+            const int st = k % stages;
+            ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (warp == 0 && k == 0) SEGKV_STAMP(7);
+            const int pos0 = (pt0 + k) * TILE;
+            consume(st, false, min(TILE, p.P - pos0), pos0);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + 8 * st);
+        }
+        if (warp == 0) SEGKV_STAMP(8);
+        if (ok) {
+            const int n_b = p.steps > 0 ? p.ucount[b] : 0;
+            const int e0 = (int)((long long)split * n_b / p.S), e1 = (int)((long long)(split + 1) * n_b / p.S);
+            const int nrt = (e1 - e0 + TILE - 1) / TILE;
+            for (int r = 0; r < nrt; ++r, ++k) {
+                const int st = k % stages;
+                ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                consume(st, true, min(TILE, e1 - (e0 + r * TILE)), 0);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8 * st);
+            }
         }
         if (!ok && lane == 0) {
             atomicOr(p.err_word, SEGKV_DEV_WAIT_LIMIT);
@@ -449,20 +589,24 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         }
     }
 
+    if (warp == 0) SEGKV_STAMP(9);
     // ==================================== epilogue ====================================
     __syncthreads();
-    if (s_abort) {
+    if (tid == 0) SEGKV_STAMP(10);
+    const bool aborted = s_abort != 0;
+    if (aborted) {
         // Something never arrived.  Give copies still in flight a bounded chance to land
-        // before the shared memory is released, then leave without touching the output.
-        if (warp == CW && lane == 0)
-            for (int k = max(0, ntiles - stages); k < ntiles; ++k)
+        // before the shared memory is released; the output is left untouched.
+        if (warp == TMA_WARP)
+            for (int k = max(0, tma_issued - stages); k < tma_issued; ++k)
                 (void)mbar_wait(full0 + 8 * (k % stages), (uint32_t)(k / stages) & 1);
-        return;
+        if (warp == GATHER_WARP) cp_async_wait_all();
     }
 
+    // ---- merge the consumer warps (each saw a different quarter of every tile) ----
     float* mrg_o = reinterpret_cast<float*>(smem);                       // [CW][8*NT][DP]
     float* mrg_ml = mrg_o + (size_t)CW * 8 * NT * DP;                    // [CW][8*NT][2]
-    if (warp < CW) {
+    if (warp < CW && !aborted) {
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
@@ -488,62 +632,157 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     __syncthreads();
 
     const int ncols = p.ncols;
-    float* ws_cta = p.ws + ((size_t)slab * p.S + split) * ncols * (D + 2);
-    for (int idx = tid; idx < ncols * D; idx += NTHREADS) {
-        const int col = idx / D, d = idx % D;
-        float mm = -INFINITY;
+    const int S = p.S;
+    // merged partial of this CTA for one float4 of one column
+    auto merged = [&](int col, int d, float& mm, float& ll) -> float4 {
+        mm = -INFINITY;
 #pragma unroll
         for (int w = 0; w < CW; ++w) mm = fmaxf(mm, mrg_ml[((size_t)w * 8 * NT + col) * 2]);
-        float ll = 0.f, o = 0.f;
+        ll = 0.f;
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int w = 0; w < CW; ++w) {
             const float mw = mrg_ml[((size_t)w * 8 * NT + col) * 2];
             const float f = (mw == -INFINITY) ? 0.f : exp2f(mw - mm);
             ll += mrg_ml[((size_t)w * 8 * NT + col) * 2 + 1] * f;
-            o += mrg_o[((size_t)w * 8 * NT + col) * DP + d] * f;
+            const float4 v = *reinterpret_cast<const float4*>(mrg_o + ((size_t)w * 8 * NT + col) * DP + d);
+            o.x += v.x * f; o.y += v.y * f; o.z += v.z * f; o.w += v.w * f;
         }
-        if (p.S == 1) {
-            const int j = col / p.G, hg = col % p.G;
-            T* orow = reinterpret_cast<T*>(p.out) + ((size_t)(b * p.W + j) * p.H + kvh * p.G + hg) * D;
-            orow[d] = Mma<T>::down(o / ll);
-        } else {
-            ws_cta[(size_t)col * (D + 2) + d] = o;
-            if (d == 0) {
-                ws_cta[(size_t)col * (D + 2) + D] = mm;
-                ws_cta[(size_t)col * (D + 2) + D + 1] = ll;
+        return o;
+    };
+    auto store_out = [&](int col, int d, float4 o) {
+        const int j = col / p.G, hg = col % p.G;
+        T* orow = reinterpret_cast<T*>(p.out) + ((size_t)(b * p.W + j) * p.H + kvh * p.G + hg) * D + d;
+        uint2 pk;
+        pk.x = Mma<T>::pack(o.x, o.y);
+        pk.y = Mma<T>::pack(o.z, o.w);
+        *reinterpret_cast<uint2*>(orow) = pk;
+    };
+
+    if (p.cluster) {
+        // ---- split merge inside the thread-block cluster, through distributed shared memory ----
+        // The (column, d) plane is cut into S equal slices; CTA r merges slice r.  Every CTA
+        // stores its part of slice r into CTA r's landing area, one cluster barrier later each
+        // CTA holds all S partials of its slice.
+        const uint32_t me = cluster_ctarank();
+        const int slice = ncols * D / S;                 // floats; a multiple of 4
+        cluster_wait_acquire();                          // every CTA of the cluster has started
+        if (!aborted) {
+            for (int it = tid; it < ncols * D4; it += NTHREADS) {
+                const int col = it / D4, d = (it % D4) * 4;
+                float mm, ll;
+                const float4 o = merged(col, d, mm, ll);
+                const int f = col * D + d;
+                const int r = f / slice;
+                st_cluster_v4(mapa_shared(smem_u32(recv_o + (size_t)me * slice + (f - r * slice)), (uint32_t)r), o);
+                if (d == 0)
+                    for (int r2 = 0; r2 < S; ++r2)
+                        st_cluster_v2(mapa_shared(smem_u32(recv_ml + ((size_t)me * ncols + col) * 2), (uint32_t)r2), mm, ll);
             }
         }
+        cluster_arrive_release();
+        cluster_wait_acquire();
+        if (tid == 0) SEGKV_STAMP(12);
+        if (aborted) return;
+        for (int i = tid; i < slice / 4; i += NTHREADS) {
+            const int f = (int)me * slice + 4 * i;
+            const int col = f / D, d = f % D;
+            float mm = -INFINITY;
+            for (int s = 0; s < S; ++s) mm = fmaxf(mm, recv_ml[((size_t)s * ncols + col) * 2]);
+            float ll = 0.f;
+            float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int s = 0; s < S; ++s) {
+                const float ms = recv_ml[((size_t)s * ncols + col) * 2];
+                const float fs = (ms == -INFINITY) ? 0.f : exp2f(ms - mm);
+                ll += recv_ml[((size_t)s * ncols + col) * 2 + 1] * fs;
+                const float4 v = *reinterpret_cast<const float4*>(recv_o + (size_t)s * slice + 4 * i);
+                o.x += v.x * fs; o.y += v.y * fs; o.z += v.z * fs; o.w += v.w * fs;
+            }
+            const float inv = 1.f / ll;
+            o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
+            store_out(col, d, o);
+        }
+        if (tid == 0) SEGKV_STAMP(13);
+        return;
     }
-    if (p.S == 1) return;
+    if (aborted) return;
 
-    // ---- split merge by the last CTA of this work group to arrive ----
-    __threadfence();
+    float* wso_cta = p.ws_o + ((size_t)slab * S + split) * ncols * D;
+    float* wsml_cta = p.ws_ml + ((size_t)slab * S + split) * ncols * 2;
+    for (int it = tid; it < ncols * D4; it += NTHREADS) {
+        const int col = it / D4, d = (it % D4) * 4;
+        float mm, ll;
+        float4 o = merged(col, d, mm, ll);
+        if (S == 1) {
+            const float inv = 1.f / ll;
+            o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
+            store_out(col, d, o);
+        } else {
+            *reinterpret_cast<float4*>(wso_cta + (size_t)col * D + d) = o;
+            if (d == 0) *reinterpret_cast<float2*>(wsml_cta + col * 2) = make_float2(mm, ll);
+        }
+    }
+    if (tid == 0) SEGKV_STAMP(11);
+    if (S == 1) return;
+
+    // ---- split merge through the global workspace: the last CTA of the work group to
+    // ---- arrive (atomic ticket, nobody waits) merges all partials
     __syncthreads();
     if (tid == 0) {
+        __threadfence();                                   // partials visible before the ticket
         const int ticket = atomicAdd(p.tickets + slab, 1);
-        s_last = (ticket == p.S - 1);
+        const int last = (ticket == S - 1);
+        if (last) __threadfence();                         // and the others' partials before reading
+        s_last = last;
     }
     __syncthreads();
+    if (tid == 0) SEGKV_STAMP(12);
     if (!s_last) return;
-    __threadfence();
-    const float* ws_slab = p.ws + (size_t)slab * p.S * ncols * (D + 2);
-    for (int idx = tid; idx < ncols * D; idx += NTHREADS) {
-        const int col = idx / D, d = idx % D;
+
+    float* c_f = reinterpret_cast<float*>(smem);           // [S][ncols] max, then scale factor
+    float* c_l = c_f + (size_t)S * ncols;
+    const float* wsml_slab = p.ws_ml + (size_t)slab * S * ncols * 2;
+    const float* wso_slab = p.ws_o + (size_t)slab * S * ncols * D;
+    for (int i = tid; i < S * ncols; i += NTHREADS) {
+        const float2 ml = __ldcg(reinterpret_cast<const float2*>(wsml_slab) + i);
+        c_f[i] = ml.x;
+        c_l[i] = ml.y;
+    }
+    __syncthreads();
+    if (tid < ncols) {
         float mm = -INFINITY;
-        for (int s = 0; s < p.S; ++s) mm = fmaxf(mm, __ldcg(ws_slab + ((size_t)s * ncols + col) * (D + 2) + D));
-        float ll = 0.f, o = 0.f;
-        for (int s = 0; s < p.S; ++s) {
-            const float* part = ws_slab + ((size_t)s * ncols + col) * (D + 2);
-            const float ms = __ldcg(part + D);
+        for (int s = 0; s < S; ++s) mm = fmaxf(mm, c_f[s * ncols + tid]);
+        float ll = 0.f;
+        for (int s = 0; s < S; ++s) {
+            const float ms = c_f[s * ncols + tid];
             const float f = (ms == -INFINITY) ? 0.f : exp2f(ms - mm);
-            ll += __ldcg(part + D + 1) * f;
-            o += __ldcg(part + d) * f;
+            ll += c_l[s * ncols + tid] * f;
+            c_f[s * ncols + tid] = f;
         }
-        const int j = col / p.G, hg = col % p.G;
-        T* orow = reinterpret_cast<T*>(p.out) + ((size_t)(b * p.W + j) * p.H + kvh * p.G + hg) * D;
-        orow[d] = Mma<T>::down(o / ll);
+        const float inv = 1.f / ll;
+        for (int s = 0; s < S; ++s) c_f[s * ncols + tid] *= inv;
+    }
+    __syncthreads();
+    for (int it = tid; it < ncols * D4; it += NTHREADS) {
+        const int col = it / D4, d = (it % D4) * 4;
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4* src = reinterpret_cast<const float4*>(wso_slab + (size_t)col * D + d);
+        const size_t sstride = (size_t)ncols * D4;            // float4 per split
+        for (int s0 = 0; s0 < S; s0 += 8) {
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                v[u] = (s0 + u < S) ? __ldcg(src + (size_t)(s0 + u) * sstride) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float f = (s0 + u < S) ? c_f[(s0 + u) * ncols + col] : 0.f;
+                o.x += v[u].x * f; o.y += v[u].y * f; o.z += v[u].z * f; o.w += v[u].w * f;
+            }
+        }
+        store_out(col, d, o);
     }
     if (tid == 0) p.tickets[slab] = 0;      // ready for the next launch
+    if (tid == 0) SEGKV_STAMP(13);
 }
 
 template <typename T, int D, int NT, int CW>
@@ -563,19 +802,46 @@ cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk,
     TiledParams p;
     p.q = a.q; p.out = a.out; p.slopes = a.slopes;
     p.kr = (const char*)a.kr; p.vr = (const char*)a.vr;
-    p.ulist = a.ulist; p.ucount = a.ucount; p.ws = a.ws; p.tickets = a.tickets; p.err_word = a.err_word;
+    p.ulist = a.ulist; p.ucount = a.ucount; p.tickets = a.tickets; p.err_word = a.err_word;
     p.P = a.prompt_len; p.steps = a.steps; p.S = a.splits; p.W = d.beams; p.G = d.group; p.H = d.heads;
     p.Hkv = d.kv_heads; p.rows = d.rows; p.max_steps = d.max_steps; p.ncols = d.beams * d.group; p.stages = stages;
     p.scale2 = 1.4426950408889634f / sqrtf((float)D);
-    const unsigned grid = (unsigned)((size_t)d.batch * d.kv_heads * a.splits);
-    kern<<<grid, 32 * (CW + 1), smem, st>>>(tmk, tmv, p);
-    return cudaGetLastError();
+    p.cluster = a.cluster ? 1 : 0;
+    p.early_prompt = (a.pdl && a.steps > 0) ? 1 : 0;
+    const size_t slabs = (size_t)d.batch * d.kv_heads;
+    p.ws_o = a.ws;
+    p.ws_ml = a.ws ? a.ws + slabs * a.splits * p.ncols * D : nullptr;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(slabs * a.splits), 1, 1);
+    cfg.blockDim = dim3(32 * (CW + 2), 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    unsigned na = 0;
+    if (p.cluster) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = (unsigned)a.splits;
+        attr[na].val.clusterDim.y = 1;
+        attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (a.pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = na ? attr : nullptr;
+    cfg.numAttrs = na;
+    return cudaLaunchKernelEx(&cfg, kern, tmk, tmv, p);
 }
 
 template <typename T>
 cudaError_t dispatch(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk, const CUtensorMap& tmv, int stages,
                      cudaStream_t st) {
     const int nt = (d.beams * d.group + 7) / 8;
+    if (a.splits < 1 || a.splits > kMaxSplits) return cudaErrorInvalidValue;
+    if (a.cluster && !tiled_cluster_ok(d, a.splits)) return cudaErrorInvalidValue;
     if (nt == 1) {
         switch (d.head_dim) {
             case 64: return launch_one<T, 64, 1, 4>(d, a, tmk, tmv, stages, st);
@@ -598,6 +864,12 @@ bool tiled_supported(const Dims& d) {
     return nt == 1 || (nt == 2 && d.head_dim <= 128);
 }
 
+// The cluster combine needs a portable cluster size and equal float4-aligned slices.
+bool tiled_cluster_ok(const Dims& d, int splits) {
+    if (splits != 2 && splits != 4 && splits != 8) return false;
+    return ((long long)d.beams * d.group * d.head_dim) % (4LL * splits) == 0;
+}
+
 int tiled_tile_keys(int head_dim) { return head_dim == 256 ? 32 : 64; }
 
 size_t tiled_smem_bytes(const Dims& d, int stages) {
@@ -616,3 +888,15 @@ cudaError_t launch_sdpa_tiled(const Dims& d, const SdpaArgs& a, const CUtensorMa
 }
 
 }  // namespace segkv_impl
+
+#ifdef SEGKV_TIMELINE
+extern "C" __attribute__((visibility("default"))) int segkv_debug_timeline(unsigned long long* host, int clear) {
+    if (cudaMemcpyFromSymbol(host, segkv_impl::g_timeline, sizeof(unsigned long long) * 1024 * 16) != cudaSuccess) return -1;
+    if (clear) {
+        void* p = nullptr;
+        cudaGetSymbolAddress(&p, segkv_impl::g_timeline);
+        cudaMemset(p, 0, sizeof(unsigned long long) * 1024 * 16);
+    }
+    return 0;
+}
+#endif

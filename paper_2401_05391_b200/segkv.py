@@ -39,9 +39,10 @@ SIGNATURES = {
     "segkv_get_error": (_int, [_vp, ctypes.POINTER(_int)]),
     "segkv_steps": (_int, [_vp]),
     "segkv_prompt_len": (_int, [_vp]),
-    "segkv_set_tuning": (_int, [_vp, _int, _int]),
+    "segkv_set_tuning": (_int, [_vp, _int, _int, _int]),
     "segkv_decode_sdpa_rowwise": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "segkv_get_splits": (_int, [_vp]),
+    "segkv_set_overlap": (_int, [_vp, _int]),
     "segkv_launch_count": (ctypes.c_longlong, [_vp]),
     "segkv_storage_bytes": (ctypes.c_size_t, [_int] * 7),
     "segkv_strerror": (ctypes.c_char_p, [_int]),
@@ -210,8 +211,8 @@ class SegKV:
         _check(lib().segkv_get_error(self._h, ctypes.byref(flags)), "segkv_get_error")
         return flags.value
 
-    def set_tuning(self, splits: int = 0, stages: int = 0) -> None:
-        _check(lib().segkv_set_tuning(self._h, splits, stages), "segkv_set_tuning")
+    def set_tuning(self, splits: int = 0, stages: int = 0, combine: int = 0) -> None:
+        _check(lib().segkv_set_tuning(self._h, splits, stages, combine), "segkv_set_tuning")
 
     def decode_sdpa_rowwise(self, q: torch.Tensor, out: Optional[torch.Tensor] = None,
                             alibi_slopes: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
@@ -223,6 +224,9 @@ class SegKV:
                                                _dev(alibi_slopes, (self.heads,), torch.float32, "alibi_slopes"),
                                                _stream_ptr(stream)), "segkv_decode_sdpa_rowwise")
         return out
+
+    def set_overlap(self, enable: bool) -> None:
+        _check(lib().segkv_set_overlap(self._h, int(enable)), "segkv_set_overlap")
 
     def get_splits(self) -> int:
         return int(lib().segkv_get_splits(self._h))

@@ -13,8 +13,8 @@ pytestmark = pytest.mark.gpu
 CHECK_STEPS = (0, 1, 2, 3, 7, 15, 16, 17, 31, 63, 127, 255)
 
 
-def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, every_step_ancestry=True):
-    r = Run(w, splits=splits, stages=stages)
+def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combine=0, every_step_ancestry=True):
+    r = Run(w, splits=splits, stages=stages, combine=combine)
     try:
         worst = 0.0
         for t in range(w.steps):
@@ -60,12 +60,20 @@ def test_ragged_small_shapes(dtype, D):
     run_workload(w, all_pairs, check_steps=(0, 1, 5, 20))
 
 
-@pytest.mark.parametrize("splits,stages", [(1, 0), (2, 2), (5, 1), (19, 3), (40, 0)])
-def test_forced_splits_and_stages(splits, stages):
-    # more splits than tiles leaves some CTAs without keys; one stage serialises the ring
+@pytest.mark.parametrize("splits,stages,combine", [(1, 0, 0), (2, 2, 1), (2, 2, 2), (4, 0, 2), (5, 1, 0), (8, 3, 1),
+                                                   (8, 0, 2), (19, 3, 0), (40, 0, 0)])
+def test_forced_splits_stages_and_combine(splits, stages, combine):
+    # more splits than tiles leaves some CTAs without keys; one stage serialises the ring;
+    # combine 1 = workspace + ticket, 2 = thread-block cluster
     w = wl.CONFIGS[1].scaled(steps=40, index=30)
     run_workload(w, lambda w: sampled_pairs(w, 12), check_steps=(0, 7, 39), splits=splits, stages=stages,
-                 every_step_ancestry=False)
+                 combine=combine, every_step_ancestry=False)
+
+
+def test_cluster_combine_small_shapes():
+    for D, dt in ((64, "f16"), (256, "bf16")):
+        w = wl.Workload("cl", 2, 3, 4, 2, D, 300, 9, dt, "uniform", True, 40 + D)
+        run_workload(w, all_pairs, check_steps=(0, 8), splits=4, combine=2)
 
 
 def test_tiled_kernel_agrees_with_rowwise_kernel():
