@@ -170,15 +170,22 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 
 #ifdef SEGKV_TIMELINE
 }  // namespace
-__device__ unsigned long long g_timeline[1024 * 16];
+__device__ unsigned long long g_timeline[8 * 512 * 16];
+#define SEGKV_CLK(ev, cond)                                                                \
+    do {                                                                                   \
+        if ((cond) && (threadIdx.x & 31) == 0 && blockIdx.x < 512) {                       \
+            g_timeline[((p.dbg_launch & 7) * 512 + blockIdx.x) * 16 + (ev)] = (unsigned long long)clock64(); \
+        }                                                                                  \
+    } while (0)
 #define SEGKV_STAMP(ev)                                                                    \
     do {                                                                                   \
-        if ((threadIdx.x & 31) == 0 && blockIdx.x < 1024) {                                \
-            g_timeline[blockIdx.x * 16 + (ev)] = (ev) == 0 ? global_ns() : (unsigned long long)clock64(); \
+        if ((threadIdx.x & 31) == 0 && blockIdx.x < 512) {                                 \
+            g_timeline[((p.dbg_launch & 7) * 512 + blockIdx.x) * 16 + (ev)] = global_ns(); \
         }                                                                                  \
     } while (0)
 namespace {
 #else
+#define SEGKV_CLK(ev, cond) do {} while (0)
 #define SEGKV_STAMP(ev) do {} while (0)
 #endif
 
@@ -197,6 +204,9 @@ struct TiledParams {
     int P, steps, S, W, G, H, Hkv, rows, max_steps, ncols, stages;
     int cluster;    // 1: the S CTAs of a work group form a thread-block cluster
     int early_prompt;  // 1: prompt tiles may be fetched before the previous kernel has completed
+#ifdef SEGKV_TIMELINE
+    int dbg_launch;
+#endif
     float scale2;   // log2(e) / sqrt(D)
 };
 
@@ -460,6 +470,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             if (warp * 16 >= nvalid) return;
             const uint32_t k_src = smem_u32(ring + (size_t)st * L::STAGE_BYTES);
             const uint32_t v_src = k_src + L::TILE_BYTES;
+            SEGKV_CLK(1, warp == 0 && st == 0 && !resp && pos0 == pt0 * TILE);
             // ---- S^T = K . Q^T ----
             float sc[NT][4];
 #pragma unroll
@@ -477,6 +488,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     for (int nt = 0; nt < NT; ++nt) Mma<T>::run(sc[nt], a, qf[nt][ks][0], qf[nt][ks][1]);
                 }
             }
+            SEGKV_CLK(14, warp == 0 && st == 0 && !resp && pos0 == pt0 * TILE);
             // ---- mask, bias, online softmax ----
             uint32_t kmask[2];
             float kpos[2];
@@ -538,6 +550,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                         o_acc[nt][mt][3] *= alpha[nt][1];
                     }
             }
+            SEGKV_CLK(15, warp == 0 && st == 0 && !resp && pos0 == pt0 * TILE);
             // ---- O^T += V^T . P^T ----
             {
                 const int key = warp * 16 + (lane & 7) + 8 * (lane >> 4);
@@ -552,6 +565,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     for (int nt = 0; nt < NT; ++nt) Mma<T>::run(o_acc[nt][mt], a, pfrag[nt][0], pfrag[nt][1]);
                 }
             }
+            SEGKV_CLK(11, warp == 0 && st == 0 && !resp && pos0 == pt0 * TILE);
         };
 
         bool ok = true;
@@ -808,6 +822,10 @@ cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk,
     p.scale2 = 1.4426950408889634f / sqrtf((float)D);
     p.cluster = a.cluster ? 1 : 0;
     p.early_prompt = (a.pdl && a.steps > 0) ? 1 : 0;
+#ifdef SEGKV_TIMELINE
+    static int launch_id = 0;
+    p.dbg_launch = launch_id++;
+#endif
     const size_t slabs = (size_t)d.batch * d.kv_heads;
     p.ws_o = a.ws;
     p.ws_ml = a.ws ? a.ws + slabs * a.splits * p.ncols * D : nullptr;
@@ -891,11 +909,11 @@ cudaError_t launch_sdpa_tiled(const Dims& d, const SdpaArgs& a, const CUtensorMa
 
 #ifdef SEGKV_TIMELINE
 extern "C" __attribute__((visibility("default"))) int segkv_debug_timeline(unsigned long long* host, int clear) {
-    if (cudaMemcpyFromSymbol(host, segkv_impl::g_timeline, sizeof(unsigned long long) * 1024 * 16) != cudaSuccess) return -1;
+    if (cudaMemcpyFromSymbol(host, segkv_impl::g_timeline, sizeof(unsigned long long) * 8 * 512 * 16) != cudaSuccess) return -1;
     if (clear) {
         void* p = nullptr;
         cudaGetSymbolAddress(&p, segkv_impl::g_timeline);
-        cudaMemset(p, 0, sizeof(unsigned long long) * 1024 * 16);
+        cudaMemset(p, 0, sizeof(unsigned long long) * 8 * 512 * 16);
     }
     return 0;
 }
