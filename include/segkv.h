@@ -130,6 +130,41 @@ SEGKV_API int segkv_append(segkv_t h, int step, const int32_t* beam_parent, cons
 SEGKV_API int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_slopes, void* stream);
 
 /*
+ * segkv_decode_sdpa for callers that must not allocate device memory.  (The
+ * paper has no counterpart: this is a deployment variant of the same kernel.)
+ *
+ * Who needs it: segkv_decode_sdpa may grow its split workspace with cudaMalloc
+ * when the launch shape changes.  A caller inside a serving loop whose memory
+ * pool owns the whole device, a caller whose next request must not stall
+ * behind the device-wide synchronisation an allocation implies, or a caller
+ * that is not allowed to call the CUDA allocator at all (a plug-in running
+ * under someone else's allocator policy) cannot afford that.  This entry point
+ * calls no allocator: the partial outputs of the splits, their max/sum pairs
+ * and the arrival counters of the workspace merge live in an 8 MiB array that
+ * is part of the library image; every GPU that loads the library holds those
+ * 8 MiB until the process exits.
+ *
+ * Arguments, results and errors are those of segkv_decode_sdpa; the output
+ * agrees with it within the path's tolerance (the splits are always merged
+ * through the workspace, never inside a cluster, so the summation order can
+ * differ).  In addition:
+ *   - ECAPACITY when batch*kv_heads*splits*beams*(heads/kv_heads)*(head_dim+2)
+ *     floats plus the counters exceed the 8 MiB (segkv_last_cuda_error() says
+ *     so); nothing is launched then.  Fewer splits (segkv_set_tuning) shrink
+ *     the need; one split needs none.  EINVAL for shapes with more than 16
+ *     query columns per kv head, which the tiled kernel does not take;
+ *   - the first call on each device looks the array's device address up
+ *     (cudaGetSymbolAddress, with the handle's device current).  Make that
+ *     first call before any stream capture begins;
+ *   - all handles and all calls share the one array, and it keeps what the
+ *     last call left: the counters are cleared on the stream at the start of
+ *     every call, and two calls that overlap on the GPU (different streams, or
+ *     this and another handle) corrupt each other's partials.  Order them.
+ */
+SEGKV_API int segkv_decode_sdpa_static(segkv_t h, const void* q, void* out, const float* alibi_slopes,
+                                       void* stream);
+
+/*
  * One whole decode step from HOST memory: copies beam_parent, k_new, v_new, q
  * (and slopes, if given) to the device, runs segkv_append + segkv_decode_sdpa,
  * copies `out` back and waits for it.  All pointers are host pointers (pinned

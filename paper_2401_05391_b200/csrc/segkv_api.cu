@@ -334,6 +334,29 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
     return SEGKV_OK;
 }
 
+int segkv_decode_sdpa_static(segkv_t h, const void* q, void* out, const float* alibi_slopes, void* stream) {
+    if (!h || !q || !out || !aligned16(q) || !aligned16(out)) return SEGKV_EINVAL;
+    if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SEGKV_EINVAL;
+    if (h->prompt_len < 0) return SEGKV_ESTATE;
+    if (h->prompt_len + h->steps <= 0) return SEGKV_ESTATE;
+    if (!tiled_supported(h->d)) return SEGKV_EINVAL;
+    int splits, stages;
+    bool cluster;
+    choose_tiling(h, &splits, &stages, &cluster);
+    SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, splits);
+    a.pdl = h->overlap;
+    int too_big = 0;
+    SEGKV_CUDA(launch_sdpa_tiled_static(h->d, a, h->tm_kp, h->tm_vp, stages, (cudaStream_t)stream, &too_big));
+    if (too_big) {
+        snprintf(g_cuda_err, sizeof g_cuda_err,
+                 "segkv_decode_sdpa_static: %d splits of this shape need more than the %zu bytes of built-in scratch",
+                 splits, tiled_static_scratch_bytes());
+        return SEGKV_ECAPACITY;
+    }
+    h->launches++;
+    return SEGKV_OK;
+}
+
 int segkv_step_host(segkv_t h, int step, const int32_t* beam_parent, const void* k_new, const void* v_new,
                     const void* q, void* out, const float* alibi_slopes, void* stream) {
     if (!h || !k_new || !v_new || !q || !out) return SEGKV_EINVAL;

@@ -109,4 +109,9 @@ size_t tiled_smem_bytes(const Dims& d, int stages);      // dynamic shared memor
 cudaError_t launch_sdpa_tiled(const Dims& d, const SdpaArgs& a, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                               int stages, cudaStream_t st);
 
+// Same kernel with its split workspace in a fixed device array of the module (no allocation).
+size_t tiled_static_scratch_bytes();
+cudaError_t launch_sdpa_tiled_static(const Dims& d, SdpaArgs a, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                     int stages, cudaStream_t st, int* too_big);
+
 }  // namespace segkv_impl

@@ -907,6 +907,56 @@ cudaError_t launch_sdpa_tiled(const Dims& d, const SdpaArgs& a, const CUtensorMa
 
 }  // namespace segkv_impl
 
+// ---------------------------------------------------------------------------
+// Variant of the launcher for callers that must not allocate: the split
+// workspace (partial outputs, their max/sum and the arrival tickets of the
+// workspace combine) lives in a fixed array that is part of the loaded module.
+// ---------------------------------------------------------------------------
+namespace segkv_impl {
+
+constexpr size_t kStaticScratchBytes = (size_t)8 << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+size_t tiled_static_scratch_bytes() { return kStaticScratchBytes; }
+
+// Returns cudaSuccess with *too_big = 1 (nothing launched) when the launch shape needs
+// more scratch than the array holds.
+cudaError_t launch_sdpa_tiled_static(const Dims& d, SdpaArgs a, const CUtensorMap& tmk, const CUtensorMap& tmv,
+                                     int stages, cudaStream_t st, int* too_big) {
+    *too_big = 0;
+    // In host code the array's name is only a handle for the runtime, not a device address:
+    // ask for the address once per device (with that device current) and keep it.
+    static void* base_of[64] = {nullptr};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    void* base = (dev >= 0 && dev < 64) ? base_of[dev] : nullptr;
+    if (!base) {
+        e = cudaGetSymbolAddress(&base, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) base_of[dev] = base;
+    }
+    const size_t slabs = (size_t)d.batch * d.kv_heads;
+    const size_t ticket_bytes = (slabs * sizeof(int) + 255) & ~(size_t)255;
+    const size_t ws_bytes = slabs * a.splits * d.beams * d.group * (d.head_dim + 2) * sizeof(float);
+    if (a.splits > 1) {
+        if (ticket_bytes + ws_bytes > kStaticScratchBytes) {
+            *too_big = 1;
+            return cudaSuccess;
+        }
+        // the tickets must read zero at the start of every launch; the array keeps whatever
+        // the last call (of any handle) left there
+        e = cudaMemsetAsync(base, 0, ticket_bytes, st);
+        if (e != cudaSuccess) return e;
+    }
+    a.tickets = reinterpret_cast<int*>(base);
+    a.ws = reinterpret_cast<float*>(static_cast<unsigned char*>(base) + ticket_bytes);
+    a.cluster = false;
+    return launch_sdpa_tiled(d, a, tmk, tmv, stages, st);
+}
+
+}  // namespace segkv_impl
+
 #ifdef SEGKV_TIMELINE
 extern "C" __attribute__((visibility("default"))) int segkv_debug_timeline(unsigned long long* host, int clear) {
     if (cudaMemcpyFromSymbol(host, segkv_impl::g_timeline, sizeof(unsigned long long) * 8 * 512 * 16) != cudaSuccess) return -1;

@@ -31,6 +31,7 @@ SIGNATURES = {
     "segkv_prefill_write": (_int, [_vp, _vp, _vp, _int, _vp]),
     "segkv_append": (_int, [_vp, _int, _vp, _vp, _vp, _vp]),
     "segkv_decode_sdpa": (_int, [_vp, _vp, _vp, _vp, _vp]),
+    "segkv_decode_sdpa_static": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "segkv_step_host": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "segkv_reset": (_int, [_vp, _int]),
     "segkv_truncate_last": (_int, [_vp]),
@@ -169,6 +170,17 @@ class SegKV:
         _check(lib().segkv_decode_sdpa(self._h, _dev(q, shape, self.dtype, "q"), _dev(out, shape, self.dtype, "out"),
                                        _dev(alibi_slopes, (self.heads,), torch.float32, "alibi_slopes"),
                                        _stream_ptr(stream)), "segkv_decode_sdpa")
+        return out
+
+    def decode_sdpa_static(self, q: torch.Tensor, out: torch.Tensor,
+                           alibi_slopes: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """segkv_decode_sdpa_static: same attention, split workspace in the library's built-in
+        device array, no allocation by the library (``out`` must be given for the same reason)."""
+        shape = (self.rows, self.heads, self.head_dim)
+        _check(lib().segkv_decode_sdpa_static(self._h, _dev(q, shape, self.dtype, "q"),
+                                              _dev(out, shape, self.dtype, "out"),
+                                              _dev(alibi_slopes, (self.heads,), torch.float32, "alibi_slopes"),
+                                              _stream_ptr(stream)), "segkv_decode_sdpa_static")
         return out
 
     def step_host(self, step: int, beam_parent, k_new, v_new, q, out, alibi_slopes=None, stream=None) -> torch.Tensor:
