@@ -68,17 +68,28 @@ def unique_bytes(w, prompt_len, unique_rows_total):
 
 # --------------------------------------------------------------------------- clocks
 class ClockSampler:
-    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+    """nvidia-smi clock samples, kept only if taken inside the [begin(), end()] load window."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index):
         self.proc = None
+        self.t0 = self.t1 = None
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(index)],
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50", "-i", str(index)],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
+
+    def begin(self):
+        self.t0 = time.time()
+
+    def end(self):
+        self.t1 = time.time()
+
+    def samples_in_window(self):
+        return 0 if self.t0 is None else int((time.time() - self.t0) / 0.05)
 
     def stop(self):
         if self.proc is None:
@@ -89,17 +100,21 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
             out, _ = self.proc.communicate()
+        import datetime
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in out.splitlines():
             parts = [p.strip() for p in line.split(",")]
-            if len(parts) != 6:
+            if len(parts) != 7:
                 continue
             try:
-                sm.append(float(parts[0])); mx.append(float(parts[1]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                if self.t0 is not None and not (self.t0 <= ts <= (self.t1 or ts)):
+                    continue
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
             except ValueError:
                 continue
-            for n, v in zip(names, parts[2:]):
+            for n, v in zip(names, parts[3:]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
@@ -180,6 +195,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2401_05391_b200 import workloads as wl
+    from paper_2401_05391_b200 import sharding
     from paper_2401_05391_b200.segkv import SegKV
 
     rank = int(os.environ.get("RANK", "0"))
@@ -197,7 +213,8 @@ def run_ours(args):
     T = args.at_step or w.steps
     t = T - 1
     # every rank holds its own requests (weak scaling: requests are independent, no exchange)
-    w_rank = w.scaled(index=w.index + 100 * rank) if world > 1 else w
+    w_rank = sharding.rank_workload(w, rank, world)
+    sampler = ClockSampler(f"GPU-{torch.cuda.get_device_properties(dev).uuid}") if rank == 0 else None
     parents = torch.from_numpy(wl.make_parents(w_rank)).to(dev)
     slopes = wl.alibi_slopes(w.heads).to(dev) if w.alibi else None
 
@@ -263,28 +280,36 @@ def run_ours(args):
         e1.record(stream)
         stream.synchronize()
         torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
+        ms = sharding.max_over_ranks(e0.elapsed_time(e1), dev)
         if world > 1:
-            tt = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
             dist.barrier()
-            ms = float(tt.item())
         return ms
 
     # ---- the timed region: K whole steps (append + attention, all layers)
     run_step, graphed = make_runner(True)
     launches0 = sum(h[0].launch_count for h in handles)
-    sampler = ClockSampler(f"GPU-{torch.cuda.get_device_properties(dev).uuid}") if rank == 0 else None
+    if sampler:
+        sampler.begin()
     ms_total = timed(run_step, args.steps, args.warmup)
     # ---- the attention kernel alone, same rotation over cold layers (roofline numerator)
     run_sdpa, _ = make_runner(False)
     ms_sdpa = timed(run_sdpa, args.steps, max(3, args.warmup))
-    clocks = sampler.stop() if sampler else None
+    clocks = None
+    if sampler:
+        # the timed loops can be shorter than nvidia-smi's sampling period: keep the same load up
+        # (untimed) until a handful of samples fall inside the window
+        t_end = time.time() + 3.0
+        while sampler.samples_in_window() < 12 and time.time() < t_end:
+            for _ in range(20):
+                run_step()
+            stream.synchronize()
+        sampler.end()
+        clocks = sampler.stop()
     launches_per_step = 2 * L
     ms_per_step = ms_total / args.steps
     us_layer = ms_per_step * 1e3 / L
     us_sdpa = ms_sdpa / args.steps * 1e3 / L
-    value = world * L * ubytes / (ms_per_step * 1e-3) / 1e9
+    value = sharding.whole_job_rate(L * ubytes, world, ms_per_step * 1e-3) / 1e9
 
     # ---- end to end from host memory through segkv_step_host
     e2e = None
@@ -309,14 +334,11 @@ def run_ours(args):
             host_step()
         torch.cuda.synchronize()
         sec = (time.perf_counter() - t0) / n_e2e
-        if world > 1:
-            tt = torch.tensor([sec], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            sec = float(tt.item())
+        sec = sharding.max_over_ranks(sec, dev)
         q, k = handles[0][1], handles[0][2]
         h2d = L * (q.numel() * 2 + 2 * k.numel() * 2 + (w.rows * 4 if t > 0 else 0) + (w.heads * 4 if hs is not None else 0))
         d2h = L * q.numel() * 2
-        e2e = {"value": world * L * ubytes / sec / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": sharding.whole_job_rate(L * ubytes, world, sec) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "us_per_step_per_layer": sec * 1e6 / L}
 
     if rank != 0:
