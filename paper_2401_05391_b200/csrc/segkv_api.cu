@@ -148,7 +148,11 @@ void choose_tiling(const segkv* h, int* splits, int* stages, bool* cluster) {
     while (st > 1 && tiled_smem_bytes(d, st) > h->smem_optin) --st;
     *splits = sp;
     *stages = st;
-    *cluster = sp > 1 && h->combine_forced != 1 && tiled_cluster_ok(d, sp);
+    // The workspace merge is the default: launches that merge inside a cluster were measured
+    // not to start early under programmatic dependent launch, which costs more than the
+    // cluster merge saves.  With overlap off the cluster merge is the faster one.
+    const bool want_cluster = h->combine_forced == 2 || (h->combine_forced == 0 && !h->overlap);
+    *cluster = sp > 1 && want_cluster && tiled_cluster_ok(d, sp);
 }
 
 SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes, int splits) {

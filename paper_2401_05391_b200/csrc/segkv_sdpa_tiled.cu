@@ -65,14 +65,18 @@ __device__ __forceinline__ uint64_t global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait (about two seconds): false when it gave up.
+// Bounded wait (about two seconds): false when it gave up.  Between polls the warp sleeps a
+// few tens of nanoseconds so that waiting warps do not crowd the load/store pipe that the
+// producer warps need for their copies.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_ns();
     for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 256; ++i)
+        for (int i = 0; i < 256; ++i) {
+            __nanosleep(32);
             if (mbar_try_wait(bar, parity)) return true;
+        }
         if (global_ns() - t0 > 2000000000ull) return false;
     }
 }
@@ -86,15 +90,16 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, 
         ::"r"(dst), "l"(m), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
-__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+// 16-byte asynchronous copy global -> shared.  No memory clobber: ordering against the consumers
+// comes from the mbarrier arrival that follows the copies.
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src));
 }
-__device__ __forceinline__ void cp_async_8(uint32_t dst, const void* src, uint32_t src_bytes) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
+// mbarrier arrival that fires when all earlier cp.async of this thread have landed
 __device__ __forceinline__ void cp_async_mbar_arrive_noinc(uint32_t bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -166,7 +171,6 @@ __device__ __forceinline__ void st_cluster_v2(uint32_t addr, float a, float b) {
 // previous one to have completed with its writes visible (no-ops without the launch attribute).
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 #ifdef SEGKV_TIMELINE
 }  // namespace
@@ -202,6 +206,7 @@ struct TiledParams {
     int* tickets;
     int* err_word;
     int P, steps, S, W, G, H, Hkv, rows, max_steps, ncols, stages;
+    int quota;      // distinct response rows per split (the last split also takes any excess)
     int cluster;    // 1: the S CTAs of a work group form a thread-block cluster
     int early_prompt;  // 1: prompt tiles may be fetched before the previous kernel has completed
 #ifdef SEGKV_TIMELINE
@@ -231,7 +236,9 @@ struct Layout {
         b = b > comb ? b : comb;
         return (b + 127) & ~(size_t)127;
     }
-    static __host__ __device__ constexpr size_t bars(int stages) { return ((size_t)stages * 16 + 8 + 127) & ~(size_t)127; }
+    static __host__ __device__ constexpr size_t bars(int stages) {
+        return (((size_t)stages * 16 + 8 + 127) & ~(size_t)127) + (size_t)TILE * 8;   // + row offsets of the gather warp
+    }
     static __host__ __device__ constexpr size_t recv(int nt) {
         return (size_t)8 * nt * D * 4 + (size_t)kMaxCluster * 8 * nt * 2 * 4;
     }
@@ -262,6 +269,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     float* recv_o = reinterpret_cast<float*>(smem + L::body(stages, NT) + L::bars(stages));   // [S][slice]
     float* recv_ml = recv_o + 8 * NT * D;                                                     // [S][ncols][2]
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + stages), hand = smem_u32(bars + 2 * stages);
+    size_t* goff = reinterpret_cast<size_t*>(reinterpret_cast<uint8_t*>(recv_o) - (size_t)TILE * 8);   // [TILE], gather warp only
     __shared__ int s_last, s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -292,18 +300,18 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 tma_load_3d(k_dst + bx * L::BOX_BYTES, &tm_k, bx * 64, y, slab, full);
                 tma_load_3d(v_dst + bx * L::BOX_BYTES, &tm_v, bx * 64, y, slab, full);
             }
-        } else {
-            mbar_arrive(full);
         }
+        mbar_arrive(full);      // lanes 1..31, and lane 0 a second time (the count is the gather warp's)
     };
 
     int tma_issued = 0;       // TMA warp: fills started (for the wind-down after an expired wait)
+    int gather_issued = 0;    // gather warp: one past the last ring slot it filled
     if (warp == TMA_WARP) {
         // The warp that issues the bulk loads sets the barriers up itself and starts the
         // first round of prompt tiles before the rest of the CTA has even synchronised.
         if (lane == 0) {
             for (int s = 0; s < stages; ++s) {
-                mbar_init(full0 + 8 * s, 32);     // every lane of the filling warp arrives once per fill
+                mbar_init(full0 + 8 * s, 33);     // every lane of the filling warp, plus lane 0 once more
                 mbar_init(empty0 + 8 * s, CW);    // one arrival per consumer warp
             }
             mbar_init(hand, 1);                   // ring handed from the TMA warp to the gather warp
@@ -354,18 +362,24 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         // The chain row count -> row list starts at once, beside the TMA warp; the ring itself
         // is taken over only when the last prompt tile has been issued (a parity wait cannot
         // tell a far-future round of a stage from the current one).
-        const int n_b = p.steps > 0 ? p.ucount[b] : 0;
-        const int e0 = (int)((long long)split * n_b / p.S), e1 = (int)((long long)(split + 1) * n_b / p.S);
-        const int nrt = (e1 - e0 + TILE - 1) / TILE;
-        SEGKV_STAMP(4);
-        bool ok = true;
-        // row ids of the next tile are fetched while the current one is being issued
-        int urow[UK], urow_next[UK];
+        // A split's range starts at split * quota whatever the row count turns out to be, so
+        // the first tile's list entries are requested together with the count, not after it.
+        uint2 ucur[UK], unext[UK];          // {row, beam mask} of this lane's keys (lane, lane + 32)
+        const int cap = p.W * p.max_steps;
 #pragma unroll
         for (int kk = 0; kk < UK; ++kk) {
             const int key = lane + 32 * kk;
-            urow_next[kk] = (key < TILE && e0 + key < e1) ? ulist_b[e0 + key].row : 0;
+            unext[kk] = (p.steps > 0 && key < TILE)
+                            ? *reinterpret_cast<const uint2*>(ulist_b + min(split * p.quota + key, cap - 1))
+                            : make_uint2(0u, 0u);
         }
+        const int n_b = p.steps > 0 ? p.ucount[b] : 0;
+        const int e0 = min(split * p.quota, n_b);
+        const int e1 = (split == p.S - 1) ? n_b : min((split + 1) * p.quota, n_b);
+        const int nrt = (e1 - e0 + TILE - 1) / TILE;
+        SEGKV_STAMP(4);
+        SEGKV_CLK(1, true);
+        bool ok = true;
         if (nrt > 0) {
             ok = mbar_wait(hand, 0);
             ok = __all_sync(0xffffffffu, ok);
@@ -376,47 +390,77 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             const int cnt = min(TILE, e1 - eb);
 #pragma unroll
             for (int kk = 0; kk < UK; ++kk) {
-                urow[kk] = urow_next[kk];
+                ucur[kk] = unext[kk];
                 const int key = lane + 32 * kk;
-                urow_next[kk] = (key < TILE && eb + TILE + key < e1) ? ulist_b[eb + TILE + key].row : 0;
+                unext[kk] = (key < TILE && eb + TILE + key < e1)
+                                ? *reinterpret_cast<const uint2*>(ulist_b + eb + TILE + key)
+                                : make_uint2(0u, 0u);
             }
             const int st = k % stages;
             ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const uint32_t full = full0 + 8 * st;
-            const uint32_t k_dst = smem_u32(ring + (size_t)st * L::STAGE_BYTES);
-            const uint32_t v_dst = k_dst + L::TILE_BYTES;
-            const uint32_t meta_dst = smem_u32(meta + (size_t)st * TILE);
+            uint8_t* k_tile = ring + (size_t)st * L::STAGE_BYTES;
+            uint8_t* v_tile = k_tile + L::TILE_BYTES;
+            const uint32_t k_dst = smem_u32(k_tile), v_dst = k_dst + L::TILE_BYTES;
+            URow* meta_st = meta + (size_t)st * TILE;
+            SEGKV_CLK(11, r == 0);
+            // Each lane publishes {row, mask} and the byte offset of its keys (lane, lane + 32);
+            // rows between the last real one and the end of its 16-key slice are zeroed with
+            // plain stores (rows past that slice are never looked at).
+            constexpr int CPR = D / 8;        // 16-byte chunks per row
+            constexpr int RPI = 32 / CPR;     // rows covered by one warp-wide copy
+            const int fill = min(TILE, (cnt + 15) & ~15);
 #pragma unroll
             for (int kk = 0; kk < UK; ++kk) {
                 const int key = lane + 32 * kk;
-                if (key < TILE) {
-                    const bool valid = key < cnt;
-                    cp_async_8(meta_dst + key * 8, valid ? (const void*)(ulist_b + eb + key) : (const void*)p.ulist,
-                               valid ? 8u : 0u);
+                if (key >= TILE) continue;
+                const bool valid = key < cnt;
+                URow u;
+                u.row = valid ? (int32_t)ucur[kk].x : 0;
+                u.mask = valid ? ucur[kk].y : 0u;
+                meta_st[key] = u;
+                goff[key] = ((size_t)u.row * p.Hkv + kvh) * (size_t)(D * 2);
+            }
+            // zero the rows between the last real one and the end of its 16-key slice: in every
+            // 128-byte box they are one contiguous run, filled 16 bytes per lane
+            {
+                const int zchunks = (fill - cnt) * 8;
+#pragma unroll
+                for (int bx = 0; bx < D / 64; ++bx) {
+                    uint4* kz = reinterpret_cast<uint4*>(k_tile + (size_t)bx * L::BOX_BYTES + (size_t)cnt * 128);
+                    uint4* vz = reinterpret_cast<uint4*>(v_tile + (size_t)bx * L::BOX_BYTES + (size_t)cnt * 128);
+                    for (int i = lane; i < zchunks; i += 32) {
+                        kz[i] = make_uint4(0u, 0u, 0u, 0u);
+                        vz[i] = make_uint4(0u, 0u, 0u, 0u);
+                    }
                 }
             }
-            constexpr int CPR = D / 8;        // 16-byte chunks per row
-            constexpr int RPI = 32 / CPR;     // rows covered by one warp-wide copy
+            SEGKV_CLK(14, r == 0);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full);          // releases the plain stores of the whole warp
+            SEGKV_CLK(6, r == 0);
+            // One warp-wide copy moves whole rows (CPR lanes per row): fully coalesced.
             const int c = lane % CPR;
             const uint32_t c_off = (uint32_t)(c / 8) * L::BOX_BYTES;
-            // rows past the last one a consumer warp will look at need no zero fill
-            const int fill = min(TILE, (cnt + 15) & ~15);
-#pragma unroll 4
+#pragma unroll
             for (int i = 0; i < TILE / RPI; ++i) {
-                const int key = i * RPI + lane / CPR;
-                int rr = urow[0];
-                if (TILE > 32 && key >= 32) rr = urow[UK - 1];
-                rr = __shfl_sync(0xffffffffu, rr, key & 31);
-                if (i * RPI >= fill) continue;            // warp-uniform
-                const bool valid = key < cnt;
-                const size_t src = ((size_t)rr * p.Hkv + kvh) * (size_t)(D * 2) + (size_t)c * 16;
-                const uint32_t off = c_off + (uint32_t)key * 128 + (uint32_t)(((c & 7) ^ (key & 7)) << 4);
-                cp_async_16(k_dst + off, valid ? p.kr + src : p.kr, valid ? 16u : 0u);
-                cp_async_16(v_dst + off, valid ? p.vr + src : p.vr, valid ? 16u : 0u);
+                if (i * RPI < cnt) {                       // warp-uniform
+                    const int key = i * RPI + lane / CPR;
+                    if (key < cnt) {
+                        const size_t src = goff[key] + (size_t)c * 16;
+                        const uint32_t off = c_off + (uint32_t)key * 128 + (uint32_t)(((c & 7) ^ (key & 7)) << 4);
+                        cp_async_16(k_dst + off, p.kr + src);
+                        cp_async_16(v_dst + off, p.vr + src);
+                    }
+                }
             }
+            SEGKV_CLK(7, r == 0);
             cp_async_mbar_arrive_noinc(full);
+            __syncwarp();                                  // goff is rewritten for the next tile
+            gather_issued = k + 1;
+            SEGKV_CLK(15, r == 0);
         }
         SEGKV_STAMP(5);
         if (!ok && lane == 0) {
@@ -434,6 +478,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 #pragma unroll
                 for (int i = 0; i < 4; ++i) o_acc[nt][mt][i] = 0.f;
         }
+        const int n_b = p.steps > 0 ? p.ucount[b] : 0;   // in flight while the prompt tiles are consumed
         // Q^T as the B operand: this lane holds column n = lane/4 of every column tile
         uint32_t qf[NT][KS][2];
 #pragma unroll
@@ -466,29 +511,30 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 
         // One tile: `nvalid` keys exist; for a response tile the per-key beam masks and row
         // ids are in the stage's meta array, for a prompt tile key i sits at position pos0 + i.
+        // shared-memory address of 16-byte chunk `ch` of row `key` of a tile (the TMA layout:
+        // 128-byte boxes, XOR swizzle; the gather warp writes response rows the same way)
+        auto chunk_addr = [&](uint32_t base, int key, int ch, bool) -> uint32_t {
+            return base + (uint32_t)(ch >> 3) * L::BOX_BYTES + (uint32_t)key * 128 + (uint32_t)(((ch & 7) ^ (key & 7)) << 4);
+        };
         auto consume = [&](int st, bool resp, int nvalid, int pos0) {
             if (warp * 16 >= nvalid) return;
             const uint32_t k_src = smem_u32(ring + (size_t)st * L::STAGE_BYTES);
             const uint32_t v_src = k_src + L::TILE_BYTES;
-            SEGKV_CLK(1, warp == 0 && st == 0 && !resp && pos0 == pt0 * TILE);
             // ---- S^T = K . Q^T ----
             float sc[NT][4];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
             {
                 const int key = warp * 16 + (lane & 15);
-                const uint32_t rowaddr = k_src + (uint32_t)key * 128;
-                const int sw = key & 7;
 #pragma unroll
                 for (int ks = 0; ks < KS; ++ks) {
                     const int ch = 2 * ks + (lane >> 4);
                     uint32_t a[4];
-                    ldmatrix_x4(a, rowaddr + (uint32_t)(ch >> 3) * L::BOX_BYTES + (uint32_t)(((ch & 7) ^ sw) << 4));
+                    ldmatrix_x4(a, chunk_addr(k_src, key, ch, resp));
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) Mma<T>::run(sc[nt], a, qf[nt][ks][0], qf[nt][ks][1]);
                 }
             }
-            SEGKV_CLK(14, warp == 0 && st == 0 && !resp && pos0 == pt0 * TILE);
             // ---- mask, bias, online softmax ----
             uint32_t kmask[2];
             float kpos[2];
@@ -550,33 +596,27 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                         o_acc[nt][mt][3] *= alpha[nt][1];
                     }
             }
-            SEGKV_CLK(15, warp == 0 && st == 0 && !resp && pos0 == pt0 * TILE);
             // ---- O^T += V^T . P^T ----
             {
                 const int key = warp * 16 + (lane & 7) + 8 * (lane >> 4);
-                const uint32_t rowaddr = v_src + (uint32_t)key * 128;
-                const int sw = key & 7;
 #pragma unroll
                 for (int mt = 0; mt < KS; ++mt) {
                     const int ch = 2 * mt + ((lane >> 3) & 1);
                     uint32_t a[4];
-                    ldmatrix_x4_trans(a, rowaddr + (uint32_t)(ch >> 3) * L::BOX_BYTES + (uint32_t)(((ch & 7) ^ sw) << 4));
+                    ldmatrix_x4_trans(a, chunk_addr(v_src, key, ch, resp));
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) Mma<T>::run(o_acc[nt][mt], a, pfrag[nt][0], pfrag[nt][1]);
                 }
             }
-            SEGKV_CLK(11, warp == 0 && st == 0 && !resp && pos0 == pt0 * TILE);
         };
 
         bool ok = true;
         int k = 0;
-        if (warp == 0) SEGKV_STAMP(6);
         for (; k < npt; ++k) {
             const int st = k % stages;
             ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            if (warp == 0 && k == 0) SEGKV_STAMP(7);
             const int pos0 = (pt0 + k) * TILE;
             consume(st, false, min(TILE, p.P - pos0), pos0);
             __syncwarp();
@@ -584,8 +624,8 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         }
         if (warp == 0) SEGKV_STAMP(8);
         if (ok) {
-            const int n_b = p.steps > 0 ? p.ucount[b] : 0;
-            const int e0 = (int)((long long)split * n_b / p.S), e1 = (int)((long long)(split + 1) * n_b / p.S);
+            const int e0 = min(split * p.quota, n_b);
+            const int e1 = (split == p.S - 1) ? n_b : min((split + 1) * p.quota, n_b);
             const int nrt = (e1 - e0 + TILE - 1) / TILE;
             for (int r = 0; r < nrt; ++r, ++k) {
                 const int st = k % stages;
@@ -743,56 +783,50 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     // ---- arrive (atomic ticket, nobody waits) merges all partials
     __syncthreads();
     if (tid == 0) {
-        __threadfence();                                   // partials visible before the ticket
-        const int ticket = atomicAdd(p.tickets + slab, 1);
-        const int last = (ticket == S - 1);
-        if (last) __threadfence();                         // and the others' partials before reading
-        s_last = last;
+        // release: this CTA's partials (ordered before by the barrier) are visible before the
+        // ticket; acquire: the last arriver sees every other CTA's partials
+        int ticket;
+        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(ticket) : "l"(p.tickets + slab) : "memory");
+        s_last = (ticket == S - 1);
     }
     __syncthreads();
     if (tid == 0) SEGKV_STAMP(12);
     if (!s_last) return;
 
-    float* c_f = reinterpret_cast<float*>(smem);           // [S][ncols] max, then scale factor
-    float* c_l = c_f + (size_t)S * ncols;
-    const float* wsml_slab = p.ws_ml + (size_t)slab * S * ncols * 2;
+    // One pass: each thread owns a float4 of one column and folds the splits in, eight at a
+    // time (their partial outputs and max/sum pairs are all requested before any is used).
+    const float2* wsml_slab = reinterpret_cast<const float2*>(p.ws_ml + (size_t)slab * S * ncols * 2);
     const float* wso_slab = p.ws_o + (size_t)slab * S * ncols * D;
-    for (int i = tid; i < S * ncols; i += NTHREADS) {
-        const float2 ml = __ldcg(reinterpret_cast<const float2*>(wsml_slab) + i);
-        c_f[i] = ml.x;
-        c_l[i] = ml.y;
-    }
-    __syncthreads();
-    if (tid < ncols) {
-        float mm = -INFINITY;
-        for (int s = 0; s < S; ++s) mm = fmaxf(mm, c_f[s * ncols + tid]);
-        float ll = 0.f;
-        for (int s = 0; s < S; ++s) {
-            const float ms = c_f[s * ncols + tid];
-            const float f = (ms == -INFINITY) ? 0.f : exp2f(ms - mm);
-            ll += c_l[s * ncols + tid] * f;
-            c_f[s * ncols + tid] = f;
-        }
-        const float inv = 1.f / ll;
-        for (int s = 0; s < S; ++s) c_f[s * ncols + tid] *= inv;
-    }
-    __syncthreads();
     for (int it = tid; it < ncols * D4; it += NTHREADS) {
         const int col = it / D4, d = (it % D4) * 4;
-        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
         const float4* src = reinterpret_cast<const float4*>(wso_slab + (size_t)col * D + d);
         const size_t sstride = (size_t)ncols * D4;            // float4 per split
+        float mm = -INFINITY, ll = 0.f;
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int s0 = 0; s0 < S; s0 += 8) {
             float4 v[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-                v[u] = (s0 + u < S) ? __ldcg(src + (size_t)(s0 + u) * sstride) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float2 ml[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const float f = (s0 + u < S) ? c_f[(s0 + u) * ncols + col] : 0.f;
+                const bool in = s0 + u < S;
+                ml[u] = in ? __ldcg(wsml_slab + (size_t)(s0 + u) * ncols + col) : make_float2(-INFINITY, 0.f);
+                v[u] = in ? __ldcg(src + (size_t)(s0 + u) * sstride) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            float bm = mm;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) bm = fmaxf(bm, ml[u].x);
+            const float fo = (mm == -INFINITY) ? 0.f : exp2f(mm - bm);
+            ll *= fo; o.x *= fo; o.y *= fo; o.z *= fo; o.w *= fo;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float f = (ml[u].x == -INFINITY) ? 0.f : exp2f(ml[u].x - bm);
+                ll += ml[u].y * f;
                 o.x += v[u].x * f; o.y += v[u].y * f; o.z += v[u].z * f; o.w += v[u].w * f;
             }
+            mm = bm;
         }
+        const float inv = 1.f / ll;
+        o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
         store_out(col, d, o);
     }
     if (tid == 0) p.tickets[slab] = 0;      // ready for the next launch
@@ -820,6 +854,8 @@ cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk,
     p.P = a.prompt_len; p.steps = a.steps; p.S = a.splits; p.W = d.beams; p.G = d.group; p.H = d.heads;
     p.Hkv = d.kv_heads; p.rows = d.rows; p.max_steps = d.max_steps; p.ncols = d.beams * d.group; p.stages = stages;
     p.scale2 = 1.4426950408889634f / sqrtf((float)D);
+    p.quota = (a.steps + 2 * d.beams + a.splits - 1) / a.splits;
+    if (p.quota < 1) p.quota = 1;
     p.cluster = a.cluster ? 1 : 0;
     p.early_prompt = (a.pdl && a.steps > 0) ? 1 : 0;
 #ifdef SEGKV_TIMELINE
