@@ -42,6 +42,7 @@ def parse():
     ap.add_argument("--workload", default="llama2-7b")
     ap.add_argument("--layers", type=int, default=0, help="distinct cache handles per step (0 = per-workload default)")
     ap.add_argument("--at-step", type=int, default=0, help="decode step to time, 1-based (0 = the workload's last)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling a smaller case)")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--combine", type=int, default=0, help="0 auto, 1 workspace+ticket, 2 cluster")
@@ -209,7 +210,9 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     w = wl.by_name(args.workload)
-    L = args.layers or DEFAULT_LAYERS.get(w.name, 1)
+    if args.batch:
+        w = w.scaled(batch=args.batch, name=f"{w.name}[batch={args.batch}]")
+    L = args.layers or DEFAULT_LAYERS.get(w.name.split("[")[0], 1)
     T = args.at_step or w.steps
     t = T - 1
     # every rank holds its own requests (weak scaling: requests are independent, no exchange)
