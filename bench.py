@@ -30,6 +30,9 @@ sys.path.insert(0, ROOT)
 
 METRIC = "decode_sdpa_unique_kv_bandwidth"
 UNIT = "GB/s"
+# dram__bytes_read.sum + dram__bytes_write.sum per attention launch from the ncu captures summarised
+# under profiles/ (the OPT-30B figure is the batch-4 capture scaled by 16; traffic grows with the batch)
+NCU_TRAFFIC_BYTES = {"llama2-7b": 19.190e6, "opt-30b": 16 * (267.04e6 + 5.1e6)}
 DEFAULT_LAYERS = {"tiny": 32, "llama2-7b": 32, "llama2-13b": 32, "gptj-6b": 4, "opt-30b": 1, "bloom-176b": 1}
 
 
@@ -366,7 +369,7 @@ def run_ours(args):
         "pct_of_8000_GBps": 100.0 * achieved / 8000.0,
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "segkv decode attention",
+                     "traffic": NCU_TRAFFIC_BYTES.get(w.name) if T == w.steps else None, "peak_kind": f"of {peak_kind}", "kernel": "segkv decode attention",
                      "bytes_per_launch": ubytes, "us_per_launch": us_sdpa},
         "e2e": e2e,
         "clocks": clocks,
