@@ -2,8 +2,8 @@
 """Benchmark of the segment-KV decode attention path on B200.
 
 One *step* is one decode step of an L-layer stack of attention layers of the
-chosen shape: per layer, append the step's K/V rows (which also updates the
-beam-index table) and run the fused decode attention.  All layers are distinct
+chosen shape: per layer one `segkv_decode_step` call, which appends the step's
+K/V rows, updates the beam-index table and runs the decode attention in one launch.  All layers are distinct
 cache handles, so a step touches L x (unique KV bytes) of HBM, far more than
 the L2 holds, and every timed kernel reads cold data.
 
@@ -246,26 +246,33 @@ def run_ours(args):
     par_t = parents[t] if t > 0 else None
     stream = torch.cuda.Stream()
 
-    def layer_pass(append: bool):
+    def layer_pass(mode: str):
+        # "step": the whole hot path in the library's fused call; "two": the same as two calls
+        # (append, then attention); "sdpa": the attention kernel alone on the state already there
         for h, q, k, v, out in handles:
-            if append:
+            if mode == "step":
+                h.truncate_last()
+                h.decode_step(t, par_t, k, v, q, out, slopes, stream=stream)
+            elif mode == "two":
                 h.truncate_last()
                 h.append(t, par_t, k, v, stream=stream)
-            h.decode_sdpa(q, out, slopes, stream=stream)
+                h.decode_sdpa(q, out, slopes, stream=stream)
+            else:
+                h.decode_sdpa(q, out, slopes, stream=stream)
 
-    def make_runner(append: bool):
+    def make_runner(mode: str):
         with torch.cuda.stream(stream):
-            layer_pass(append)                               # lazy initialisation outside any capture
+            layer_pass(mode)                                 # lazy initialisation outside any capture
         stream.synchronize()
         if args.no_graph:
-            return lambda: layer_pass(append), False
+            return lambda: layer_pass(mode), False
         g = torch.cuda.CUDAGraph()
         try:
             with torch.cuda.graph(g, stream=stream):
-                layer_pass(append)
+                layer_pass(mode)
         except Exception as e:                               # report, never hide
             sys.stderr.write(f"[bench] CUDA graph capture failed ({e}); timing direct launches\n")
-            return lambda: layer_pass(append), False
+            return lambda: layer_pass(mode), False
 
         def replay():
             with torch.cuda.stream(stream):
@@ -291,15 +298,18 @@ def run_ours(args):
             dist.barrier()
         return ms
 
-    # ---- the timed region: K whole steps (append + attention, all layers)
-    run_step, graphed = make_runner(True)
+    # ---- the timed region: K whole steps (append + beam-index update + attention, all layers)
+    run_step, graphed = make_runner("step")
     launches0 = sum(h[0].launch_count for h in handles)
     if sampler:
         sampler.begin()
     ms_total = timed(run_step, args.steps, args.warmup)
     # ---- the attention kernel alone, same rotation over cold layers (roofline numerator)
-    run_sdpa, _ = make_runner(False)
+    run_sdpa, _ = make_runner("sdpa")
     ms_sdpa = timed(run_sdpa, args.steps, max(3, args.warmup))
+    # ---- for comparison: the same step as two library calls (append, then attention)
+    run_two, _ = make_runner("two")
+    ms_two = timed(run_two, args.steps, max(3, args.warmup))
     clocks = None
     if sampler:
         # the timed loops can be shorter than nvidia-smi's sampling period: keep the same load up
@@ -311,7 +321,7 @@ def run_ours(args):
             stream.synchronize()
         sampler.end()
         clocks = sampler.stop()
-    launches_per_step = 2 * L
+    launches_per_step = L
     ms_per_step = ms_total / args.steps
     us_layer = ms_per_step * 1e3 / L
     us_sdpa = ms_sdpa / args.steps * 1e3 / L
@@ -364,6 +374,7 @@ def run_ours(args):
                    "splits": handles[0][0].get_splits(), "parallelism": f"replica x{world}" if world > 1 else "1 gpu"},
         "us_per_step_per_layer": us_layer,
         "us_sdpa_per_layer": us_sdpa,
+        "us_per_step_per_layer_two_calls": ms_two / args.steps * 1e3 / L,
         "unique_kv_bytes_per_layer": ubytes,
         "logical_kv_bytes_per_layer": logical_bytes,
         "pct_of_8000_GBps": 100.0 * achieved / 8000.0,

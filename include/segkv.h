@@ -130,6 +130,21 @@ SEGKV_API int segkv_append(segkv_t h, int step, const int32_t* beam_parent, cons
 SEGKV_API int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_slopes, void* stream);
 
 /*
+ * One decode step in ONE launch: exactly segkv_append(step, ...) followed by
+ * segkv_decode_sdpa(q, out, ...), fused (Section 3.1-3.3 taken together: the
+ * step's Key_t/Value_t, its beam indices and the attention over prompt +
+ * responses).  The attention kernel derives the new beam-index column from
+ * `beam_parent` and the previous step's table while it gathers, reads the new
+ * rows straight from k_new / v_new, and stores rows, parents and table for the
+ * following steps.  Saves a launch and a dependent memory round trip per layer.
+ * Arguments, layouts and errors are those of the two calls; shapes with more
+ * than 16 query columns per kv head fall back to the two launches.
+ */
+SEGKV_API int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const void* k_new,
+                                const void* v_new, const void* q, void* out, const float* alibi_slopes,
+                                void* stream);
+
+/*
  * segkv_decode_sdpa for callers that must not allocate device memory.  (The
  * paper has no counterpart: this is a deployment variant of the same kernel.)
  *
@@ -166,7 +181,7 @@ SEGKV_API int segkv_decode_sdpa_static(segkv_t h, const void* q, void* out, cons
 
 /*
  * One whole decode step from HOST memory: copies beam_parent, k_new, v_new, q
- * (and slopes, if given) to the device, runs segkv_append + segkv_decode_sdpa,
+ * (and slopes, if given) to the device, runs segkv_decode_step,
  * copies `out` back and waits for it.  All pointers are host pointers (pinned
  * memory makes the copies asynchronous); layouts as in the device calls.
  * Staging buffers are part of the handle.  Errors: as the two calls.

@@ -155,6 +155,16 @@ void choose_tiling(const segkv* h, int* splits, int* stages, bool* cluster) {
     *cluster = sp > 1 && want_cluster && tiled_cluster_ok(d, sp);
 }
 
+// The attention kernel's separate form walks per-request lists of distinct rows that the append
+// kernel makes; fused steps skip them, so they are re-derived from the table when needed.
+int ensure_lists(segkv* h, cudaStream_t st) {
+    if (h->lists_valid || h->steps == 0) return SEGKV_OK;
+    SEGKV_CUDA(launch_rebuild_lists(h->d, h->steps, h->anc[(h->steps - 1) & 1], h->ulist, h->ucount, st));
+    h->launches++;
+    h->lists_valid = true;
+    return SEGKV_OK;
+}
+
 SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes, int splits) {
     SdpaArgs a;
     a.q = q;
@@ -175,6 +185,13 @@ SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes
     a.splits = splits;
     a.cluster = false;
     a.pdl = false;
+    a.prompt_immutable = h->steps > 0;     // the first append after a prefill is a fully serialised launch
+    a.fused = false;
+    a.parent = nullptr;
+    a.k_new = a.v_new = nullptr;
+    a.kr_new_slab = a.vr_new_slab = nullptr;
+    a.anc_dst = nullptr;
+    a.parent_row = nullptr;
     return a;
 }
 
@@ -245,9 +262,9 @@ int segkv_create(segkv_t* out, int batch, int beams, int heads, int kv_heads, in
     SEGKV_TRY(dmalloc(&h->anc[1], (size_t)max_steps * d.rows * sizeof(int32_t)));
     SEGKV_TRY(dmalloc(&h->ulist, (size_t)max_steps * d.rows * sizeof(URow)));
     SEGKV_TRY(dmalloc(&h->ucount, (size_t)batch * sizeof(int32_t)));
+    SEGKV_TRY(cudaMemset(h->ucount, 0, (size_t)batch * sizeof(int32_t)));
     SEGKV_TRY(dmalloc(&h->err_word, sizeof(int)));
     SEGKV_TRY(dmalloc(&h->tickets, (size_t)batch * kv_heads * sizeof(int)));
-    SEGKV_TRY(cudaMemset(h->ucount, 0, (size_t)batch * sizeof(int32_t)));
     SEGKV_TRY(cudaMemset(h->err_word, 0, sizeof(int)));
     SEGKV_TRY(cudaMemset(h->tickets, 0, (size_t)batch * kv_heads * sizeof(int)));
     const size_t qbytes = (size_t)d.rows * heads * head_dim * eb;
@@ -306,6 +323,7 @@ int segkv_append(segkv_t h, int step, const int32_t* beam_parent, const void* k_
     h->launches++;
     h->steps = step + 1;
     h->truncated = false;
+    h->lists_valid = true;
     return SEGKV_OK;
 }
 
@@ -319,6 +337,10 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
         SEGKV_CUDA(launch_sdpa_rowwise(h->d, a, (cudaStream_t)stream));
         h->launches++;
         return SEGKV_OK;
+    }
+    {
+        int rc = ensure_lists(h, (cudaStream_t)stream);
+        if (rc != SEGKV_OK) return rc;
     }
     int splits, stages;
     bool cluster;
@@ -344,6 +366,10 @@ int segkv_decode_sdpa_static(segkv_t h, const void* q, void* out, const float* a
     if (h->prompt_len < 0) return SEGKV_ESTATE;
     if (h->prompt_len + h->steps <= 0) return SEGKV_ESTATE;
     if (!tiled_supported(h->d)) return SEGKV_EINVAL;
+    {
+        int rc = ensure_lists(h, (cudaStream_t)stream);     // a kernel launch at most, never an allocation
+        if (rc != SEGKV_OK) return rc;
+    }
     int splits, stages;
     bool cluster;
     choose_tiling(h, &splits, &stages, &cluster);
@@ -358,6 +384,65 @@ int segkv_decode_sdpa_static(segkv_t h, const void* q, void* out, const float* a
         return SEGKV_ECAPACITY;
     }
     h->launches++;
+    return SEGKV_OK;
+}
+
+int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const void* k_new, const void* v_new,
+                      const void* q, void* out, const float* alibi_slopes, void* stream) {
+    if (!h || step < 0 || !k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return SEGKV_EINVAL;
+    if (!q || !out || !aligned16(q) || !aligned16(out)) return SEGKV_EINVAL;
+    if (step > 0 && (!beam_parent || (reinterpret_cast<uintptr_t>(beam_parent) & 3u))) return SEGKV_EINVAL;
+    if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SEGKV_EINVAL;
+    if (h->prompt_len < 0) return SEGKV_ESTATE;
+    if (step != h->steps) return SEGKV_ESTATE;
+    if (step >= h->d.max_steps) return SEGKV_ECAPACITY;
+    if (!tiled_supported(h->d)) {
+        // shapes the tiled kernel does not take: the two separate launches
+        int rc = segkv_append(h, step, beam_parent, k_new, v_new, stream);
+        if (rc != SEGKV_OK) return rc;
+        return segkv_decode_sdpa(h, q, out, alibi_slopes, stream);
+    }
+    const Dims& d = h->d;
+    h->steps = step + 1;                 // the launch shape is chosen for the step being added
+    int splits, stages;
+    bool cluster;
+    choose_tiling(h, &splits, &stages, &cluster);
+    h->steps = step;
+    if (splits == 1 && !h->fuse_always) {
+        // Work groups that fill the GPU on their own are bandwidth-bound: the separate append is
+        // then ~1 % of the step and the list it makes keeps the response tiles dense and cheap
+        // to build, so the two launches are the faster form.
+        int rc = segkv_append(h, step, beam_parent, k_new, v_new, stream);
+        if (rc != SEGKV_OK) return rc;
+        return segkv_decode_sdpa(h, q, out, alibi_slopes, stream);
+    }
+    if (h->combine_forced == 2 && splits > 1 && !cluster) return SEGKV_EINVAL;
+    if (!cluster && splits > h->ws_splits) {
+        SEGKV_CUDA(cudaDeviceSynchronize());
+        int rc = alloc_workspace(h, splits);
+        if (rc != SEGKV_OK) return rc;
+    }
+    SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, splits);
+    const size_t slab_bytes = (size_t)d.rows * d.kv_heads * d.head_dim * 2;
+    a.steps = step + 1;
+    a.anc = h->anc[(step + 1) & 1];      // table of step-1 (unused at step 0)
+    a.cluster = cluster;
+    // the first step after a prefill is fully serialised; from then on the prompt cannot change
+    a.pdl = h->overlap && step > 0;
+    a.prompt_immutable = step > 0;
+    a.fused = true;
+    a.parent = step > 0 ? beam_parent : nullptr;
+    a.k_new = k_new;
+    a.v_new = v_new;
+    a.kr_new_slab = (char*)h->kr + (size_t)step * slab_bytes;
+    a.vr_new_slab = (char*)h->vr + (size_t)step * slab_bytes;
+    a.anc_dst = h->anc[step & 1];
+    a.parent_row = h->parent + (size_t)step * d.rows;
+    SEGKV_CUDA(launch_sdpa_tiled(d, a, h->tm_kp, h->tm_vp, stages, (cudaStream_t)stream));
+    h->launches++;
+    h->steps = step + 1;
+    h->truncated = false;
+    h->lists_valid = false;              // the fused kernel does not make the distinct-row lists
     return SEGKV_OK;
 }
 
@@ -378,9 +463,8 @@ int segkv_step_host(segkv_t h, int step, const int32_t* beam_parent, const void*
     if (alibi_slopes)
         SEGKV_CUDA(cudaMemcpyAsync(h->st_slopes, alibi_slopes, (size_t)d.heads * sizeof(float),
                                    cudaMemcpyHostToDevice, st));
-    int rc = segkv_append(h, step, step > 0 ? h->st_parent : nullptr, h->st_k, h->st_v, stream);
-    if (rc != SEGKV_OK) return rc;
-    rc = segkv_decode_sdpa(h, h->st_q, h->st_out, alibi_slopes ? h->st_slopes : nullptr, stream);
+    int rc = segkv_decode_step(h, step, step > 0 ? h->st_parent : nullptr, h->st_k, h->st_v, h->st_q, h->st_out,
+                               alibi_slopes ? h->st_slopes : nullptr, stream);
     if (rc != SEGKV_OK) return rc;
     SEGKV_CUDA(cudaMemcpyAsync(out, h->st_out, qbytes, cudaMemcpyDeviceToHost, st));
     SEGKV_CUDA(cudaStreamSynchronize(st));
@@ -422,14 +506,29 @@ int segkv_get_ancestry(segkv_t h, int32_t* host_out, void* stream) {
 int segkv_get_unique_rows(segkv_t h, int32_t* host_out, void* stream) {
     if (!h || !host_out) return SEGKV_EINVAL;
     if (h->truncated) return SEGKV_ESTATE;
-    if (h->steps == 0) {
-        memset(host_out, 0, (size_t)h->d.batch * sizeof(int32_t));
-        return SEGKV_OK;
+    const Dims& d = h->d;
+    memset(host_out, 0, (size_t)d.batch * sizeof(int32_t));
+    if (h->steps == 0) return SEGKV_OK;
+    // count on the host what the attention kernel de-duplicates on the fly
+    int32_t* anc = (int32_t*)malloc((size_t)d.rows * h->steps * sizeof(int32_t));
+    if (!anc) return SEGKV_ENOMEM;
+    int rc = segkv_get_ancestry(h, anc, stream);
+    if (rc == SEGKV_OK) {
+        for (int b = 0; b < d.batch; ++b) {
+            int n = 0;
+            for (int s = 0; s < h->steps; ++s)
+                for (int j = 0; j < d.beams; ++j) {
+                    bool first = true;
+                    const int32_t rj = anc[(size_t)(b * d.beams + j) * h->steps + s];
+                    for (int i = 0; i < j && first; ++i)
+                        first = anc[(size_t)(b * d.beams + i) * h->steps + s] != rj;
+                    n += first ? 1 : 0;
+                }
+            host_out[b] = n;
+        }
     }
-    SEGKV_CUDA(cudaMemcpyAsync(host_out, h->ucount, (size_t)h->d.batch * sizeof(int32_t), cudaMemcpyDeviceToHost,
-                               (cudaStream_t)stream));
-    SEGKV_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
-    return SEGKV_OK;
+    free(anc);
+    return rc;
 }
 
 int segkv_get_error(segkv_t h, int* device_flags) {
@@ -450,6 +549,7 @@ int segkv_set_tuning(segkv_t h, int splits, int stages, int combine) {
     h->splits_forced = splits;
     h->stages_forced = stages;
     h->combine_forced = combine;
+    h->fuse_always = splits == 1;        // an explicit single split still exercises the fused kernel
     return SEGKV_OK;
 }
 

@@ -81,7 +81,7 @@ append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __
               const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, uint4* __restrict__ kr_slab,
               uint4* __restrict__ vr_slab, long long slab_chunks, int32_t* __restrict__ parent_row,
               const int32_t* __restrict__ anc_prev, int32_t* __restrict__ anc_cur, URow* __restrict__ ulist,
-              int32_t* __restrict__ ucount, int* __restrict__ err_word) {
+              int32_t* __restrict__ ucount, int* __restrict__ err_word, int rebuild) {
     // Programmatic dependent launch: the next kernel may start its prologue now; this one
     // touches nothing until the previous kernel of the stream has completed.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -109,7 +109,7 @@ append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __
     __shared__ int s_base;
     if (tid < W) {
         int p = tid;
-        if (step > 0) {
+        if (step > 0 && !rebuild) {
             p = beam_parent[b * W + tid];
             if (p < 0 || p >= W) {
                 atomicOr(err_word, SEGKV_DEV_BAD_PARENT);
@@ -130,10 +130,14 @@ append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __
         if (s < n) {
 #pragma unroll 4
             for (int j = 0; j < W; ++j) {
-                int v = (s == step) ? b * W + j
-                                    : anc_prev[(size_t)(b * W + s_par[j]) * max_steps + s];
+                int v;
+                if (rebuild) {
+                    v = anc_cur[(size_t)(b * W + j) * max_steps + s];    // the table is already this step's
+                } else {
+                    v = (s == step) ? b * W + j : anc_prev[(size_t)(b * W + s_par[j]) * max_steps + s];
+                    anc_cur[(size_t)(b * W + j) * max_steps + s] = v;
+                }
                 r[j] = v;
-                anc_cur[(size_t)(b * W + j) * max_steps + s] = v;
             }
             for (int j = 0; j < W; ++j) {
                 bool first = true;
@@ -203,7 +207,18 @@ cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, c
     const int32_t* bp = step > 0 ? beam_parent : nullptr;
     return cudaLaunchKernelEx(&cfg, append_kernel, d.batch, d.beams, d.rows, d.max_steps, step, bp,
                               (const uint4*)k_new, (const uint4*)v_new, kr_slab, vr_slab, slab_chunks,
-                              parent_tab + (size_t)step * d.rows, anc_prev, anc_cur, ulist, ucount, err_word);
+                              parent_tab + (size_t)step * d.rows, anc_prev, anc_cur, ulist, ucount, err_word, 0);
+}
+
+// The distinct-row lists of the newest step from its beam-index table alone: the table blocks of
+// the append kernel in read-only mode (used after fused decode steps, which skip the lists).
+cudaError_t launch_rebuild_lists(const Dims& d, int steps, const int32_t* anc_cur, URow* ulist, int32_t* ucount,
+                                 cudaStream_t st) {
+    if (steps <= 0) return cudaSuccess;
+    append_kernel<<<(unsigned)d.batch, kBtThreads, 0, st>>>(
+        d.batch, d.beams, d.rows, d.max_steps, steps - 1, nullptr, nullptr, nullptr, nullptr, nullptr, 0, nullptr,
+        nullptr, const_cast<int32_t*>(anc_cur), ulist, ucount, nullptr, 1);
+    return cudaGetLastError();
 }
 
 }  // namespace segkv_impl

@@ -12,10 +12,11 @@ namespace segkv_impl {
 constexpr int kMaxCols = 32;       // beams * (heads/kv_heads) handled by one CTA
 constexpr int kMaxSplits = 64;     // CTAs that may share one (request, kv head) work group
 constexpr int kMaxCluster = 8;     // largest portable thread-block cluster
+constexpr int kMaxTiledBeams = 16;  // beams the tiled kernel handles (16 query columns at most)
 
-// One entry of the per-request list of DISTINCT response rows: `row` indexes the
-// response segment's [step*rows + slot] axis, `mask` has bit j set when beam j of
-// the request reads this row.
+// {row, mask} pairs.  In the per-request list of DISTINCT response rows `row` indexes the
+// response segment's [step*rows + slot] axis; in the per-key record of a response tile in
+// shared memory it is the key's step.  `mask` has bit j set when beam j reads the row.
 struct URow {
     int32_t row;
     uint32_t mask;
@@ -43,6 +44,7 @@ struct segkv {
     int stages_forced;   // 0 = automatic
     int combine_forced;  // 0 = automatic, 1 = global workspace + ticket, 2 = cluster
     bool overlap;        // programmatic dependent launch between consecutive kernels
+    bool fuse_always;    // segkv_decode_step uses the fused kernel even for a single split
     long long launches;
     // device storage (owned)
     void* kp;            // [batch, kv_heads, max_prompt, D]
@@ -51,8 +53,9 @@ struct segkv {
     void* vr;
     int32_t* parent;     // [max_steps, rows]
     int32_t* anc[2];     // [rows, max_steps], generation t lives in anc[t & 1]
-    segkv_impl::URow* ulist;   // [batch, beams*max_steps]
+    segkv_impl::URow* ulist;   // [batch, beams*max_steps] distinct response rows per request
     int32_t* ucount;     // [batch]
+    bool lists_valid;    // ulist/ucount describe the newest step (a fused step does not update them)
     int* err_word;       // device error word
     float* ws;           // split workspace
     size_t ws_bytes;
@@ -77,6 +80,9 @@ cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, c
                           const void* v_new, void* kr, void* vr, int32_t* parent_tab,
                           const int32_t* anc_prev, int32_t* anc_cur, URow* ulist, int32_t* ucount,
                           int* err_word, int sm_count, bool pdl, cudaStream_t st);
+// Re-derive the distinct-row lists from the current beam-index table (after fused steps).
+cudaError_t launch_rebuild_lists(const Dims& d, int steps, const int32_t* anc_cur, URow* ulist, int32_t* ucount,
+                                 cudaStream_t st);
 
 struct SdpaArgs {
     const void* q;
@@ -86,7 +92,7 @@ struct SdpaArgs {
     const void* vp;
     const void* kr;
     const void* vr;
-    const int32_t* anc;      // generation of the newest step
+    const int32_t* anc;      // beam-index table (fused step: the previous step's)
     const URow* ulist;
     const int32_t* ucount;
     float* ws;
@@ -95,6 +101,16 @@ struct SdpaArgs {
     int prompt_len, steps, splits;
     bool cluster;            // merge the splits inside a thread-block cluster
     bool pdl;                // launch with programmatic stream serialisation
+    bool prompt_immutable;   // a fully serialised launch has followed the last prompt store
+    // fused decode step (append + beam-index update + attention in one launch)
+    bool fused;
+    const int32_t* parent;   // [rows] device, NULL at step 0
+    const void* k_new;
+    const void* v_new;
+    void* kr_new_slab;
+    void* vr_new_slab;
+    int32_t* anc_dst;
+    int32_t* parent_row;
 };
 
 // Plain gather kernel: one CTA per (beam slot, head), fp32 ALU; kept for shapes

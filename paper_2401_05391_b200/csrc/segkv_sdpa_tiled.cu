@@ -205,6 +205,17 @@ struct TiledParams {
     float* ws_ml;   // [slab][S][ncols][2]   running max (base-2 domain) and sum
     int* tickets;
     int* err_word;
+    // fused decode step only: the step's inputs and the cache locations they are stored to
+    const int32_t* anc_prev; // beam-index table of the previous step
+    const int32_t* parent;   // [rows] beam parents of the new step (NULL at step 0)
+    const char* k_new;       // [rows, Hkv, D]
+    const char* v_new;
+    char* kr_new_slab;       // slab of the new step inside the response segment
+    char* vr_new_slab;
+    int32_t* anc_dst;        // table of the new step
+    int32_t* parent_row;     // row of the parent table
+    int fused;      // 1: steps-1 is a new step whose rows come from k_new / v_new and whose beam-index
+                    //    column is derived here from `parent` and the previous table
     int P, steps, S, W, G, H, Hkv, rows, max_steps, ncols, stages;
     int quota;      // distinct response rows per split (the last split also takes any excess)
     int cluster;    // 1: the S CTAs of a work group form a thread-block cluster
@@ -237,7 +248,8 @@ struct Layout {
         return (b + 127) & ~(size_t)127;
     }
     static __host__ __device__ constexpr size_t bars(int stages) {
-        return (((size_t)stages * 16 + 8 + 127) & ~(size_t)127) + (size_t)TILE * 8;   // + row offsets of the gather warp
+        // mbarriers, per-stage {count, last} of response tiles, then the gather warp's row pointers
+        return (((size_t)stages * 24 + 8 + 127) & ~(size_t)127) + (size_t)TILE * 16;
     }
     static __host__ __device__ constexpr size_t recv(int nt) {
         return (size_t)8 * nt * D * 4 + (size_t)kMaxCluster * 8 * nt * 2 * 4;
@@ -247,7 +259,7 @@ struct Layout {
     }
 };
 
-template <typename T, int D, int NT, int CW>
+template <typename T, int D, int NT, int CW, bool FUSED>
 __global__ void __launch_bounds__(32 * (CW + 2), NT > 1 ? 1 : 2)
 sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                   const TiledParams p) {
@@ -269,7 +281,9 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     float* recv_o = reinterpret_cast<float*>(smem + L::body(stages, NT) + L::bars(stages));   // [S][slice]
     float* recv_ml = recv_o + 8 * NT * D;                                                     // [S][ncols][2]
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + stages), hand = smem_u32(bars + 2 * stages);
-    size_t* goff = reinterpret_cast<size_t*>(reinterpret_cast<uint8_t*>(recv_o) - (size_t)TILE * 8);   // [TILE], gather warp only
+    int2* tile_hdr = reinterpret_cast<int2*>(bars + 2 * stages + 1);                           // [stages] {count, last}
+    const char** gk = reinterpret_cast<const char**>(reinterpret_cast<uint8_t*>(recv_o) - (size_t)TILE * 16);  // [TILE] K row pointers
+    const char** gv = gk + TILE;                                                               // [TILE] V row pointers
     __shared__ int s_last, s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -286,6 +300,8 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     const int pt0 = (int)((long long)split * ntp / p.S), pt1 = (int)((long long)(split + 1) * ntp / p.S);
     const int npt = pt1 - pt0;
     const URow* ulist_b = p.ulist + (size_t)b * p.W * p.max_steps;
+    // fused step: response steps are cut evenly over the splits (known from the launch shape alone)
+    const int rs0 = (int)((long long)split * p.steps / p.S), rs1 = (int)((long long)(split + 1) * p.steps / p.S);
 
     auto issue_prompt_tile = [&](int k) {
         const int st = k % stages;
@@ -305,7 +321,6 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     };
 
     int tma_issued = 0;       // TMA warp: fills started (for the wind-down after an expired wait)
-    int gather_issued = 0;    // gather warp: one past the last ring slot it filled
     if (warp == TMA_WARP) {
         // The warp that issues the bulk loads sets the barriers up itself and starts the
         // first round of prompt tiles before the rest of the CTA has even synchronised.
@@ -358,111 +373,208 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             s_abort = 1;
         }
     } else if (warp == GATHER_WARP) {
-        // ================== response tiles: gather the request's distinct rows ==================
-        // The chain row count -> row list starts at once, beside the TMA warp; the ring itself
-        // is taken over only when the last prompt tile has been issued (a parity wait cannot
-        // tell a far-future round of a stage from the current one).
-        // A split's range starts at split * quota whatever the row count turns out to be, so
-        // the first tile's list entries are requested together with the count, not after it.
-        uint2 ucur[UK], unext[UK];          // {row, beam mask} of this lane's keys (lane, lane + 32)
-        const int cap = p.W * p.max_steps;
-#pragma unroll
-        for (int kk = 0; kk < UK; ++kk) {
-            const int key = lane + 32 * kk;
-            unext[kk] = (p.steps > 0 && key < TILE)
-                            ? *reinterpret_cast<const uint2*>(ulist_b + min(split * p.quota + key, cap - 1))
-                            : make_uint2(0u, 0u);
-        }
-        const int n_b = p.steps > 0 ? p.ucount[b] : 0;
-        const int e0 = min(split * p.quota, n_b);
-        const int e1 = (split == p.S - 1) ? n_b : min((split + 1) * p.quota, n_b);
-        const int nrt = (e1 - e0 + TILE - 1) / TILE;
-        SEGKV_STAMP(4);
-        SEGKV_CLK(1, true);
-        bool ok = true;
-        if (nrt > 0) {
-            ok = mbar_wait(hand, 0);
-            ok = __all_sync(0xffffffffu, ok);
-        }
-        for (int r = 0; r < nrt && ok; ++r) {
-            const int k = npt + r;
-            const int eb = e0 + r * TILE;
-            const int cnt = min(TILE, e1 - eb);
-#pragma unroll
-            for (int kk = 0; kk < UK; ++kk) {
-                ucur[kk] = unext[kk];
-                const int key = lane + 32 * kk;
-                unext[kk] = (key < TILE && eb + TILE + key < e1)
-                                ? *reinterpret_cast<const uint2*>(ulist_b + eb + TILE + key)
-                                : make_uint2(0u, 0u);
-            }
-            const int st = k % stages;
-            ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+        // ================== response tiles: index select fused into the load ==================
+        // A tile holds up to TILE distinct response rows of the request, each with its step and
+        // the set of beams that read it (rows shared by several beams are fetched once).  The
+        // ring is taken over from the TMA warp only when the last prompt tile has been issued
+        // (a parity wait cannot tell a far-future round of a stage from the current one).
+        constexpr int CPR = D / 8;        // 16-byte chunks per row
+        constexpr int RPI = 32 / CPR;     // rows covered by one warp-wide copy
+        // Publish the tile whose per-key meta and row pointers (gk, gv) have been written:
+        // zero the rows between the last real one and the end of its 16-key slice (rows past
+        // that slice are never looked at), release the plain stores, then copy the rows.
+        auto publish_tile = [&](int st, int cnt, bool last) {
             const uint32_t full = full0 + 8 * st;
             uint8_t* k_tile = ring + (size_t)st * L::STAGE_BYTES;
             uint8_t* v_tile = k_tile + L::TILE_BYTES;
             const uint32_t k_dst = smem_u32(k_tile), v_dst = k_dst + L::TILE_BYTES;
-            URow* meta_st = meta + (size_t)st * TILE;
-            SEGKV_CLK(11, r == 0);
-            // Each lane publishes {row, mask} and the byte offset of its keys (lane, lane + 32);
-            // rows between the last real one and the end of its 16-key slice are zeroed with
-            // plain stores (rows past that slice are never looked at).
-            constexpr int CPR = D / 8;        // 16-byte chunks per row
-            constexpr int RPI = 32 / CPR;     // rows covered by one warp-wide copy
             const int fill = min(TILE, (cnt + 15) & ~15);
+            const int zchunks = (fill - cnt) * 8;      // in every 128-byte box the run is contiguous
 #pragma unroll
-            for (int kk = 0; kk < UK; ++kk) {
-                const int key = lane + 32 * kk;
-                if (key >= TILE) continue;
-                const bool valid = key < cnt;
-                URow u;
-                u.row = valid ? (int32_t)ucur[kk].x : 0;
-                u.mask = valid ? ucur[kk].y : 0u;
-                meta_st[key] = u;
-                goff[key] = ((size_t)u.row * p.Hkv + kvh) * (size_t)(D * 2);
-            }
-            // zero the rows between the last real one and the end of its 16-key slice: in every
-            // 128-byte box they are one contiguous run, filled 16 bytes per lane
-            {
-                const int zchunks = (fill - cnt) * 8;
-#pragma unroll
-                for (int bx = 0; bx < D / 64; ++bx) {
-                    uint4* kz = reinterpret_cast<uint4*>(k_tile + (size_t)bx * L::BOX_BYTES + (size_t)cnt * 128);
-                    uint4* vz = reinterpret_cast<uint4*>(v_tile + (size_t)bx * L::BOX_BYTES + (size_t)cnt * 128);
-                    for (int i = lane; i < zchunks; i += 32) {
-                        kz[i] = make_uint4(0u, 0u, 0u, 0u);
-                        vz[i] = make_uint4(0u, 0u, 0u, 0u);
-                    }
+            for (int bx = 0; bx < D / 64; ++bx) {
+                uint4* kz = reinterpret_cast<uint4*>(k_tile + (size_t)bx * L::BOX_BYTES + (size_t)cnt * 128);
+                uint4* vz = reinterpret_cast<uint4*>(v_tile + (size_t)bx * L::BOX_BYTES + (size_t)cnt * 128);
+                for (int i = lane; i < zchunks; i += 32) {
+                    kz[i] = make_uint4(0u, 0u, 0u, 0u);
+                    vz[i] = make_uint4(0u, 0u, 0u, 0u);
                 }
             }
-            SEGKV_CLK(14, r == 0);
+            if (lane == 0) tile_hdr[st] = make_int2(cnt, last ? 1 : 0);
             __syncwarp();
             if (lane == 0) mbar_arrive(full);          // releases the plain stores of the whole warp
-            SEGKV_CLK(6, r == 0);
-            // One warp-wide copy moves whole rows (CPR lanes per row): fully coalesced.
+            // one warp-wide copy moves whole rows (CPR lanes per row): fully coalesced
             const int c = lane % CPR;
             const uint32_t c_off = (uint32_t)(c / 8) * L::BOX_BYTES;
 #pragma unroll
             for (int i = 0; i < TILE / RPI; ++i) {
-                if (i * RPI < cnt) {                       // warp-uniform
+                if (i * RPI < cnt) {                   // warp-uniform
                     const int key = i * RPI + lane / CPR;
                     if (key < cnt) {
-                        const size_t src = goff[key] + (size_t)c * 16;
                         const uint32_t off = c_off + (uint32_t)key * 128 + (uint32_t)(((c & 7) ^ (key & 7)) << 4);
-                        cp_async_16(k_dst + off, p.kr + src);
-                        cp_async_16(v_dst + off, p.vr + src);
+                        if constexpr (FUSED) {             // rows may sit in the caller's k_new / v_new
+                            cp_async_16(k_dst + off, gk[key] + c * 16);
+                            cp_async_16(v_dst + off, gv[key] + c * 16);
+                        } else {                           // one offset serves both segments
+                            const size_t src = reinterpret_cast<size_t>(gk[key]) + (size_t)c * 16;
+                            cp_async_16(k_dst + off, p.kr + src);
+                            cp_async_16(v_dst + off, p.vr + src);
+                        }
                     }
                 }
             }
-            SEGKV_CLK(7, r == 0);
             cp_async_mbar_arrive_noinc(full);
-            __syncwarp();                                  // goff is rewritten for the next tile
-            gather_issued = k + 1;
-            SEGKV_CLK(15, r == 0);
+            __syncwarp();                              // gk / gv are rewritten for the next tile
+        };
+        bool ok = true;
+        if constexpr (!FUSED) {
+            // ---- rows from the request's list of distinct rows (made by the append kernel) ----
+            // A split's range starts at split * quota whatever the row count turns out to be, so
+            // the first tile's list entries are requested together with the count, not after it.
+            uint2 ucur[UK], unext[UK];          // {row, beam mask} of this lane's keys (lane, lane + 32)
+            const int cap = p.W * p.max_steps;
+#pragma unroll
+            for (int kk = 0; kk < UK; ++kk) {
+                const int key = lane + 32 * kk;
+                unext[kk] = (p.steps > 0 && key < TILE)
+                                ? *reinterpret_cast<const uint2*>(ulist_b + min(split * p.quota + key, cap - 1))
+                                : make_uint2(0u, 0u);
+            }
+            const int n_b = p.steps > 0 ? p.ucount[b] : 0;
+            const int e0 = min(split * p.quota, n_b);
+            const int e1 = (split == p.S - 1) ? n_b : min((split + 1) * p.quota, n_b);
+            const int nrt = (e1 - e0 + TILE - 1) / TILE;
+            SEGKV_STAMP(4);
+            if (nrt > 0) {
+                ok = mbar_wait(hand, 0);
+                ok = __all_sync(0xffffffffu, ok);
+            }
+            for (int r = 0; r < nrt && ok; ++r) {
+                const int k = npt + r;
+                const int eb = e0 + r * TILE;
+                const int cnt = min(TILE, e1 - eb);
+#pragma unroll
+                for (int kk = 0; kk < UK; ++kk) {
+                    ucur[kk] = unext[kk];
+                    const int key = lane + 32 * kk;
+                    unext[kk] = (key < TILE && eb + TILE + key < e1)
+                                    ? *reinterpret_cast<const uint2*>(ulist_b + eb + TILE + key)
+                                    : make_uint2(0u, 0u);
+                }
+                const int st = k % stages;
+                ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                URow* meta_st = meta + (size_t)st * TILE;
+#pragma unroll
+                for (int kk = 0; kk < UK; ++kk) {
+                    const int key = lane + 32 * kk;
+                    if (key >= TILE) continue;
+                    const bool valid = key < cnt;
+                    const int row = valid ? (int)ucur[kk].x : 0;         // step * rows + slot
+                    URow u;
+                    u.row = row / p.rows;                                // consumers need the step only
+                    u.mask = valid ? ucur[kk].y : 0u;
+                    meta_st[key] = u;
+                    gk[key] = reinterpret_cast<const char*>(((size_t)row * p.Hkv + kvh) * (size_t)(D * 2));  // byte offset
+                }
+                publish_tile(st, cnt, r == nrt - 1);
+            }
+            SEGKV_STAMP(5);
+        } else {
+            // ---- fused decode step: rows from the beam-index table, derived on the fly ----
+            // The new step's column of the table (Section 3.3) is anc_t[j][s] = anc_{t-1}[parent[j]][s]
+            // for s < t and anc_t[j][t] = j.  One lane takes one (step, beam) pair; the lanes of a step
+            // compare rows to keep each distinct row once with its beam mask, a warp prefix sum packs
+            // the steps of a window densely into the tile, and the column is stored for later steps.
+            const int Wb = p.W;
+            int Wp = 1;
+            while (Wp < Wb) Wp <<= 1;                     // lanes per step (a power of two, <= 16)
+            const int spw = 32 / Wp;                      // steps per window
+            const int ls = lane / Wp, j = lane % Wp;
+            const int gbase = lane - j;                   // first lane of this lane's step
+            const int t_new = p.steps - 1;                // the step whose rows are still in k_new / v_new
+            int par = j;
+            if (p.steps > 1 && j < Wb) {
+                par = p.parent[b * Wb + j];
+                if (par < 0 || par >= Wb) {
+                    if (kvh == 0 && split == 0) atomicOr(p.err_word, SEGKV_DEV_BAD_PARENT);
+                    par = par < 0 ? 0 : Wb - 1;
+                }
+            }
+            const size_t slab_bytes = (size_t)p.rows * p.Hkv * (size_t)(D * 2);
+            SEGKV_STAMP(4);
+            if (rs1 > rs0) {
+                ok = mbar_wait(hand, 0);
+                ok = __all_sync(0xffffffffu, ok);
+            }
+            int sbeg = rs0, fillpos = 0, k = npt, st = 0;
+            bool open = false;
+            while (ok && sbeg < rs1) {
+                const int s = sbeg + ls;
+                const int nact = min(spw, rs1 - sbeg);        // steps in this window
+                const bool active = ls < nact && j < Wb;
+                int row = -1 - lane;                          // inactive lanes match nobody
+                if (active) row = (s == t_new) ? b * Wb + j : p.anc_prev[(size_t)(b * Wb + par) * p.max_steps + s];
+                bool first = active;
+                uint32_t mask = 0;
+                for (int i = 0; i < Wp; ++i) {
+                    const int ri = __shfl_sync(0xffffffffu, row, gbase + i);
+                    if (ri == row) {
+                        mask |= 1u << i;
+                        if (i < j) first = false;
+                    }
+                }
+                int incl = first ? 1 : 0;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += n;
+                }
+                // whole steps only: a step fits if its last lane's running count still fits
+                const int step_end = __shfl_sync(0xffffffffu, incl, gbase + Wp - 1);
+                const uint32_t fitmask = __ballot_sync(0xffffffffu, ls < nact && j == 0 && fillpos + step_end <= TILE);
+                const int nfit = __popc(fitmask);             // leading steps (the count is monotone)
+                if (!open) {
+                    st = k % stages;
+                    ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    open = true;
+                }
+                if (ls < nfit && active) {
+                    if (first) {
+                        const int pos = fillpos + incl - 1;
+                        URow u;
+                        u.row = s;
+                        u.mask = mask;
+                        meta[(size_t)st * TILE + pos] = u;
+                        const size_t off = ((size_t)row * p.Hkv + kvh) * (size_t)(D * 2);
+                        gk[pos] = (s == t_new ? p.k_new : p.kr + (size_t)s * slab_bytes) + off;
+                        gv[pos] = (s == t_new ? p.v_new : p.vr + (size_t)s * slab_bytes) + off;
+                    }
+                    if (kvh == 0) p.anc_dst[(size_t)(b * Wb + j) * p.max_steps + s] = row;
+                }
+                if (nfit > 0) fillpos += __shfl_sync(0xffffffffu, incl, nfit * Wp - 1);
+                sbeg += nfit;
+                if (nfit < nact || fillpos + Wb > TILE || sbeg >= rs1) {
+                    publish_tile(st, fillpos, sbeg >= rs1);
+                    ++k;
+                    open = false;
+                    fillpos = 0;
+                }
+            }
+            SEGKV_STAMP(5);
+            // store what the step appends: the parent ids and the new K/V rows of this work group
+            if (kvh == 0 && split == 0 && lane < Wb)
+                p.parent_row[b * Wb + lane] = p.steps > 1 ? p.parent[b * Wb + lane] : lane;
+            if (split == p.S - 1) {
+                for (int i = lane; i < Wb * CPR; i += 32) {
+                    const size_t off = ((size_t)(b * Wb + i / CPR) * p.Hkv + kvh) * (size_t)(D * 2) + (size_t)(i % CPR) * 16;
+                    *reinterpret_cast<uint4*>(p.kr_new_slab + off) = *reinterpret_cast<const uint4*>(p.k_new + off);
+                    *reinterpret_cast<uint4*>(p.vr_new_slab + off) = *reinterpret_cast<const uint4*>(p.v_new + off);
+                }
+            }
         }
-        SEGKV_STAMP(5);
         if (!ok && lane == 0) {
             atomicOr(p.err_word, SEGKV_DEV_WAIT_LIMIT);
             s_abort = 1;
@@ -478,7 +590,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 #pragma unroll
                 for (int i = 0; i < 4; ++i) o_acc[nt][mt][i] = 0.f;
         }
-        const int n_b = p.steps > 0 ? p.ucount[b] : 0;   // in flight while the prompt tiles are consumed
+        const int n_b = (p.steps > 0 && !FUSED) ? p.ucount[b] : 0;   // in flight while the prompt tiles are consumed
         // Q^T as the B operand: this lane holds column n = lane/4 of every column tile
         uint32_t qf[NT][KS][2];
 #pragma unroll
@@ -542,9 +654,9 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             for (int r = 0; r < 2; ++r) {
                 const int key = key_lo + 8 * r;
                 if (resp) {
-                    const URow u = meta[(size_t)st * TILE + key];
+                    const URow u = meta[(size_t)st * TILE + key];       // {step, beams that read the row}
                     kmask[r] = key < nvalid ? u.mask : 0u;
-                    kpos[r] = (float)(p.P + u.row / p.rows - qpos);
+                    kpos[r] = (float)(p.P + u.row - qpos);
                 } else {
                     kmask[r] = key < nvalid ? 0xffffffffu : 0u;
                     kpos[r] = (float)(pos0 + key - qpos);
@@ -623,7 +735,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             if (lane == 0) mbar_arrive(empty0 + 8 * st);
         }
         if (warp == 0) SEGKV_STAMP(8);
-        if (ok) {
+        if (ok && !FUSED) {
             const int e0 = min(split * p.quota, n_b);
             const int e1 = (split == p.S - 1) ? n_b : min((split + 1) * p.quota, n_b);
             const int nrt = (e1 - e0 + TILE - 1) / TILE;
@@ -635,6 +747,21 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 consume(st, true, min(TILE, e1 - (e0 + r * TILE)), 0);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8 * st);
+            }
+        } else if (ok && rs1 > rs0) {
+            // fused step: how many response tiles there are and how full each is only the gather
+            // warp knows; it says so in the tile's header
+            for (;;) {
+                const int st = k % stages;
+                ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const int2 hd = tile_hdr[st];
+                consume(st, true, hd.x, 0);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8 * st);
+                ++k;
+                if (hd.y) break;
             }
         }
         if (!ok && lane == 0) {
@@ -833,12 +960,12 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     if (tid == 0) SEGKV_STAMP(13);
 }
 
-template <typename T, int D, int NT, int CW>
+template <typename T, int D, int NT, int CW, bool FUSED>
 cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk, const CUtensorMap& tmv, int stages,
                        cudaStream_t st) {
     using L = Layout<D, CW>;
     const size_t smem = L::bytes(stages, NT);
-    auto kern = sdpa_tiled_kernel<T, D, NT, CW>;
+    auto kern = sdpa_tiled_kernel<T, D, NT, CW, FUSED>;
     static size_t configured[64] = {0};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -851,13 +978,17 @@ cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk,
     p.q = a.q; p.out = a.out; p.slopes = a.slopes;
     p.kr = (const char*)a.kr; p.vr = (const char*)a.vr;
     p.ulist = a.ulist; p.ucount = a.ucount; p.tickets = a.tickets; p.err_word = a.err_word;
+    p.fused = a.fused ? 1 : 0;
+    p.anc_prev = a.anc; p.parent = a.parent; p.k_new = (const char*)a.k_new; p.v_new = (const char*)a.v_new;
+    p.kr_new_slab = (char*)a.kr_new_slab; p.vr_new_slab = (char*)a.vr_new_slab;
+    p.anc_dst = a.anc_dst; p.parent_row = a.parent_row;
     p.P = a.prompt_len; p.steps = a.steps; p.S = a.splits; p.W = d.beams; p.G = d.group; p.H = d.heads;
     p.Hkv = d.kv_heads; p.rows = d.rows; p.max_steps = d.max_steps; p.ncols = d.beams * d.group; p.stages = stages;
     p.scale2 = 1.4426950408889634f / sqrtf((float)D);
     p.quota = (a.steps + 2 * d.beams + a.splits - 1) / a.splits;
     if (p.quota < 1) p.quota = 1;
     p.cluster = a.cluster ? 1 : 0;
-    p.early_prompt = (a.pdl && a.steps > 0) ? 1 : 0;
+    p.early_prompt = (a.pdl && a.prompt_immutable) ? 1 : 0;
 #ifdef SEGKV_TIMELINE
     static int launch_id = 0;
     p.dbg_launch = launch_id++;
@@ -898,14 +1029,19 @@ cudaError_t dispatch(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk, c
     if (a.cluster && !tiled_cluster_ok(d, a.splits)) return cudaErrorInvalidValue;
     if (nt == 1) {
         switch (d.head_dim) {
-            case 64: return launch_one<T, 64, 1, 4>(d, a, tmk, tmv, stages, st);
-            case 128: return launch_one<T, 128, 1, 4>(d, a, tmk, tmv, stages, st);
-            case 256: return launch_one<T, 256, 1, 2>(d, a, tmk, tmv, stages, st);
+            case 64: return a.fused ? launch_one<T, 64, 1, 4, true>(d, a, tmk, tmv, stages, st)
+                                    : launch_one<T, 64, 1, 4, false>(d, a, tmk, tmv, stages, st);
+            case 128: return a.fused ? launch_one<T, 128, 1, 4, true>(d, a, tmk, tmv, stages, st)
+                                    : launch_one<T, 128, 1, 4, false>(d, a, tmk, tmv, stages, st);
+            case 256: return a.fused ? launch_one<T, 256, 1, 2, true>(d, a, tmk, tmv, stages, st)
+                                    : launch_one<T, 256, 1, 2, false>(d, a, tmk, tmv, stages, st);
         }
     } else if (nt == 2) {
         switch (d.head_dim) {
-            case 64: return launch_one<T, 64, 2, 4>(d, a, tmk, tmv, stages, st);
-            case 128: return launch_one<T, 128, 2, 4>(d, a, tmk, tmv, stages, st);
+            case 64: return a.fused ? launch_one<T, 64, 2, 4, true>(d, a, tmk, tmv, stages, st)
+                                    : launch_one<T, 64, 2, 4, false>(d, a, tmk, tmv, stages, st);
+            case 128: return a.fused ? launch_one<T, 128, 2, 4, true>(d, a, tmk, tmv, stages, st)
+                                    : launch_one<T, 128, 2, 4, false>(d, a, tmk, tmv, stages, st);
         }
     }
     return cudaErrorInvalidValue;

@@ -31,6 +31,7 @@ SIGNATURES = {
     "segkv_prefill_write": (_int, [_vp, _vp, _vp, _int, _vp]),
     "segkv_append": (_int, [_vp, _int, _vp, _vp, _vp, _vp]),
     "segkv_decode_sdpa": (_int, [_vp, _vp, _vp, _vp, _vp]),
+    "segkv_decode_step": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "segkv_decode_sdpa_static": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "segkv_step_host": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "segkv_reset": (_int, [_vp, _int]),
@@ -170,6 +171,20 @@ class SegKV:
         _check(lib().segkv_decode_sdpa(self._h, _dev(q, shape, self.dtype, "q"), _dev(out, shape, self.dtype, "out"),
                                        _dev(alibi_slopes, (self.heads,), torch.float32, "alibi_slopes"),
                                        _stream_ptr(stream)), "segkv_decode_sdpa")
+        return out
+
+    def decode_step(self, step: int, beam_parent: Optional[torch.Tensor], k_new: torch.Tensor, v_new: torch.Tensor,
+                    q: torch.Tensor, out: Optional[torch.Tensor] = None,
+                    alibi_slopes: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        kv = (self.rows, self.kv_heads, self.head_dim)
+        qs = (self.rows, self.heads, self.head_dim)
+        if out is None:
+            out = torch.empty(qs, dtype=self.dtype, device=q.device)
+        _check(lib().segkv_decode_step(self._h, step, _dev(beam_parent, (self.rows,), torch.int32, "beam_parent"),
+                                       _dev(k_new, kv, self.dtype, "k_new"), _dev(v_new, kv, self.dtype, "v_new"),
+                                       _dev(q, qs, self.dtype, "q"), _dev(out, qs, self.dtype, "out"),
+                                       _dev(alibi_slopes, (self.heads,), torch.float32, "alibi_slopes"),
+                                       _stream_ptr(stream)), "segkv_decode_step")
         return out
 
     def decode_sdpa_static(self, q: torch.Tensor, out: torch.Tensor,

@@ -40,6 +40,17 @@ class Run:
         self.k_steps.append(k); self.v_steps.append(v); self.q_steps.append(q)
         return t
 
+    def step_fused(self):
+        """Append the next step and attend in one fused launch; returns (t, out, q)."""
+        t = self.h.steps
+        q, k, v = wl.make_step(self.w, t, self.device)
+        out = torch.full((self.w.rows, self.w.heads, self.w.head_dim), float("nan"),
+                         dtype=self.w.torch_dtype, device=self.device)
+        self.h.decode_step(t, self.parents_dev[t] if t > 0 else None, k, v, q, out, self.slopes)
+        torch.cuda.synchronize()
+        self.k_steps.append(k); self.v_steps.append(v); self.q_steps.append(q)
+        return t, out, q
+
     def advance_to(self, t: int):
         while self.h.steps <= t:
             self.append_next()

@@ -33,6 +33,86 @@ def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combi
         r.close()
 
 
+def run_workload_fused(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combine=0):
+    """Same as run_workload but every step is one fused segkv_decode_step launch."""
+    r = Run(w, splits=splits, stages=stages, combine=combine)
+    try:
+        for t in range(w.steps):
+            _, out, q = r.step_fused()
+            if t in check_steps or t == w.steps - 1:
+                ref = r.oracle_ancestry(t)
+                assert np.array_equal(r.h.get_ancestry(), ref), f"beam-index table differs at step {t}"
+                assert np.array_equal(r.h.get_unique_rows(), unique_rows_from_ancestry(ref, w.batch, w.beams))
+                r.check(out, q, t, pairs_fn(w))
+        assert r.h.get_error() == 0
+    finally:
+        r.close()
+
+
+def test_fused_step_tiny_every_step():
+    w = wl.CONFIGS[0]
+    run_workload_fused(w, all_pairs, check_steps=tuple(range(w.steps)))
+
+
+def test_fused_step_llama2_7b_shape():
+    run_workload_fused(wl.CONFIGS[1], all_pairs)
+
+
+@pytest.mark.parametrize("idx", [2, 3, 4])
+def test_fused_step_large_shapes_sampled(idx):
+    run_workload_fused(wl.CONFIGS[idx], lambda w: sampled_pairs(w, 24), check_steps=(0, 1, 17, 127, 255))
+
+
+@pytest.mark.parametrize("dtype,D,splits,combine", [("f16", 64, 4, 1), ("bf16", 128, 4, 2), ("f16", 256, 4, 1),
+                                                    ("f16", 128, 1, 0), ("bf16", 64, 7, 0)])
+def test_fused_step_ragged_shapes(dtype, D, splits, combine):
+    # a forced single split still runs the fused kernel (several response tiles per CTA)
+    w = wl.Workload("ragged-fused", 3, 3, 6, 2, D, 150, 40, dtype, "uniform", dtype == "bf16", 60 + D // 64)
+    run_workload_fused(w, all_pairs, check_steps=(0, 1, 5, 20, 39), splits=splits, combine=combine)
+
+
+def test_fused_step_long_response_single_split():
+    # 200 steps x 4 beams through one CTA per work group: windows, tile spill-over, ring reuse
+    w = wl.Workload("long-fused", 2, 4, 2, 2, 128, 100, 200, "f16", "half_identity", False, 66)
+    run_workload_fused(w, all_pairs, check_steps=(0, 15, 16, 17, 63, 64, 65, 130, 199), splits=1)
+
+
+def test_fused_and_separate_calls_mix():
+    """A fused step leaves the cache, parents and table exactly as append would: later separate
+    calls (and the other way round) continue from it."""
+    w = wl.CONFIGS[0].scaled(steps=12, prompt_len=70, index=61)
+    r = Run(w)
+    try:
+        for t in range(w.steps):
+            if t % 3 == 0:
+                r.append_next()
+                out, q = r.decode()
+            else:
+                _, out, q = r.step_fused()
+                again, _ = r.decode(q)                     # the separate kernel on the state the fused step left
+                # same result up to the order in which keys are summed (the two forms cut the
+                # response rows into tiles differently)
+                assert torch.allclose(out.float(), again.float(), atol=2e-3, rtol=1e-2)
+            assert np.array_equal(r.h.get_ancestry(), r.oracle_ancestry(t))
+            r.check(out, q, t, all_pairs(w))
+        # re-time a fused step: drop it, run it again, same bits
+        r.h.truncate_last()
+        t = w.steps - 1
+        out2 = r.h.decode_step(t, r.parents_dev[t], r.k_steps[t], r.v_steps[t], q, None, r.slopes)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
+    finally:
+        r.close()
+
+
+def test_fused_step_wide_beam_and_single_beam():
+    run_workload_fused(wl.Workload("w1f", 2, 1, 4, 4, 128, 77, 9, "f16", "uniform", False, 62), all_pairs)
+    run_workload_fused(wl.Workload("w8f", 2, 8, 2, 2, 64, 77, 40, "f16", "uniform", False, 63), all_pairs,
+                       check_steps=(0, 3, 39))
+    run_workload_fused(wl.Workload("w16f", 1, 16, 2, 2, 64, 40, 24, "f16", "uniform", False, 64), all_pairs,
+                       check_steps=(0, 3, 23))
+
+
 def test_tiny_every_step_all_outputs():
     w = wl.CONFIGS[0]
     run_workload(w, all_pairs, check_steps=tuple(range(w.steps)))
