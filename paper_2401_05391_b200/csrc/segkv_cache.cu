@@ -82,10 +82,11 @@ append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __
               uint4* __restrict__ vr_slab, long long slab_chunks, int32_t* __restrict__ parent_row,
               const int32_t* __restrict__ anc_prev, int32_t* __restrict__ anc_cur, URow* __restrict__ ulist,
               int32_t* __restrict__ ucount, int* __restrict__ err_word, int rebuild) {
-    // Programmatic dependent launch: the next kernel may start its prologue now; this one
-    // touches nothing until the previous kernel of the stream has completed.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Programmatic dependent launch: this kernel touches nothing until the previous kernel of
+    // the stream has completed, and only then lets the next one start its prologue (so a kernel
+    // that starts early always finds everything older than its predecessor complete).
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if ((int)blockIdx.x >= B) {
         // ---- copy blocks -------------------------------------------------
         const long long nb = gridDim.x - B;

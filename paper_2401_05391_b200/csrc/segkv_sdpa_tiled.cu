@@ -288,7 +288,6 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) { SEGKV_STAMP(0); SEGKV_STAMP(1); }
-    grid_launch_dependents();
     const int split = blockIdx.x % p.S;
     const int slab = blockIdx.x / p.S;           // b * Hkv + kvh
     const int b = slab / p.Hkv, kvh = slab % p.Hkv;
@@ -350,7 +349,11 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     }
     if (p.cluster) cluster_arrive_relaxed();     // "this CTA has started" (waited for before any remote store)
     __syncthreads();
-    grid_wait();      // everything else (q, row lists, response rows, outputs) follows the previous kernel
+    // Everything else (q, row lists, parents, response rows, outputs) follows the previous kernel.
+    // The next kernel is let go only after this wait, so a kernel that starts early behind this
+    // one finds every kernel before this one's predecessor complete.
+    grid_wait();
+    grid_launch_dependents();
     if (tid == 0) SEGKV_STAMP(2);
 
     // consumer state (declared here so that the epilogue sees it)
@@ -380,31 +383,15 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         // (a parity wait cannot tell a far-future round of a stage from the current one).
         constexpr int CPR = D / 8;        // 16-byte chunks per row
         constexpr int RPI = 32 / CPR;     // rows covered by one warp-wide copy
-        // Publish the tile whose per-key meta and row pointers (gk, gv) have been written:
-        // zero the rows between the last real one and the end of its 16-key slice (rows past
-        // that slice are never looked at), release the plain stores, then copy the rows.
-        auto publish_tile = [&](int st, int cnt, bool last) {
+        // Copy rows [0, cnt) of the tile whose row pointers (gk, gv) have been written.  One
+        // warp-wide copy moves whole rows (CPR lanes per row): fully coalesced.  The arrival on
+        // the stage's full barrier fires when this lane's copies have landed.
+        auto copy_rows = [&](int st, int cnt) {
             const uint32_t full = full0 + 8 * st;
-            uint8_t* k_tile = ring + (size_t)st * L::STAGE_BYTES;
-            uint8_t* v_tile = k_tile + L::TILE_BYTES;
-            const uint32_t k_dst = smem_u32(k_tile), v_dst = k_dst + L::TILE_BYTES;
-            const int fill = min(TILE, (cnt + 15) & ~15);
-            const int zchunks = (fill - cnt) * 8;      // in every 128-byte box the run is contiguous
-#pragma unroll
-            for (int bx = 0; bx < D / 64; ++bx) {
-                uint4* kz = reinterpret_cast<uint4*>(k_tile + (size_t)bx * L::BOX_BYTES + (size_t)cnt * 128);
-                uint4* vz = reinterpret_cast<uint4*>(v_tile + (size_t)bx * L::BOX_BYTES + (size_t)cnt * 128);
-                for (int i = lane; i < zchunks; i += 32) {
-                    kz[i] = make_uint4(0u, 0u, 0u, 0u);
-                    vz[i] = make_uint4(0u, 0u, 0u, 0u);
-                }
-            }
-            if (lane == 0) tile_hdr[st] = make_int2(cnt, last ? 1 : 0);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(full);          // releases the plain stores of the whole warp
-            // one warp-wide copy moves whole rows (CPR lanes per row): fully coalesced
+            const uint32_t k_dst = smem_u32(ring + (size_t)st * L::STAGE_BYTES), v_dst = k_dst + L::TILE_BYTES;
             const int c = lane % CPR;
             const uint32_t c_off = (uint32_t)(c / 8) * L::BOX_BYTES;
+            __syncwarp();                              // gk / gv written by other lanes
 #pragma unroll
             for (int i = 0; i < TILE / RPI; ++i) {
                 if (i * RPI < cnt) {                   // warp-uniform
@@ -424,6 +411,31 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             }
             cp_async_mbar_arrive_noinc(full);
             __syncwarp();                              // gk / gv are rewritten for the next tile
+        };
+        // Complete a tile of cnt keys whose per-key meta has been written: zero the rows between
+        // the last real one and the end of its 16-key slice (rows past that slice are never
+        // looked at), say how full the tile is, and release the plain stores of the whole warp.
+        auto finish_tile = [&](int st, int cnt, bool last) {
+            uint8_t* k_tile = ring + (size_t)st * L::STAGE_BYTES;
+            uint8_t* v_tile = k_tile + L::TILE_BYTES;
+            const int fill = min(TILE, (cnt + 15) & ~15);
+            const int zchunks = (fill - cnt) * 8;      // in every 128-byte box the run is contiguous
+#pragma unroll
+            for (int bx = 0; bx < D / 64; ++bx) {
+                uint4* kz = reinterpret_cast<uint4*>(k_tile + (size_t)bx * L::BOX_BYTES + (size_t)cnt * 128);
+                uint4* vz = reinterpret_cast<uint4*>(v_tile + (size_t)bx * L::BOX_BYTES + (size_t)cnt * 128);
+                for (int i = lane; i < zchunks; i += 32) {
+                    kz[i] = make_uint4(0u, 0u, 0u, 0u);
+                    vz[i] = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+            if (lane == 0) tile_hdr[st] = make_int2(cnt, last ? 1 : 0);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full0 + 8 * st);
+        };
+        auto publish_tile = [&](int st, int cnt, bool last) {
+            copy_rows(st, cnt);
+            finish_tile(st, cnt, last);
         };
         bool ok = true;
         if constexpr (!FUSED) {
@@ -493,76 +505,95 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             const int ls = lane / Wp, j = lane % Wp;
             const int gbase = lane - j;                   // first lane of this lane's step
             const int t_new = p.steps - 1;                // the step whose rows are still in k_new / v_new
-            int par = j;
-            if (p.steps > 1 && j < Wb) {
-                par = p.parent[b * Wb + j];
-                if (par < 0 || par >= Wb) {
-                    if (kvh == 0 && split == 0) atomicOr(p.err_word, SEGKV_DEV_BAD_PARENT);
-                    par = par < 0 ? 0 : Wb - 1;
+            constexpr int PF = 4;                         // windows whose table entries are fetched at once
+            // Every lane fetches the previous table's entry of its OWN slot j; the entry of its
+            // parent slot is then one shuffle away, so the table read does not wait for the parent
+            // ids: both requests are in flight together.
+            auto fetch_windows = [&](int w0, int (&rowb)[PF]) {
+#pragma unroll
+                for (int u = 0; u < PF; ++u) {
+                    const int s = rs0 + (w0 + u) * spw + ls;
+                    rowb[u] = 0;
+                    if (s < rs1 && j < Wb && s != t_new) rowb[u] = p.anc_prev[(size_t)(b * Wb + j) * p.max_steps + s];
                 }
-            }
+            };
             const size_t slab_bytes = (size_t)p.rows * p.Hkv * (size_t)(D * 2);
+            int rowb[PF];
+            int par = j;
+            par = (p.steps > 1 && j < Wb) ? p.parent[b * Wb + j] : j;
+            fetch_windows(0, rowb);
+            if (j < Wb && (par < 0 || par >= Wb)) {       // first use of the parent ids
+                if (kvh == 0 && split == 0) atomicOr(p.err_word, SEGKV_DEV_BAD_PARENT);
+                par = par < 0 ? 0 : Wb - 1;
+            }
             SEGKV_STAMP(4);
             if (rs1 > rs0) {
                 ok = mbar_wait(hand, 0);
                 ok = __all_sync(0xffffffffu, ok);
             }
-            int sbeg = rs0, fillpos = 0, k = npt, st = 0;
+            // Windows of spw steps at fixed positions; the table entries of four windows are
+            // requested at once, so a split of up to 4 * spw steps pays one memory round trip.
+            // A window (at most 32 rows) is never cut: if it does not fit, the tile is published
+            // first and the window opens the next one.
+            const int nwin = (rs1 - rs0 + spw - 1) / spw;
+            int fillpos = 0, k = npt, st = 0;
             bool open = false;
-            while (ok && sbeg < rs1) {
-                const int s = sbeg + ls;
-                const int nact = min(spw, rs1 - sbeg);        // steps in this window
-                const bool active = ls < nact && j < Wb;
-                int row = -1 - lane;                          // inactive lanes match nobody
-                if (active) row = (s == t_new) ? b * Wb + j : p.anc_prev[(size_t)(b * Wb + par) * p.max_steps + s];
-                bool first = active;
-                uint32_t mask = 0;
-                for (int i = 0; i < Wp; ++i) {
-                    const int ri = __shfl_sync(0xffffffffu, row, gbase + i);
-                    if (ri == row) {
-                        mask |= 1u << i;
-                        if (i < j) first = false;
-                    }
-                }
-                int incl = first ? 1 : 0;
+            for (int w0 = 0; w0 < nwin && ok; w0 += PF) {
+                if (w0 > 0) fetch_windows(w0, rowb);
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int n = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += n;
-                }
-                // whole steps only: a step fits if its last lane's running count still fits
-                const int step_end = __shfl_sync(0xffffffffu, incl, gbase + Wp - 1);
-                const uint32_t fitmask = __ballot_sync(0xffffffffu, ls < nact && j == 0 && fillpos + step_end <= TILE);
-                const int nfit = __popc(fitmask);             // leading steps (the count is monotone)
-                if (!open) {
-                    st = k % stages;
-                    ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    open = true;
-                }
-                if (ls < nfit && active) {
-                    if (first) {
-                        const int pos = fillpos + incl - 1;
-                        URow u;
-                        u.row = s;
-                        u.mask = mask;
-                        meta[(size_t)st * TILE + pos] = u;
-                        const size_t off = ((size_t)row * p.Hkv + kvh) * (size_t)(D * 2);
-                        gk[pos] = (s == t_new ? p.k_new : p.kr + (size_t)s * slab_bytes) + off;
-                        gv[pos] = (s == t_new ? p.v_new : p.vr + (size_t)s * slab_bytes) + off;
+                for (int u = 0; u < PF; ++u) {
+                    if (w0 + u >= nwin || !ok) break;             // warp-uniform
+                    const int s = rs0 + (w0 + u) * spw + ls;
+                    const bool active = s < rs1 && j < Wb;
+                    int row = __shfl_sync(0xffffffffu, rowb[u], gbase + par);     // anc_{t-1}[parent[j]][s]
+                    if (s == t_new) row = b * Wb + j;
+                    if (!active) row = -1 - lane;                                 // matches nobody
+                    bool first = active;
+                    uint32_t mask = 0;
+                    for (int i = 0; i < Wp; ++i) {
+                        const int ri = __shfl_sync(0xffffffffu, row, gbase + i);
+                        if (ri == row) {
+                            mask |= 1u << i;
+                            if (i < j) first = false;
+                        }
                     }
-                    if (kvh == 0) p.anc_dst[(size_t)(b * Wb + j) * p.max_steps + s] = row;
-                }
-                if (nfit > 0) fillpos += __shfl_sync(0xffffffffu, incl, nfit * Wp - 1);
-                sbeg += nfit;
-                if (nfit < nact || fillpos + Wb > TILE || sbeg >= rs1) {
-                    publish_tile(st, fillpos, sbeg >= rs1);
-                    ++k;
-                    open = false;
-                    fillpos = 0;
+                    int incl = first ? 1 : 0;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const int n = __shfl_up_sync(0xffffffffu, incl, o);
+                        if (lane >= o) incl += n;
+                    }
+                    const int total = __shfl_sync(0xffffffffu, incl, 31);
+                    if (open && fillpos + total > TILE) {
+                        publish_tile(st, fillpos, false);
+                        ++k;
+                        open = false;
+                        fillpos = 0;
+                    }
+                    if (!open) {
+                        st = k % stages;
+                        ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                        open = true;
+                    }
+                    if (active) {
+                        if (first) {
+                            const int pos = fillpos + incl - 1;
+                            URow uu;
+                            uu.row = s;
+                            uu.mask = mask;
+                            meta[(size_t)st * TILE + pos] = uu;
+                            const size_t off = ((size_t)row * p.Hkv + kvh) * (size_t)(D * 2);
+                            gk[pos] = (s == t_new ? p.k_new : p.kr + (size_t)s * slab_bytes) + off;
+                            gv[pos] = (s == t_new ? p.v_new : p.vr + (size_t)s * slab_bytes) + off;
+                        }
+                        if (kvh == 0) p.anc_dst[(size_t)(b * Wb + j) * p.max_steps + s] = row;
+                    }
+                    fillpos += total;
                 }
             }
+            if (ok && open) publish_tile(st, fillpos, true);
             SEGKV_STAMP(5);
             // store what the step appends: the parent ids and the new K/V rows of this work group
             if (kvh == 0 && split == 0 && lane < Wb)
