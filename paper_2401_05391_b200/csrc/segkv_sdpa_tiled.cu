@@ -9,13 +9,23 @@
 //    heads of the kv head's group) of its work group, so a K/V byte staged in
 //    shared memory is used by every beam: prompt bytes cross HBM once, not BW
 //    times (Section 4.2.1: "accesses only 1/BW amount data in HBM").
-//  * one producer warp feeds a ring of shared-memory stages.  Prompt tiles come
-//    by TMA (cp.async.bulk.tensor, 128-byte swizzle) from the head-major prompt
-//    segment; response tiles are gathered row by row with 16-byte cp.async
-//    through the request's list of DISTINCT response rows (the index select of
-//    Section 3.3 folded into the load), written into the same swizzled layout.
-//    Every row carries the set of beams that read it; scores of other beams
-//    are masked, so a row shared by several beams is also fetched once.
+//  * two producer warps feed a ring of shared-memory stages.  The TMA warp
+//    fetches prompt tiles (cp.async.bulk.tensor, 128-byte swizzle) from the
+//    head-major prompt segment; it sets the mbarriers up itself and issues the
+//    first ring before the CTA has synchronised.  The gather warp copies
+//    response rows one by one with 16-byte cp.async (16 lanes per 256-byte
+//    row) into the same swizzled layout: the index select of Section 3.3
+//    folded into the load.  Every row carries its step and the set of beams
+//    that read it; scores of other beams are masked, so a row shared by
+//    several beams is fetched once.
+//      - separate form (segkv_decode_sdpa): the rows come from the request's
+//        list of DISTINCT rows that the append kernel made;
+//      - fused form (segkv_decode_step, template FUSED): one lane per (step,
+//        beam) reads the previous step's beam-index table, resolves the new
+//        parents with a shuffle (anc_t[j][s] = anc_{t-1}[parent[j]][s]),
+//        removes duplicates among the lanes of a step, packs the distinct rows
+//        with a warp prefix sum, stores the new table column, and takes the
+//        new step's rows straight from the caller's k_new / v_new.
 //  * consumer warps take 16 keys of a tile each.  Scores are a small GEMM on
 //    tensor cores with the KEYS on the M side: S^T[16 keys, 8 cols] = K . Q^T
 //    (mma.sync m16n8k16, fp32 accumulate), so the BW=4 beams pad only to 8.
@@ -23,8 +33,14 @@
 //    (movmatrix) and O^T[16 d, 8 cols] += V^T . P^T, V^T read with
 //    ldmatrix.trans.  Each warp keeps its own running max / sum / O^T.
 //  * epilogue: warps merge through shared memory; with more than one split the
-//    partial (m, l, O) goes to a workspace and the last CTA of the work group
-//    to arrive (atomic ticket, no waiting) merges the splits and writes out.
+//    partial (m, l, O) goes to a global workspace and the last CTA of the work
+//    group to arrive (acq_rel ticket, nobody waits) folds the splits in one
+//    pass, or, on request, the splits form a thread-block cluster and exchange
+//    slices of the (column, d) plane through distributed shared memory.
+//  * programmatic dependent launch: prompt tiles are requested before the
+//    previous kernel of the stream has finished (nothing in a decode loop
+//    writes the prompt segment); everything else follows griddepcontrol.wait,
+//    and dependents are released only after that wait.
 //
 // All mbarrier waits are bounded: on expiry the kernel sets
 // SEGKV_DEV_WAIT_LIMIT in the error word and winds down.
