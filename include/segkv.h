@@ -78,6 +78,25 @@ enum {
 SEGKV_API int segkv_create(segkv_t* out, int batch, int beams, int heads, int kv_heads, int head_dim,
                  int max_prompt, int max_steps, int dtype);
 
+/*
+ * Like segkv_create, but the response segment grows with the response
+ * (Section 3.2: N_step is raised in steps of 16 so that short responses do not
+ * pay for the model's maximum length): storage for `chunk_steps` more steps is
+ * allocated when step chunk_steps, 2*chunk_steps, ... is appended, and the K/V
+ * held after n steps follow Eq. 3 with step = chunk_steps.  Unlike the paper's
+ * scheme nothing is copied or freed when the capacity grows: the chunks are
+ * separate allocations that the kernels address through a small table.
+ * max_steps stays the upper bound (it sizes the index tables).  chunk_steps 0,
+ * or >= max_steps, is segkv_create.  The append / decode-step call that opens
+ * a chunk calls cudaMalloc.  Errors: as segkv_create.
+ */
+SEGKV_API int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_heads, int head_dim,
+                                   int max_prompt, int max_steps, int chunk_steps, int dtype);
+
+/* K/V bytes the handle holds right now: batch * (max_prompt + beams * steps held) * 2*kv_heads*head_dim*2
+ * (Eq. 3 for one layer; "steps held" is max_steps, or the chunks opened so far). */
+SEGKV_API long long segkv_allocated_kv_bytes(segkv_t h);
+
 /* Free everything the handle owns.  Synchronises the device.  NULL is allowed. */
 SEGKV_API int segkv_destroy(segkv_t h);
 

@@ -81,11 +81,46 @@ int make_prompt_map(const segkv* h, void* base, int prompt_len, CUtensorMap* out
 }
 
 void free_all(segkv* h) {
-    void* ptrs[] = {h->kp, h->vp, h->kr, h->vr, h->parent, h->anc[0], h->anc[1], h->ulist, h->ucount,
+    void* ptrs[] = {h->kp, h->vp, h->kr, h->k_chunks_dev, h->parent, h->anc[0], h->anc[1], h->ulist, h->ucount,
                     h->err_word, h->ws, h->tickets, h->st_q, h->st_out, h->st_k, h->st_v, h->st_parent,
                     h->st_slopes};
     for (void* p : ptrs)
         if (p) cudaFree(p);
+    for (int c = 0; c < h->nchunks; ++c)
+        if (h->k_chunks_host[c]) cudaFree(h->k_chunks_host[c]);
+    free(h->k_chunks_host);
+}
+
+size_t slab_bytes_of(const Dims& d) { return (size_t)d.rows * d.kv_heads * d.head_dim * 2; }
+
+// Device address of the K slab of response step `step` (its V slab is vdelta behind).
+char* k_slab_of(const segkv* h, int step) {
+    const Dims& d = h->d;
+    if (d.chunk_steps == 0) return (char*)h->kr + (size_t)step * slab_bytes_of(d);
+    const int c = step / d.chunk_steps;
+    return (char*)h->k_chunks_host[c] + (size_t)(step - c * d.chunk_steps) * slab_bytes_of(d);
+}
+
+long long vdelta_of(const segkv* h) {
+    const Dims& d = h->d;
+    return (long long)((size_t)(d.chunk_steps ? d.chunk_steps : d.max_steps) * slab_bytes_of(d));
+}
+
+// Growing capacity (Section 3.2): make sure the chunk that holds `step` exists.  A new chunk is
+// one allocation {K part, V part}; its address is appended to the device table on the stream.
+int ensure_chunk(segkv* h, int step, cudaStream_t st) {
+    const Dims& d = h->d;
+    if (d.chunk_steps == 0) return SEGKV_OK;
+    const int need = step / d.chunk_steps + 1;
+    while (h->nchunks < need) {
+        void* p = nullptr;
+        SEGKV_CUDA(cudaMalloc(&p, 2 * (size_t)d.chunk_steps * slab_bytes_of(d)));
+        h->k_chunks_host[h->nchunks] = p;
+        SEGKV_CUDA(cudaMemcpyAsync(h->k_chunks_dev + h->nchunks, h->k_chunks_host + h->nchunks, sizeof(void*),
+                                   cudaMemcpyHostToDevice, st));
+        h->nchunks++;
+    }
+    return SEGKV_OK;
 }
 
 template <typename T>
@@ -174,6 +209,8 @@ SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes
     a.vp = h->vp;
     a.kr = h->kr;
     a.vr = h->vr;
+    a.k_chunks = (const void* const*)h->k_chunks_dev;
+    a.vdelta = vdelta_of(h);
     a.anc = h->anc[h->steps > 0 ? ((h->steps - 1) & 1) : 0];
     a.ulist = h->ulist;
     a.ucount = h->ucount;
@@ -208,6 +245,14 @@ size_t segkv_storage_bytes(int batch, int beams, int kv_heads, int head_dim, int
     return (size_t)batch * ((size_t)max_prompt + (size_t)beams * max_steps) * token;
 }
 
+long long segkv_allocated_kv_bytes(segkv_t h) {
+    if (!h) return SEGKV_EINVAL;
+    const Dims& d = h->d;
+    const size_t token = 2 * (size_t)d.kv_heads * d.head_dim * 2;
+    const size_t steps_held = d.chunk_steps ? (size_t)h->nchunks * d.chunk_steps : (size_t)d.max_steps;
+    return (long long)((size_t)d.batch * ((size_t)d.max_prompt + (size_t)d.beams * steps_held) * token);
+}
+
 const char* segkv_strerror(int code) {
     switch (code) {
         case SEGKV_OK: return "ok";
@@ -225,15 +270,22 @@ const char* segkv_last_cuda_error(void) { return g_cuda_err; }
 
 int segkv_create(segkv_t* out, int batch, int beams, int heads, int kv_heads, int head_dim, int max_prompt,
                  int max_steps, int dtype) {
+    return segkv_create_growing(out, batch, beams, heads, kv_heads, head_dim, max_prompt, max_steps, 0, dtype);
+}
+
+int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_heads, int head_dim, int max_prompt,
+                         int max_steps, int chunk_steps, int dtype) {
     if (!out) return SEGKV_EINVAL;
     if (!dims_ok(batch, beams, heads, kv_heads, head_dim, max_prompt, max_steps, dtype)) return SEGKV_EINVAL;
+    if (chunk_steps < 0) return SEGKV_EINVAL;
+    if (chunk_steps >= max_steps) chunk_steps = 0;      // one chunk would hold everything: fixed capacity
     segkv* h = new (std::nothrow) segkv();
     if (!h) return SEGKV_ENOMEM;
     memset(h, 0, sizeof *h);
     Dims& d = h->d;
     d.batch = batch; d.beams = beams; d.heads = heads; d.kv_heads = kv_heads; d.head_dim = head_dim;
     d.group = heads / kv_heads; d.max_prompt = max_prompt; d.max_steps = max_steps;
-    d.rows = batch * beams; d.dtype = dtype;
+    d.rows = batch * beams; d.dtype = dtype; d.chunk_steps = chunk_steps;
     h->prompt_len = -1;
     h->overlap = true;
 
@@ -255,8 +307,15 @@ int segkv_create(segkv_t* out, int batch, int beams, int heads, int kv_heads, in
     const size_t resp_bytes = (size_t)max_steps * d.rows * kv_heads * head_dim * eb;
     SEGKV_TRY(dmalloc(&h->kp, prompt_bytes));
     SEGKV_TRY(dmalloc(&h->vp, prompt_bytes));
-    SEGKV_TRY(dmalloc(&h->kr, resp_bytes));
-    SEGKV_TRY(dmalloc(&h->vr, resp_bytes));
+    if (chunk_steps == 0) {
+        SEGKV_TRY(dmalloc(&h->kr, 2 * resp_bytes));                      // K, then V, in one allocation
+        h->vr = (char*)h->kr + resp_bytes;
+    } else {
+        h->nchunks_max = (max_steps + chunk_steps - 1) / chunk_steps;
+        h->k_chunks_host = (void**)calloc((size_t)h->nchunks_max, sizeof(void*));
+        if (!h->k_chunks_host) return fail(SEGKV_ENOMEM);
+        SEGKV_TRY(dmalloc(&h->k_chunks_dev, (size_t)h->nchunks_max * sizeof(void*)));
+    }
     SEGKV_TRY(dmalloc(&h->parent, (size_t)max_steps * d.rows * sizeof(int32_t)));
     SEGKV_TRY(dmalloc(&h->anc[0], (size_t)max_steps * d.rows * sizeof(int32_t)));
     SEGKV_TRY(dmalloc(&h->anc[1], (size_t)max_steps * d.rows * sizeof(int32_t)));
@@ -317,7 +376,12 @@ int segkv_append(segkv_t h, int step, const int32_t* beam_parent, const void* k_
     if (h->prompt_len < 0) return SEGKV_ESTATE;
     if (step != h->steps) return SEGKV_ESTATE;
     if (step >= h->d.max_steps) return SEGKV_ECAPACITY;
-    SEGKV_CUDA(launch_append(h->d, step, beam_parent, k_new, v_new, h->kr, h->vr, h->parent,
+    {
+        int rc = ensure_chunk(h, step, (cudaStream_t)stream);
+        if (rc != SEGKV_OK) return rc;
+    }
+    SEGKV_CUDA(launch_append(h->d, step, beam_parent, k_new, v_new, k_slab_of(h, step),
+                             k_slab_of(h, step) + vdelta_of(h), h->parent,
                              h->anc[(step + 1) & 1], h->anc[step & 1], h->ulist, h->ucount, h->err_word,
                              h->sm_count, h->overlap && step > 0, (cudaStream_t)stream));
     h->launches++;
@@ -422,8 +486,11 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
         int rc = alloc_workspace(h, splits);
         if (rc != SEGKV_OK) return rc;
     }
+    {
+        int rc = ensure_chunk(h, step, (cudaStream_t)stream);
+        if (rc != SEGKV_OK) return rc;
+    }
     SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, splits);
-    const size_t slab_bytes = (size_t)d.rows * d.kv_heads * d.head_dim * 2;
     a.steps = step + 1;
     a.anc = h->anc[(step + 1) & 1];      // table of step-1 (unused at step 0)
     a.cluster = cluster;
@@ -434,8 +501,8 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     a.parent = step > 0 ? beam_parent : nullptr;
     a.k_new = k_new;
     a.v_new = v_new;
-    a.kr_new_slab = (char*)h->kr + (size_t)step * slab_bytes;
-    a.vr_new_slab = (char*)h->vr + (size_t)step * slab_bytes;
+    a.kr_new_slab = k_slab_of(h, step);
+    a.vr_new_slab = k_slab_of(h, step) + vdelta_of(h);
     a.anc_dst = h->anc[step & 1];
     a.parent_row = h->parent + (size_t)step * d.rows;
     SEGKV_CUDA(launch_sdpa_tiled(d, a, h->tm_kp, h->tm_vp, stages, (cudaStream_t)stream));

@@ -183,7 +183,7 @@ append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __
 }
 
 cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, const void* k_new,
-                          const void* v_new, void* kr, void* vr, int32_t* parent_tab,
+                          const void* v_new, void* kr_slab_v, void* vr_slab_v, int32_t* parent_tab,
                           const int32_t* anc_prev, int32_t* anc_cur, URow* ulist, int32_t* ucount,
                           int* err_word, int sm_count, bool pdl, cudaStream_t st) {
     const long long slab_elems = (long long)d.rows * d.kv_heads * d.head_dim;
@@ -191,8 +191,8 @@ cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, c
     long long copy_blocks = (slab_chunks + kBtThreads * 4 - 1) / (kBtThreads * 4);
     if (copy_blocks < 1) copy_blocks = 1;
     if (copy_blocks > (long long)sm_count * 8) copy_blocks = (long long)sm_count * 8;
-    uint4* kr_slab = (uint4*)((char*)kr + (size_t)step * slab_elems * 2);
-    uint4* vr_slab = (uint4*)((char*)vr + (size_t)step * slab_elems * 2);
+    uint4* kr_slab = (uint4*)kr_slab_v;     // slab of this step inside the response segment
+    uint4* vr_slab = (uint4*)vr_slab_v;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(d.batch + copy_blocks), 1, 1);
     cfg.blockDim = dim3(kBtThreads, 1, 1);

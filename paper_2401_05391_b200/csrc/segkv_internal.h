@@ -26,6 +26,7 @@ struct Dims {
     int batch, beams, heads, kv_heads, head_dim, group;  // group = heads / kv_heads
     int max_prompt, max_steps;
     int rows;                                            // batch * beams
+    int chunk_steps;                                     // response capacity grows in chunks of this many steps (0: fixed)
     int dtype;
 };
 
@@ -49,8 +50,12 @@ struct segkv {
     // device storage (owned)
     void* kp;            // [batch, kv_heads, max_prompt, D]
     void* vp;
-    void* kr;            // [max_steps, rows, kv_heads, D]
-    void* vr;
+    void* kr;            // [max_steps, rows, kv_heads, D]; K and V of the response segment are ONE
+    void* vr;            // allocation (V right behind K), so a V row is its K row plus a constant
+    // growing capacity (Section 3.2): chunks of chunk_steps steps, each {K part, V part} in one allocation
+    void** k_chunks_host;    // [nchunks_max] device pointers, host copy
+    void** k_chunks_dev;     // the same table on the device
+    int nchunks, nchunks_max;
     int32_t* parent;     // [max_steps, rows]
     int32_t* anc[2];     // [rows, max_steps], generation t lives in anc[t & 1]
     segkv_impl::URow* ulist;   // [batch, beams*max_steps] distinct response rows per request
@@ -77,7 +82,7 @@ cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v
                                      int prompt_len, cudaStream_t st);
 
 cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, const void* k_new,
-                          const void* v_new, void* kr, void* vr, int32_t* parent_tab,
+                          const void* v_new, void* kr_slab, void* vr_slab, int32_t* parent_tab,
                           const int32_t* anc_prev, int32_t* anc_cur, URow* ulist, int32_t* ucount,
                           int* err_word, int sm_count, bool pdl, cudaStream_t st);
 // Re-derive the distinct-row lists from the current beam-index table (after fused steps).
@@ -90,8 +95,10 @@ struct SdpaArgs {
     const float* slopes;
     const void* kp;
     const void* vp;
-    const void* kr;
+    const void* kr;          // response K (fixed capacity) or NULL (growing: see k_chunks)
     const void* vr;
+    const void* const* k_chunks;   // device table of chunk base pointers (growing capacity)
+    long long vdelta;        // bytes from a response K row to its V row
     const int32_t* anc;      // beam-index table (fused step: the previous step's)
     const URow* ulist;
     const int32_t* ucount;

@@ -51,7 +51,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kWarps * 32)
 sdpa_rowwise_kernel(const T* __restrict__ q, T* __restrict__ out, const float* __restrict__ slopes,
                     const T* __restrict__ kp, const T* __restrict__ vp, const T* __restrict__ kr,
-                    const T* __restrict__ vr, const int32_t* __restrict__ anc, int P, int steps, int W, int H,
+                    const T* const* __restrict__ k_chunks, int chunk_steps, long long vdelta_elems,
+                    const int32_t* __restrict__ anc, int P, int steps, int W, int H,
                     int Hkv, int group, int max_prompt, int max_steps, int rows) {
     constexpr int E = D / 32;
     const int h = blockIdx.x, g = blockIdx.y;
@@ -71,19 +72,24 @@ sdpa_rowwise_kernel(const T* __restrict__ q, T* __restrict__ out, const float* _
     for (int e = 0; e < E; ++e) acc[e] = 0.f;
 
     for (int i = warp; i < L; i += kWarps) {
-        size_t off;
+        const T* krow;
+        const T* vrow;
         if (i < P) {
-            off = (((size_t)b * Hkv + kvh) * max_prompt + i) * D;
+            const size_t off = (((size_t)b * Hkv + kvh) * max_prompt + i) * D;
+            krow = kp + off;
+            vrow = vp + off;
         } else {
-            int s = i - P;
-            int r = anc[(size_t)g * max_steps + s];
-            off = (((size_t)s * rows + r) * Hkv + kvh) * D;
+            const int s = i - P;
+            const int r = anc[(size_t)g * max_steps + s];
+            const size_t slab = (size_t)rows * Hkv * D;          // elements of one step
+            const T* base = kr + (size_t)s * slab;                // one array, or the chunk that holds step s
+            if (chunk_steps) base = k_chunks[s / chunk_steps] + (size_t)(s % chunk_steps) * slab;
+            krow = base + ((size_t)r * Hkv + kvh) * D;
+            vrow = krow + vdelta_elems;                           // V rows sit a constant behind their K rows
         }
-        const T* kbase = i < P ? kp : kr;
-        const T* vbase = i < P ? vp : vr;
         float kf[E], vf[E];
-        load_row<T, E>(kbase + off + lane * E, kf);
-        load_row<T, E>(vbase + off + lane * E, vf);
+        load_row<T, E>(krow + lane * E, kf);
+        load_row<T, E>(vrow + lane * E, vf);
         float dot = 0.f;
 #pragma unroll
         for (int e = 0; e < E; ++e) dot = fmaf(qf[e], kf[e], dot);
@@ -126,7 +132,8 @@ cudaError_t dispatch(const Dims& d, const SdpaArgs& a, cudaStream_t st) {
 #define SEGKV_ROWWISE(DD)                                                                               \
     sdpa_rowwise_kernel<T, DD><<<grid, block, 0, st>>>(                                                 \
         (const T*)a.q, (T*)a.out, a.slopes, (const T*)a.kp, (const T*)a.vp, (const T*)a.kr,             \
-        (const T*)a.vr, a.anc, a.prompt_len, a.steps, d.beams, d.heads, d.kv_heads, d.group,            \
+        (const T* const*)a.k_chunks, d.chunk_steps, a.vdelta / 2, a.anc, a.prompt_len, a.steps, d.beams, \
+        d.heads, d.kv_heads, d.group,                                                                  \
         d.max_prompt, d.max_steps, d.rows)
     switch (d.head_dim) {
         case 64: SEGKV_ROWWISE(64); break;

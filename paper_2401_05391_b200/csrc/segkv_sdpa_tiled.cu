@@ -213,8 +213,9 @@ struct TiledParams {
     const void* q;
     void* out;
     const float* slopes;
-    const char* kr;
-    const char* vr;
+    const char* kr;          // response K, fixed capacity (V row = K row + vdelta)
+    const char* const* k_chunks;   // growing capacity: chunk base pointers, chunk_steps steps each
+    long long vdelta;
     const URow* ulist;
     const int32_t* ucount;
     float* ws_o;    // [slab][S][ncols][D]   un-normalised partial outputs (ticket combine only)
@@ -233,6 +234,7 @@ struct TiledParams {
     int fused;      // 1: steps-1 is a new step whose rows come from k_new / v_new and whose beam-index
                     //    column is derived here from `parent` and the previous table
     int P, steps, S, W, G, H, Hkv, rows, max_steps, ncols, stages;
+    int chunk_steps;   // 0: the response segment is one array
     int quota;      // distinct response rows per split (the last split also takes any excess)
     int cluster;    // 1: the S CTAs of a work group form a thread-block cluster
     int early_prompt;  // 1: prompt tiles may be fetched before the previous kernel has completed
@@ -399,6 +401,13 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         // (a parity wait cannot tell a far-future round of a stage from the current one).
         constexpr int CPR = D / 8;        // 16-byte chunks per row
         constexpr int RPI = 32 / CPR;     // rows covered by one warp-wide copy
+        const size_t slab_bytes = (size_t)p.rows * p.Hkv * (size_t)(D * 2);
+        // K slab of response step s: in the one array, or in the chunk that holds the step
+        auto k_slab = [&](int s) -> const char* {
+            if (p.chunk_steps == 0) return p.kr + (size_t)s * slab_bytes;
+            const int c = s / p.chunk_steps;
+            return p.k_chunks[c] + (size_t)(s - c * p.chunk_steps) * slab_bytes;
+        };
         // Copy rows [0, cnt) of the tile whose row pointers (gk, gv) have been written.  One
         // warp-wide copy moves whole rows (CPR lanes per row): fully coalesced.  The arrival on
         // the stage's full barrier fires when this lane's copies have landed.
@@ -417,10 +426,10 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                         if constexpr (FUSED) {             // rows may sit in the caller's k_new / v_new
                             cp_async_16(k_dst + off, gk[key] + c * 16);
                             cp_async_16(v_dst + off, gv[key] + c * 16);
-                        } else {                           // one offset serves both segments
-                            const size_t src = reinterpret_cast<size_t>(gk[key]) + (size_t)c * 16;
-                            cp_async_16(k_dst + off, p.kr + src);
-                            cp_async_16(v_dst + off, p.vr + src);
+                        } else {                           // a V row sits a constant behind its K row
+                            const char* src = gk[key] + c * 16;
+                            cp_async_16(k_dst + off, src);
+                            cp_async_16(v_dst + off, src + p.vdelta);
                         }
                     }
                 }
@@ -503,7 +512,8 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     u.row = row / p.rows;                                // consumers need the step only
                     u.mask = valid ? ucur[kk].y : 0u;
                     meta_st[key] = u;
-                    gk[key] = reinterpret_cast<const char*>(((size_t)row * p.Hkv + kvh) * (size_t)(D * 2));  // byte offset
+                    const int sidx = u.row;
+                    gk[key] = k_slab(sidx) + ((size_t)(row - sidx * p.rows) * p.Hkv + kvh) * (size_t)(D * 2);
                 }
                 publish_tile(st, cnt, r == nrt - 1);
             }
@@ -533,7 +543,6 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     if (s < rs1 && j < Wb && s != t_new) rowb[u] = p.anc_prev[(size_t)(b * Wb + j) * p.max_steps + s];
                 }
             };
-            const size_t slab_bytes = (size_t)p.rows * p.Hkv * (size_t)(D * 2);
             int rowb[PF];
             int par = j;
             par = (p.steps > 1 && j < Wb) ? p.parent[b * Wb + j] : j;
@@ -601,8 +610,9 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                             uu.mask = mask;
                             meta[(size_t)st * TILE + pos] = uu;
                             const size_t off = ((size_t)row * p.Hkv + kvh) * (size_t)(D * 2);
-                            gk[pos] = (s == t_new ? p.k_new : p.kr + (size_t)s * slab_bytes) + off;
-                            gv[pos] = (s == t_new ? p.v_new : p.vr + (size_t)s * slab_bytes) + off;
+                            const char* ksl = (s == t_new) ? p.k_new : k_slab(s);
+                            gk[pos] = ksl + off;
+                            gv[pos] = (s == t_new ? p.v_new : ksl + p.vdelta) + off;
                         }
                         if (kvh == 0) p.anc_dst[(size_t)(b * Wb + j) * p.max_steps + s] = row;
                     }
@@ -1023,7 +1033,8 @@ cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk,
     }
     TiledParams p;
     p.q = a.q; p.out = a.out; p.slopes = a.slopes;
-    p.kr = (const char*)a.kr; p.vr = (const char*)a.vr;
+    p.kr = (const char*)a.kr; p.k_chunks = (const char* const*)a.k_chunks; p.vdelta = a.vdelta;
+    p.chunk_steps = d.chunk_steps;
     p.ulist = a.ulist; p.ucount = a.ucount; p.tickets = a.tickets; p.err_word = a.err_word;
     p.fused = a.fused ? 1 : 0;
     p.anc_prev = a.anc; p.parent = a.parent; p.k_new = (const char*)a.k_new; p.v_new = (const char*)a.v_new;

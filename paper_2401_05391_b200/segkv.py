@@ -27,6 +27,8 @@ _vp, _int, _i32p = ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int32)
 # name -> (restype, argtypes); one entry per symbol include/segkv.h declares
 SIGNATURES = {
     "segkv_create": (_int, [ctypes.POINTER(_vp)] + [_int] * 8),
+    "segkv_create_growing": (_int, [ctypes.POINTER(_vp)] + [_int] * 9),
+    "segkv_allocated_kv_bytes": (ctypes.c_longlong, [_vp]),
     "segkv_destroy": (_int, [_vp]),
     "segkv_prefill_write": (_int, [_vp, _vp, _vp, _int, _vp]),
     "segkv_append": (_int, [_vp, _int, _vp, _vp, _vp, _vp]),
@@ -121,15 +123,20 @@ def segkv_strerror(code: int) -> str:
 class SegKV:
     """One attention layer's segment KV cache; methods mirror the C entry points."""
 
-    def __init__(self, batch, beams, heads, kv_heads, head_dim, max_prompt, max_steps, dtype=torch.float16):
+    def __init__(self, batch, beams, heads, kv_heads, head_dim, max_prompt, max_steps, dtype=torch.float16,
+                 chunk_steps: int = 0):
         self.batch, self.beams, self.heads, self.kv_heads = batch, beams, heads, kv_heads
         self.head_dim, self.max_prompt, self.max_steps = head_dim, max_prompt, max_steps
         self.dtype = dtype
         self.rows = batch * beams
         code = {torch.float16: SEGKV_F16, torch.bfloat16: SEGKV_BF16}.get(dtype, -1)
         self._h = _vp()
-        _check(lib().segkv_create(ctypes.byref(self._h), batch, beams, heads, kv_heads, head_dim,
-                                  max_prompt, max_steps, code), "segkv_create")
+        if chunk_steps:
+            _check(lib().segkv_create_growing(ctypes.byref(self._h), batch, beams, heads, kv_heads, head_dim,
+                                              max_prompt, max_steps, chunk_steps, code), "segkv_create_growing")
+        else:
+            _check(lib().segkv_create(ctypes.byref(self._h), batch, beams, heads, kv_heads, head_dim,
+                                      max_prompt, max_steps, code), "segkv_create")
 
     # ------------------------------------------------------------ life cycle
     def destroy(self) -> None:
@@ -257,6 +264,10 @@ class SegKV:
 
     def get_splits(self) -> int:
         return int(lib().segkv_get_splits(self._h))
+
+    @property
+    def allocated_kv_bytes(self) -> int:
+        return int(lib().segkv_allocated_kv_bytes(self._h))
 
     @property
     def launch_count(self) -> int:

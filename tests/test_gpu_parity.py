@@ -113,6 +113,37 @@ def test_fused_step_wide_beam_and_single_beam():
                        check_steps=(0, 3, 23))
 
 
+@pytest.mark.parametrize("fused", [False, True])
+def test_growing_capacity_matches_fixed_capacity_and_eq3(fused):
+    """Response capacity in 16-step chunks (the paper's N_step policy): same bits as the fixed-capacity
+    cache at every step, and the K/V bytes held follow Eq. 3."""
+    import oracle
+    w = wl.Workload("grow", 2, 4, 4, 2, 128, 96, 50, "f16", "uniform", False, 67)
+    a, b = Run(w), Run(w, chunk_steps=16)
+    try:
+        tok = oracle.cache_token(1, w.kv_heads, w.head_dim, 2)
+        for t in range(w.steps):
+            if fused:
+                _, oa, q = a.step_fused()
+                _, ob, _ = b.step_fused()
+            else:
+                a.append_next(); b.append_next()
+                oa, q = a.decode()
+                ob, _ = b.decode(q)
+            assert torch.equal(oa.view(torch.int16), ob.view(torch.int16)), f"step {t}"
+            assert b.h.allocated_kv_bytes == oracle.cache_segment(w.batch, w.beams, w.prompt_len, t + 1, tok, 16)
+            assert a.h.allocated_kv_bytes == sk.segkv_storage_bytes(w.batch, w.beams, w.kv_heads, w.head_dim,
+                                                                   w.prompt_len, w.steps, sk.SEGKV_F16)
+        assert np.array_equal(a.h.get_ancestry(), b.h.get_ancestry())
+        b.check(ob, q, w.steps - 1, all_pairs(w))
+        x = b.h.decode_sdpa_rowwise(q, None, None)           # the per-beam kernel walks the chunks too
+        torch.cuda.synchronize()
+        assert torch.allclose(x.float(), ob.float(), atol=4e-3, rtol=2e-2)
+        assert a.h.get_error() == 0 and b.h.get_error() == 0
+    finally:
+        a.close(); b.close()
+
+
 def test_tiny_every_step_all_outputs():
     w = wl.CONFIGS[0]
     run_workload(w, all_pairs, check_steps=tuple(range(w.steps)))
