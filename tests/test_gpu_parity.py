@@ -218,6 +218,60 @@ def test_single_beam_and_wide_beam():
                  check_steps=(0, 3, 39))
 
 
+def test_sixteen_query_columns_and_the_rowwise_fallback():
+    # 16 columns per kv head (two column tiles) is the most the tiled kernel takes ...
+    run_workload(wl.Workload("c16", 2, 4, 8, 2, 128, 130, 20, "f16", "uniform", True, 24), all_pairs,
+                 check_steps=(0, 7, 19))
+    run_workload(wl.Workload("c16b", 1, 16, 2, 2, 64, 70, 20, "bf16", "uniform", False, 25), all_pairs,
+                 check_steps=(0, 19))
+    # ... beyond that (here 32 beams) the per-beam kernel serves segkv_decode_sdpa and segkv_decode_step
+    w = wl.Workload("w32", 1, 32, 2, 2, 64, 40, 12, "f16", "uniform", False, 26)
+    run_workload(w, all_pairs, check_steps=(0, 5, 11))
+    run_workload_fused(w, all_pairs, check_steps=(0, 5, 11))
+
+
+@pytest.mark.parametrize("kind", ["identity", "collapse", "cycle"])
+def test_degenerate_parent_tables(kind):
+    """identity: beams never mix (every response row is read by one beam); collapse: every beam
+    extends beam 0 (one shared row per step); cycle: the beams rotate."""
+    w = wl.Workload("deg-" + kind, 2, 4, 4, 4, 128, 90, 33, "f16", "uniform", False, 27)
+    j = np.tile(np.arange(w.beams), w.batch)
+    row = {"identity": j, "collapse": np.zeros_like(j), "cycle": (j + 1) % w.beams}[kind]
+    par = np.tile(row, (w.steps, 1)).astype(np.int32)
+    for fused in (False, True):
+        r = Run(w, parents=par)
+        try:
+            for t in range(w.steps):
+                if fused:
+                    _, out, q = r.step_fused()
+                else:
+                    r.append_next()
+            if not fused:
+                out, q = r.decode()
+            t = w.steps - 1
+            assert np.array_equal(r.h.get_ancestry(), r.oracle_ancestry(t))
+            uniq = r.h.get_unique_rows()
+            if kind == "identity" or kind == "cycle":
+                assert (uniq == w.beams * w.steps).all()
+            else:
+                assert (uniq == w.steps + w.beams - 1).all()       # one row per step, W at the newest
+            r.check(out, q, t, all_pairs(w))
+        finally:
+            r.close()
+
+
+def test_one_key_only():
+    # a single prompt key and no response: the output is that key's value row, for every beam
+    w = wl.Workload("one", 2, 4, 2, 2, 128, 1, 1, "f16", "uniform", False, 28)
+    r = Run(w)
+    try:
+        out, q = r.decode()
+        want = r.vp[:, 0].repeat_interleave(w.beams, dim=0)        # [rows, kv_heads, D]
+        assert torch.equal(out.view(torch.int16), want.view(torch.int16))
+    finally:
+        r.close()
+
+
 def test_repeat_is_bit_identical_and_every_output_is_written():
     w = wl.CONFIGS[1].scaled(steps=24)
     r = Run(w)
