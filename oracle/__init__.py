@@ -53,6 +53,8 @@ def _load():
         lib.segkv_oracle_ancestry.restype = None
         lib.segkv_oracle_decode.argtypes = [c_int] * 8 + [u16p] * 5 + [i32p, f32p, i32p, c_int, f64p, f64p]
         lib.segkv_oracle_decode.restype = c_int
+        lib.segkv_oracle_prefill.argtypes = [c_int] * 6 + [u16p] * 3 + [f32p, i32p, c_int, f64p]
+        lib.segkv_oracle_prefill.restype = c_int
         lib.segkv_oracle_cache_token.argtypes = [c_int] * 4
         lib.segkv_oracle_cache_token.restype = ctypes.c_double
         lib.segkv_oracle_cache_standard.argtypes = [c_int, c_int, ctypes.c_long, ctypes.c_long, ctypes.c_double]
@@ -154,6 +156,36 @@ def decode_sdpa(dtype: str, batch: int, beams: int, heads: int, kv_heads: int, h
         if return_probs:
             probs = probs.reshape(rows, heads, L)
     return (out, probs) if return_probs else out
+
+
+def prefill_sdpa(dtype: str, batch: int, heads: int, kv_heads: int, head_dim: int, q: np.ndarray, k: np.ndarray,
+                 v: np.ndarray, slopes: Optional[np.ndarray] = None, rows: Optional[Sequence] = None) -> np.ndarray:
+    """Causal prefill attention.  q ``[batch, N, heads, D]``, k, v ``[batch, N, kv_heads, D]`` (uint16
+    bits).  ``rows`` = list of (b, i, h) to evaluate (default: all); returns float64 ``[nrows, D]``
+    (``[batch, N, heads, D]`` when all rows are asked for)."""
+    N = int(q.shape[1])
+    q = _u16(q, (batch, N, heads, head_dim))
+    k = _u16(k, (batch, N, kv_heads, head_dim))
+    v = _u16(v, (batch, N, kv_heads, head_dim))
+    if slopes is not None:
+        slopes = np.ascontiguousarray(slopes, dtype=np.float32)
+        if slopes.shape != (heads,):
+            raise ValueError("slopes must be [heads]")
+    all_rows = rows is None
+    if all_rows:
+        bb, ii, hh = np.meshgrid(np.arange(batch), np.arange(N), np.arange(heads), indexing="ij")
+        rows_a = np.stack([bb.ravel(), ii.ravel(), hh.ravel()], axis=1)
+    else:
+        rows_a = np.asarray(rows).reshape(-1, 3)
+    rows_a = np.ascontiguousarray(rows_a, dtype=np.int32)
+    out = np.empty((rows_a.shape[0], head_dim), dtype=np.float64)
+    rc = _load().segkv_oracle_prefill(DTYPES[dtype], batch, N, heads, kv_heads, head_dim,
+                                      _ptr(q, ctypes.c_uint16), _ptr(k, ctypes.c_uint16), _ptr(v, ctypes.c_uint16),
+                                      _ptr(slopes, ctypes.c_float), _ptr(rows_a, ctypes.c_int32), rows_a.shape[0],
+                                      _ptr(out, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("segkv_oracle_prefill rejected its arguments")
+    return out.reshape(batch, N, heads, head_dim) if all_rows else out
 
 
 def cache_token(layers: int, heads: int, head_dim: int, elem_bytes: int) -> float:

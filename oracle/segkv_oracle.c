@@ -164,6 +164,48 @@ int segkv_oracle_decode(int dtype, int BS, int BW, int H, int Hkv, int D, int P,
 }
 
 /*
+ * Prefill attention (Section 3.1 / 3.3: the prefill kernel is the special case of the decode
+ * kernel that sees only query and prompt key/value, batch-first in and out): causal
+ * self-attention of every prompt position over the positions up to itself,
+ *     out[b,i,h,:] = softmax_{j<=i}( q[b,i,h,:] . k[b,j,kvh,:] / sqrt(D) + bias ) . v[b,j,kvh,:]
+ * with bias = slope[h] * (j - i) when slopes are given.  q, out: [BS, N, H, D]; k, v: [BS, N, Hkv, D]
+ * (token-major, 16-bit storage as raw bits).  `rows` lists (b, i, h) triples; out is [nrows][D].
+ */
+int segkv_oracle_prefill(int dtype, int BS, int N, int H, int Hkv, int D, const uint16_t* q,
+                         const uint16_t* k, const uint16_t* v, const float* slopes, const int32_t* rows,
+                         int nrows, double* out) {
+    if (BS <= 0 || N <= 0 || H <= 0 || Hkv <= 0 || H % Hkv || D <= 0) return -1;
+    int group = H / Hkv, fail = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int ir = 0; ir < nrows; ++ir) {
+        int b = rows[3 * ir], i = rows[3 * ir + 1], h = rows[3 * ir + 2];
+        if (b < 0 || b >= BS || i < 0 || i >= N || h < 0 || h >= H) { fail = 1; continue; }
+        int kvh = h / group, L = i + 1;
+        double* sc = (double*)malloc(sizeof(double) * (size_t)L);
+        double inv = 1.0 / sqrt((double)D), mx = -INFINITY;
+        for (int j = 0; j < L; ++j) {
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d)
+                dot += widen(dtype, q[(((long)b * N + i) * H + h) * D + d]) *
+                       widen(dtype, k[(((long)b * N + j) * Hkv + kvh) * D + d]);
+            double s = dot * inv;
+            if (slopes) s += (double)slopes[h] * (double)(j - i);
+            sc[j] = s;
+            if (s > mx) mx = s;
+        }
+        double den = 0.0;
+        for (int j = 0; j < L; ++j) { sc[j] = exp(sc[j] - mx); den += sc[j]; }
+        for (int d = 0; d < D; ++d) {
+            double acc = 0.0;
+            for (int j = 0; j < L; ++j) acc += sc[j] / den * widen(dtype, v[(((long)b * N + j) * Hkv + kvh) * D + d]);
+            out[(long)ir * D + d] = acc;
+        }
+        free(sc);
+    }
+    return fail ? -1 : 0;
+}
+
+/*
  * KV-cache sizes in bytes (Section 3.2).  Eq. 1: one token's K and V over all
  * layers.  Eq. 2: the standard contiguous cache, prompt copied per beam.
  * Eq. 3: the segment cache, prompt once per request, response capacity grown

@@ -386,3 +386,43 @@ def test_oracle_rejects_global_parent_ids():
     par = np.array([[0, 1, 0, 1], [0, 1, 2, 3], [0, 0, 0, 0]], dtype=np.int32)
     with pytest.raises(ValueError):
         oracle.ancestry(par, B, W, T - 1)
+
+
+# ------------------------------------------------------------------ prefill
+def test_prefill_equals_textbook_causal_attention():
+    B, N, H, Hkv, D = 2, 9, 4, 2, 16
+    for dtype, name in ((torch.float16, "f16"), (torch.bfloat16, "bf16")):
+        q = draw((B, N, H, D), dtype, 201); k = draw((B, N, Hkv, D), dtype, 202); v = draw((B, N, Hkv, D), dtype, 203)
+        slopes = np.array([0.5, 0.25, 0.125, 0.0625], np.float32)
+        for sl in (None, slopes):
+            got = oracle.prefill_sdpa(name, B, H, Hkv, D, bits(q), bits(k), bits(v), slopes=sl)
+            for b in range(B):
+                for h in range(H):
+                    S = f64(q)[b, :, h] @ f64(k)[b, :, h // (H // Hkv)].T / np.sqrt(D)
+                    if sl is not None:
+                        S = S + float(sl[h]) * (np.arange(N)[None, :] - np.arange(N)[:, None])
+                    S[np.triu_indices(N, k=1)] = -np.inf
+                    np.testing.assert_allclose(got[b, :, h], softmax_rows(S) @ f64(v)[b, :, h // (H // Hkv)],
+                                               rtol=1e-12, atol=1e-13)
+
+
+def test_prefill_row_is_the_decode_oracle_on_the_prefix():
+    """Prefill position i = decode attention of one beam over the first i+1 prompt keys (the paper
+    calls the prefill kernel the special case of the decode kernel), incl. the ALiBi convention."""
+    B, N, H, Hkv, D = 2, 7, 2, 1, 8
+    q = draw((B, N, H, D), torch.float16, 211); k = draw((B, N, Hkv, D), torch.float16, 212)
+    v = draw((B, N, Hkv, D), torch.float16, 213)
+    slopes = np.array([0.3, 0.7], np.float32)
+    got = oracle.prefill_sdpa("f16", B, H, Hkv, D, bits(q), bits(k), bits(v), slopes=slopes)
+    for i in (0, 3, N - 1):
+        dec = oracle.decode_sdpa("f16", B, 1, H, Hkv, D, bits(q[:, i].contiguous()), bits(k[:, :i + 1].contiguous()),
+                                 bits(v[:, :i + 1].contiguous()), None, None, None, -1, slopes=slopes)
+        np.testing.assert_allclose(got[:, i], dec, rtol=1e-12, atol=1e-13)
+
+
+def test_prefill_first_position_returns_its_own_value():
+    B, N, H, Hkv, D = 1, 5, 2, 2, 8
+    q = draw((B, N, H, D), torch.float16, 221); k = draw((B, N, Hkv, D), torch.float16, 222)
+    v = draw((B, N, Hkv, D), torch.float16, 223)
+    got = oracle.prefill_sdpa("f16", B, H, Hkv, D, bits(q), bits(k), bits(v), rows=[(0, 0, 0), (0, 0, 1)])
+    np.testing.assert_allclose(got, f64(v)[0, 0], rtol=0, atol=1e-15)
