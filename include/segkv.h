@@ -111,6 +111,23 @@ SEGKV_API int segkv_destroy(segkv_t h);
 SEGKV_API int segkv_prefill_write(segkv_t h, const void* k, const void* v, int prompt_len, void* stream);
 
 /*
+ * Prefill attention (Section 3.1: at prefill Query_0/Key_0/Value_0 arrive batch-first and the
+ * customised SDPA kernel takes and returns that layout; Section 3.3: it is the special case of
+ * the decode kernel that sees only query and prompt key/value).  Causal self-attention of every
+ * prompt position over the positions up to itself, K/V read from the prompt segment that
+ * segkv_prefill_write has stored:
+ *     out[b,i,hd,:] = softmax_{j<=i}(q[b,i,hd,:] . K[b,j,:] / sqrt(head_dim) + bias) . V[b,j,:]
+ *   q, out: device [batch, prompt_len, heads, head_dim] (token-major, like k and v of the write);
+ *   alibi_slopes: device float [heads] or NULL; bias = slope[hd] * (j - i).
+ * fp16/bf16 operands, fp32 scores/softmax/accumulation, output rounded to nearest-even.
+ * Errors: EINVAL (also head_dim 256, which this kernel does not take), ESTATE (no prompt
+ * stored), ECUDA.  segkv_prefill is segkv_prefill_write followed by segkv_prefill_sdpa.
+ */
+SEGKV_API int segkv_prefill_sdpa(segkv_t h, const void* q, void* out, const float* alibi_slopes, void* stream);
+SEGKV_API int segkv_prefill(segkv_t h, const void* k, const void* v, const void* q, void* out, int prompt_len,
+                            const float* alibi_slopes, void* stream);
+
+/*
  * Decode step `step` (0-based), before its attention call: write the step's
  * new K/V rows into slab `step` of the response segment (Section 3.1: Key_t,
  * Value_t kept in place in the pre-allocated buffer), record the beam parents

@@ -369,6 +369,26 @@ int segkv_prefill_write(segkv_t h, const void* k, const void* v, int prompt_len,
     return SEGKV_OK;
 }
 
+int segkv_prefill_sdpa(segkv_t h, const void* q, void* out, const float* alibi_slopes, void* stream) {
+    if (!h || !q || !out || !aligned16(q) || !aligned16(out)) return SEGKV_EINVAL;
+    if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SEGKV_EINVAL;
+    if (h->prompt_len <= 0 || !h->tm_valid) return SEGKV_ESTATE;
+    if (!prefill_sdpa_supported(h->d)) return SEGKV_EINVAL;
+    PrefillArgs a;
+    a.q = q; a.out = out; a.slopes = alibi_slopes; a.err_word = h->err_word;
+    a.prompt_len = h->prompt_len; a.tm_k = &h->tm_kp; a.tm_v = &h->tm_vp;
+    SEGKV_CUDA(launch_prefill_sdpa(h->d, a, (cudaStream_t)stream));
+    h->launches++;
+    return SEGKV_OK;
+}
+
+int segkv_prefill(segkv_t h, const void* k, const void* v, const void* q, void* out, int prompt_len,
+                  const float* alibi_slopes, void* stream) {
+    int rc = segkv_prefill_write(h, k, v, prompt_len, stream);
+    if (rc != SEGKV_OK) return rc;
+    return segkv_prefill_sdpa(h, q, out, alibi_slopes, stream);
+}
+
 int segkv_append(segkv_t h, int step, const int32_t* beam_parent, const void* k_new, const void* v_new,
                  void* stream) {
     if (!h || step < 0 || !k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return SEGKV_EINVAL;

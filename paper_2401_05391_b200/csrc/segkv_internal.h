@@ -137,4 +137,17 @@ size_t tiled_static_scratch_bytes();
 cudaError_t launch_sdpa_tiled_static(const Dims& d, SdpaArgs a, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                      int stages, cudaStream_t st, int* too_big);
 
+// Causal prefill attention over the prompt segment (tile rows must be 64: head_dim 64 or 128).
+struct PrefillArgs {
+    const void* q;
+    void* out;
+    const float* slopes;
+    int* err_word;
+    int prompt_len;
+    const CUtensorMap* tm_k;
+    const CUtensorMap* tm_v;
+};
+bool prefill_sdpa_supported(const Dims& d);
+cudaError_t launch_prefill_sdpa(const Dims& d, const PrefillArgs& a, cudaStream_t st);
+
 }  // namespace segkv_impl

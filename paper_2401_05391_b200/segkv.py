@@ -31,6 +31,8 @@ SIGNATURES = {
     "segkv_allocated_kv_bytes": (ctypes.c_longlong, [_vp]),
     "segkv_destroy": (_int, [_vp]),
     "segkv_prefill_write": (_int, [_vp, _vp, _vp, _int, _vp]),
+    "segkv_prefill_sdpa": (_int, [_vp, _vp, _vp, _vp, _vp]),
+    "segkv_prefill": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _vp]),
     "segkv_append": (_int, [_vp, _int, _vp, _vp, _vp, _vp]),
     "segkv_decode_sdpa": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "segkv_decode_step": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -162,6 +164,29 @@ class SegKV:
         shape = (self.batch, p, self.kv_heads, self.head_dim)
         _check(lib().segkv_prefill_write(self._h, _dev(k, shape, self.dtype, "k"), _dev(v, shape, self.dtype, "v"),
                                          p, _stream_ptr(stream)), "segkv_prefill_write")
+
+    def prefill_sdpa(self, q: torch.Tensor, out: Optional[torch.Tensor] = None,
+                     alibi_slopes: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        shape = (self.batch, self.prompt_len, self.heads, self.head_dim)
+        if out is None:
+            out = torch.empty(shape, dtype=self.dtype, device=q.device)
+        _check(lib().segkv_prefill_sdpa(self._h, _dev(q, shape, self.dtype, "q"), _dev(out, shape, self.dtype, "out"),
+                                        _dev(alibi_slopes, (self.heads,), torch.float32, "alibi_slopes"),
+                                        _stream_ptr(stream)), "segkv_prefill_sdpa")
+        return out
+
+    def prefill(self, k: torch.Tensor, v: torch.Tensor, q: torch.Tensor, out: Optional[torch.Tensor] = None,
+                alibi_slopes: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        p = int(k.shape[1])
+        kv = (self.batch, p, self.kv_heads, self.head_dim)
+        qs = (self.batch, p, self.heads, self.head_dim)
+        if out is None:
+            out = torch.empty(qs, dtype=self.dtype, device=q.device)
+        _check(lib().segkv_prefill(self._h, _dev(k, kv, self.dtype, "k"), _dev(v, kv, self.dtype, "v"),
+                                   _dev(q, qs, self.dtype, "q"), _dev(out, qs, self.dtype, "out"), p,
+                                   _dev(alibi_slopes, (self.heads,), torch.float32, "alibi_slopes"),
+                                   _stream_ptr(stream)), "segkv_prefill")
+        return out
 
     def append(self, step: int, beam_parent: Optional[torch.Tensor], k_new: torch.Tensor, v_new: torch.Tensor,
                stream=None) -> None:

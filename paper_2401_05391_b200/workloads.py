@@ -124,6 +124,12 @@ def make_prompt(w: Workload, device="cpu", prompt_len: Optional[int] = None):
             _normal(shape, w, device, w.seed * 1000 + 2))
 
 
+def make_prefill_query(w: Workload, device="cpu", prompt_len: Optional[int] = None) -> torch.Tensor:
+    """Prefill queries, token-major ``[batch, prompt_len, heads, head_dim]``."""
+    p = w.prompt_len if prompt_len is None else prompt_len
+    return _normal((w.batch, p, w.heads, w.head_dim), w, device, w.seed * 1000 + 3)
+
+
 def make_step(w: Workload, step: int, device="cpu"):
     """Step ``step``'s q ``[rows, heads, D]`` and new k, v ``[rows, kv_heads, D]``.
 

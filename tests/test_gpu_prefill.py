@@ -1,0 +1,106 @@
+"""GPU parity of the prefill attention against the CPU oracle, through the C-ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2401_05391_b200 import segkv as sk
+from paper_2401_05391_b200 import workloads as wl
+
+from _harness import ATOL, RTOL
+
+pytestmark = pytest.mark.gpu
+
+
+def check_rows(w, q, kp, vp, out, slopes, rows):
+    ref = oracle.prefill_sdpa(w.dtype, w.batch, w.heads, w.kv_heads, w.head_dim, wl.to_bits(q), wl.to_bits(kp),
+                              wl.to_bits(vp), slopes=None if slopes is None else slopes.cpu().numpy(), rows=rows)
+    got = np.stack([out[b, i, h].to(torch.float64).cpu().numpy() for b, i, h in rows])
+    assert np.isfinite(got).all()
+    err = np.abs(got - ref)
+    # The stated tolerance, plus for bf16 the bound of rounding the softmax weights to 8 mantissa
+    # bits before P.V: sum_j p_j * 2^-9 * |v_j| <= 2^-9 * max|v|.  It only shows on the first rows,
+    # where one or two keys carry all the weight and their values can cancel in the reference.
+    atol = ATOL + (2.0 ** -9 * float(vp.abs().max()) if w.dtype == "bf16" else 0.0)
+    assert (err <= atol + RTOL * np.abs(ref)).all(), f"max err {err.max():.3e}"
+
+
+def run_prefill(w, rows_fn):
+    h = sk.SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, w.steps, w.torch_dtype)
+    try:
+        kp, vp = wl.make_prompt(w, "cuda")
+        q = wl.make_prefill_query(w, "cuda")
+        slopes = wl.alibi_slopes(w.heads).cuda() if w.alibi else None
+        out = torch.full_like(q, float("nan"))
+        h.prefill(kp, vp, q, out, slopes)
+        torch.cuda.synchronize()
+        assert not torch.isnan(out.float()).any(), "unwritten outputs"
+        check_rows(w, q, kp, vp, out, slopes, rows_fn(w))
+        assert h.get_error() == 0
+        return h, q, kp, vp, out, slopes
+    except Exception:
+        h.destroy()
+        raise
+
+
+def all_rows(w):
+    return [(b, i, h) for b in range(w.batch) for i in range(w.prompt_len) for h in range(w.heads)]
+
+
+def sampled_rows(w, n=192, seed=0):
+    rng = np.random.default_rng(w.seed + seed)
+    rows = {(0, 0, 0), (w.batch - 1, w.prompt_len - 1, w.heads - 1), (0, 63, 0), (0, 64, 0), (0, w.prompt_len - 1, 0)}
+    while len(rows) < n:
+        rows.add((int(rng.integers(w.batch)), int(rng.integers(w.prompt_len)), int(rng.integers(w.heads))))
+    return sorted(r for r in rows if r[1] < w.prompt_len)
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("D,P", [(64, 150), (128, 150), (128, 64), (128, 65), (64, 1)])
+def test_prefill_ragged_small_shapes(dtype, D, P):
+    # several tiles and a ragged tail, GQA, ALiBi on the bf16 variants
+    w = wl.Workload("pf", 2, 3, 6, 2, D, P, 2, dtype, "uniform", dtype == "bf16", 80 + D // 64)
+    h = run_prefill(w, all_rows)[0]
+    h.destroy()
+
+
+def test_prefill_llama2_7b_shape_sampled():
+    h = run_prefill(wl.CONFIGS[1], lambda w: sampled_rows(w, 256))[0]
+    h.destroy()
+
+
+def test_prefill_bloom_shape_cut_to_batch_2_sampled():
+    h = run_prefill(wl.CONFIGS[4].scaled(batch=2), lambda w: sampled_rows(w, 256))[0]
+    h.destroy()
+
+
+def test_prefill_last_row_agrees_with_the_decode_kernel_on_the_prompt():
+    """The prefill kernel is the decode kernel's special case: its last row is what the decode
+    kernel returns for a query that sees only the prompt."""
+    w = wl.Workload("pfdec", 2, 4, 4, 2, 128, 200, 2, "f16", "uniform", True, 83)
+    h, q, kp, vp, out, slopes = run_prefill(w, lambda w: sampled_rows(w, 64))
+    try:
+        qd = q[:, -1].repeat_interleave(w.beams, dim=0).contiguous()        # [rows, heads, D]
+        od = h.decode_sdpa(qd, None, slopes)
+        torch.cuda.synchronize()
+        want = out[:, -1].repeat_interleave(w.beams, dim=0)
+        assert torch.allclose(od.float(), want.float(), atol=2e-3, rtol=1e-2)
+    finally:
+        h.destroy()
+
+
+def test_prefill_argument_and_state_errors():
+    h = sk.SegKV(1, 2, 2, 2, 256, 16, 4, torch.float16)
+    q = torch.zeros(1, 16, 2, 256, dtype=torch.float16, device="cuda")
+    kv = torch.zeros(1, 16, 2, 256, dtype=torch.float16, device="cuda")
+    with pytest.raises(sk.SegKVError) as e:
+        h.prefill(kv, kv, q)
+    assert e.value.code == sk.SEGKV_EINVAL                   # head_dim 256 is not taken
+    h.destroy()
+    h = sk.SegKV(1, 2, 2, 2, 64, 16, 4, torch.float16)
+    with pytest.raises(sk.SegKVError) as e:
+        lib = sk.lib()
+        rc = lib.segkv_prefill_sdpa(h._h, q.data_ptr(), q.data_ptr(), None, None)
+        sk._check(rc, "segkv_prefill_sdpa")
+    assert e.value.code == sk.SEGKV_ESTATE                   # no prompt stored yet
+    h.destroy()
