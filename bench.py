@@ -49,6 +49,7 @@ def parse():
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--combine", type=int, default=0, help="0 auto, 1 workspace+ticket, 2 cluster")
+    ap.add_argument("--prefill", action="store_true", help="time the prefill attention instead of the decode step")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="turn programmatic dependent launch off")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -398,8 +399,63 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_prefill(args):
+    """Prefill attention of the workload's prompt (one JSON line of its own; tensor-core bound)."""
+    import torch
+    from paper_2401_05391_b200 import workloads as wl
+    from paper_2401_05391_b200.segkv import SegKV
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    w = wl.by_name(args.workload)
+    if args.batch:
+        w = w.scaled(batch=args.batch, name=f"{w.name}[batch={args.batch}]")
+    L = args.layers or DEFAULT_LAYERS.get(w.name.split("[")[0], 1)
+    handles = []
+    for layer in range(L):
+        wl_layer = w.scaled(index=w.index + 1000 * layer)
+        h = SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, 1, w.torch_dtype)
+        kp, vp = wl.make_prompt(wl_layer, dev)
+        h.prefill_write(kp, vp)
+        del kp, vp
+        q = wl.make_prefill_query(wl_layer, dev)
+        handles.append((h, q, torch.empty_like(q)))
+    slopes = wl.alibi_slopes(w.heads).to(dev) if w.alibi else None
+    stream = torch.cuda.Stream()
+
+    def one_pass():
+        for h, q, o in handles:
+            h.prefill_sdpa(q, o, slopes, stream=stream)
+    for _ in range(max(3, args.warmup)):
+        one_pass()
+    stream.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        one_pass()
+    e1.record(stream)
+    stream.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps / L
+    n = w.prompt_len
+    flops = 4.0 * w.head_dim * (n * (n + 1) / 2) * w.batch * w.heads          # causal: only the visible keys
+    tflops = flops / (ms * 1e-3) / 1e12
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak, kind = (float(json.load(open(path))["bf16_tflops"]), "measured") if os.path.exists(path) else (1590.0, "fallback")
+    print(json.dumps({
+        "metric": "prefill_sdpa_causal_tflops", "value": tflops, "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "dtype": w.dtype,
+        "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.batch, "heads": w.heads, "kv_heads": w.kv_heads,
+                   "head_dim": w.head_dim, "prompt_len": n, "layers_rotated": L},
+        "roofline": {"bound": "tensor", "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak,
+                     "traffic": None, "peak_kind": f"of {kind} (bf16 GEMM burst; fp16 has the same nominal rate)",
+                     "kernel": "segkv prefill attention (mma.sync m16n8k16)"},
+        "gpu_launches": args.steps * L}))
+
+
 def main():
     args = parse()
+    if args.prefill and args.impl != "reference":
+        return run_prefill(args)
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -14,7 +14,7 @@ namespace {
 thread_local char g_cuda_err[256] = "";
 
 int cuda_fail(cudaError_t e, const char* what) {
-    snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s (%s)", what, cudaGetErrorName(e), cudaGetErrorString(e));
+    snprintf(g_cuda_err, sizeof g_cuda_err, "%.120s: %.40s (%.80s)", what, cudaGetErrorName(e), cudaGetErrorString(e));
     return e == cudaErrorMemoryAllocation ? SEGKV_ENOMEM : SEGKV_ECUDA;
 }
 

@@ -4,8 +4,8 @@
 //     out[b,i,h,:] = softmax_{j<=i}( q[b,i,h,:] . K[b,j,:] / sqrt(D) + bias ) . V[b,j,:],
 // with K/V read from the head-major prompt segment that segkv_prefill_write has just stored.
 //
-// Dense work, so it is laid out as a flash-attention forward: a CTA owns 64 query rows of one
-// (request, head), four consumer warps take 16 rows each, a producer warp streams 64-key K/V
+// Dense work, so it is laid out as a flash-attention forward: a CTA owns 128 query rows of one
+// (request, head), eight consumer warps take 16 rows each, a producer warp streams 64-key K/V
 // tiles through a TMA-fed, 128-byte-swizzled shared-memory ring (the same tensor maps and tile
 // layout as the decode kernel).  S = Q.K^T and O += P.V run on tensor cores (mma.sync
 // m16n8k16, fp32 accumulate; Q fragments stay in registers, P is re-used as the A operand
@@ -29,7 +29,8 @@ struct PrefillParams {
     float scale2;        // log2(e) / sqrt(D)
 };
 
-constexpr int kBM = 64;  // query rows per CTA
+constexpr int kPW = 8;             // consumer warps
+constexpr int kBM = 16 * kPW;  // query rows per CTA
 constexpr int kBN = 64;  // keys per tile
 
 template <int D>
@@ -41,7 +42,7 @@ struct PrefillLayout {
 };
 
 template <typename T, int D>
-__global__ void __launch_bounds__(160, 1)
+__global__ void __launch_bounds__(32 * (kPW + 1), 1)
 prefill_sdpa_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                     const PrefillParams p) {
     using L = PrefillLayout<D>;
@@ -59,12 +60,12 @@ prefill_sdpa_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     const int h = blockIdx.y, b = blockIdx.z;
     const int kvh = h / p.G;
     const int slab = b * p.Hkv + kvh;
-    const int nkt = qt + 1;                                      // causal: key tiles 0..qt
+    const int nkt = min((p.N + kBN - 1) / kBN, ((qt + 1) * kBM + kBN - 1) / kBN);   // causal: tiles up to the CTA's last row
 
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(full0 + 8 * s, 1);
-            mbar_init(empty0 + 8 * s, 4);
+            mbar_init(empty0 + 8 * s, kPW);
         }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -72,7 +73,7 @@ prefill_sdpa_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     }
     __syncthreads();
 
-    if (warp == 4) {
+    if (warp == kPW) {
         // ------------------------------- producer warp -------------------------------
         if (lane == 0) {
             prefetch_tmap(&tm_k);
@@ -129,6 +130,12 @@ prefill_sdpa_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         if (!ok) break;
         const uint32_t k_src = smem_u32(smem + (size_t)st * L::STAGE_BYTES);
         const uint32_t v_src = k_src + L::TILE_BYTES;
+        const int wrow_lo = qt * kBM + warp * 16;                // this warp's rows: wrow_lo .. wrow_lo + 15
+        if (kt * kBN > wrow_lo + 15) {                           // tile entirely above the diagonal for this warp
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8 * st);
+            continue;
+        }
         auto chunk_addr = [&](uint32_t base, int key, int ch) -> uint32_t {
             return base + (uint32_t)(ch >> 3) * L::BOX_BYTES + (uint32_t)key * 128 + (uint32_t)(((ch & 7) ^ (key & 7)) << 4);
         };
@@ -152,18 +159,30 @@ prefill_sdpa_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         }
         // ---- scale, ALiBi, causal mask (diagonal tile only), online softmax ----
         const int key0 = kt * kBN + (lane & 3) * 2;              // key of sc[nt][0] is key0 + 8*nt
-        const bool diag = kt == qt;
+        const bool diag = kt * kBN + kBN - 1 > wrow_lo;          // some key of the tile is above some row of the warp
         float tmax[2] = {-INFINITY, -INFINITY};
+        if (diag || p.slopes) {
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
+            for (int nt = 0; nt < 8; ++nt) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int key = key0 + 8 * nt + (i & 1);
-                const int row = (i & 2) ? row1 : row0;
-                float v = sc[nt][i] * p.scale2 + slope2 * (float)(key - row);
-                if (diag && key > row) v = -INFINITY;
-                sc[nt][i] = v;
-                tmax[i >> 1] = fmaxf(tmax[i >> 1], v);
+                for (int i = 0; i < 4; ++i) {
+                    const int key = key0 + 8 * nt + (i & 1);
+                    const int row = (i & 2) ? row1 : row0;
+                    float v = sc[nt][i] * p.scale2 + slope2 * (float)(key - row);
+                    if (diag && key > row) v = -INFINITY;
+                    sc[nt][i] = v;
+                    tmax[i >> 1] = fmaxf(tmax[i >> 1], v);
+                }
+            }
+        } else {                                                 // the common tile: scale only
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float v = sc[nt][i] * p.scale2;
+                    sc[nt][i] = v;
+                    tmax[i >> 1] = fmaxf(tmax[i >> 1], v);
+                }
             }
         }
         float alpha[2];
@@ -188,12 +207,14 @@ prefill_sdpa_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         }
         l_run[0] = l_run[0] * alpha[0] + lsum[0];
         l_run[1] = l_run[1] * alpha[1] + lsum[1];
+        if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {
 #pragma unroll
-        for (int dt = 0; dt < DT; ++dt) {
-            o_acc[dt][0] *= alpha[0];
-            o_acc[dt][1] *= alpha[0];
-            o_acc[dt][2] *= alpha[1];
-            o_acc[dt][3] *= alpha[1];
+            for (int dt = 0; dt < DT; ++dt) {
+                o_acc[dt][0] *= alpha[0];
+                o_acc[dt][1] *= alpha[0];
+                o_acc[dt][2] *= alpha[1];
+                o_acc[dt][3] *= alpha[1];
+            }
         }
         // ---- O[16 rows, D] += P . V, P taken from the score accumulators as the A operand ----
         {
@@ -263,7 +284,7 @@ cudaError_t launch_prefill(const Dims& d, const PrefillArgs& a, cudaStream_t st)
     p.N = a.prompt_len; p.H = d.heads; p.Hkv = d.kv_heads; p.G = d.group; p.stages = stages;
     p.scale2 = 1.4426950408889634f / sqrtf((float)D);
     dim3 grid((unsigned)((a.prompt_len + kBM - 1) / kBM), (unsigned)d.heads, (unsigned)d.batch);
-    kern<<<grid, 160, smem, st>>>(*a.tm_k, *a.tm_v, p);
+    kern<<<grid, 32 * (kPW + 1), smem, st>>>(*a.tm_k, *a.tm_v, p);
     return cudaGetLastError();
 }
 
