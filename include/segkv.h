@@ -120,8 +120,7 @@ SEGKV_API int segkv_prefill_write(segkv_t h, const void* k, const void* v, int p
  *   q, out: device [batch, prompt_len, heads, head_dim] (token-major, like k and v of the write);
  *   alibi_slopes: device float [heads] or NULL; bias = slope[hd] * (j - i).
  * fp16/bf16 operands, fp32 scores/softmax/accumulation, output rounded to nearest-even.
- * Errors: EINVAL (also head_dim 256, which this kernel does not take), ESTATE (no prompt
- * stored), ECUDA.  segkv_prefill is segkv_prefill_write followed by segkv_prefill_sdpa.
+ * Errors: EINVAL, ESTATE (no prompt stored), ECUDA.  segkv_prefill is segkv_prefill_write followed by segkv_prefill_sdpa.
  */
 SEGKV_API int segkv_prefill_sdpa(segkv_t h, const void* q, void* out, const float* alibi_slopes, void* stream);
 SEGKV_API int segkv_prefill(segkv_t h, const void* k, const void* v, const void* q, void* out, int prompt_len,

@@ -56,7 +56,7 @@ def sampled_rows(w, n=192, seed=0):
 
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
-@pytest.mark.parametrize("D,P", [(64, 150), (128, 150), (128, 64), (128, 65), (64, 1)])
+@pytest.mark.parametrize("D,P", [(64, 150), (128, 150), (128, 64), (128, 65), (64, 1), (256, 150), (256, 33), (128, 300)])
 def test_prefill_ragged_small_shapes(dtype, D, P):
     # several tiles and a ragged tail, GQA, ALiBi on the bf16 variants
     w = wl.Workload("pf", 2, 3, 6, 2, D, P, 2, dtype, "uniform", dtype == "bf16", 80 + D // 64)
@@ -66,6 +66,11 @@ def test_prefill_ragged_small_shapes(dtype, D, P):
 
 def test_prefill_llama2_7b_shape_sampled():
     h = run_prefill(wl.CONFIGS[1], lambda w: sampled_rows(w, 256))[0]
+    h.destroy()
+
+
+def test_prefill_gptj_shape_cut_to_batch_2_sampled():
+    h = run_prefill(wl.CONFIGS[2].scaled(batch=2), lambda w: sampled_rows(w, 256))[0]
     h.destroy()
 
 
@@ -90,17 +95,12 @@ def test_prefill_last_row_agrees_with_the_decode_kernel_on_the_prompt():
 
 
 def test_prefill_argument_and_state_errors():
-    h = sk.SegKV(1, 2, 2, 2, 256, 16, 4, torch.float16)
-    q = torch.zeros(1, 16, 2, 256, dtype=torch.float16, device="cuda")
-    kv = torch.zeros(1, 16, 2, 256, dtype=torch.float16, device="cuda")
-    with pytest.raises(sk.SegKVError) as e:
-        h.prefill(kv, kv, q)
-    assert e.value.code == sk.SEGKV_EINVAL                   # head_dim 256 is not taken
-    h.destroy()
     h = sk.SegKV(1, 2, 2, 2, 64, 16, 4, torch.float16)
+    q = torch.zeros(1, 16, 2, 64, dtype=torch.float16, device="cuda")
     with pytest.raises(sk.SegKVError) as e:
-        lib = sk.lib()
-        rc = lib.segkv_prefill_sdpa(h._h, q.data_ptr(), q.data_ptr(), None, None)
+        rc = sk.lib().segkv_prefill_sdpa(h._h, q.data_ptr(), q.data_ptr(), None, None)
         sk._check(rc, "segkv_prefill_sdpa")
     assert e.value.code == sk.SEGKV_ESTATE                   # no prompt stored yet
+    rc = sk.lib().segkv_prefill_sdpa(h._h, None, q.data_ptr(), None, None)
+    assert rc == sk.SEGKV_EINVAL
     h.destroy()
