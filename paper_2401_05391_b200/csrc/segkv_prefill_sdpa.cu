@@ -46,7 +46,7 @@ struct PrefillLayout {
 };
 
 template <typename T, int D, int kPW, int kBN, bool QSMEM>
-__global__ void __launch_bounds__(32 * (kPW + 1), 1)
+__global__ void __launch_bounds__(32 * (kPW + 1), (kPW <= 4 && D <= 128) ? 2 : 1)
 prefill_sdpa_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                     const PrefillParams p) {
     using L = PrefillLayout<D, kPW, kBN, QSMEM>;
@@ -325,11 +325,11 @@ cudaError_t launch_prefill_sdpa(const Dims& d, const PrefillArgs& a, cudaStream_
     const bool bf = d.dtype == SEGKV_BF16;
     switch (d.head_dim) {
         case 64:
-            return bf ? launch_prefill<__nv_bfloat16, 64, 8, 64, false>(d, a, st)
-                      : launch_prefill<__half, 64, 8, 64, false>(d, a, st);
+            return bf ? launch_prefill<__nv_bfloat16, 64, 4, 64, false>(d, a, st)
+                      : launch_prefill<__half, 64, 4, 64, false>(d, a, st);
         case 128:
-            return bf ? launch_prefill<__nv_bfloat16, 128, 8, 64, false>(d, a, st)
-                      : launch_prefill<__half, 128, 8, 64, false>(d, a, st);
+            return bf ? launch_prefill<__nv_bfloat16, 128, 4, 64, false>(d, a, st)
+                      : launch_prefill<__half, 128, 4, 64, false>(d, a, st);
         case 256:   // 32-key tiles (the prompt segment's box for this head size), Q staged in shared memory
             return bf ? launch_prefill<__nv_bfloat16, 256, 4, 32, true>(d, a, st)
                       : launch_prefill<__half, 256, 4, 32, true>(d, a, st);
