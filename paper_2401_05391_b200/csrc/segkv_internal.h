@@ -149,5 +149,8 @@ struct PrefillArgs {
 };
 bool prefill_sdpa_supported(const Dims& d);
 cudaError_t launch_prefill_sdpa(const Dims& d, const PrefillArgs& a, cudaStream_t st);
+// the same operation on tcgen05 tensor cores with TMEM accumulators (head_dim 128)
+bool prefill_tc5_supported(const Dims& d);
+cudaError_t launch_prefill_tc5(const Dims& d, const PrefillArgs& a, cudaStream_t st);
 
 }  // namespace segkv_impl

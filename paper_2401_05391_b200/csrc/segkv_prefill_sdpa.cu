@@ -322,6 +322,7 @@ cudaError_t launch_prefill(const Dims& d, const PrefillArgs& a, cudaStream_t st)
 bool prefill_sdpa_supported(const Dims& d) { return d.head_dim == 64 || d.head_dim == 128 || d.head_dim == 256; }
 
 cudaError_t launch_prefill_sdpa(const Dims& d, const PrefillArgs& a, cudaStream_t st) {
+    if (prefill_tc5_supported(d)) return launch_prefill_tc5(d, a, st);
     const bool bf = d.dtype == SEGKV_BF16;
     switch (d.head_dim) {
         case 64:
