@@ -287,6 +287,16 @@ SEGKV_API int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, con
  */
 SEGKV_API int segkv_set_overlap(segkv_t h, int enable);
 
+/*
+ * Override the CTA shape of the prefill attention kernel for head_dim 128
+ * (the tcgen05 kernel): `row_groups` = groups of 128 query rows that one CTA
+ * works on side by side (1 or 2; each group has its own softmax warps and
+ * tensor-memory accumulators, all share the K/V tile ring).  0 = choose from
+ * the grid size (the default).  EINVAL for any other value.  Other head sizes
+ * ignore it.  A launch-shape knob: the paper has no counterpart.
+ */
+SEGKV_API int segkv_set_prefill_tuning(segkv_t h, int row_groups);
+
 /* Kernels launched by the handle since creation (each launch counted once). */
 SEGKV_API long long segkv_launch_count(segkv_t h);
 

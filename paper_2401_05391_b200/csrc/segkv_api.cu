@@ -288,6 +288,7 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
     d.rows = batch * beams; d.dtype = dtype; d.chunk_steps = chunk_steps;
     h->prompt_len = -1;
     h->overlap = true;
+    h->prefill_groups = 0;
 
     int rc = SEGKV_OK;
     auto fail = [&](int code) { free_all(h); delete h; return code; };
@@ -377,6 +378,7 @@ int segkv_prefill_sdpa(segkv_t h, const void* q, void* out, const float* alibi_s
     PrefillArgs a;
     a.q = q; a.out = out; a.slopes = alibi_slopes; a.err_word = h->err_word;
     a.prompt_len = h->prompt_len; a.tm_k = &h->tm_kp; a.tm_v = &h->tm_vp;
+    a.row_groups = h->prefill_groups;
     SEGKV_CUDA(launch_prefill_sdpa(h->d, a, (cudaStream_t)stream));
     h->launches++;
     return SEGKV_OK;
@@ -663,6 +665,12 @@ int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, const float* 
 int segkv_set_overlap(segkv_t h, int enable) {
     if (!h) return SEGKV_EINVAL;
     h->overlap = enable != 0;
+    return SEGKV_OK;
+}
+
+int segkv_set_prefill_tuning(segkv_t h, int row_groups) {
+    if (!h || row_groups < 0 || row_groups > 2) return SEGKV_EINVAL;
+    h->prefill_groups = row_groups;
     return SEGKV_OK;
 }
 

@@ -45,6 +45,7 @@ struct segkv {
     int stages_forced;   // 0 = automatic
     int combine_forced;  // 0 = automatic, 1 = global workspace + ticket, 2 = cluster
     bool overlap;        // programmatic dependent launch between consecutive kernels
+    int prefill_groups;  // 0 = automatic; 1 or 2 row groups per CTA of the tcgen05 prefill kernel
     bool fuse_always;    // segkv_decode_step uses the fused kernel even for a single split
     long long launches;
     // device storage (owned)
@@ -146,6 +147,7 @@ struct PrefillArgs {
     int prompt_len;
     const CUtensorMap* tm_k;
     const CUtensorMap* tm_v;
+    int row_groups;      // 0 = automatic
 };
 bool prefill_sdpa_supported(const Dims& d);
 cudaError_t launch_prefill_sdpa(const Dims& d, const PrefillArgs& a, cudaStream_t st);

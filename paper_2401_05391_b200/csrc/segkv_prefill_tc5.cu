@@ -3,22 +3,29 @@
 // Same operation as segkv_prefill_sdpa.cu (paper Section 3.1 / 3.3: causal attention of the
 // prompt, batch-first in and out, K/V from the prompt segment), laid out for tcgen05:
 //
-//   * a CTA owns 128 query rows of one (request, head): one row per TMEM lane;
-//   * Q [128 x 128] is staged once in shared memory in the 128-byte-swizzled K-major layout,
-//     K/V tiles of 64 keys arrive by TMA in the same layout (the prompt segment's tensor maps);
-//   * one elected thread issues the MMAs: S = Q.K^T (M 128, N 64, eight K-steps of 16) into one
-//     of two 64-column TMEM buffers, and O += P.V (M 128, N 128, four K-steps) into a 128-column
-//     TMEM accumulator; V is consumed as an MN-major B operand straight from its row-major tile;
-//   * four softmax warps own one row per thread: they read S with tcgen05.ld (no shuffles for
-//     the row max / sum), write P as bf16/fp16 into a swizzled shared-memory tile that the next
-//     MMA takes as its A operand, and rescale O in tensor memory only when a row's maximum has
-//     grown by more than 2^8 since the reference it is using (the sum uses the same reference,
-//     so the result is exact);
-//   * S is double-buffered, so Q.K^T of tile j+1 runs under the softmax of tile j and P.V of
-//     tile j under the softmax of tile j+1.
+//   * a CTA owns one or two groups of 128 query rows of one (request, head): one row per TMEM
+//     lane and per softmax thread;
+//   * Q [128 x 128] of each group is staged once in shared memory in the 128-byte-swizzled
+//     K-major layout; K and V tiles of 128 keys arrive by TMA in the same layout (the prompt
+//     segment's tensor maps), through separate rings: a K tile is needed one step before the V
+//     tile of the same keys;
+//   * one elected thread issues the MMAs: S = Q.K^T (M 128, N 128, eight K-steps of 16) into a
+//     128-column TMEM buffer and O += P.V (M 128, N 128, eight K-steps) into a 128-column TMEM
+//     accumulator.  P never touches shared memory: the softmax threads write it, rounded to the
+//     16-bit type, over the first 64 columns of the S buffer it came from, and the MMA takes its
+//     A operand from tensor memory.  V is consumed as an MN-major B operand straight from its
+//     row-major tile.  Both operands in shared memory would make every MMA wait for 8 KB of
+//     shared-memory reads; with P in tensor memory P.V reads only V;
+//   * the softmax threads read S with tcgen05.ld (no shuffles for the row max / sum) and
+//     rescale O in tensor memory only when a row's maximum has grown by more than 2^8 since the
+//     reference it is using (the sum uses the same reference, so the result is exact);
+//   * with two groups per CTA each has one S buffer and the tensor cores work for one group
+//     while the other is in its softmax; with one group S is double-buffered so that Q.K^T of
+//     tile j+1 runs under the softmax of tile j.
 //
-// Every mbarrier wait is bounded; on expiry the kernel flags SEGKV_DEV_WAIT_LIMIT, skips the
-// output and still releases its tensor memory.
+// Tensor memory (512 columns): S buffers at 0 and 128, O accumulators at 256 (+128 for the
+// second group).  Every mbarrier wait is bounded; on expiry the kernel flags
+// SEGKV_DEV_WAIT_LIMIT, skips the output and still releases its tensor memory.
 #include "segkv_internal.h"
 #include "segkv_ptx.cuh"
 
@@ -29,13 +36,14 @@ namespace {
 using namespace ptx;
 
 constexpr int kD = 128;        // head_dim of this kernel
-constexpr int kRows = 128;     // query rows per CTA (TMEM lanes)
-constexpr int kKeys = 64;      // keys per K/V tile
-constexpr int kStages = 3;
-constexpr int kBoxKV = kKeys * 128;          // one 64-element-wide box of a K/V tile
-constexpr int kTileKV = kKeys * kD * 2;      // bytes of a K (or V) tile
-constexpr int kBoxQ = kRows * 128;           // one box of the Q tile
-constexpr int kTmemCols = 256;               // S0 [0,64)  S1 [64,128)  O [128,256)
+constexpr int kRows = 128;     // query rows per group (TMEM lanes)
+constexpr int kKeys = 128;     // keys per K/V tile
+constexpr int kBoxRows = 64;   // rows of one TMA box of the prompt segment's tensor map
+constexpr int kBoxBytes = kBoxRows * 128;    // one TMA box: 64 rows x 64 elements
+constexpr int kHalfTile = kKeys * 128;       // 64 of the 128 head-dim elements of all keys of a tile
+constexpr int kTileKV = 2 * kHalfTile;       // bytes of a K (or a V) tile
+constexpr int kBoxQ = kRows * 128;           // 64 of the 128 head-dim elements of a group's Q rows
+constexpr int kTmemCols = 512;
 
 struct Tc5Params {
     const void* q;
@@ -47,15 +55,13 @@ struct Tc5Params {
     uint32_t idesc_qk, idesc_pv;
 };
 
-// shared memory: | K/V ring (kStages x 32 KB) | Q 32 KB | P 16 KB | barriers | tmem slot |
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * 2 * kTileKV + 2 * kBoxQ + kBoxQ + 256;
-
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+// D[tmem] (+)= A[smem] . B[smem]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
@@ -63,8 +69,17 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
         : "memory");
 }
+// D[tmem] (+)= A[tmem] . B[smem]; A is M x 16 of a 16-bit type, two elements per 32-bit column
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
 // 32 lanes x 32 columns of 32-bit words: this thread's TMEM lane, 32 consecutive columns
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
@@ -75,7 +90,7 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr));
 }
-__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t* r) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
         "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
@@ -84,6 +99,14 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32])
           "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
           "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
           "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -99,155 +122,253 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     return ((uint64_t)hi << 32) | lo;
 }
 
-template <typename T>
-__global__ void __launch_bounds__(192, 1)
+// Critical-path wait: poll without sleeping first (the hardware suspends the thread inside
+// try_wait for a while), then fall back to the bounded, sleeping wait.
+__device__ __forceinline__ bool mbar_wait_hot(uint32_t bar, uint32_t parity) {
+#pragma unroll 1
+    for (int i = 0; i < 4096; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait(bar, parity);
+}
+
+#ifdef SEGKV_TC5_TIMELINE
+}  // namespace
+__device__ long long g_tc5_tl[3 * 64 * 8];
+#define TC5_STAMP(role, kt, ev)                                                                   \
+    do {                                                                                          \
+        if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (kt) < 64)                   \
+            g_tc5_tl[((role) * 64 + (kt)) * 8 + (ev)] = clock64();                                \
+    } while (0)
+namespace {
+#else
+#define TC5_STAMP(role, kt, ev) do {} while (0)
+#endif
+
+template <int NG>
+struct Tc5Layout {
+    static constexpr int NB = NG == 1 ? 2 : 1;                   // S buffers per group
+    static constexpr int kThreads = 32 * (4 * NG + 2);
+    static constexpr int kStagesK = 3;
+    static constexpr int kStagesV = NG == 1 ? 3 : 2;
+    static constexpr int kRingK = kStagesK * kTileKV;
+    static constexpr int kRingV = kStagesV * kTileKV;
+    static constexpr int kQ = NG * 2 * kBoxQ;
+    static constexpr int kBars = 2 * kStagesK + 2 * kStagesV + 4 * NG;   // K full/empty, V full/empty, per group: S0 S1 P O
+    static constexpr size_t kBytes = 1024 + (size_t)kRingK + kRingV + kQ + 8 * kBars + 64;
+};
+
+template <typename T, int NG>
+__global__ void __launch_bounds__(Tc5Layout<NG>::kThreads, 1)
 prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    const Tc5Params p) {
+    using L = Tc5Layout<NG>;
+    constexpr int NB = L::NB, SK = L::kStagesK, SV = L::kStagesV;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* q_smem = smem + (size_t)kStages * 2 * kTileKV;      // two boxes [128 rows][64 elements], swizzled
-    uint8_t* p_smem = q_smem + 2 * kBoxQ;                         // one box [128 rows][64 keys], swizzled
-    uint64_t* bars = reinterpret_cast<uint64_t*>(p_smem + kBoxQ);
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kStages);
-    const uint32_t bar_s0 = smem_u32(bars + 2 * kStages);         // two: S buffer written
-    const uint32_t bar_p = bar_s0 + 16;                           // P tile written, S buffer read
-    const uint32_t bar_o = bar_s0 + 24;                           // P.V of a tile complete
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+    uint8_t* k_ring = smem;                                       // tile: two halves [128 keys][64 elements]
+    uint8_t* v_ring = k_ring + L::kRingK;
+    uint8_t* q_smem = v_ring + L::kRingV;                         // per group two halves [128 rows][64 elements]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(q_smem + L::kQ);
+    const uint32_t kfull0 = smem_u32(bars), kempty0 = kfull0 + 8 * SK;
+    const uint32_t vfull0 = kempty0 + 8 * SK, vempty0 = vfull0 + 8 * SV;
+    const uint32_t gbar0 = vempty0 + 8 * SV;                      // group g: +32 g; S buffer 0, S buffer 1, P, O
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + L::kBars);
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;          // longest tiles first
     const int h = blockIdx.y, b = blockIdx.z;
     const int slab = b * p.Hkv + h / p.G;
-    const int nkt = min((p.N + kKeys - 1) / kKeys, ((qt + 1) * kRows + kKeys - 1) / kKeys);
+    const int row_cta = qt * kRows * NG;
+    const int nkt_all = (p.N + kKeys - 1) / kKeys;
+    // key tiles of group g: up to its diagonal tile (causal); none when the group lies past the prompt
+    auto group_tiles = [&](int g) -> int {
+        const int base = row_cta + g * kRows;
+        return base < p.N ? min(nkt_all, base / kKeys + 1) : 0;
+    };
+    int nkt = 0;
+#pragma unroll
+    for (int g = 0; g < NG; ++g) nkt = max(nkt, group_tiles(g));
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(full0 + 8 * s, 1);
-            mbar_init(empty0 + 8 * s, 1);
+        for (int s = 0; s < 2 * SK + 2 * SV; ++s) mbar_init(kfull0 + 8 * s, 1);
+        for (int g = 0; g < NG; ++g) {
+            mbar_init(gbar0 + 32 * g, 1);
+            mbar_init(gbar0 + 32 * g + 8, 1);
+            mbar_init(gbar0 + 32 * g + 16, 128);
+            mbar_init(gbar0 + 32 * g + 24, 1);
         }
-        mbar_init(bar_s0, 1);
-        mbar_init(bar_s0 + 8, 1);
-        mbar_init(bar_p, 128);
-        mbar_init(bar_o, 1);
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
-    if (warp == 5) {                                              // this warp owns the tensor memory
+    if (warp == 4 * NG + 1) {                                     // this warp owns the tensor memory
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(tmem_slot)), "n"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // stage Q (rows past the prompt as zeros): element (r, d) -> box d/64, row r, 16-byte chunk
-    // ((d%64)/8) ^ (r%8): the layout TMA's 128-byte swizzle would have produced
+    // stage Q (rows past the prompt as zeros): element (r, d) of a group -> half d/64, row r, 16-byte
+    // chunk ((d%64)/8) ^ (r%8): the layout TMA's 128-byte swizzle would have produced
     const T* qbase = reinterpret_cast<const T*>(p.q) + ((size_t)b * p.N * p.H + h) * kD;
     const size_t qstride = (size_t)p.H * kD;
-    for (int i = tid; i < kRows * 16; i += 192) {
-        const int r = i >> 4, c = i & 15, grow = qt * kRows + r;
+    for (int i = tid; i < NG * kRows * 16; i += L::kThreads) {
+        const int rr = i >> 4, c = i & 15, grow = row_cta + rr;
+        const int g = rr / kRows, r = rr % kRows;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (grow < p.N) v = *reinterpret_cast<const uint4*>(qbase + (size_t)grow * qstride + c * 8);
-        *reinterpret_cast<uint4*>(q_smem + (size_t)(c >> 3) * kBoxQ + (size_t)r * 128 + (size_t)(((c ^ r) & 7) << 4)) = v;
+        *reinterpret_cast<uint4*>(q_smem + (size_t)(2 * g + (c >> 3)) * kBoxQ + (size_t)r * 128 +
+                                  (size_t)(((c ^ r) & 7) << 4)) = v;
     }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const uint32_t tm_o = tmem + 128;                             // O accumulator columns
 
-    if (warp == 4) {
+    if (warp == 4 * NG) {
         // ------------------------------- TMA producer -------------------------------
         if (lane == 0) {
             prefetch_tmap(&tm_k);
             prefetch_tmap(&tm_v);
-            for (int kt = 0; kt < nkt; ++kt) {
-                const int st = kt % kStages;
-                if (!mbar_wait(empty0 + 8 * st, (((uint32_t)(kt / kStages)) & 1) ^ 1)) { s_abort = 1; break; }
-                const uint32_t full = full0 + 8 * st;
-                const uint32_t k_dst = smem_u32(smem + (size_t)st * 2 * kTileKV);
-                const uint32_t v_dst = k_dst + kTileKV;
-                mbar_arrive_expect_tx(full, 2u * kTileKV);
+            auto load_tile = [&](const CUtensorMap* tm, uint8_t* dst_tile, int kt, uint32_t full) {
+                const uint32_t dst = smem_u32(dst_tile);
+                mbar_arrive_expect_tx(full, (uint32_t)kTileKV);
 #pragma unroll
-                for (int bx = 0; bx < 2; ++bx) {
-                    tma_load_3d(k_dst + bx * kBoxKV, &tm_k, bx * 64, kt * kKeys, slab, full);
-                    tma_load_3d(v_dst + bx * kBoxKV, &tm_v, bx * 64, kt * kKeys, slab, full);
-                }
+                for (int half = 0; half < 2; ++half)
+#pragma unroll
+                    for (int rb = 0; rb < kKeys / kBoxRows; ++rb)
+                        tma_load_3d(dst + half * kHalfTile + rb * kBoxBytes, tm, half * 64,
+                                    kt * kKeys + rb * kBoxRows, slab, full);
+            };
+            for (int kt = 0; kt < nkt; ++kt) {
+                const int sk = kt % SK, sv = kt % SV;
+                if (!mbar_wait(kempty0 + 8 * sk, (((uint32_t)(kt / SK)) & 1) ^ 1)) { s_abort = 1; break; }
+                load_tile(&tm_k, k_ring + (size_t)sk * kTileKV, kt, kfull0 + 8 * sk);
+                if (!mbar_wait(vempty0 + 8 * sv, (((uint32_t)(kt / SV)) & 1) ^ 1)) { s_abort = 1; break; }
+                load_tile(&tm_v, v_ring + (size_t)sv * kTileKV, kt, vfull0 + 8 * sv);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 4 * NG + 1) {
         // -------------------------------- MMA issuer --------------------------------
         if (lane == 0) {
-            const uint32_t q_addr = smem_u32(q_smem), p_addr = smem_u32(p_smem);
-            auto issue_qk = [&](int kt) -> bool {                 // S[kt & 1] = Q . K_kt^T
-                const int st = kt % kStages;
-                if (!mbar_wait(full0 + 8 * st, ((uint32_t)(kt / kStages)) & 1)) return false;
-                tc_fence_after();
-                const uint32_t k_addr = smem_u32(smem + (size_t)st * 2 * kTileKV);
+            int gt[NG];
+#pragma unroll
+            for (int g = 0; g < NG; ++g) gt[g] = group_tiles(g);
+            auto issue_qk = [&](int g, int kt, int buf) {         // S_g[buf] = Q_g . K_kt^T
+                const uint32_t q_addr = smem_u32(q_smem) + (uint32_t)g * 2 * kBoxQ;
+                const uint32_t k_addr = smem_u32(k_ring + (size_t)(kt % SK) * kTileKV);
 #pragma unroll
                 for (int ks = 0; ks < kD / 16; ++ks) {
                     const uint32_t off = (uint32_t)(ks & 3) * 32;
-                    tc_mma(tmem + (uint32_t)(kt & 1) * 64,
-                           smem_desc(q_addr + (ks >> 2) * kBoxQ + off, 16, 1024),
-                           smem_desc(k_addr + (ks >> 2) * kBoxKV + off, 16, 1024), p.idesc_qk, ks > 0);
+                    tc_mma_ss(tmem + 128u * (uint32_t)(g + buf),
+                              smem_desc(q_addr + (ks >> 2) * kBoxQ + off, 16, 1024),
+                              smem_desc(k_addr + (ks >> 2) * kHalfTile + off, 16, 1024), p.idesc_qk, ks > 0);
                 }
-                tc_commit(bar_s0 + 8 * (kt & 1));
-                return true;
+                tc_commit(gbar0 + 32 * g + 8 * buf);
             };
-            bool ok = issue_qk(0);
-            for (int kt = 0; kt < nkt && ok; ++kt) {
-                if (kt + 1 < nkt) ok = issue_qk(kt + 1);          // runs under the softmax of tile kt
-                if (!ok) break;
-                ok = mbar_wait(bar_p, (uint32_t)kt & 1);
-                if (!ok) break;
+            auto wait_k = [&](int kt) -> bool {
+                const bool ok = mbar_wait_hot(kfull0 + 8 * (kt % SK), ((uint32_t)(kt / SK)) & 1);
                 tc_fence_after();
-                const int st = kt % kStages;
-                const uint32_t v_addr = smem_u32(smem + (size_t)st * 2 * kTileKV) + kTileKV;
+                return ok;
+            };
+            bool ok = wait_k(0);
+            if (ok) {
 #pragma unroll
-                for (int kk = 0; kk < kKeys / 16; ++kk)           // O += P[:, 16 keys] . V[16 keys, :]
-                    tc_mma(tm_o, smem_desc(p_addr + kk * 32, 16, 1024),
-                           smem_desc(v_addr + kk * 2048, kBoxKV, 1024), p.idesc_pv, (kt > 0 || kk > 0));
-                tc_commit(empty0 + 8 * st);                       // K/V stage free once these MMAs are done
-                tc_commit(bar_o);
+                for (int g = 0; g < NG; ++g)
+                    if (gt[g] > 0) issue_qk(g, 0, 0);
+                tc_commit(kempty0);                               // K stage free once these MMAs are done
+            }
+            for (int kt = 0; kt < nkt && ok; ++kt) {
+                TC5_STAMP(2, kt, 0);
+                if (NB == 2 && kt + 1 < nkt) {                    // next tile's scores run under this tile's softmax
+                    ok = wait_k(kt + 1);
+                    if (!ok) break;
+#pragma unroll
+                    for (int g = 0; g < NG; ++g)
+                        if (kt + 1 < gt[g]) issue_qk(g, kt + 1, (kt + 1) & 1);
+                    tc_commit(kempty0 + 8 * ((kt + 1) % SK));
+                }
+                TC5_STAMP(2, kt, 1);
+                const int sv = kt % SV;
+                const uint32_t v_addr = smem_u32(v_ring + (size_t)sv * kTileKV);
+                ok = mbar_wait_hot(vfull0 + 8 * sv, ((uint32_t)(kt / SV)) & 1);
+                if (!ok) break;
+                TC5_STAMP(2, kt, 2);
+                bool k_next = false;
+#pragma unroll
+                for (int g = 0; g < NG; ++g) {
+                    if (kt >= gt[g]) continue;
+                    ok = mbar_wait_hot(gbar0 + 32 * g + 16, (uint32_t)kt & 1);   // P_g written over its S buffer
+                    if (!ok) break;
+                    TC5_STAMP(2, kt, 3 + 2 * g);
+                    tc_fence_after();
+                    const uint32_t p_tmem = tmem + 128u * (uint32_t)(g + (NB == 2 ? (kt & 1) : 0));
+#pragma unroll
+                    for (int kk = 0; kk < kKeys / 16; ++kk)       // O_g += P_g[:, 16 keys] . V[16 keys, :]
+                        tc_mma_ts(tmem + 256u + 128u * (uint32_t)g, p_tmem + kk * 8,
+                                  smem_desc(v_addr + kk * 2048, kHalfTile, 1024), p.idesc_pv, (kt > 0 || kk > 0));
+                    tc_commit(gbar0 + 32 * g + 24);
+                    if (NB == 1 && kt + 1 < gt[g]) {              // the group's next scores, behind its P.V in the pipe
+                        if (!k_next) {
+                            ok = wait_k(kt + 1);
+                            if (!ok) break;
+                            k_next = true;
+                        }
+                        issue_qk(g, kt + 1, 0);
+                    }
+                    TC5_STAMP(2, kt, 4 + 2 * g);
+                }
+                if (!ok) break;
+                tc_commit(vempty0 + 8 * sv);                      // stages free once every MMA so far is done
+                if (NB == 1 && kt + 1 < nkt) tc_commit(kempty0 + 8 * ((kt + 1) % SK));
             }
             if (!ok) s_abort = 1;
         }
     } else {
         // ------------------------------ softmax warps: one row per thread ------------------------------
-        const int row = qt * kRows + tid;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;    // this warp's TMEM lanes
+        const int g = warp >> 2, r = tid & (kRows - 1);
+        const int row = row_cta + g * kRows + r;
+        const int my_tiles = group_tiles(g);
+        const uint32_t bar_s0 = gbar0 + 32 * g, bar_p = bar_s0 + 16, bar_o = bar_s0 + 24;
+        const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);     // this warp's TMEM lanes
+        const uint32_t tm_o = tm_lane + 256u + 128u * (uint32_t)g;
         const float slope2 = p.slopes ? p.slopes[h] * 1.4426950408889634f : 0.f;
+        const bool stamp = lane == 0 && (warp & 3) == 0;
         float m_ref = -INFINITY, l_run = 0.f;
         bool ok = true;
-        for (int kt = 0; kt < nkt; ++kt) {
-            ok = mbar_wait(bar_s0 + 8 * (kt & 1), ((uint32_t)(kt >> 1)) & 1);
+        for (int kt = 0; kt < my_tiles; ++kt) {
+            const int buf = NB == 2 ? (kt & 1) : 0;
+            const uint32_t tm_s = tm_lane + 128u * (uint32_t)(g + buf);
+            ok = mbar_wait_hot(bar_s0 + 8 * buf, (uint32_t)(NB == 2 ? (kt >> 1) : kt) & 1);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
+            if (stamp) TC5_STAMP(g, kt, 0);
             tc_fence_after();
-            uint32_t sr[2][32];
-            tc_ld32(tmem + lane_base + (uint32_t)(kt & 1) * 64, sr[0]);
-            tc_ld32(tmem + lane_base + (uint32_t)(kt & 1) * 64 + 32, sr[1]);
+            uint32_t sr[kKeys];
+#pragma unroll
+            for (int c = 0; c < kKeys / 32; ++c) tc_ld32(tm_s + 32 * c, sr + 32 * c);
             tc_wait_ld();
+            if (stamp) TC5_STAMP(g, kt, 1);
+            float* sv = reinterpret_cast<float*>(sr);
             const int key0 = kt * kKeys;
-            const bool diag = key0 + kKeys - 1 > qt * kRows;       // some key above some row of the CTA
-            float tmax = -INFINITY;
-            float* sv = reinterpret_cast<float*>(&sr[0][0]);
-            if (diag || p.slopes) {
+            const bool diag = key0 + kKeys - 1 > row_cta + g * kRows;   // the group's diagonal tile
+            const bool general = diag || p.slopes != nullptr;
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            if (general) {
 #pragma unroll
                 for (int i = 0; i < kKeys; ++i) {
                     const int key = key0 + i;
                     float v = sv[i] * p.scale2 + slope2 * (float)(key - row);
                     if (diag && key > row) v = -INFINITY;
                     sv[i] = v;
-                    tmax = fmaxf(tmax, v);
+                    mx[i & 3] = fmaxf(mx[i & 3], v);
                 }
             } else {
 #pragma unroll
-                for (int i = 0; i < kKeys; ++i) {
-                    sv[i] *= p.scale2;
-                    tmax = fmaxf(tmax, sv[i]);
-                }
+                for (int i = 0; i < kKeys; ++i) mx[i & 3] = fmaxf(mx[i & 3], sv[i]);
             }
+            float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            if (!general) tmax *= p.scale2;
             // a new reference only when the maximum has grown by more than 2^8: exponentials stay
             // below 2^8 of the reference, the sum and O use the same reference
             const bool need = tmax > m_ref + 8.f;
@@ -256,54 +377,54 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 alpha = exp2f(m_ref - tmax);                       // 0 on the first tile
                 m_ref = tmax;
             }
-            float lsum = 0.f;
+            float ls[4] = {0.f, 0.f, 0.f, 0.f};
             uint32_t pk[kKeys / 2];
+            const float sc = general ? 1.f : p.scale2, nm = -m_ref;
 #pragma unroll
             for (int i = 0; i < kKeys; i += 2) {
-                const float e0 = exp2f(sv[i] - m_ref), e1 = exp2f(sv[i + 1] - m_ref);
-                lsum += e0 + e1;
+                const float e0 = exp2f(fmaf(sv[i], sc, nm)), e1 = exp2f(fmaf(sv[i + 1], sc, nm));
+                ls[(i >> 1) & 3] += e0 + e1;
                 pk[i >> 1] = Mma<T>::pack(e0, e1);
             }
-            l_run = l_run * alpha + lsum;
-            if (kt > 0) {
-                ok = mbar_wait(bar_o, (uint32_t)(kt - 1) & 1);     // P.V of the previous tile done: P free, O stable
+            l_run = l_run * alpha + ((ls[0] + ls[1]) + (ls[2] + ls[3]));
+            if (stamp) TC5_STAMP(g, kt, 2);
+            if (kt > 0 && __any_sync(0xffffffffu, need)) {
+                ok = mbar_wait_hot(bar_o, (uint32_t)(kt - 1) & 1); // P.V of the previous tile done: O stable
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, need)) {
 #pragma unroll
-                    for (int c = 0; c < kD / 32; ++c) {
-                        uint32_t orr[32];
-                        tc_ld32(tm_o + lane_base + c * 32, orr);
-                        tc_wait_ld();
+                for (int c = 0; c < kD / 32; ++c) {
+                    uint32_t orr[32];
+                    tc_ld32(tm_o + c * 32, orr);
+                    tc_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
-                        tc_st32(tm_o + lane_base + c * 32, orr);
-                    }
-                    tc_wait_st();
+                    for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+                    tc_st32(tm_o + c * 32, orr);
                 }
+                if (stamp) TC5_STAMP(g, kt, 3);
             }
-            // P row -> shared memory, K-major with the 128-byte swizzle (eight 16-byte chunks)
+            // P over the first 64 columns of the S buffer: two 16-bit weights per column, the A
+            // operand layout of the MMA that follows.  S has been read completely above.
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<uint4*>(p_smem + (size_t)tid * 128 + (size_t)(((c ^ tid) & 7) << 4)) =
-                    make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-            fence_proxy_async();
+            for (int c = 0; c < kKeys / 32; ++c) tc_st16(tm_s + 16 * c, pk + 16 * c);
+            tc_wait_st();
             tc_fence_before();
             mbar_arrive(bar_p);
+            if (stamp) TC5_STAMP(g, kt, 4);
         }
-        if (ok) {
-            ok = mbar_wait(bar_o, (uint32_t)(nkt - 1) & 1);
+        if (ok && my_tiles > 0) {
+            ok = mbar_wait_hot(bar_o, (uint32_t)(my_tiles - 1) & 1);
             ok = __all_sync(0xffffffffu, ok);
         }
-        if (ok) {
+        if (ok && my_tiles > 0) {
             tc_fence_after();
             const float inv = 1.f / l_run;
             T* orow = reinterpret_cast<T*>(p.out) + ((size_t)b * p.N * p.H + h) * kD + (size_t)row * qstride;
 #pragma unroll
             for (int c = 0; c < kD / 32; ++c) {
                 uint32_t orr[32];
-                tc_ld32(tm_o + lane_base + c * 32, orr);
+                tc_ld32(tm_o + c * 32, orr);
                 tc_wait_ld();
                 if (row < p.N) {
 #pragma unroll
@@ -315,17 +436,34 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                             Mma<T>::pack(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv));
                 }
             }
-        } else if (lane == 0) {
+        } else if (!ok && lane == 0) {
             s_abort = 1;
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == 4 * NG + 1) {
         __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(kTmemCols) : "memory");
         if (lane == 0 && s_abort) atomicOr(p.err_word, SEGKV_DEV_WAIT_LIMIT);
     }
+}
+
+template <typename T, int NG>
+cudaError_t launch_tc5(const Dims& d, const PrefillArgs& a, const Tc5Params& p, cudaStream_t st) {
+    using L = Tc5Layout<NG>;
+    auto kern = prefill_tc5_kernel<T, NG>;
+    static bool configured[64] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    dim3 grid((unsigned)((a.prompt_len + kRows * NG - 1) / (kRows * NG)), (unsigned)d.heads, (unsigned)d.batch);
+    kern<<<grid, L::kThreads, L::kBytes, st>>>(*a.tm_k, *a.tm_v, p);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -335,17 +473,6 @@ bool prefill_tc5_supported(const Dims& d) { return d.head_dim == kD; }
 cudaError_t launch_prefill_tc5(const Dims& d, const PrefillArgs& a, cudaStream_t st) {
     if (d.head_dim != kD) return cudaErrorInvalidValue;
     const bool bf = d.dtype == SEGKV_BF16;
-    static bool configured[64][2] = {{false}};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !configured[dev][bf]) {
-        cudaError_t e = bf ? cudaFuncSetAttribute(prefill_tc5_kernel<__nv_bfloat16>,
-                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes)
-                           : cudaFuncSetAttribute(prefill_tc5_kernel<__half>,
-                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e != cudaSuccess) return e;
-        configured[dev][bf] = true;
-    }
     Tc5Params p;
     p.q = a.q; p.out = a.out; p.slopes = a.slopes; p.err_word = a.err_word;
     p.N = a.prompt_len; p.H = d.heads; p.Hkv = d.kv_heads; p.G = d.group;
@@ -355,10 +482,23 @@ cudaError_t launch_prefill_tc5(const Dims& d, const PrefillArgs& a, cudaStream_t
     const uint32_t common = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kRows >> 4) << 24);
     p.idesc_qk = common | ((uint32_t)(kKeys >> 3) << 17);                 // A, B both K-major
     p.idesc_pv = common | (1u << 16) | ((uint32_t)(kD >> 3) << 17);       // B (= V) MN-major
-    dim3 grid((unsigned)((a.prompt_len + kRows - 1) / kRows), (unsigned)d.heads, (unsigned)d.batch);
-    if (bf) prefill_tc5_kernel<__nv_bfloat16><<<grid, 192, kSmemBytes, st>>>(*a.tm_k, *a.tm_v, p);
-    else prefill_tc5_kernel<__half><<<grid, 192, kSmemBytes, st>>>(*a.tm_k, *a.tm_v, p);
-    return cudaGetLastError();
+    // two row groups per CTA once there are enough 256-row CTAs to fill the machine a few times over
+    int sms = 148;
+    {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    const long ctas2 = (long)((a.prompt_len + 2 * kRows - 1) / (2 * kRows)) * d.heads * d.batch;
+    const bool two = a.row_groups ? a.row_groups == 2 : ctas2 >= 2L * sms;
+    if (two) return bf ? launch_tc5<__nv_bfloat16, 2>(d, a, p, st) : launch_tc5<__half, 2>(d, a, p, st);
+    return bf ? launch_tc5<__nv_bfloat16, 1>(d, a, p, st) : launch_tc5<__half, 1>(d, a, p, st);
 }
 
 }  // namespace segkv_impl
+
+#ifdef SEGKV_TC5_TIMELINE
+extern "C" __attribute__((visibility("default"))) int segkv_debug_tc5_timeline(long long* host) {
+    return cudaMemcpyFromSymbol(host, segkv_impl::g_tc5_tl, sizeof(long long) * 3 * 64 * 8) == cudaSuccess ? 0 : -1;
+}
+#endif

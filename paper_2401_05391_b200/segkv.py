@@ -49,6 +49,7 @@ SIGNATURES = {
     "segkv_decode_sdpa_rowwise": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "segkv_get_splits": (_int, [_vp]),
     "segkv_set_overlap": (_int, [_vp, _int]),
+    "segkv_set_prefill_tuning": (_int, [_vp, _int]),
     "segkv_launch_count": (ctypes.c_longlong, [_vp]),
     "segkv_storage_bytes": (ctypes.c_size_t, [_int] * 7),
     "segkv_strerror": (ctypes.c_char_p, [_int]),
@@ -286,6 +287,9 @@ class SegKV:
 
     def set_overlap(self, enable: bool) -> None:
         _check(lib().segkv_set_overlap(self._h, int(enable)), "segkv_set_overlap")
+
+    def set_prefill_tuning(self, row_groups: int = 0) -> None:
+        _check(lib().segkv_set_prefill_tuning(self._h, row_groups), "segkv_set_prefill_tuning")
 
     def get_splits(self) -> int:
         return int(lib().segkv_get_splits(self._h))

@@ -25,9 +25,10 @@ def check_rows(w, q, kp, vp, out, slopes, rows):
     assert (err <= atol + RTOL * np.abs(ref)).all(), f"max err {err.max():.3e}"
 
 
-def run_prefill(w, rows_fn):
+def run_prefill(w, rows_fn, row_groups=0):
     h = sk.SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, w.steps, w.torch_dtype)
     try:
+        h.set_prefill_tuning(row_groups)
         kp, vp = wl.make_prompt(w, "cuda")
         q = wl.make_prefill_query(w, "cuda")
         slopes = wl.alibi_slopes(w.heads).cuda() if w.alibi else None
@@ -61,6 +62,24 @@ def test_prefill_ragged_small_shapes(dtype, D, P):
     # several tiles and a ragged tail, GQA, ALiBi on the bf16 variants
     w = wl.Workload("pf", 2, 3, 6, 2, D, P, 2, dtype, "uniform", dtype == "bf16", 80 + D // 64)
     h = run_prefill(w, all_rows)[0]
+    h.destroy()
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("row_groups", [1, 2])
+@pytest.mark.parametrize("P", [64, 128, 129, 150, 256, 257, 300, 520, 777])
+def test_prefill_head_dim_128_row_groups(dtype, row_groups, P):
+    # the tcgen05 kernel with one and with two 128-row groups per CTA: prompts that leave the
+    # second group empty (64, 128), with one row (129), exact tiles (256), ragged (150, 257, 300, 777)
+    # and spanning CTAs (520, 777)
+    w = wl.Workload("pf", 2, 3, 4, 2, 128, P, 2, dtype, "uniform", dtype == "bf16", 90 + row_groups)
+    h = run_prefill(w, all_rows if P <= 300 else (lambda w: sampled_rows(w, 400)), row_groups)[0]
+    h.destroy()
+
+
+@pytest.mark.parametrize("row_groups", [1, 2])
+def test_prefill_llama2_7b_shape_row_groups_sampled(row_groups):
+    h = run_prefill(wl.CONFIGS[1], lambda w: sampled_rows(w, 256), row_groups)[0]
     h.destroy()
 
 
