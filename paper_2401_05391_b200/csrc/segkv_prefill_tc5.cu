@@ -157,6 +157,23 @@ struct Tc5Layout {
     static constexpr size_t kBytes = 1024 + (size_t)kRingK + kRingV + kQ + 8 * kBars + 64;
 };
 
+// Row maximum of one tile's scores.  BIAS: sv[i] <- sv[i] * scale2 + slope2 * (key_i - row), the
+// maximum is in log2 units; otherwise sv keeps the raw dot products and the maximum is raw.
+// MASK: keys above the row (i > lim) are set to -inf first.
+template <bool BIAS, bool MASK>
+__device__ __forceinline__ float score_max(float* sv, float scale2, float slope2, float bias0, int lim) {
+    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+    for (int i = 0; i < kKeys; ++i) {
+        float v = sv[i];
+        if (BIAS) v = fmaf(v, scale2, fmaf(slope2, (float)i, bias0));
+        if (MASK) v = i > lim ? -INFINITY : v;
+        if (BIAS || MASK) sv[i] = v;
+        mx[i & 3] = fmaxf(mx[i & 3], v);
+    }
+    return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+}
+
 template <typename T, int NG>
 __global__ void __launch_bounds__(Tc5Layout<NG>::kThreads, 1)
 prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -190,8 +207,31 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 #pragma unroll
     for (int g = 0; g < NG; ++g) nkt = max(nkt, group_tiles(g));
 
-    if (tid == 0) {
+    // K/V tile -> its ring stage; the barrier gets the byte count first
+    auto load_tile = [&](const CUtensorMap* tm, uint8_t* dst_tile, int kt, uint32_t full) {
+        const uint32_t dst = smem_u32(dst_tile);
+        mbar_arrive_expect_tx(full, (uint32_t)kTileKV);
+#pragma unroll
+        for (int half = 0; half < 2; ++half)
+#pragma unroll
+            for (int rb = 0; rb < kKeys / kBoxRows; ++rb)
+                tma_load_3d(dst + half * kHalfTile + rb * kBoxBytes, tm, half * 64, kt * kKeys + rb * kBoxRows, slab, full);
+    };
+    constexpr int kEarly = SK < SV ? SK : SV;                     // tiles requested before anything else happens
+    if (warp == 4 * NG && lane == 0) {
+        // the producer sets up the ring barriers itself and requests the first tiles at once: they
+        // do not depend on Q, which the other warps stage meanwhile
         for (int s = 0; s < 2 * SK + 2 * SV; ++s) mbar_init(kfull0 + 8 * s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+        prefetch_tmap(&tm_k);
+        prefetch_tmap(&tm_v);
+        for (int kt = 0; kt < min(nkt, kEarly); ++kt) {
+            load_tile(&tm_k, k_ring + (size_t)kt * kTileKV, kt, kfull0 + 8 * kt);
+            load_tile(&tm_v, v_ring + (size_t)kt * kTileKV, kt, vfull0 + 8 * kt);
+        }
+    }
+    if (tid == 0) {
         for (int g = 0; g < NG; ++g) {
             mbar_init(gbar0 + 32 * g, 1);
             mbar_init(gbar0 + 32 * g + 8, 1);
@@ -228,19 +268,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (warp == 4 * NG) {
         // ------------------------------- TMA producer -------------------------------
         if (lane == 0) {
-            prefetch_tmap(&tm_k);
-            prefetch_tmap(&tm_v);
-            auto load_tile = [&](const CUtensorMap* tm, uint8_t* dst_tile, int kt, uint32_t full) {
-                const uint32_t dst = smem_u32(dst_tile);
-                mbar_arrive_expect_tx(full, (uint32_t)kTileKV);
-#pragma unroll
-                for (int half = 0; half < 2; ++half)
-#pragma unroll
-                    for (int rb = 0; rb < kKeys / kBoxRows; ++rb)
-                        tma_load_3d(dst + half * kHalfTile + rb * kBoxBytes, tm, half * 64,
-                                    kt * kKeys + rb * kBoxRows, slab, full);
-            };
-            for (int kt = 0; kt < nkt; ++kt) {
+            for (int kt = kEarly; kt < nkt; ++kt) {
                 const int sk = kt % SK, sv = kt % SV;
                 if (!mbar_wait(kempty0 + 8 * sk, (((uint32_t)(kt / SK)) & 1) ^ 1)) { s_abort = 1; break; }
                 load_tile(&tm_k, k_ring + (size_t)sk * kTileKV, kt, kfull0 + 8 * sk);
@@ -352,23 +380,16 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             float* sv = reinterpret_cast<float*>(sr);
             const int key0 = kt * kKeys;
             const bool diag = key0 + kKeys - 1 > row_cta + g * kRows;   // the group's diagonal tile
-            const bool general = diag || p.slopes != nullptr;
-            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            if (general) {
-#pragma unroll
-                for (int i = 0; i < kKeys; ++i) {
-                    const int key = key0 + i;
-                    float v = sv[i] * p.scale2 + slope2 * (float)(key - row);
-                    if (diag && key > row) v = -INFINITY;
-                    sv[i] = v;
-                    mx[i & 3] = fmaxf(mx[i & 3], v);
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < kKeys; ++i) mx[i & 3] = fmaxf(mx[i & 3], sv[i]);
-            }
-            float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-            if (!general) tmax *= p.scale2;
+            // scores in log2 units: s * scale2 (+ ALiBi bias); the scale is folded into the exponent's
+            // FMA unless a bias has to be added first; keys above the row (diagonal tile) become -inf
+            const bool biased = p.slopes != nullptr;
+            const int lim = row - key0;                            // key index i of this tile is visible iff i <= lim
+            const float bias0 = slope2 * (float)(key0 - row);
+            float tmax;
+            if (biased) tmax = diag ? score_max<true, true>(sv, p.scale2, slope2, bias0, lim)
+                                    : score_max<true, false>(sv, p.scale2, slope2, bias0, lim);
+            else tmax = (diag ? score_max<false, true>(sv, p.scale2, slope2, bias0, lim)
+                              : score_max<false, false>(sv, p.scale2, slope2, bias0, lim)) * p.scale2;
             // a new reference only when the maximum has grown by more than 2^8: exponentials stay
             // below 2^8 of the reference, the sum and O use the same reference
             const bool need = tmax > m_ref + 8.f;
@@ -379,7 +400,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             }
             float ls[4] = {0.f, 0.f, 0.f, 0.f};
             uint32_t pk[kKeys / 2];
-            const float sc = general ? 1.f : p.scale2, nm = -m_ref;
+            const float sc = biased ? 1.f : p.scale2, nm = -m_ref;
 #pragma unroll
             for (int i = 0; i < kKeys; i += 2) {
                 const float e0 = exp2f(fmaf(sv[i], sc, nm)), e1 = exp2f(fmaf(sv[i + 1], sc, nm));
