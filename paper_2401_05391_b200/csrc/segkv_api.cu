@@ -80,6 +80,31 @@ int make_prompt_map(const segkv* h, void* base, int prompt_len, CUtensorMap* out
     return SEGKV_OK;
 }
 
+// Tensor map over the prefill query [batch][prompt_len][heads][D] (token-major): one box is 64
+// elements of one head for 128 consecutive tokens; tokens >= prompt_len read as zero.
+int make_query_map(const segkv* h, const void* q, int prompt_len, CUtensorMap* out) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled entry point not available");
+        return SEGKV_ECUDA;
+    }
+    const Dims& d = h->d;
+    const cuuint64_t row = (cuuint64_t)d.head_dim * 2;
+    cuuint64_t dims[4] = {(cuuint64_t)d.head_dim, (cuuint64_t)d.heads, (cuuint64_t)prompt_len, (cuuint64_t)d.batch};
+    cuuint64_t strides[3] = {row, row * d.heads, row * d.heads * prompt_len};
+    cuuint32_t box[4] = {64, 1, 128, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUtensorMapDataType dt = d.dtype == SEGKV_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    CUresult r = fn(out, dt, 4, const_cast<void*>(q), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled (query) failed with CUresult %d", (int)r);
+        return SEGKV_ECUDA;
+    }
+    return SEGKV_OK;
+}
+
 void free_all(segkv* h) {
     void* ptrs[] = {h->kp, h->vp, h->kr, h->k_chunks_dev, h->parent, h->anc[0], h->anc[1], h->ulist, h->ucount,
                     h->err_word, h->ws, h->tickets, h->st_q, h->st_out, h->st_k, h->st_v, h->st_parent,
@@ -379,6 +404,13 @@ int segkv_prefill_sdpa(segkv_t h, const void* q, void* out, const float* alibi_s
     a.q = q; a.out = out; a.slopes = alibi_slopes; a.err_word = h->err_word;
     a.prompt_len = h->prompt_len; a.tm_k = &h->tm_kp; a.tm_v = &h->tm_vp;
     a.row_groups = h->prefill_groups;
+    CUtensorMap tm_q;
+    a.tm_q = nullptr;
+    if (prefill_tc5_supported(h->d)) {
+        int rc = make_query_map(h, q, h->prompt_len, &tm_q);
+        if (rc != SEGKV_OK) return rc;
+        a.tm_q = &tm_q;
+    }
     SEGKV_CUDA(launch_prefill_sdpa(h->d, a, (cudaStream_t)stream));
     h->launches++;
     return SEGKV_OK;

@@ -147,6 +147,7 @@ struct PrefillArgs {
     int prompt_len;
     const CUtensorMap* tm_k;
     const CUtensorMap* tm_v;
+    const CUtensorMap* tm_q;   // over q as [batch][prompt_len][heads][D], box 64 elements x 128 tokens; NULL if unused
     int row_groups;      // 0 = automatic
 };
 bool prefill_sdpa_supported(const Dims& d);

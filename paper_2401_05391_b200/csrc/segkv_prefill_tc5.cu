@@ -50,7 +50,7 @@ struct Tc5Params {
     void* out;
     const float* slopes;
     int* err_word;
-    int N, H, Hkv, G;
+    int N, H, Hkv, G, B;
     float scale2;
     uint32_t idesc_qk, idesc_pv;
 };
@@ -136,7 +136,8 @@ __device__ __forceinline__ bool mbar_wait_hot(uint32_t bar, uint32_t parity) {
 __device__ long long g_tc5_tl[3 * 64 * 8];
 #define TC5_STAMP(role, kt, ev)                                                                   \
     do {                                                                                          \
-        if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (kt) < 64)                   \
+        if ((SEGKV_TC5_TIMELINE != 2 || ((role) == 2 && (ev) == 0)) &&                            \
+            blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (kt) < 64)                   \
             g_tc5_tl[((role) * 64 + (kt)) * 8 + (ev)] = clock64();                                \
     } while (0)
 namespace {
@@ -153,7 +154,7 @@ struct Tc5Layout {
     static constexpr int kRingK = kStagesK * kTileKV;
     static constexpr int kRingV = kStagesV * kTileKV;
     static constexpr int kQ = NG * 2 * kBoxQ;
-    static constexpr int kBars = 2 * kStagesK + 2 * kStagesV + 4 * NG;   // K full/empty, V full/empty, per group: S0 S1 P O
+    static constexpr int kBars = 2 * kStagesK + 2 * kStagesV + 6 * NG;   // K full/empty, V full/empty, per group: S0 S1 P O Qfull Qempty
     static constexpr size_t kBytes = 1024 + (size_t)kRingK + kRingV + kQ + 8 * kBars + 64;
 };
 
@@ -174,10 +175,15 @@ __device__ __forceinline__ float score_max(float* sv, float scale2, float slope2
     return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
 }
 
+// One CTA per SM walks a static list of work items (128*NG query rows of one (request, head)),
+// longest first and dealt round-robin, so that the tail of one item overlaps the head of the
+// next: the producer runs ahead through the K/V rings and reloads a group's Q as soon as the
+// group's last Q.K^T has been read, and the first Q.K^T of the next item executes while the
+// softmax threads are still storing the previous output.
 template <typename T, int NG>
 __global__ void __launch_bounds__(Tc5Layout<NG>::kThreads, 1)
-prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                   const Tc5Params p) {
+prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                   const __grid_constant__ CUtensorMap tm_v, const Tc5Params p) {
     using L = Tc5Layout<NG>;
     constexpr int NB = L::NB, SK = L::kStagesK, SV = L::kStagesV;
     extern __shared__ uint8_t smem_raw[];
@@ -188,55 +194,32 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     uint64_t* bars = reinterpret_cast<uint64_t*>(q_smem + L::kQ);
     const uint32_t kfull0 = smem_u32(bars), kempty0 = kfull0 + 8 * SK;
     const uint32_t vfull0 = kempty0 + 8 * SK, vempty0 = vfull0 + 8 * SV;
-    const uint32_t gbar0 = vempty0 + 8 * SV;                      // group g: +32 g; S buffer 0, S buffer 1, P, O
+    const uint32_t gbar0 = vempty0 + 8 * SV;                      // group g: +48 g; S buffer 0, S buffer 1, P, O, Q full, Q empty
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + L::kBars);
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;          // longest tiles first
-    const int h = blockIdx.y, b = blockIdx.z;
-    const int slab = b * p.Hkv + h / p.G;
-    const int row_cta = qt * kRows * NG;
     const int nkt_all = (p.N + kKeys - 1) / kKeys;
-    // key tiles of group g: up to its diagonal tile (causal); none when the group lies past the prompt
-    auto group_tiles = [&](int g) -> int {
-        const int base = row_cta + g * kRows;
+    const int nqt = (p.N + kRows * NG - 1) / (kRows * NG);
+    const int hb_count = p.H * p.B;
+    const int n_items = nqt * hb_count;
+    // item w -> query tile (longest first), head, request
+    auto item_qt = [&](int w) { return nqt - 1 - w / hb_count; };
+    // key tiles of group g of query tile qt: up to its diagonal tile (causal); none past the prompt
+    auto group_tiles = [&](int qt, int g) -> int {
+        const int base = (qt * NG + g) * kRows;
         return base < p.N ? min(nkt_all, base / kKeys + 1) : 0;
     };
-    int nkt = 0;
-#pragma unroll
-    for (int g = 0; g < NG; ++g) nkt = max(nkt, group_tiles(g));
 
-    // K/V tile -> its ring stage; the barrier gets the byte count first
-    auto load_tile = [&](const CUtensorMap* tm, uint8_t* dst_tile, int kt, uint32_t full) {
-        const uint32_t dst = smem_u32(dst_tile);
-        mbar_arrive_expect_tx(full, (uint32_t)kTileKV);
-#pragma unroll
-        for (int half = 0; half < 2; ++half)
-#pragma unroll
-            for (int rb = 0; rb < kKeys / kBoxRows; ++rb)
-                tma_load_3d(dst + half * kHalfTile + rb * kBoxBytes, tm, half * 64, kt * kKeys + rb * kBoxRows, slab, full);
-    };
-    constexpr int kEarly = SK < SV ? SK : SV;                     // tiles requested before anything else happens
-    if (warp == 4 * NG && lane == 0) {
-        // the producer sets up the ring barriers itself and requests the first tiles at once: they
-        // do not depend on Q, which the other warps stage meanwhile
-        for (int s = 0; s < 2 * SK + 2 * SV; ++s) mbar_init(kfull0 + 8 * s, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        fence_proxy_async();
-        prefetch_tmap(&tm_k);
-        prefetch_tmap(&tm_v);
-        for (int kt = 0; kt < min(nkt, kEarly); ++kt) {
-            load_tile(&tm_k, k_ring + (size_t)kt * kTileKV, kt, kfull0 + 8 * kt);
-            load_tile(&tm_v, v_ring + (size_t)kt * kTileKV, kt, vfull0 + 8 * kt);
-        }
-    }
     if (tid == 0) {
+        for (int s = 0; s < 2 * SK + 2 * SV; ++s) mbar_init(kfull0 + 8 * s, 1);
         for (int g = 0; g < NG; ++g) {
-            mbar_init(gbar0 + 32 * g, 1);
-            mbar_init(gbar0 + 32 * g + 8, 1);
-            mbar_init(gbar0 + 32 * g + 16, 128);
-            mbar_init(gbar0 + 32 * g + 24, 1);
+            mbar_init(gbar0 + 48 * g, 1);
+            mbar_init(gbar0 + 48 * g + 8, 1);
+            mbar_init(gbar0 + 48 * g + 16, 128);
+            mbar_init(gbar0 + 48 * g + 24, 1);
+            mbar_init(gbar0 + 48 * g + 32, 1);
+            mbar_init(gbar0 + 48 * g + 40, 1);
         }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -247,19 +230,6 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                      ::"r"(smem_u32(tmem_slot)), "n"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // stage Q (rows past the prompt as zeros): element (r, d) of a group -> half d/64, row r, 16-byte
-    // chunk ((d%64)/8) ^ (r%8): the layout TMA's 128-byte swizzle would have produced
-    const T* qbase = reinterpret_cast<const T*>(p.q) + ((size_t)b * p.N * p.H + h) * kD;
-    const size_t qstride = (size_t)p.H * kD;
-    for (int i = tid; i < NG * kRows * 16; i += L::kThreads) {
-        const int rr = i >> 4, c = i & 15, grow = row_cta + rr;
-        const int g = rr / kRows, r = rr % kRows;
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (grow < p.N) v = *reinterpret_cast<const uint4*>(qbase + (size_t)grow * qstride + c * 8);
-        *reinterpret_cast<uint4*>(q_smem + (size_t)(2 * g + (c >> 3)) * kBoxQ + (size_t)r * 128 +
-                                  (size_t)(((c ^ r) & 7) << 4)) = v;
-    }
-    fence_proxy_async();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -268,177 +238,237 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (warp == 4 * NG) {
         // ------------------------------- TMA producer -------------------------------
         if (lane == 0) {
-            for (int kt = kEarly; kt < nkt; ++kt) {
-                const int sk = kt % SK, sv = kt % SV;
-                if (!mbar_wait(kempty0 + 8 * sk, (((uint32_t)(kt / SK)) & 1) ^ 1)) { s_abort = 1; break; }
-                load_tile(&tm_k, k_ring + (size_t)sk * kTileKV, kt, kfull0 + 8 * sk);
-                if (!mbar_wait(vempty0 + 8 * sv, (((uint32_t)(kt / SV)) & 1) ^ 1)) { s_abort = 1; break; }
-                load_tile(&tm_v, v_ring + (size_t)sv * kTileKV, kt, vfull0 + 8 * sv);
+            prefetch_tmap(&tm_q);
+            prefetch_tmap(&tm_k);
+            prefetch_tmap(&tm_v);
+            auto load_tile = [&](const CUtensorMap* tm, uint8_t* dst_tile, int kt, int slab, uint32_t full) {
+                const uint32_t dst = smem_u32(dst_tile);
+                mbar_arrive_expect_tx(full, (uint32_t)kTileKV);
+#pragma unroll
+                for (int half = 0; half < 2; ++half)
+#pragma unroll
+                    for (int rb = 0; rb < kKeys / kBoxRows; ++rb)
+                        tma_load_3d(dst + half * kHalfTile + rb * kBoxBytes, tm, half * 64,
+                                    kt * kKeys + rb * kBoxRows, slab, full);
+            };
+            uint32_t T = 0;                                       // K/V tiles requested so far (ring position)
+            uint32_t qi[NG];                                      // items group g has taken part in: Q barrier phases
+#pragma unroll
+            for (int g = 0; g < NG; ++g) qi[g] = 0;
+            bool ok = true;
+            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+                const int qt = item_qt(w), hb = w % hb_count, h = hb % p.H, b = hb / p.H;
+                const int slab = b * p.Hkv + h / p.G;
+                int nkt = 0;
+#pragma unroll
+                for (int g = 0; g < NG; ++g) {
+                    const int gt = group_tiles(qt, g);
+                    nkt = max(nkt, gt);
+                    if (gt == 0) continue;
+                    // the group's Q rows (past the prompt: zeros), once its previous Q is no longer read
+                    ok = mbar_wait(gbar0 + 48 * g + 40, (qi[g] & 1) ^ 1);
+                    if (!ok) break;
+                    ++qi[g];
+                    const uint32_t qfull = gbar0 + 48 * g + 32;
+                    const uint32_t dst = smem_u32(q_smem) + (uint32_t)g * 2 * kBoxQ;
+                    mbar_arrive_expect_tx(qfull, 2u * kBoxQ);
+                    tma_load_4d(dst, &tm_q, 0, h, (qt * NG + g) * kRows, b, qfull);
+                    tma_load_4d(dst + kBoxQ, &tm_q, 64, h, (qt * NG + g) * kRows, b, qfull);
+                }
+                for (int kt = 0; kt < nkt && ok; ++kt, ++T) {
+                    const uint32_t sk = T % SK, sv = T % SV;
+                    ok = mbar_wait(kempty0 + 8 * sk, ((T / SK) & 1) ^ 1);
+                    if (!ok) break;
+                    load_tile(&tm_k, k_ring + (size_t)sk * kTileKV, kt, slab, kfull0 + 8 * sk);
+                    ok = mbar_wait(vempty0 + 8 * sv, ((T / SV) & 1) ^ 1);
+                    if (!ok) break;
+                    load_tile(&tm_v, v_ring + (size_t)sv * kTileKV, kt, slab, vfull0 + 8 * sv);
+                }
             }
+            if (!ok) s_abort = 1;
         }
     } else if (warp == 4 * NG + 1) {
         // -------------------------------- MMA issuer --------------------------------
         if (lane == 0) {
-            int gt[NG];
+            uint32_t T = 0;                                       // ring position of the item's first K/V tile
+            uint32_t n[NG], qi[NG];                               // tiles / items of group g so far: barrier phases
 #pragma unroll
-            for (int g = 0; g < NG; ++g) gt[g] = group_tiles(g);
-            auto issue_qk = [&](int g, int kt, int buf) {         // S_g[buf] = Q_g . K_kt^T
-                const uint32_t q_addr = smem_u32(q_smem) + (uint32_t)g * 2 * kBoxQ;
-                const uint32_t k_addr = smem_u32(k_ring + (size_t)(kt % SK) * kTileKV);
-#pragma unroll
-                for (int ks = 0; ks < kD / 16; ++ks) {
-                    const uint32_t off = (uint32_t)(ks & 3) * 32;
-                    tc_mma_ss(tmem + 128u * (uint32_t)(g + buf),
-                              smem_desc(q_addr + (ks >> 2) * kBoxQ + off, 16, 1024),
-                              smem_desc(k_addr + (ks >> 2) * kHalfTile + off, 16, 1024), p.idesc_qk, ks > 0);
-                }
-                tc_commit(gbar0 + 32 * g + 8 * buf);
-            };
-            auto wait_k = [&](int kt) -> bool {
-                const bool ok = mbar_wait_hot(kfull0 + 8 * (kt % SK), ((uint32_t)(kt / SK)) & 1);
-                tc_fence_after();
-                return ok;
-            };
-            bool ok = wait_k(0);
-            if (ok) {
-#pragma unroll
-                for (int g = 0; g < NG; ++g)
-                    if (gt[g] > 0) issue_qk(g, 0, 0);
-                tc_commit(kempty0);                               // K stage free once these MMAs are done
-            }
-            for (int kt = 0; kt < nkt && ok; ++kt) {
-                TC5_STAMP(2, kt, 0);
-                if (NB == 2 && kt + 1 < nkt) {                    // next tile's scores run under this tile's softmax
-                    ok = wait_k(kt + 1);
-                    if (!ok) break;
-#pragma unroll
-                    for (int g = 0; g < NG; ++g)
-                        if (kt + 1 < gt[g]) issue_qk(g, kt + 1, (kt + 1) & 1);
-                    tc_commit(kempty0 + 8 * ((kt + 1) % SK));
-                }
-                TC5_STAMP(2, kt, 1);
-                const int sv = kt % SV;
-                const uint32_t v_addr = smem_u32(v_ring + (size_t)sv * kTileKV);
-                ok = mbar_wait_hot(vfull0 + 8 * sv, ((uint32_t)(kt / SV)) & 1);
-                if (!ok) break;
-                TC5_STAMP(2, kt, 2);
-                bool k_next = false;
+            for (int g = 0; g < NG; ++g) n[g] = qi[g] = 0;
+            bool ok = true;
+            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+                const int qt = item_qt(w);
+                int gt[NG], nkt = 0;
 #pragma unroll
                 for (int g = 0; g < NG; ++g) {
-                    if (kt >= gt[g]) continue;
-                    ok = mbar_wait_hot(gbar0 + 32 * g + 16, (uint32_t)kt & 1);   // P_g written over its S buffer
-                    if (!ok) break;
-                    TC5_STAMP(2, kt, 3 + 2 * g);
-                    tc_fence_after();
-                    const uint32_t p_tmem = tmem + 128u * (uint32_t)(g + (NB == 2 ? (kt & 1) : 0));
-#pragma unroll
-                    for (int kk = 0; kk < kKeys / 16; ++kk)       // O_g += P_g[:, 16 keys] . V[16 keys, :]
-                        tc_mma_ts(tmem + 256u + 128u * (uint32_t)g, p_tmem + kk * 8,
-                                  smem_desc(v_addr + kk * 2048, kHalfTile, 1024), p.idesc_pv, (kt > 0 || kk > 0));
-                    tc_commit(gbar0 + 32 * g + 24);
-                    if (NB == 1 && kt + 1 < gt[g]) {              // the group's next scores, behind its P.V in the pipe
-                        if (!k_next) {
-                            ok = wait_k(kt + 1);
-                            if (!ok) break;
-                            k_next = true;
-                        }
-                        issue_qk(g, kt + 1, 0);
-                    }
-                    TC5_STAMP(2, kt, 4 + 2 * g);
+                    gt[g] = group_tiles(qt, g);
+                    nkt = max(nkt, gt[g]);
                 }
+                // S_g[buf] = Q_g . K^T for the group's tile kt; after its last one the group's Q may be replaced
+                auto issue_qk = [&](int g, int kt, int buf) {
+                    const uint32_t q_addr = smem_u32(q_smem) + (uint32_t)g * 2 * kBoxQ;
+                    const uint32_t k_addr = smem_u32(k_ring + (size_t)((T + kt) % SK) * kTileKV);
+#pragma unroll
+                    for (int ks = 0; ks < kD / 16; ++ks) {
+                        const uint32_t off = (uint32_t)(ks & 3) * 32;
+                        tc_mma_ss(tmem + 128u * (uint32_t)(g + buf),
+                                  smem_desc(q_addr + (ks >> 2) * kBoxQ + off, 16, 1024),
+                                  smem_desc(k_addr + (ks >> 2) * kHalfTile + off, 16, 1024), p.idesc_qk, ks > 0);
+                    }
+                    tc_commit(gbar0 + 48 * g + 8 * buf);
+                    if (kt + 1 == gt[g]) tc_commit(gbar0 + 48 * g + 40);
+                };
+                auto wait_k = [&](int kt) -> bool {
+                    const bool r = mbar_wait_hot(kfull0 + 8 * ((T + kt) % SK), ((T + kt) / SK) & 1);
+                    tc_fence_after();
+                    return r;
+                };
+#pragma unroll
+                for (int g = 0; g < NG; ++g)
+                    if (gt[g] > 0 && ok) ok = mbar_wait_hot(gbar0 + 48 * g + 32, qi[g]++ & 1);   // Q_g landed
+                if (ok) ok = wait_k(0);
                 if (!ok) break;
-                tc_commit(vempty0 + 8 * sv);                      // stages free once every MMA so far is done
-                if (NB == 1 && kt + 1 < nkt) tc_commit(kempty0 + 8 * ((kt + 1) % SK));
+#pragma unroll
+                for (int g = 0; g < NG; ++g)
+                    if (gt[g] > 0) issue_qk(g, 0, NB == 2 ? (int)(n[g] & 1) : 0);
+                tc_commit(kempty0 + 8 * (T % SK));                // K stage free once these MMAs are done
+                for (int kt = 0; kt < nkt && ok; ++kt) {
+                    TC5_STAMP(2, kt, 0);
+                    if (NB == 2 && kt + 1 < nkt) {                // next tile's scores run under this tile's softmax
+                        ok = wait_k(kt + 1);
+                        if (!ok) break;
+#pragma unroll
+                        for (int g = 0; g < NG; ++g)
+                            if (kt + 1 < gt[g]) issue_qk(g, kt + 1, (int)((n[g] + 1) & 1));
+                        tc_commit(kempty0 + 8 * ((T + kt + 1) % SK));
+                    }
+                    const uint32_t sv = (T + kt) % SV;
+                    const uint32_t v_addr = smem_u32(v_ring + (size_t)sv * kTileKV);
+                    ok = mbar_wait_hot(vfull0 + 8 * sv, ((T + kt) / SV) & 1);
+                    if (!ok) break;
+                    bool k_next = false;
+#pragma unroll
+                    for (int g = 0; g < NG; ++g) {
+                        if (kt >= gt[g]) continue;
+                        ok = mbar_wait_hot(gbar0 + 48 * g + 16, n[g] & 1);   // P_g written over its S buffer
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t p_tmem = tmem + 128u * (uint32_t)(g + (NB == 2 ? (int)(n[g] & 1) : 0));
+#pragma unroll
+                        for (int kk = 0; kk < kKeys / 16; ++kk)   // O_g += P_g[:, 16 keys] . V[16 keys, :]
+                            tc_mma_ts(tmem + 256u + 128u * (uint32_t)g, p_tmem + kk * 8,
+                                      smem_desc(v_addr + kk * 2048, kHalfTile, 1024), p.idesc_pv, (kt > 0 || kk > 0));
+                        tc_commit(gbar0 + 48 * g + 24);
+                        ++n[g];
+                        if (NB == 1 && kt + 1 < gt[g]) {          // the group's next scores, behind its P.V in the pipe
+                            if (!k_next) {
+                                ok = wait_k(kt + 1);
+                                if (!ok) break;
+                                k_next = true;
+                            }
+                            issue_qk(g, kt + 1, 0);
+                        }
+                    }
+                    if (!ok) break;
+                    tc_commit(vempty0 + 8 * sv);                  // stages free once every MMA so far is done
+                    if (NB == 1 && kt + 1 < nkt) tc_commit(kempty0 + 8 * ((T + kt + 1) % SK));
+                }
+                T += (uint32_t)nkt;
             }
             if (!ok) s_abort = 1;
         }
     } else {
         // ------------------------------ softmax warps: one row per thread ------------------------------
         const int g = warp >> 2, r = tid & (kRows - 1);
-        const int row = row_cta + g * kRows + r;
-        const int my_tiles = group_tiles(g);
-        const uint32_t bar_s0 = gbar0 + 32 * g, bar_p = bar_s0 + 16, bar_o = bar_s0 + 24;
+        const uint32_t bar_s0 = gbar0 + 48 * g, bar_p = bar_s0 + 16, bar_o = bar_s0 + 24;
         const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);     // this warp's TMEM lanes
         const uint32_t tm_o = tm_lane + 256u + 128u * (uint32_t)g;
-        const float slope2 = p.slopes ? p.slopes[h] * 1.4426950408889634f : 0.f;
         const bool stamp = lane == 0 && (warp & 3) == 0;
-        float m_ref = -INFINITY, l_run = 0.f;
+        const size_t qstride = (size_t)p.H * kD;
+        uint32_t n = 0;                                           // tiles of this group so far: barrier phases
         bool ok = true;
-        for (int kt = 0; kt < my_tiles; ++kt) {
-            const int buf = NB == 2 ? (kt & 1) : 0;
-            const uint32_t tm_s = tm_lane + 128u * (uint32_t)(g + buf);
-            ok = mbar_wait_hot(bar_s0 + 8 * buf, (uint32_t)(NB == 2 ? (kt >> 1) : kt) & 1);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            if (stamp) TC5_STAMP(g, kt, 0);
-            tc_fence_after();
-            uint32_t sr[kKeys];
-#pragma unroll
-            for (int c = 0; c < kKeys / 32; ++c) tc_ld32(tm_s + 32 * c, sr + 32 * c);
-            tc_wait_ld();
-            if (stamp) TC5_STAMP(g, kt, 1);
-            float* sv = reinterpret_cast<float*>(sr);
-            const int key0 = kt * kKeys;
-            const bool diag = key0 + kKeys - 1 > row_cta + g * kRows;   // the group's diagonal tile
-            // scores in log2 units: s * scale2 (+ ALiBi bias); the scale is folded into the exponent's
-            // FMA unless a bias has to be added first; keys above the row (diagonal tile) become -inf
-            const bool biased = p.slopes != nullptr;
-            const int lim = row - key0;                            // key index i of this tile is visible iff i <= lim
-            const float bias0 = slope2 * (float)(key0 - row);
-            float tmax;
-            if (biased) tmax = diag ? score_max<true, true>(sv, p.scale2, slope2, bias0, lim)
-                                    : score_max<true, false>(sv, p.scale2, slope2, bias0, lim);
-            else tmax = (diag ? score_max<false, true>(sv, p.scale2, slope2, bias0, lim)
-                              : score_max<false, false>(sv, p.scale2, slope2, bias0, lim)) * p.scale2;
-            // a new reference only when the maximum has grown by more than 2^8: exponentials stay
-            // below 2^8 of the reference, the sum and O use the same reference
-            const bool need = tmax > m_ref + 8.f;
-            float alpha = 1.f;
-            if (need) {
-                alpha = exp2f(m_ref - tmax);                       // 0 on the first tile
-                m_ref = tmax;
-            }
-            float ls[4] = {0.f, 0.f, 0.f, 0.f};
-            uint32_t pk[kKeys / 2];
-            const float sc = biased ? 1.f : p.scale2, nm = -m_ref;
-#pragma unroll
-            for (int i = 0; i < kKeys; i += 2) {
-                const float e0 = exp2f(fmaf(sv[i], sc, nm)), e1 = exp2f(fmaf(sv[i + 1], sc, nm));
-                ls[(i >> 1) & 3] += e0 + e1;
-                pk[i >> 1] = Mma<T>::pack(e0, e1);
-            }
-            l_run = l_run * alpha + ((ls[0] + ls[1]) + (ls[2] + ls[3]));
-            if (stamp) TC5_STAMP(g, kt, 2);
-            if (kt > 0 && __any_sync(0xffffffffu, need)) {
-                ok = mbar_wait_hot(bar_o, (uint32_t)(kt - 1) & 1); // P.V of the previous tile done: O stable
+        for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+            const int qt = item_qt(w), hb = w % hb_count, h = hb % p.H, b = hb / p.H;
+            const int my_tiles = group_tiles(qt, g);
+            if (my_tiles == 0) continue;
+            const int row0 = (qt * NG + g) * kRows, row = row0 + r;
+            const float slope2 = p.slopes ? p.slopes[h] * 1.4426950408889634f : 0.f;
+            float m_ref = -INFINITY, l_run = 0.f;
+            for (int kt = 0; kt < my_tiles; ++kt, ++n) {
+                const int buf = NB == 2 ? (int)(n & 1) : 0;
+                const uint32_t tm_s = tm_lane + 128u * (uint32_t)(g + buf);
+                ok = mbar_wait_hot(bar_s0 + 8 * buf, (NB == 2 ? (n >> 1) : n) & 1);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+                if (stamp) TC5_STAMP(g, kt, 0);
                 tc_fence_after();
+                uint32_t sr[kKeys];
 #pragma unroll
-                for (int c = 0; c < kD / 32; ++c) {
-                    uint32_t orr[32];
-                    tc_ld32(tm_o + c * 32, orr);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
-                    tc_st32(tm_o + c * 32, orr);
+                for (int c = 0; c < kKeys / 32; ++c) tc_ld32(tm_s + 32 * c, sr + 32 * c);
+                tc_wait_ld();
+                if (stamp) TC5_STAMP(g, kt, 1);
+                float* sv = reinterpret_cast<float*>(sr);
+                const int key0 = kt * kKeys;
+                const bool diag = key0 + kKeys - 1 > row0;         // the group's diagonal tile
+                // scores in log2 units: s * scale2 (+ ALiBi bias); the scale is folded into the exponent's
+                // FMA unless a bias has to be added first; keys above the row (diagonal tile) become -inf
+                const bool biased = p.slopes != nullptr;
+                const int lim = row - key0;                        // key index i of this tile is visible iff i <= lim
+                const float bias0 = slope2 * (float)(key0 - row);
+                float tmax;
+                if (biased) tmax = diag ? score_max<true, true>(sv, p.scale2, slope2, bias0, lim)
+                                        : score_max<true, false>(sv, p.scale2, slope2, bias0, lim);
+                else tmax = (diag ? score_max<false, true>(sv, p.scale2, slope2, bias0, lim)
+                                  : score_max<false, false>(sv, p.scale2, slope2, bias0, lim)) * p.scale2;
+                // a new reference only when the maximum has grown by more than 2^8: exponentials stay
+                // below 2^8 of the reference, the sum and O use the same reference
+                const bool need = tmax > m_ref + 8.f;
+                float alpha = 1.f;
+                if (need) {
+                    alpha = exp2f(m_ref - tmax);                   // 0 on the first tile
+                    m_ref = tmax;
                 }
-                if (stamp) TC5_STAMP(g, kt, 3);
-            }
-            // P over the first 64 columns of the S buffer: two 16-bit weights per column, the A
-            // operand layout of the MMA that follows.  S has been read completely above.
+                float ls[4] = {0.f, 0.f, 0.f, 0.f};
+                uint32_t pk[kKeys / 2];
+                const float sc = biased ? 1.f : p.scale2, nm = -m_ref;
 #pragma unroll
-            for (int c = 0; c < kKeys / 32; ++c) tc_st16(tm_s + 16 * c, pk + 16 * c);
-            tc_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar_p);
-            if (stamp) TC5_STAMP(g, kt, 4);
-        }
-        if (ok && my_tiles > 0) {
-            ok = mbar_wait_hot(bar_o, (uint32_t)(my_tiles - 1) & 1);
+                for (int i = 0; i < kKeys; i += 2) {
+                    const float e0 = exp2f(fmaf(sv[i], sc, nm)), e1 = exp2f(fmaf(sv[i + 1], sc, nm));
+                    ls[(i >> 1) & 3] += e0 + e1;
+                    pk[i >> 1] = Mma<T>::pack(e0, e1);
+                }
+                l_run = l_run * alpha + ((ls[0] + ls[1]) + (ls[2] + ls[3]));
+                if (stamp) TC5_STAMP(g, kt, 2);
+                if (kt > 0 && __any_sync(0xffffffffu, need)) {
+                    ok = mbar_wait_hot(bar_o, (n - 1) & 1);        // P.V of the previous tile done: O stable
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < kD / 32; ++c) {
+                        uint32_t orr[32];
+                        tc_ld32(tm_o + c * 32, orr);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+                        tc_st32(tm_o + c * 32, orr);
+                    }
+                    if (stamp) TC5_STAMP(g, kt, 3);
+                }
+                // P over the first 64 columns of the S buffer: two 16-bit weights per column, the A
+                // operand layout of the MMA that follows.  S has been read completely above.
+#pragma unroll
+                for (int c = 0; c < kKeys / 32; ++c) tc_st16(tm_s + 16 * c, pk + 16 * c);
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar_p);
+                if (stamp) TC5_STAMP(g, kt, 4);
+            }
+            if (!ok) break;
+            // the item's output: O / l, once the last P.V has landed.  The next item's first P.V
+            // cannot overwrite O before these loads: it waits for this thread's next P arrival.
+            ok = mbar_wait_hot(bar_o, (n - 1) & 1);
             ok = __all_sync(0xffffffffu, ok);
-        }
-        if (ok && my_tiles > 0) {
+            if (!ok) break;
             tc_fence_after();
             const float inv = 1.f / l_run;
             T* orow = reinterpret_cast<T*>(p.out) + ((size_t)b * p.N * p.H + h) * kD + (size_t)row * qstride;
@@ -457,9 +487,8 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                             Mma<T>::pack(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv));
                 }
             }
-        } else if (!ok && lane == 0) {
-            s_abort = 1;
         }
+        if (!ok && lane == 0) s_abort = 1;
     }
     tc_fence_before();
     __syncthreads();
@@ -471,7 +500,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 }
 
 template <typename T, int NG>
-cudaError_t launch_tc5(const Dims& d, const PrefillArgs& a, const Tc5Params& p, cudaStream_t st) {
+cudaError_t launch_tc5(const Dims& d, const PrefillArgs& a, const Tc5Params& p, int sms, cudaStream_t st) {
     using L = Tc5Layout<NG>;
     auto kern = prefill_tc5_kernel<T, NG>;
     static bool configured[64] = {false};
@@ -482,8 +511,9 @@ cudaError_t launch_tc5(const Dims& d, const PrefillArgs& a, const Tc5Params& p, 
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-    dim3 grid((unsigned)((a.prompt_len + kRows * NG - 1) / (kRows * NG)), (unsigned)d.heads, (unsigned)d.batch);
-    kern<<<grid, L::kThreads, L::kBytes, st>>>(*a.tm_k, *a.tm_v, p);
+    const long items = (long)((a.prompt_len + kRows * NG - 1) / (kRows * NG)) * d.heads * d.batch;
+    const unsigned grid = (unsigned)(items < sms ? items : sms);  // one CTA per SM: the shared memory allows no more
+    kern<<<grid, L::kThreads, L::kBytes, st>>>(*a.tm_q, *a.tm_k, *a.tm_v, p);
     return cudaGetLastError();
 }
 
@@ -496,7 +526,7 @@ cudaError_t launch_prefill_tc5(const Dims& d, const PrefillArgs& a, cudaStream_t
     const bool bf = d.dtype == SEGKV_BF16;
     Tc5Params p;
     p.q = a.q; p.out = a.out; p.slopes = a.slopes; p.err_word = a.err_word;
-    p.N = a.prompt_len; p.H = d.heads; p.Hkv = d.kv_heads; p.G = d.group;
+    p.N = a.prompt_len; p.H = d.heads; p.Hkv = d.kv_heads; p.G = d.group; p.B = d.batch;
     p.scale2 = 1.4426950408889634f / sqrtf((float)kD);
     // instruction descriptor: fp32 accumulate, A/B format, operand majors, N >> 3, M >> 4
     const uint32_t fmt = bf ? 1u : 0u;
@@ -512,8 +542,8 @@ cudaError_t launch_prefill_tc5(const Dims& d, const PrefillArgs& a, cudaStream_t
     }
     const long ctas2 = (long)((a.prompt_len + 2 * kRows - 1) / (2 * kRows)) * d.heads * d.batch;
     const bool two = a.row_groups ? a.row_groups == 2 : ctas2 >= 2L * sms;
-    if (two) return bf ? launch_tc5<__nv_bfloat16, 2>(d, a, p, st) : launch_tc5<__half, 2>(d, a, p, st);
-    return bf ? launch_tc5<__nv_bfloat16, 1>(d, a, p, st) : launch_tc5<__half, 1>(d, a, p, st);
+    if (two) return bf ? launch_tc5<__nv_bfloat16, 2>(d, a, p, sms, st) : launch_tc5<__half, 2>(d, a, p, sms, st);
+    return bf ? launch_tc5<__nv_bfloat16, 1>(d, a, p, sms, st) : launch_tc5<__half, 1>(d, a, p, sms, st);
 }
 
 }  // namespace segkv_impl
