@@ -50,6 +50,8 @@ def parse():
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--combine", type=int, default=0, help="0 auto, 1 workspace+ticket, 2 cluster")
     ap.add_argument("--prefill", action="store_true", help="time the prefill attention instead of the decode step")
+    ap.add_argument("--prefill-groups", type=int, default=0,
+                    help="128-row groups per CTA of the head_dim-128 prefill kernel (1 or 2; 0 = automatic)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="turn programmatic dependent launch off")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -416,6 +418,8 @@ def run_prefill(args):
         h = SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, 1, w.torch_dtype)
         kp, vp = wl.make_prompt(wl_layer, dev)
         h.prefill_write(kp, vp)
+        if args.prefill_groups:
+            h.set_prefill_tuning(args.prefill_groups)
         del kp, vp
         q = wl.make_prefill_query(wl_layer, dev)
         handles.append((h, q, torch.empty_like(q)))
@@ -448,7 +452,8 @@ def run_prefill(args):
                    "head_dim": w.head_dim, "prompt_len": n, "layers_rotated": L},
         "roofline": {"bound": "tensor", "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak,
                      "traffic": None, "peak_kind": f"of {kind} (bf16 GEMM burst; fp16 has the same nominal rate)",
-                     "kernel": "segkv prefill attention (mma.sync m16n8k16)"},
+                     "kernel": ("segkv prefill attention (tcgen05, S/P/O in tensor memory, persistent CTAs)"
+                                if w.head_dim == 128 else "segkv prefill attention (mma.sync m16n8k16)")},
         "gpu_launches": args.steps * L}))
 
 

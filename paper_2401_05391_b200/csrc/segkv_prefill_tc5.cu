@@ -137,7 +137,7 @@ __device__ long long g_tc5_tl[3 * 64 * 8];
 #define TC5_STAMP(role, kt, ev)                                                                   \
     do {                                                                                          \
         if ((SEGKV_TC5_TIMELINE != 2 || ((role) == 2 && (ev) == 0)) &&                            \
-            blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (kt) < 64)                   \
+            w == 0 && (kt) < 64)                                                                 \
             g_tc5_tl[((role) * 64 + (kt)) * 8 + (ev)] = clock64();                                \
     } while (0)
 namespace {
@@ -251,7 +251,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         tma_load_3d(dst + half * kHalfTile + rb * kBoxBytes, tm, half * 64,
                                     kt * kKeys + rb * kBoxRows, slab, full);
             };
-            uint32_t T = 0;                                       // K/V tiles requested so far (ring position)
+            uint32_t tp = 0;                                       // K/V tiles requested so far (ring position)
             uint32_t qi[NG];                                      // items group g has taken part in: Q barrier phases
 #pragma unroll
             for (int g = 0; g < NG; ++g) qi[g] = 0;
@@ -275,12 +275,12 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     tma_load_4d(dst, &tm_q, 0, h, (qt * NG + g) * kRows, b, qfull);
                     tma_load_4d(dst + kBoxQ, &tm_q, 64, h, (qt * NG + g) * kRows, b, qfull);
                 }
-                for (int kt = 0; kt < nkt && ok; ++kt, ++T) {
-                    const uint32_t sk = T % SK, sv = T % SV;
-                    ok = mbar_wait(kempty0 + 8 * sk, ((T / SK) & 1) ^ 1);
+                for (int kt = 0; kt < nkt && ok; ++kt, ++tp) {
+                    const uint32_t sk = tp % SK, sv = tp % SV;
+                    ok = mbar_wait(kempty0 + 8 * sk, ((tp / SK) & 1) ^ 1);
                     if (!ok) break;
                     load_tile(&tm_k, k_ring + (size_t)sk * kTileKV, kt, slab, kfull0 + 8 * sk);
-                    ok = mbar_wait(vempty0 + 8 * sv, ((T / SV) & 1) ^ 1);
+                    ok = mbar_wait(vempty0 + 8 * sv, ((tp / SV) & 1) ^ 1);
                     if (!ok) break;
                     load_tile(&tm_v, v_ring + (size_t)sv * kTileKV, kt, slab, vfull0 + 8 * sv);
                 }
@@ -290,7 +290,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     } else if (warp == 4 * NG + 1) {
         // -------------------------------- MMA issuer --------------------------------
         if (lane == 0) {
-            uint32_t T = 0;                                       // ring position of the item's first K/V tile
+            uint32_t tp = 0;                                       // ring position of the item's first K/V tile
             uint32_t n[NG], qi[NG];                               // tiles / items of group g so far: barrier phases
 #pragma unroll
             for (int g = 0; g < NG; ++g) n[g] = qi[g] = 0;
@@ -306,7 +306,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 // S_g[buf] = Q_g . K^T for the group's tile kt; after its last one the group's Q may be replaced
                 auto issue_qk = [&](int g, int kt, int buf) {
                     const uint32_t q_addr = smem_u32(q_smem) + (uint32_t)g * 2 * kBoxQ;
-                    const uint32_t k_addr = smem_u32(k_ring + (size_t)((T + kt) % SK) * kTileKV);
+                    const uint32_t k_addr = smem_u32(k_ring + (size_t)((tp + kt) % SK) * kTileKV);
 #pragma unroll
                     for (int ks = 0; ks < kD / 16; ++ks) {
                         const uint32_t off = (uint32_t)(ks & 3) * 32;
@@ -318,7 +318,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     if (kt + 1 == gt[g]) tc_commit(gbar0 + 48 * g + 40);
                 };
                 auto wait_k = [&](int kt) -> bool {
-                    const bool r = mbar_wait_hot(kfull0 + 8 * ((T + kt) % SK), ((T + kt) / SK) & 1);
+                    const bool r = mbar_wait_hot(kfull0 + 8 * ((tp + kt) % SK), ((tp + kt) / SK) & 1);
                     tc_fence_after();
                     return r;
                 };
@@ -330,7 +330,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
                 for (int g = 0; g < NG; ++g)
                     if (gt[g] > 0) issue_qk(g, 0, NB == 2 ? (int)(n[g] & 1) : 0);
-                tc_commit(kempty0 + 8 * (T % SK));                // K stage free once these MMAs are done
+                tc_commit(kempty0 + 8 * (tp % SK));                // K stage free once these MMAs are done
                 for (int kt = 0; kt < nkt && ok; ++kt) {
                     TC5_STAMP(2, kt, 0);
                     if (NB == 2 && kt + 1 < nkt) {                // next tile's scores run under this tile's softmax
@@ -339,11 +339,11 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
                         for (int g = 0; g < NG; ++g)
                             if (kt + 1 < gt[g]) issue_qk(g, kt + 1, (int)((n[g] + 1) & 1));
-                        tc_commit(kempty0 + 8 * ((T + kt + 1) % SK));
+                        tc_commit(kempty0 + 8 * ((tp + kt + 1) % SK));
                     }
-                    const uint32_t sv = (T + kt) % SV;
+                    const uint32_t sv = (tp + kt) % SV;
                     const uint32_t v_addr = smem_u32(v_ring + (size_t)sv * kTileKV);
-                    ok = mbar_wait_hot(vfull0 + 8 * sv, ((T + kt) / SV) & 1);
+                    ok = mbar_wait_hot(vfull0 + 8 * sv, ((tp + kt) / SV) & 1);
                     if (!ok) break;
                     bool k_next = false;
 #pragma unroll
@@ -351,6 +351,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         if (kt >= gt[g]) continue;
                         ok = mbar_wait_hot(gbar0 + 48 * g + 16, n[g] & 1);   // P_g written over its S buffer
                         if (!ok) break;
+                        TC5_STAMP(2, kt, 1 + 3 * g);
                         tc_fence_after();
                         const uint32_t p_tmem = tmem + 128u * (uint32_t)(g + (NB == 2 ? (int)(n[g] & 1) : 0));
 #pragma unroll
@@ -358,6 +359,10 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             tc_mma_ts(tmem + 256u + 128u * (uint32_t)g, p_tmem + kk * 8,
                                       smem_desc(v_addr + kk * 2048, kHalfTile, 1024), p.idesc_pv, (kt > 0 || kk > 0));
                         tc_commit(gbar0 + 48 * g + 24);
+#if defined(SEGKV_TC5_TIMELINE) && SEGKV_TC5_TIMELINE == 3
+                        mbar_wait_hot(gbar0 + 48 * g + 24, n[g] & 1);   // measurement only: serialise on P.V
+                        TC5_STAMP(2, kt, 2 + 3 * g);
+#endif
                         ++n[g];
                         if (NB == 1 && kt + 1 < gt[g]) {          // the group's next scores, behind its P.V in the pipe
                             if (!k_next) {
@@ -366,13 +371,17 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                                 k_next = true;
                             }
                             issue_qk(g, kt + 1, 0);
+#if defined(SEGKV_TC5_TIMELINE) && SEGKV_TC5_TIMELINE == 3
+                            mbar_wait_hot(gbar0 + 48 * g, n[g] & 1);    // measurement only: serialise on Q.K^T
+                            TC5_STAMP(2, kt, 3 + 3 * g);
+#endif
                         }
                     }
                     if (!ok) break;
                     tc_commit(vempty0 + 8 * sv);                  // stages free once every MMA so far is done
-                    if (NB == 1 && kt + 1 < nkt) tc_commit(kempty0 + 8 * ((T + kt + 1) % SK));
+                    if (NB == 1 && kt + 1 < nkt) tc_commit(kempty0 + 8 * ((tp + kt + 1) % SK));
                 }
-                T += (uint32_t)nkt;
+                tp += (uint32_t)nkt;
             }
             if (!ok) s_abort = 1;
         }
