@@ -50,7 +50,7 @@ struct Tc5Params {
     void* out;
     const float* slopes;
     int* err_word;
-    int N, H, Hkv, G, B;
+    int N, H, Hkv, G, B, snake;
     float scale2;
     uint32_t idesc_qk, idesc_pv;
 };
@@ -203,6 +203,13 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const int nqt = (p.N + kRows * NG - 1) / (kRows * NG);
     const int hb_count = p.H * p.B;
     const int n_items = nqt * hb_count;
+    // The CTA's item of round j: the list is sorted longest first and dealt out round-robin; with
+    // only a few rounds, in snake order (every other round reversed), which evens out the total
+    // length per CTA.
+    auto round_item = [&](int j) -> int {
+        const int G = (int)gridDim.x, c = (int)blockIdx.x;
+        return j * G + ((p.snake && (j & 1)) ? G - 1 - c : c);
+    };
     // item w -> query tile (longest first), head, request
     auto item_qt = [&](int w) { return nqt - 1 - w / hb_count; };
     // key tiles of group g of query tile qt: up to its diagonal tile (causal); none past the prompt
@@ -256,7 +263,9 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
             for (int g = 0; g < NG; ++g) qi[g] = 0;
             bool ok = true;
-            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+            for (int j = 0; j * (int)gridDim.x < n_items && ok; ++j) {
+                const int w = round_item(j);
+                if (w >= n_items) continue;
                 const int qt = item_qt(w), hb = w % hb_count, h = hb % p.H, b = hb / p.H;
                 const int slab = b * p.Hkv + h / p.G;
                 int nkt = 0;
@@ -295,7 +304,9 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
             for (int g = 0; g < NG; ++g) n[g] = qi[g] = 0;
             bool ok = true;
-            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+            for (int j = 0; j * (int)gridDim.x < n_items && ok; ++j) {
+                const int w = round_item(j);
+                if (w >= n_items) continue;
                 const int qt = item_qt(w);
                 int gt[NG], nkt = 0;
 #pragma unroll
@@ -395,7 +406,9 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const size_t qstride = (size_t)p.H * kD;
         uint32_t n = 0;                                           // tiles of this group so far: barrier phases
         bool ok = true;
-        for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+        for (int j = 0; j * (int)gridDim.x < n_items && ok; ++j) {
+            const int w = round_item(j);
+            if (w >= n_items) continue;
             const int qt = item_qt(w), hb = w % hb_count, h = hb % p.H, b = hb / p.H;
             const int my_tiles = group_tiles(qt, g);
             if (my_tiles == 0) continue;
@@ -522,7 +535,9 @@ cudaError_t launch_tc5(const Dims& d, const PrefillArgs& a, const Tc5Params& p, 
     }
     const long items = (long)((a.prompt_len + kRows * NG - 1) / (kRows * NG)) * d.heads * d.batch;
     const unsigned grid = (unsigned)(items < sms ? items : sms);  // one CTA per SM: the shared memory allows no more
-    kern<<<grid, L::kThreads, L::kBytes, st>>>(*a.tm_q, *a.tm_k, *a.tm_v, p);
+    Tc5Params pp = p;
+    pp.snake = items < 8L * sms;
+    kern<<<grid, L::kThreads, L::kBytes, st>>>(*a.tm_q, *a.tm_k, *a.tm_v, pp);
     return cudaGetLastError();
 }
 
