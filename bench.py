@@ -49,6 +49,9 @@ def parse():
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--combine", type=int, default=0, help="0 auto, 1 workspace+ticket, 2 cluster")
+    ap.add_argument("--prompt-layout", default="head_major", choices=["head_major", "token_major", "seq_first"],
+                    help="memory layout of the prompt segment (the paper's Fig. 6 compares layouts)")
+    ap.add_argument("--beams", type=int, default=0, help="override the workload's beam width")
     ap.add_argument("--prefill", action="store_true", help="time the prefill attention instead of the decode step")
     ap.add_argument("--prefill-groups", type=int, default=0,
                     help="128-row groups per CTA of the head_dim-128 prefill kernel (1 or 2; 0 = automatic)")
@@ -218,6 +221,8 @@ def run_ours(args):
     w = wl.by_name(args.workload)
     if args.batch:
         w = w.scaled(batch=args.batch, name=f"{w.name}[batch={args.batch}]")
+    if args.beams:
+        w = w.scaled(beams=args.beams, name=f"{w.name}[beams={args.beams}]")
     L = args.layers or DEFAULT_LAYERS.get(w.name.split("[")[0], 1)
     T = args.at_step or w.steps
     t = T - 1
@@ -235,6 +240,8 @@ def run_ours(args):
             h.set_tuning(args.splits, args.stages, args.combine)
         if args.no_overlap:
             h.set_overlap(False)
+        if args.prompt_layout != "head_major":
+            h.set_prompt_layout(args.prompt_layout)
         kp, vp = wl.make_prompt(wl_layer, dev)
         h.prefill_write(kp, vp)
         del kp, vp
@@ -377,6 +384,7 @@ def run_ours(args):
         "config": {"workload": w.name, "batch": w.batch, "beams": w.beams, "heads": w.heads, "kv_heads": w.kv_heads,
                    "head_dim": w.head_dim, "prompt_len": w.prompt_len, "at_step": T, "layers_per_step": L,
                    "l2": f"{L} distinct layer caches per step, {L * ubytes / 1e6:.0f} MB > L2", "cuda_graph": graphed, "dependent_launch": not args.no_overlap,
+                   "prompt_layout": args.prompt_layout,
                    "splits": handles[0][0].get_splits(), "parallelism": f"replica x{world}" if world > 1 else "1 gpu"},
         "us_per_step_per_layer": us_layer,
         "us_sdpa_per_layer": us_sdpa,
@@ -411,11 +419,15 @@ def run_prefill(args):
     w = wl.by_name(args.workload)
     if args.batch:
         w = w.scaled(batch=args.batch, name=f"{w.name}[batch={args.batch}]")
+    if args.beams:
+        w = w.scaled(beams=args.beams, name=f"{w.name}[beams={args.beams}]")
     L = args.layers or DEFAULT_LAYERS.get(w.name.split("[")[0], 1)
     handles = []
     for layer in range(L):
         wl_layer = w.scaled(index=w.index + 1000 * layer)
         h = SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, 1, w.torch_dtype)
+        if args.prompt_layout != "head_major":
+            h.set_prompt_layout(args.prompt_layout)
         kp, vp = wl.make_prompt(wl_layer, dev)
         h.prefill_write(kp, vp)
         if args.prefill_groups:

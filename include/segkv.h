@@ -288,6 +288,21 @@ SEGKV_API int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, con
 SEGKV_API int segkv_set_overlap(segkv_t h, int enable);
 
 /*
+ * Memory layout of the prompt segment inside the handle (Section 4.1 / Fig. 6
+ * of the paper compares prompt layouts for the decode kernel):
+ *   SEGKV_PROMPT_HEAD_MAJOR  [batch, kv_heads, max_prompt, head_dim]  (default)
+ *   SEGKV_PROMPT_TOKEN_MAJOR [batch, max_prompt, kv_heads, head_dim]  (the paper's [BS, Np, H, D])
+ *   SEGKV_PROMPT_SEQ_FIRST   [max_prompt, batch, kv_heads, head_dim]  (sequence-first)
+ * Every kernel reaches the prompt through a 4-D tensor map (or the strides) of
+ * the chosen layout; results do not depend on it.  Only allowed while no prompt
+ * is stored (before segkv_prefill_write, or after segkv_reset(h, 0)): ESTATE
+ * otherwise; EINVAL for an unknown layout.  The inputs of segkv_prefill_write
+ * stay token-major whatever the internal layout.
+ */
+enum { SEGKV_PROMPT_HEAD_MAJOR = 0, SEGKV_PROMPT_TOKEN_MAJOR = 1, SEGKV_PROMPT_SEQ_FIRST = 2 };
+SEGKV_API int segkv_set_prompt_layout(segkv_t h, int layout);
+
+/*
  * Override the CTA shape of the prefill attention kernel for head_dim 128
  * (the tcgen05 kernel): `row_groups` = groups of 128 query rows that one CTA
  * works on side by side (1 or 2; each group has its own softmax warps and

@@ -55,9 +55,10 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// Tensor map over one prompt array seen as [batch*kv_heads][prompt_len][D]:
-// rows >= prompt_len read as zero, a box never crosses a (request, head) slab.
-// Box = 64 elements (128 bytes, one swizzle span) x one tile of rows.
+// Tensor map over one prompt array seen as [batch][prompt_len][kv_heads][D] in coordinates
+// (d, head, token, request), with the strides of the handle's prompt layout: tokens >=
+// prompt_len read as zero, a box holds one (request, head).
+// Box = 64 elements (128 bytes, one swizzle span) x one tile of tokens.
 int make_prompt_map(const segkv* h, void* base, int prompt_len, CUtensorMap* out) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) {
@@ -65,12 +66,13 @@ int make_prompt_map(const segkv* h, void* base, int prompt_len, CUtensorMap* out
         return SEGKV_ECUDA;
     }
     const Dims& d = h->d;
-    cuuint64_t dims[3] = {(cuuint64_t)d.head_dim, (cuuint64_t)prompt_len, (cuuint64_t)d.batch * d.kv_heads};
-    cuuint64_t strides[2] = {(cuuint64_t)d.head_dim * 2, (cuuint64_t)d.max_prompt * d.head_dim * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)tiled_tile_keys(d.head_dim), 1};
-    cuuint32_t estr[3] = {1, 1, 1};
+    const PromptStrides ps = prompt_strides(d);
+    cuuint64_t dims[4] = {(cuuint64_t)d.head_dim, (cuuint64_t)d.kv_heads, (cuuint64_t)prompt_len, (cuuint64_t)d.batch};
+    cuuint64_t strides[3] = {(cuuint64_t)ps.h * 2, (cuuint64_t)ps.p * 2, (cuuint64_t)ps.b * 2};
+    cuuint32_t box[4] = {64, 1, (cuuint32_t)tiled_tile_keys(d.head_dim), 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
     CUtensorMapDataType dt = d.dtype == SEGKV_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
-    CUresult r = fn(out, dt, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    CUresult r = fn(out, dt, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -314,6 +316,7 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
     h->prompt_len = -1;
     h->overlap = true;
     h->prefill_groups = 0;
+    d.prompt_layout = SEGKV_PROMPT_HEAD_MAJOR;
 
     int rc = SEGKV_OK;
     auto fail = [&](int code) { free_all(h); delete h; return code; };
@@ -697,6 +700,13 @@ int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, const float* 
 int segkv_set_overlap(segkv_t h, int enable) {
     if (!h) return SEGKV_EINVAL;
     h->overlap = enable != 0;
+    return SEGKV_OK;
+}
+
+int segkv_set_prompt_layout(segkv_t h, int layout) {
+    if (!h || layout < SEGKV_PROMPT_HEAD_MAJOR || layout > SEGKV_PROMPT_SEQ_FIRST) return SEGKV_EINVAL;
+    if (h->prompt_len >= 0) return SEGKV_ESTATE;     // a prompt is stored in the current layout
+    h->d.prompt_layout = layout;
     return SEGKV_OK;
 }
 

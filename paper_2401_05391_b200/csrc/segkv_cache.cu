@@ -14,7 +14,8 @@ namespace segkv_impl {
 // ---------------------------------------------------------------------------
 __global__ void prefill_transpose_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v,
                                          uint4* __restrict__ kp, uint4* __restrict__ vp, int B, int P,
-                                         int Hkv, int chunks /* D*2/16 */, int max_prompt) {
+                                         int Hkv, int chunks /* D*2/16 */, long long sb, long long sh,
+                                         long long sp /* strides in 16-byte chunks */) {
     const long long total = (long long)B * P * Hkv * chunks;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
@@ -24,7 +25,7 @@ __global__ void prefill_transpose_kernel(const uint4* __restrict__ k, const uint
         r /= Hkv;
         int p = (int)(r % P);
         int b = (int)(r / P);
-        long long dst = (((long long)b * Hkv + h) * max_prompt + p) * chunks + c;
+        long long dst = b * sb + h * sh + p * sp + c;
         kp[dst] = k[i];
         vp[dst] = v[i];
     }
@@ -33,6 +34,7 @@ __global__ void prefill_transpose_kernel(const uint4* __restrict__ k, const uint
 cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v, void* kp, void* vp,
                                      int prompt_len, cudaStream_t st) {
     const int chunks = d.head_dim * 2 / 16;
+    const PromptStrides ps = prompt_strides(d);
     long long total = (long long)d.batch * prompt_len * d.kv_heads * chunks;
     if (total == 0) return cudaSuccess;
     int threads = 256;
@@ -40,7 +42,7 @@ cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v
     if (blocks > 148 * 32) blocks = 148 * 32;
     prefill_transpose_kernel<<<(unsigned)blocks, threads, 0, st>>>(
         (const uint4*)k, (const uint4*)v, (uint4*)kp, (uint4*)vp, d.batch, prompt_len, d.kv_heads, chunks,
-        d.max_prompt);
+        ps.b / 8, ps.h / 8, ps.p / 8);
     return cudaGetLastError();
 }
 

@@ -28,7 +28,20 @@ struct Dims {
     int rows;                                            // batch * beams
     int chunk_steps;                                     // response capacity grows in chunks of this many steps (0: fixed)
     int dtype;
+    int prompt_layout;                                   // SEGKV_PROMPT_HEAD_MAJOR / _TOKEN_MAJOR / _SEQ_FIRST
 };
+
+// Element strides of the prompt segment for a request, a kv head and a token in the handle's
+// prompt layout (head_dim is always the contiguous dimension).
+struct PromptStrides { long long b, h, p; };
+inline PromptStrides prompt_strides(const Dims& d) {
+    const long long D = d.head_dim, Hkv = d.kv_heads, P = d.max_prompt, B = d.batch;
+    switch (d.prompt_layout) {
+        case 1: return {P * Hkv * D, D, Hkv * D};        // [B, P, Hkv, D]
+        case 2: return {Hkv * D, D, B * Hkv * D};        // [P, B, Hkv, D]
+        default: return {Hkv * P * D, P * D, D};         // [B, Hkv, P, D]
+    }
+}
 
 }  // namespace segkv_impl
 
@@ -49,7 +62,7 @@ struct segkv {
     bool fuse_always;    // segkv_decode_step uses the fused kernel even for a single split
     long long launches;
     // device storage (owned)
-    void* kp;            // [batch, kv_heads, max_prompt, D]
+    void* kp;            // [batch, kv_heads, max_prompt, D] (or the layout chosen by segkv_set_prompt_layout)
     void* vp;
     void* kr;            // [max_steps, rows, kv_heads, D]; K and V of the response segment are ONE
     void* vr;            // allocation (V right behind K), so a V row is its K row plus a constant

@@ -66,7 +66,6 @@ prefill_sdpa_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;        // longest tiles first
     const int h = blockIdx.y, b = blockIdx.z;
     const int kvh = h / p.G;
-    const int slab = b * p.Hkv + kvh;
     const int nkt = min((p.N + kBN - 1) / kBN, ((qt + 1) * kBM + kBN - 1) / kBN);   // causal: tiles up to the CTA's last row
 
     if (tid == 0) {
@@ -96,8 +95,8 @@ prefill_sdpa_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 mbar_arrive_expect_tx(full, (uint32_t)L::STAGE_BYTES);
 #pragma unroll
                 for (int bx = 0; bx < D / 64; ++bx) {
-                    tma_load_3d(k_dst + bx * L::BOX_BYTES, &tm_k, bx * 64, kt * kBN, slab, full);
-                    tma_load_3d(v_dst + bx * L::BOX_BYTES, &tm_v, bx * 64, kt * kBN, slab, full);
+                    tma_load_4d(k_dst + bx * L::BOX_BYTES, &tm_k, bx * 64, kvh, kt * kBN, b, full);
+                    tma_load_4d(v_dst + bx * L::BOX_BYTES, &tm_v, bx * 64, kvh, kt * kBN, b, full);
                 }
             }
             if (!ok) s_abort = 1;

@@ -248,15 +248,15 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             prefetch_tmap(&tm_q);
             prefetch_tmap(&tm_k);
             prefetch_tmap(&tm_v);
-            auto load_tile = [&](const CUtensorMap* tm, uint8_t* dst_tile, int kt, int slab, uint32_t full) {
+            auto load_tile = [&](const CUtensorMap* tm, uint8_t* dst_tile, int kt, int kvh, int b, uint32_t full) {
                 const uint32_t dst = smem_u32(dst_tile);
                 mbar_arrive_expect_tx(full, (uint32_t)kTileKV);
 #pragma unroll
                 for (int half = 0; half < 2; ++half)
 #pragma unroll
                     for (int rb = 0; rb < kKeys / kBoxRows; ++rb)
-                        tma_load_3d(dst + half * kHalfTile + rb * kBoxBytes, tm, half * 64,
-                                    kt * kKeys + rb * kBoxRows, slab, full);
+                        tma_load_4d(dst + half * kHalfTile + rb * kBoxBytes, tm, half * 64, kvh,
+                                    kt * kKeys + rb * kBoxRows, b, full);
             };
             uint32_t tp = 0;                                       // K/V tiles requested so far (ring position)
             uint32_t qi[NG];                                      // items group g has taken part in: Q barrier phases
@@ -267,7 +267,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const int w = round_item(j);
                 if (w >= n_items) continue;
                 const int qt = item_qt(w), hb = w % hb_count, h = hb % p.H, b = hb / p.H;
-                const int slab = b * p.Hkv + h / p.G;
+                const int kvh = h / p.G;
                 int nkt = 0;
 #pragma unroll
                 for (int g = 0; g < NG; ++g) {
@@ -288,10 +288,10 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     const uint32_t sk = tp % SK, sv = tp % SV;
                     ok = mbar_wait(kempty0 + 8 * sk, ((tp / SK) & 1) ^ 1);
                     if (!ok) break;
-                    load_tile(&tm_k, k_ring + (size_t)sk * kTileKV, kt, slab, kfull0 + 8 * sk);
+                    load_tile(&tm_k, k_ring + (size_t)sk * kTileKV, kt, kvh, b, kfull0 + 8 * sk);
                     ok = mbar_wait(vempty0 + 8 * sv, ((tp / SV) & 1) ^ 1);
                     if (!ok) break;
-                    load_tile(&tm_v, v_ring + (size_t)sv * kTileKV, kt, slab, vfull0 + 8 * sv);
+                    load_tile(&tm_v, v_ring + (size_t)sv * kTileKV, kt, kvh, b, vfull0 + 8 * sv);
                 }
             }
             if (!ok) s_abort = 1;

@@ -53,7 +53,7 @@ sdpa_rowwise_kernel(const T* __restrict__ q, T* __restrict__ out, const float* _
                     const T* __restrict__ kp, const T* __restrict__ vp, const T* __restrict__ kr,
                     const T* const* __restrict__ k_chunks, int chunk_steps, long long vdelta_elems,
                     const int32_t* __restrict__ anc, int P, int steps, int W, int H,
-                    int Hkv, int group, int max_prompt, int max_steps, int rows) {
+                    int Hkv, int group, PromptStrides ps, int max_steps, int rows) {
     constexpr int E = D / 32;
     const int h = blockIdx.x, g = blockIdx.y;
     const int b = g / W, kvh = h / group;
@@ -75,7 +75,7 @@ sdpa_rowwise_kernel(const T* __restrict__ q, T* __restrict__ out, const float* _
         const T* krow;
         const T* vrow;
         if (i < P) {
-            const size_t off = (((size_t)b * Hkv + kvh) * max_prompt + i) * D;
+            const size_t off = (size_t)(b * ps.b + kvh * ps.h + i * ps.p);
             krow = kp + off;
             vrow = vp + off;
         } else {
@@ -134,7 +134,7 @@ cudaError_t dispatch(const Dims& d, const SdpaArgs& a, cudaStream_t st) {
         (const T*)a.q, (T*)a.out, a.slopes, (const T*)a.kp, (const T*)a.vp, (const T*)a.kr,             \
         (const T* const*)a.k_chunks, d.chunk_steps, a.vdelta / 2, a.anc, a.prompt_len, a.steps, d.beams, \
         d.heads, d.kv_heads, d.group,                                                                  \
-        d.max_prompt, d.max_steps, d.rows)
+        prompt_strides(d), d.max_steps, d.rows)
     switch (d.head_dim) {
         case 64: SEGKV_ROWWISE(64); break;
         case 128: SEGKV_ROWWISE(128); break;

@@ -228,8 +228,8 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             const int y = (pt0 + k) * TILE;
 #pragma unroll
             for (int bx = 0; bx < D / 64; ++bx) {
-                tma_load_3d(k_dst + bx * L::BOX_BYTES, &tm_k, bx * 64, y, slab, full);
-                tma_load_3d(v_dst + bx * L::BOX_BYTES, &tm_v, bx * 64, y, slab, full);
+                tma_load_4d(k_dst + bx * L::BOX_BYTES, &tm_k, bx * 64, kvh, y, b, full);
+                tma_load_4d(v_dst + bx * L::BOX_BYTES, &tm_v, bx * 64, kvh, y, b, full);
             }
         }
         mbar_arrive(full);      // lanes 1..31, and lane 0 a second time (the count is the gather warp's)

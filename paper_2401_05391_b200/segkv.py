@@ -50,6 +50,7 @@ SIGNATURES = {
     "segkv_get_splits": (_int, [_vp]),
     "segkv_set_overlap": (_int, [_vp, _int]),
     "segkv_set_prefill_tuning": (_int, [_vp, _int]),
+    "segkv_set_prompt_layout": (_int, [_vp, _int]),
     "segkv_launch_count": (ctypes.c_longlong, [_vp]),
     "segkv_storage_bytes": (ctypes.c_size_t, [_int] * 7),
     "segkv_strerror": (ctypes.c_char_p, [_int]),
@@ -287,6 +288,12 @@ class SegKV:
 
     def set_overlap(self, enable: bool) -> None:
         _check(lib().segkv_set_overlap(self._h, int(enable)), "segkv_set_overlap")
+
+    PROMPT_LAYOUTS = {"head_major": 0, "token_major": 1, "seq_first": 2}
+
+    def set_prompt_layout(self, layout) -> None:
+        code = self.PROMPT_LAYOUTS[layout] if isinstance(layout, str) else int(layout)
+        _check(lib().segkv_set_prompt_layout(self._h, code), "segkv_set_prompt_layout")
 
     def set_prefill_tuning(self, row_groups: int = 0) -> None:
         _check(lib().segkv_set_prefill_tuning(self._h, row_groups), "segkv_set_prefill_tuning")

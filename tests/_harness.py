@@ -14,13 +14,15 @@ ATOL, RTOL = 2e-3, 1e-2   # |gpu - ref| <= ATOL + RTOL*|ref|, the path's stated 
 
 class Run:
     def __init__(self, w: wl.Workload, device="cuda", max_steps=None, max_prompt=None, parents=None,
-                 splits=0, stages=0, combine=0, chunk_steps=0):
+                 splits=0, stages=0, combine=0, chunk_steps=0, prompt_layout=None):
         self.w, self.device = w, device
         self.h = SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim,
                        w.prompt_len if max_prompt is None else max_prompt,
                        w.steps if max_steps is None else max_steps, w.torch_dtype, chunk_steps=chunk_steps)
         if splits or stages or combine:
             self.h.set_tuning(splits, stages, combine)
+        if prompt_layout is not None:
+            self.h.set_prompt_layout(prompt_layout)
         self.parents = wl.make_parents(w) if parents is None else np.ascontiguousarray(parents, np.int32)
         self.parents_dev = torch.from_numpy(self.parents).to(device)
         self.slopes = wl.alibi_slopes(w.heads).to(device) if w.alibi else None

@@ -13,8 +13,9 @@ pytestmark = pytest.mark.gpu
 CHECK_STEPS = (0, 1, 2, 3, 7, 15, 16, 17, 31, 63, 127, 255)
 
 
-def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combine=0, every_step_ancestry=True):
-    r = Run(w, splits=splits, stages=stages, combine=combine)
+def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combine=0, every_step_ancestry=True,
+                 prompt_layout=None):
+    r = Run(w, splits=splits, stages=stages, combine=combine, prompt_layout=prompt_layout)
     try:
         worst = 0.0
         for t in range(w.steps):
@@ -33,9 +34,9 @@ def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combi
         r.close()
 
 
-def run_workload_fused(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combine=0):
+def run_workload_fused(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combine=0, prompt_layout=None):
     """Same as run_workload but every step is one fused segkv_decode_step launch."""
-    r = Run(w, splits=splits, stages=stages, combine=combine)
+    r = Run(w, splits=splits, stages=stages, combine=combine, prompt_layout=prompt_layout)
     try:
         for t in range(w.steps):
             _, out, q = r.step_fused()
@@ -185,6 +186,50 @@ def test_cluster_combine_small_shapes():
     for D, dt in ((64, "f16"), (256, "bf16")):
         w = wl.Workload("cl", 2, 3, 4, 2, D, 300, 9, dt, "uniform", True, 40 + D)
         run_workload(w, all_pairs, check_steps=(0, 8), splits=4, combine=2)
+
+
+@pytest.mark.parametrize("layout", ["token_major", "seq_first"])
+@pytest.mark.parametrize("dtype,D", [("f16", 64), ("bf16", 128), ("f16", 256)])
+def test_prompt_layouts_ragged_shapes(layout, dtype, D):
+    # the prompt segment kept token-major ([B, P, Hkv, D], the paper's) or sequence-first instead of
+    # head-major: separate calls and the fused step, GQA, ragged prompt, ALiBi on the bf16 variant
+    w = wl.Workload("layout", 3, 3, 6, 2, D, 150, 9, dtype, "uniform", dtype == "bf16", 60 + D // 64)
+    run_workload(w, all_pairs, check_steps=(0, 8), prompt_layout=layout)
+    run_workload_fused(w, all_pairs, check_steps=(0, 8), splits=3, prompt_layout=layout)
+
+
+@pytest.mark.parametrize("layout", ["token_major", "seq_first"])
+def test_prompt_layouts_llama2_7b_shape_and_rowwise(layout):
+    w = wl.CONFIGS[1]
+    r = Run(w, prompt_layout=layout)
+    try:
+        r.advance_to(w.steps - 1)
+        out, q = r.decode()
+        r.check(out, q, w.steps - 1, sampled_pairs(w, 64))
+        b = r.h.decode_sdpa_rowwise(q, None, r.slopes)
+        torch.cuda.synchronize()
+        r.check(b, q, w.steps - 1, sampled_pairs(w, 64))
+        assert r.h.get_error() == 0
+    finally:
+        r.close()
+
+
+def test_prompt_layout_can_only_change_while_no_prompt_is_stored():
+    w = wl.CONFIGS[0]
+    r = Run(w)
+    try:
+        with pytest.raises(sk.SegKVError):
+            r.h.set_prompt_layout("token_major")
+        with pytest.raises(sk.SegKVError):
+            r.h.set_prompt_layout(7)
+        r.h.reset(keep_prompt=False)
+        r.h.set_prompt_layout("token_major")
+        r.h.prefill_write(r.kp, r.vp)
+        r.advance_to(2)
+        out, q = r.decode()
+        r.check(out, q, 2, all_pairs(w))
+    finally:
+        r.close()
 
 
 def test_tiled_kernel_agrees_with_rowwise_kernel():

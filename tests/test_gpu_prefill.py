@@ -25,10 +25,12 @@ def check_rows(w, q, kp, vp, out, slopes, rows):
     assert (err <= atol + RTOL * np.abs(ref)).all(), f"max err {err.max():.3e}"
 
 
-def run_prefill(w, rows_fn, row_groups=0):
+def run_prefill(w, rows_fn, row_groups=0, prompt_layout=None):
     h = sk.SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, w.steps, w.torch_dtype)
     try:
         h.set_prefill_tuning(row_groups)
+        if prompt_layout is not None:
+            h.set_prompt_layout(prompt_layout)
         kp, vp = wl.make_prompt(w, "cuda")
         q = wl.make_prefill_query(w, "cuda")
         slopes = wl.alibi_slopes(w.heads).cuda() if w.alibi else None
@@ -80,6 +82,14 @@ def test_prefill_head_dim_128_row_groups(dtype, row_groups, P):
 @pytest.mark.parametrize("row_groups", [1, 2])
 def test_prefill_llama2_7b_shape_row_groups_sampled(row_groups):
     h = run_prefill(wl.CONFIGS[1], lambda w: sampled_rows(w, 256), row_groups)[0]
+    h.destroy()
+
+
+@pytest.mark.parametrize("layout", ["token_major", "seq_first"])
+@pytest.mark.parametrize("D,P", [(64, 150), (128, 300), (256, 150)])
+def test_prefill_prompt_layouts(layout, D, P):
+    w = wl.Workload("pf", 2, 3, 6, 2, D, P, 2, "f16", "uniform", False, 95)
+    h = run_prefill(w, all_rows, prompt_layout=layout)[0]
     h.destroy()
 
 
