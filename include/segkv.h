@@ -111,6 +111,24 @@ SEGKV_API int segkv_destroy(segkv_t h);
 SEGKV_API int segkv_prefill_write(segkv_t h, const void* k, const void* v, int prompt_len, void* stream);
 
 /*
+ * The same for prompts of different lengths (the paper's experiments use one
+ * prompt length per batch; a serving batch does not).  k, v: device, token-major
+ * [batch, padded_len, kv_heads, head_dim], request b's tokens in rows
+ * [0, prompt_lens[b]) and anything at all in the padding behind them.
+ * prompt_lens: HOST int32 [batch], each in [1, padded_len]; copied before the
+ * call returns.  Every later call on the handle then uses request b's own
+ * length: the decode attention and the fused step attend to its prompt_lens[b]
+ * prompt tokens followed by the response steps, ALiBi positions count from its
+ * own length.  The padding is stored as zeros.  segkv_prompt_len returns
+ * padded_len.  segkv_prefill_sdpa still computes all padded_len rows of every
+ * request; rows at or past a request's length attend to zeros and are to be
+ * ignored.  A later segkv_prefill_write returns the handle to one length.
+ * Errors: EINVAL (NULL, a length out of range), ECAPACITY, ECUDA.
+ */
+SEGKV_API int segkv_prefill_write_ragged(segkv_t h, const void* k, const void* v, int padded_len,
+                                         const int32_t* prompt_lens, void* stream);
+
+/*
  * Prefill attention (Section 3.1: at prefill Query_0/Key_0/Value_0 arrive batch-first and the
  * customised SDPA kernel takes and returns that layout; Section 3.3: it is the special case of
  * the decode kernel that sees only query and prompt key/value).  Causal self-attention of every

@@ -108,7 +108,7 @@ int make_query_map(const segkv* h, const void* q, int prompt_len, CUtensorMap* o
 }
 
 void free_all(segkv* h) {
-    void* ptrs[] = {h->kp, h->vp, h->kr, h->k_chunks_dev, h->parent, h->anc[0], h->anc[1], h->ulist, h->ucount,
+    void* ptrs[] = {h->kp, h->vp, h->kr, h->k_chunks_dev, h->parent, h->anc[0], h->anc[1], h->ulist, h->ucount, h->plens,
                     h->err_word, h->ws, h->tickets, h->st_q, h->st_out, h->st_k, h->st_v, h->st_parent,
                     h->st_slopes};
     for (void* p : ptrs)
@@ -241,6 +241,7 @@ SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes
     a.anc = h->anc[h->steps > 0 ? ((h->steps - 1) & 1) : 0];
     a.ulist = h->ulist;
     a.ucount = h->ucount;
+    a.plens = h->ragged ? h->plens : nullptr;
     a.ws = h->ws;
     a.tickets = h->tickets;
     a.err_word = h->err_word;
@@ -316,6 +317,7 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
     h->prompt_len = -1;
     h->overlap = true;
     h->prefill_groups = 0;
+    h->ragged = false;
     d.prompt_layout = SEGKV_PROMPT_HEAD_MAJOR;
 
     int rc = SEGKV_OK;
@@ -351,6 +353,7 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
     SEGKV_TRY(dmalloc(&h->ulist, (size_t)max_steps * d.rows * sizeof(URow)));
     SEGKV_TRY(dmalloc(&h->ucount, (size_t)batch * sizeof(int32_t)));
     SEGKV_TRY(cudaMemset(h->ucount, 0, (size_t)batch * sizeof(int32_t)));
+    SEGKV_TRY(dmalloc(&h->plens, (size_t)batch * sizeof(int32_t)));
     SEGKV_TRY(dmalloc(&h->err_word, sizeof(int)));
     SEGKV_TRY(dmalloc(&h->tickets, (size_t)batch * kv_heads * sizeof(int)));
     SEGKV_TRY(cudaMemset(h->err_word, 0, sizeof(int)));
@@ -378,14 +381,40 @@ int segkv_destroy(segkv_t h) {
     return SEGKV_OK;
 }
 
+static int prefill_write_impl(segkv_t h, const void* k, const void* v, int prompt_len, const int32_t* plens_dev,
+                              void* stream);
+
 int segkv_prefill_write(segkv_t h, const void* k, const void* v, int prompt_len, void* stream) {
+    if (!h) return SEGKV_EINVAL;
+    int rc = prefill_write_impl(h, k, v, prompt_len, nullptr, stream);
+    if (rc == SEGKV_OK) h->ragged = false;
+    return rc;
+}
+
+int segkv_prefill_write_ragged(segkv_t h, const void* k, const void* v, int padded_len, const int32_t* prompt_lens,
+                               void* stream) {
+    if (!h || !prompt_lens || padded_len <= 0) return SEGKV_EINVAL;
+    if (padded_len > h->d.max_prompt) return SEGKV_ECAPACITY;
+    for (int b = 0; b < h->d.batch; ++b)
+        if (prompt_lens[b] < 1 || prompt_lens[b] > padded_len) return SEGKV_EINVAL;
+    // the lengths travel on the caller's stream, ahead of the kernel that reads them; the source
+    // is pageable host memory, so the copy has been staged by the time the call returns
+    SEGKV_CUDA(cudaMemcpyAsync(h->plens, prompt_lens, (size_t)h->d.batch * sizeof(int32_t), cudaMemcpyHostToDevice,
+                               (cudaStream_t)stream));
+    int rc = prefill_write_impl(h, k, v, padded_len, h->plens, stream);
+    if (rc == SEGKV_OK) h->ragged = true;
+    return rc;
+}
+
+static int prefill_write_impl(segkv_t h, const void* k, const void* v, int prompt_len, const int32_t* plens_dev,
+                              void* stream) {
     if (!h || prompt_len < 0) return SEGKV_EINVAL;
     if (prompt_len > h->d.max_prompt) return SEGKV_ECAPACITY;
     if (prompt_len > 0 && (!k || !v || !aligned16(k) || !aligned16(v))) return SEGKV_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     h->tm_valid = false;
     if (prompt_len > 0) {
-        SEGKV_CUDA(launch_prefill_transpose(h->d, k, v, h->kp, h->vp, prompt_len, st));
+        SEGKV_CUDA(launch_prefill_transpose(h->d, k, v, h->kp, h->vp, plens_dev, prompt_len, st));
         h->launches++;
         int rc = make_prompt_map(h, h->kp, prompt_len, &h->tm_kp);
         if (rc == SEGKV_OK) rc = make_prompt_map(h, h->vp, prompt_len, &h->tm_vp);

@@ -15,7 +15,8 @@ namespace segkv_impl {
 __global__ void prefill_transpose_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v,
                                          uint4* __restrict__ kp, uint4* __restrict__ vp, int B, int P,
                                          int Hkv, int chunks /* D*2/16 */, long long sb, long long sh,
-                                         long long sp /* strides in 16-byte chunks */) {
+                                         long long sp /* strides in 16-byte chunks */,
+                                         const int32_t* __restrict__ plens) {
     const long long total = (long long)B * P * Hkv * chunks;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
@@ -26,12 +27,15 @@ __global__ void prefill_transpose_kernel(const uint4* __restrict__ k, const uint
         int p = (int)(r % P);
         int b = (int)(r / P);
         long long dst = b * sb + h * sh + p * sp + c;
-        kp[dst] = k[i];
-        vp[dst] = v[i];
+        // ragged prompts: the padding of a shorter request is stored as zeros, so that a masked
+        // key can never put a NaN or an infinity into a weighted sum
+        const bool pad = plens && p >= plens[b];
+        kp[dst] = pad ? make_uint4(0u, 0u, 0u, 0u) : k[i];
+        vp[dst] = pad ? make_uint4(0u, 0u, 0u, 0u) : v[i];
     }
 }
 
-cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v, void* kp, void* vp,
+cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v, void* kp, void* vp, const int32_t* plens,
                                      int prompt_len, cudaStream_t st) {
     const int chunks = d.head_dim * 2 / 16;
     const PromptStrides ps = prompt_strides(d);
@@ -42,7 +46,7 @@ cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v
     if (blocks > 148 * 32) blocks = 148 * 32;
     prefill_transpose_kernel<<<(unsigned)blocks, threads, 0, st>>>(
         (const uint4*)k, (const uint4*)v, (uint4*)kp, (uint4*)vp, d.batch, prompt_len, d.kv_heads, chunks,
-        ps.b / 8, ps.h / 8, ps.p / 8);
+        ps.b / 8, ps.h / 8, ps.p / 8, plens);
     return cudaGetLastError();
 }
 

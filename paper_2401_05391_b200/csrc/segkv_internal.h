@@ -72,6 +72,8 @@ struct segkv {
     int nchunks, nchunks_max;
     int32_t* parent;     // [max_steps, rows]
     int32_t* anc[2];     // [rows, max_steps], generation t lives in anc[t & 1]
+    int32_t* plens;      // [batch] per-request prompt lengths (segkv_prefill_write_ragged)
+    bool ragged;         // plens is in use; prompt_len is then the longest
     segkv_impl::URow* ulist;   // [batch, beams*max_steps] distinct response rows per request
     int32_t* ucount;     // [batch]
     bool lists_valid;    // ulist/ucount describe the newest step (a fused step does not update them)
@@ -92,7 +94,8 @@ struct segkv {
 namespace segkv_impl {
 
 // ---- kernels (each returns the cudaError_t of its launch) -----------------
-cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v, void* kp, void* vp,
+// plens (device, [batch]) or NULL: tokens at or past a request's own length are stored as zeros
+cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v, void* kp, void* vp, const int32_t* plens,
                                      int prompt_len, cudaStream_t st);
 
 cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, const void* k_new,
@@ -116,6 +119,7 @@ struct SdpaArgs {
     const int32_t* anc;      // beam-index table (fused step: the previous step's)
     const URow* ulist;
     const int32_t* ucount;
+    const int32_t* plens;    // device [batch] prompt lengths when they differ per request, else NULL
     float* ws;
     int* tickets;
     int* err_word;

@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(kWarps * 32)
 sdpa_rowwise_kernel(const T* __restrict__ q, T* __restrict__ out, const float* __restrict__ slopes,
                     const T* __restrict__ kp, const T* __restrict__ vp, const T* __restrict__ kr,
                     const T* const* __restrict__ k_chunks, int chunk_steps, long long vdelta_elems,
-                    const int32_t* __restrict__ anc, int P, int steps, int W, int H,
+                    const int32_t* __restrict__ anc, const int32_t* __restrict__ plens, int P_all, int steps, int W, int H,
                     int Hkv, int group, PromptStrides ps, int max_steps, int rows) {
     constexpr int E = D / 32;
     const int h = blockIdx.x, g = blockIdx.y;
@@ -64,6 +64,7 @@ sdpa_rowwise_kernel(const T* __restrict__ q, T* __restrict__ out, const float* _
     const float kLog2e = 1.4426950408889634f;
     const float scale2 = kLog2e / sqrtf((float)D);
     const float slope2 = slopes ? slopes[h] * kLog2e : 0.f;
+    const int P = plens ? plens[b] : P_all;
     const int L = P + steps;
     const int qpos = L - 1;
 
@@ -132,7 +133,7 @@ cudaError_t dispatch(const Dims& d, const SdpaArgs& a, cudaStream_t st) {
 #define SEGKV_ROWWISE(DD)                                                                               \
     sdpa_rowwise_kernel<T, DD><<<grid, block, 0, st>>>(                                                 \
         (const T*)a.q, (T*)a.out, a.slopes, (const T*)a.kp, (const T*)a.vp, (const T*)a.kr,             \
-        (const T* const*)a.k_chunks, d.chunk_steps, a.vdelta / 2, a.anc, a.prompt_len, a.steps, d.beams, \
+        (const T* const*)a.k_chunks, d.chunk_steps, a.vdelta / 2, a.anc, a.plens, a.prompt_len, a.steps, d.beams, \
         d.heads, d.kv_heads, d.group,                                                                  \
         prompt_strides(d), d.max_steps, d.rows)
     switch (d.head_dim) {

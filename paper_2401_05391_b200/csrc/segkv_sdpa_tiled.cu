@@ -116,6 +116,7 @@ struct TiledParams {
     long long vdelta;
     const URow* ulist;
     const int32_t* ucount;
+    const int32_t* plens;    // per-request prompt lengths, or NULL: every request has P tokens
     float* ws_o;    // [slab][S][ncols][D]   un-normalised partial outputs (ticket combine only)
     float* ws_ml;   // [slab][S][ncols][2]   running max (base-2 domain) and sum
     int* tickets;
@@ -211,7 +212,11 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     // This CTA's share of the work group: whole prompt tiles (known from the launch shape
     // alone, so their loads start at once) and a range of the request's distinct response
     // rows (known once the row count has been read).
-    const int ntp = (p.P + TILE - 1) / TILE;
+    // prompt length of this request: the launch's, or its own when the prompts are ragged (rows
+    // between the two hold zeros); written at prefill time, so it may be read before the
+    // grid-dependency wait
+    const int P = p.plens ? __ldg(p.plens + b) : p.P;
+    const int ntp = (P + TILE - 1) / TILE;
     const int pt0 = (int)((long long)split * ntp / p.S), pt1 = (int)((long long)(split + 1) * ntp / p.S);
     const int npt = pt1 - pt0;
     const URow* ulist_b = p.ulist + (size_t)b * p.W * p.max_steps;
@@ -573,7 +578,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 beambit[nt][c] = cv ? (1u << (col / p.G)) : 0u;
                 slope2[nt][c] = (cv && p.slopes) ? p.slopes[kvh * p.G + col % p.G] * 1.4426950408889634f : 0.f;
             }
-        const int qpos = p.P + (p.steps > 0 ? p.steps - 1 : -1);
+        const int qpos = P + (p.steps > 0 ? p.steps - 1 : -1);
         const int key_lo = warp * 16 + (lane >> 2);       // tile-local key of accumulator rows 0..7
 
         // One tile: `nvalid` keys exist; for a response tile the per-key beam masks and row
@@ -611,7 +616,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 if (resp) {
                     const URow u = meta[(size_t)st * TILE + key];       // {step, beams that read the row}
                     kmask[r] = key < nvalid ? u.mask : 0u;
-                    kpos[r] = (float)(p.P + u.row - qpos);
+                    kpos[r] = (float)(P + u.row - qpos);
                 } else {
                     kmask[r] = key < nvalid ? 0xffffffffu : 0u;
                     kpos[r] = (float)(pos0 + key - qpos);
@@ -685,7 +690,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const int pos0 = (pt0 + k) * TILE;
-            consume(st, false, min(TILE, p.P - pos0), pos0);
+            consume(st, false, min(TILE, P - pos0), pos0);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + 8 * st);
         }
@@ -938,6 +943,7 @@ cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk,
     p.anc_prev = a.anc; p.parent = a.parent; p.k_new = (const char*)a.k_new; p.v_new = (const char*)a.v_new;
     p.kr_new_slab = (char*)a.kr_new_slab; p.vr_new_slab = (char*)a.vr_new_slab;
     p.anc_dst = a.anc_dst; p.parent_row = a.parent_row;
+    p.plens = a.plens;
     p.P = a.prompt_len; p.steps = a.steps; p.S = a.splits; p.W = d.beams; p.G = d.group; p.H = d.heads;
     p.Hkv = d.kv_heads; p.rows = d.rows; p.max_steps = d.max_steps; p.ncols = d.beams * d.group; p.stages = stages;
     p.scale2 = 1.4426950408889634f / sqrtf((float)D);

@@ -51,6 +51,7 @@ SIGNATURES = {
     "segkv_set_overlap": (_int, [_vp, _int]),
     "segkv_set_prefill_tuning": (_int, [_vp, _int]),
     "segkv_set_prompt_layout": (_int, [_vp, _int]),
+    "segkv_prefill_write_ragged": (_int, [_vp, _vp, _vp, _int, _vp, _vp]),
     "segkv_launch_count": (ctypes.c_longlong, [_vp]),
     "segkv_storage_bytes": (ctypes.c_size_t, [_int] * 7),
     "segkv_strerror": (ctypes.c_char_p, [_int]),
@@ -166,6 +167,18 @@ class SegKV:
         shape = (self.batch, p, self.kv_heads, self.head_dim)
         _check(lib().segkv_prefill_write(self._h, _dev(k, shape, self.dtype, "k"), _dev(v, shape, self.dtype, "v"),
                                          p, _stream_ptr(stream)), "segkv_prefill_write")
+
+    def prefill_write_ragged(self, k: torch.Tensor, v: torch.Tensor, prompt_lens, stream=None) -> None:
+        """k, v: [batch, padded_len, kv_heads, head_dim] on the device; prompt_lens: batch host integers."""
+        p = int(k.shape[1])
+        shape = (self.batch, p, self.kv_heads, self.head_dim)
+        lens = (ctypes.c_int32 * self.batch)(*[int(x) for x in prompt_lens])
+        if len(prompt_lens) != self.batch:
+            raise ValueError("prompt_lens needs one entry per request")
+        _check(lib().segkv_prefill_write_ragged(self._h, _dev(k, shape, self.dtype, "k"),
+                                                _dev(v, shape, self.dtype, "v"), p,
+                                                ctypes.cast(lens, ctypes.c_void_p), _stream_ptr(stream)),
+               "segkv_prefill_write_ragged")
 
     def prefill_sdpa(self, q: torch.Tensor, out: Optional[torch.Tensor] = None,
                      alibi_slopes: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:

@@ -14,7 +14,8 @@ ATOL, RTOL = 2e-3, 1e-2   # |gpu - ref| <= ATOL + RTOL*|ref|, the path's stated 
 
 class Run:
     def __init__(self, w: wl.Workload, device="cuda", max_steps=None, max_prompt=None, parents=None,
-                 splits=0, stages=0, combine=0, chunk_steps=0, prompt_layout=None):
+                 splits=0, stages=0, combine=0, chunk_steps=0, prompt_layout=None,
+                 prompt_lens=None):
         self.w, self.device = w, device
         self.h = SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim,
                        w.prompt_len if max_prompt is None else max_prompt,
@@ -29,7 +30,15 @@ class Run:
         self.kp = self.vp = None
         if w.prompt_len > 0:
             self.kp, self.vp = wl.make_prompt(w, device)
-        self.h.prefill_write(self.kp, self.vp)
+        self.prompt_lens = None if prompt_lens is None else [int(x) for x in prompt_lens]
+        if self.prompt_lens is not None:
+            # the padding behind each request's own prompt is poison: the library must never let it through
+            for b, n in enumerate(self.prompt_lens):
+                self.kp[b, n:] = float("nan")
+                self.vp[b, n:] = float("inf")
+            self.h.prefill_write_ragged(self.kp, self.vp, self.prompt_lens)
+        else:
+            self.h.prefill_write(self.kp, self.vp)
         self.k_steps, self.v_steps, self.q_steps = [], [], []
 
     def close(self):
@@ -79,7 +88,8 @@ class Run:
         sl = slice(b * W, (b + 1) * W)
         qb = wl.to_bits(q[sl, hd:hd + 1])
         if self.kp is not None:
-            kpb = wl.to_bits(self.kp[b:b + 1, :, kvh:kvh + 1]); vpb = wl.to_bits(self.vp[b:b + 1, :, kvh:kvh + 1])
+            n = self.kp.shape[1] if self.prompt_lens is None else self.prompt_lens[b]
+            kpb = wl.to_bits(self.kp[b:b + 1, :n, kvh:kvh + 1]); vpb = wl.to_bits(self.vp[b:b + 1, :n, kvh:kvh + 1])
         else:
             kpb = vpb = np.zeros((1, 0, 1, w.head_dim), np.uint16)
         if t >= 0:

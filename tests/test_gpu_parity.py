@@ -14,8 +14,8 @@ CHECK_STEPS = (0, 1, 2, 3, 7, 15, 16, 17, 31, 63, 127, 255)
 
 
 def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combine=0, every_step_ancestry=True,
-                 prompt_layout=None):
-    r = Run(w, splits=splits, stages=stages, combine=combine, prompt_layout=prompt_layout)
+                 prompt_layout=None, prompt_lens=None):
+    r = Run(w, splits=splits, stages=stages, combine=combine, prompt_layout=prompt_layout, prompt_lens=prompt_lens)
     try:
         worst = 0.0
         for t in range(w.steps):
@@ -34,9 +34,10 @@ def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combi
         r.close()
 
 
-def run_workload_fused(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combine=0, prompt_layout=None):
+def run_workload_fused(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combine=0, prompt_layout=None,
+                       prompt_lens=None):
     """Same as run_workload but every step is one fused segkv_decode_step launch."""
-    r = Run(w, splits=splits, stages=stages, combine=combine, prompt_layout=prompt_layout)
+    r = Run(w, splits=splits, stages=stages, combine=combine, prompt_layout=prompt_layout, prompt_lens=prompt_lens)
     try:
         for t in range(w.steps):
             _, out, q = r.step_fused()
@@ -228,6 +229,43 @@ def test_prompt_layout_can_only_change_while_no_prompt_is_stored():
         r.advance_to(2)
         out, q = r.decode()
         r.check(out, q, 2, all_pairs(w))
+    finally:
+        r.close()
+
+
+@pytest.mark.parametrize("dtype,D,layout", [("f16", 64, None), ("bf16", 128, None), ("f16", 256, None),
+                                            ("bf16", 128, "token_major")])
+def test_per_request_prompt_lengths(dtype, D, layout):
+    # every request with its own prompt length (1, a full tile, ragged, the padded length), NaN / inf in
+    # the padding, ALiBi positions counted from each request's own length on the bf16 variants
+    w = wl.Workload("plens", 5, 3, 6, 2, D, 200, 9, dtype, "uniform", dtype == "bf16", 70 + D // 64)
+    lens = [1, 64, 150, 200, 65]
+    for splits in (0, 3):
+        run_workload(w, all_pairs, check_steps=(0, 8), splits=splits, prompt_layout=layout, prompt_lens=lens)
+        run_workload_fused(w, all_pairs, check_steps=(0, 8), splits=splits, prompt_layout=layout, prompt_lens=lens)
+
+
+def test_per_request_prompt_lengths_rowwise_and_errors():
+    w = wl.Workload("plens", 3, 4, 4, 4, 128, 100, 5, "f16", "uniform", True, 77)
+    r = Run(w, prompt_lens=[100, 3, 37])
+    try:
+        r.advance_to(4)
+        out, q = r.decode()
+        r.check(out, q, 4, all_pairs(w))
+        b = r.h.decode_sdpa_rowwise(q, None, r.slopes)
+        torch.cuda.synchronize()
+        r.check(b, q, 4, all_pairs(w))
+        for bad in ([100, 0, 37], [100, 101, 37]):
+            with pytest.raises(sk.SegKVError):
+                r.h.prefill_write_ragged(r.kp, r.vp, bad)
+        # back to one length for all: the padding written above is what the requests now see
+        clean_k, clean_v = wl.make_prompt(w, "cuda")
+        r.kp, r.vp, r.prompt_lens = clean_k, clean_v, None
+        r.h.prefill_write(clean_k, clean_v)
+        r.k_steps, r.v_steps, r.q_steps = [], [], []
+        r.advance_to(1)
+        out, q = r.decode()
+        r.check(out, q, 1, all_pairs(w))
     finally:
         r.close()
 
