@@ -188,6 +188,41 @@ def prefill_sdpa(dtype: str, batch: int, heads: int, kv_heads: int, head_dim: in
     return out.reshape(batch, N, heads, head_dim) if all_rows else out
 
 
+def narrow(dtype: str, x: np.ndarray) -> np.ndarray:
+    """float64 -> fp16 / bf16 bit patterns (uint16), round to nearest even.  bf16 goes through
+    float32 first; the double rounding can only matter within 2^-24 of a bf16 tie."""
+    x = np.asarray(x, np.float64)
+    if dtype == "f16":
+        return x.astype(np.float16).view(np.uint16)
+    u = x.astype(np.float32).view(np.uint32).astype(np.uint64)
+    return ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint16)
+
+
+def rope(dtype: str, x: np.ndarray, cos: np.ndarray, sin: np.ndarray, style: str) -> np.ndarray:
+    """Rotary position embedding of key rows (Section 3.1 lists a fused RoPE kernel; the rotation
+    is the standard one): x [n, D] as bit patterns, cos / sin [n, D/2] the values for each row's
+    position.  Pair i is (x[i], x[i + D/2]) for style "half" (Llama, NeoX) and (x[2i], x[2i+1])
+    for style "interleaved" (GPT-J); each pair (a, b) becomes (a cos - b sin, b cos + a sin).
+    Computed in float64, rounded once to the 16-bit type; returns bit patterns [n, D]."""
+    xb = np.ascontiguousarray(x, np.uint16)
+    n, D = xb.shape
+    xf = widen(dtype, xb).reshape(n, D)
+    c = np.asarray(cos, np.float64).reshape(n, D // 2)
+    s = np.asarray(sin, np.float64).reshape(n, D // 2)
+    out = np.empty_like(xf)
+    if style == "half":
+        a, b = xf[:, :D // 2], xf[:, D // 2:]
+        out[:, :D // 2] = a * c - b * s
+        out[:, D // 2:] = b * c + a * s
+    elif style == "interleaved":
+        a, b = xf[:, 0::2], xf[:, 1::2]
+        out[:, 0::2] = a * c - b * s
+        out[:, 1::2] = b * c + a * s
+    else:
+        raise ValueError(style)
+    return narrow(dtype, out)
+
+
 def cache_token(layers: int, heads: int, head_dim: int, elem_bytes: int) -> float:
     """Eq. 1: K and V bytes of one token over all layers."""
     return _load().segkv_oracle_cache_token(layers, heads, head_dim, elem_bytes)

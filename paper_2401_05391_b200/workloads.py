@@ -103,6 +103,16 @@ def alibi_slopes(heads: int) -> torch.Tensor:
     return torch.pow(torch.tensor(2.0, dtype=torch.float64), -8.0 * i / heads).to(torch.float32)
 
 
+def rope_tables(positions: int, head_dim: int, base: float = 10000.0):
+    """fp32 tables cos / sin [positions, head_dim/2] of the angle ``m * base^(-2i/head_dim)`` for
+    position m and pair i: the input a rotary-embedding kernel is given (computed in float64,
+    rounded once)."""
+    m = torch.arange(positions, dtype=torch.float64)[:, None]
+    i = torch.arange(head_dim // 2, dtype=torch.float64)[None, :]
+    ang = m * torch.pow(torch.tensor(float(base), dtype=torch.float64), -2.0 * i / head_dim)
+    return torch.cos(ang).to(torch.float32), torch.sin(ang).to(torch.float32)
+
+
 def _gen(device, seed: int) -> torch.Generator:
     g = torch.Generator(device=device)
     g.manual_seed(seed)

@@ -426,3 +426,85 @@ def test_prefill_first_position_returns_its_own_value():
     v = draw((B, N, Hkv, D), torch.float16, 223)
     got = oracle.prefill_sdpa("f16", B, H, Hkv, D, bits(q), bits(k), bits(v), rows=[(0, 0, 0), (0, 0, 1)])
     np.testing.assert_allclose(got, f64(v)[0, 0], rtol=0, atol=1e-15)
+
+
+# ------------------------------------------------------------ rotary embedding
+def _complex_rotation(x, pos, base, style):
+    """Independent statement of the rotary embedding: each pair is a complex number multiplied by
+    exp(i * pos * base^(-2j/D)) (numpy complex arithmetic, not the oracle's formula)."""
+    n, D = x.shape
+    theta = base ** (-2.0 * np.arange(D // 2) / D)
+    rot = np.exp(1j * pos[:, None] * theta[None, :])
+    if style == "half":
+        z = (x[:, :D // 2] + 1j * x[:, D // 2:]) * rot
+        return np.concatenate([z.real, z.imag], axis=1)
+    z = (x[:, 0::2] + 1j * x[:, 1::2]) * rot
+    out = np.empty_like(x)
+    out[:, 0::2], out[:, 1::2] = z.real, z.imag
+    return out
+
+
+@pytest.mark.parametrize("style", ["half", "interleaved"])
+@pytest.mark.parametrize("dtype,tdt", [("f16", torch.float16), ("bf16", torch.bfloat16)])
+def test_rope_equals_complex_multiplication_and_tables_are_the_closed_form(style, dtype, tdt):
+    D, n, base = 64, 37, 10000.0
+    x = draw((n, D), tdt, 500)
+    pos = np.arange(n, dtype=np.float64) * 3 + 1
+    cos_t, sin_t = wl.rope_tables(200, D, base)
+    # the table generator against the closed form, entry by entry
+    theta = base ** (-2.0 * np.arange(D // 2) / D)
+    m = np.arange(200, dtype=np.float64)[:, None]
+    assert np.allclose(cos_t.numpy(), np.cos(m * theta[None, :]), atol=6e-8, rtol=0)
+    assert np.allclose(sin_t.numpy(), np.sin(m * theta[None, :]), atol=6e-8, rtol=0)
+    idx = pos.astype(np.int64)
+    got = oracle.widen(dtype, oracle.rope(dtype, bits(x), cos_t.numpy()[idx], sin_t.numpy()[idx], style)).reshape(n, D)
+    want = _complex_rotation(f64(x), pos, base, style)
+    ulp = 2.0 ** (-10 if dtype == "f16" else -7)
+    assert np.all(np.abs(got - want) <= ulp * np.maximum(np.abs(want), 2.0 ** -14) + 1e-6)
+
+
+@pytest.mark.parametrize("style", ["half", "interleaved"])
+def test_rope_position_zero_is_identity_and_pairs_keep_their_norm(style):
+    D, n = 32, 9
+    x = draw((n, D), torch.float16, 501)
+    one, zero = np.ones((n, D // 2)), np.zeros((n, D // 2))
+    assert np.array_equal(oracle.rope("f16", bits(x), one, zero, style), bits(x))
+    ang = np.random.default_rng(3).uniform(0, 6.28, (n, D // 2))
+    y = oracle.widen("f16", oracle.rope("f16", bits(x), np.cos(ang), np.sin(ang), style)).reshape(n, D)
+    xf = f64(x)
+    if style == "half":
+        nx, ny = xf[:, :D // 2] ** 2 + xf[:, D // 2:] ** 2, y[:, :D // 2] ** 2 + y[:, D // 2:] ** 2
+    else:
+        nx, ny = xf[:, 0::2] ** 2 + xf[:, 1::2] ** 2, y[:, 0::2] ** 2 + y[:, 1::2] ** 2
+    assert np.allclose(nx, ny, rtol=4e-3, atol=1e-5)
+    # a quarter turn maps (a, b) to (-b, a) exactly
+    q = oracle.widen("f16", oracle.rope("f16", bits(x), zero, one, style)).reshape(n, D)
+    if style == "half":
+        assert np.array_equal(q[:, :D // 2], -xf[:, D // 2:]) and np.array_equal(q[:, D // 2:], xf[:, :D // 2])
+    else:
+        assert np.array_equal(q[:, 0::2], -xf[:, 1::2]) and np.array_equal(q[:, 1::2], xf[:, 0::2])
+
+
+@pytest.mark.parametrize("style", ["half", "interleaved"])
+def test_rope_scores_depend_on_the_position_difference_only(style):
+    # <R_m q, R_n k> = <R_(m-n) q, k>: the property the embedding exists for (float64 inputs that are
+    # exactly representable, so only the final rounding of the rotated rows differs)
+    D, base = 16, 100.0
+    q, k = draw((1, D), torch.float16, 502), draw((1, D), torch.float16, 503)
+    cos_t, sin_t = [t.numpy().astype(np.float64) for t in wl.rope_tables(64, D, base)]
+
+    def rot(x, m):
+        return oracle.widen("f16", oracle.rope("f16", bits(x), cos_t[m:m + 1], sin_t[m:m + 1], style)).reshape(-1)
+    for m, n in [(5, 2), (40, 37), (13, 10)]:
+        a = float(rot(q, m) @ rot(k, n))
+        b = float(rot(q, m - n) @ f64(k).reshape(-1))
+        assert abs(a - b) <= 2e-2 * (np.abs(f64(q)).sum() * np.abs(f64(k)).max())
+
+
+def test_narrow_rounds_to_nearest_even():
+    # halfway cases and neighbours, against torch's conversions
+    vals = np.array([1.0, 1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -2.5, 65504.0,
+                     1e-5, 0.3333333333, -7.0625])
+    t = torch.from_numpy(vals)
+    assert np.array_equal(oracle.narrow("f16", vals), bits(t.to(torch.float16)))
+    assert np.array_equal(oracle.narrow("bf16", vals), bits(t.to(torch.float32).to(torch.bfloat16)))
