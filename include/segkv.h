@@ -306,6 +306,27 @@ SEGKV_API int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, con
 SEGKV_API int segkv_set_overlap(segkv_t h, int enable);
 
 /*
+ * segkv_append with the rotary position embedding applied to the new K rows on
+ * their way into the response segment (Section 3.1 lists RoPE among the fused
+ * kernels; here it rides on the copy the append does anyway).  Everything as
+ * segkv_append, and:
+ *   rope_cos, rope_sin: device float [rope_positions, head_dim/2]: cos and sin
+ *     of the rotation angle of pair i at position m, row m of the table;
+ *   style: SEGKV_ROPE_HALF pairs (x[i], x[i + head_dim/2]) (Llama, NeoX),
+ *     SEGKV_ROPE_INTERLEAVED pairs (x[2i], x[2i+1]) (GPT-J); a pair (a, b)
+ *     becomes (a cos - b sin, b cos + a sin), fp32 arithmetic, rounded once;
+ *   the position of request b's token of this step is its prompt length + step.
+ * V rows are stored as they come.  The query is NOT rotated by the library: q
+ * handed to segkv_decode_sdpa must already carry its rotation.
+ * Errors: those of segkv_append; EINVAL for NULL or misaligned tables or an
+ * unknown style; ECAPACITY if a position would fall outside the tables.
+ */
+enum { SEGKV_ROPE_HALF = 1, SEGKV_ROPE_INTERLEAVED = 2 };
+SEGKV_API int segkv_append_rope(segkv_t h, int step, const int32_t* beam_parent, const void* k_new,
+                                const void* v_new, const float* rope_cos, const float* rope_sin,
+                                int rope_positions, int style, void* stream);
+
+/*
  * Memory layout of the prompt segment inside the handle (Section 4.1 / Fig. 6
  * of the paper compares prompt layouts for the decode kernel):
  *   SEGKV_PROMPT_HEAD_MAJOR  [batch, kv_heads, max_prompt, head_dim]  (default)

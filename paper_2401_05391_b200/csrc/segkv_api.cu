@@ -455,8 +455,32 @@ int segkv_prefill(segkv_t h, const void* k, const void* v, const void* q, void* 
     return segkv_prefill_sdpa(h, q, out, alibi_slopes, stream);
 }
 
+static int append_impl(segkv_t h, int step, const int32_t* beam_parent, const void* k_new, const void* v_new,
+                       const RopeArgs* rope, void* stream);
+
 int segkv_append(segkv_t h, int step, const int32_t* beam_parent, const void* k_new, const void* v_new,
                  void* stream) {
+    return append_impl(h, step, beam_parent, k_new, v_new, nullptr, stream);
+}
+
+int segkv_append_rope(segkv_t h, int step, const int32_t* beam_parent, const void* k_new, const void* v_new,
+                      const float* rope_cos, const float* rope_sin, int rope_positions, int style, void* stream) {
+    if (!h || !rope_cos || !rope_sin || rope_positions <= 0) return SEGKV_EINVAL;
+    if (style != SEGKV_ROPE_HALF && style != SEGKV_ROPE_INTERLEAVED) return SEGKV_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(rope_cos) & 3u) || (reinterpret_cast<uintptr_t>(rope_sin) & 3u)) return SEGKV_EINVAL;
+    if (h->prompt_len < 0) return SEGKV_ESTATE;
+    if (step >= 0 && h->prompt_len + step >= rope_positions) return SEGKV_ECAPACITY;   // the longest request's position
+    RopeArgs r;
+    r.cos = rope_cos; r.sin = rope_sin;
+    r.plens = h->ragged ? h->plens : nullptr;
+    r.prompt_len = h->prompt_len;
+    r.style = style;
+    r.head_dim = h->d.head_dim; r.kv_heads = h->d.kv_heads; r.bf16 = h->d.dtype == SEGKV_BF16;
+    return append_impl(h, step, beam_parent, k_new, v_new, &r, stream);
+}
+
+static int append_impl(segkv_t h, int step, const int32_t* beam_parent, const void* k_new, const void* v_new,
+                       const RopeArgs* rope, void* stream) {
     if (!h || step < 0 || !k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return SEGKV_EINVAL;
     if (step > 0 && (!beam_parent || (reinterpret_cast<uintptr_t>(beam_parent) & 3u))) return SEGKV_EINVAL;
     if (h->prompt_len < 0) return SEGKV_ESTATE;
@@ -469,7 +493,7 @@ int segkv_append(segkv_t h, int step, const int32_t* beam_parent, const void* k_
     SEGKV_CUDA(launch_append(h->d, step, beam_parent, k_new, v_new, k_slab_of(h, step),
                              k_slab_of(h, step) + vdelta_of(h), h->parent,
                              h->anc[(step + 1) & 1], h->anc[step & 1], h->ulist, h->ucount, h->err_word,
-                             h->sm_count, h->overlap && step > 0, (cudaStream_t)stream));
+                             h->sm_count, h->overlap && step > 0, (cudaStream_t)stream, rope));
     h->launches++;
     h->steps = step + 1;
     h->truncated = false;

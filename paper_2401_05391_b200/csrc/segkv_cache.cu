@@ -2,6 +2,9 @@
 // beam-index (ancestry) update.
 #include "segkv_internal.h"
 
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
 namespace segkv_impl {
 
 // ---------------------------------------------------------------------------
@@ -82,12 +85,96 @@ __device__ __forceinline__ int warp_incl_scan(int v) {
     return v;
 }
 
+// Eight 16-bit values of one 16-byte chunk <-> fp32.
+__device__ __forceinline__ void unpack8(const uint4& v, bool bf16, float* f) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (bf16) {
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        } else {
+            const float2 t = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+            f[2 * i] = t.x;
+            f[2 * i + 1] = t.y;
+        }
+    }
+}
+__device__ __forceinline__ uint4 pack8(const float* f, bool bf16) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (bf16) {
+            const __nv_bfloat162 t = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+            w[i] = *reinterpret_cast<const uint32_t*>(&t);
+        } else {
+            const __half2 t = __floats2half2_rn(f[2 * i], f[2 * i + 1]);
+            w[i] = *reinterpret_cast<const uint32_t*>(&t);
+        }
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// The copy blocks' K rows with the rotary embedding applied on the way (fp32 arithmetic, one
+// rounding): pair i of a row is (x[i], x[i + D/2]) (half-split) or (x[2i], x[2i+1])
+// (interleaved) and turns by the angle whose cos / sin the tables hold for the row's position.
+__device__ __forceinline__ void rope_copy(const RopeArgs& r, int W, int step, const uint4* __restrict__ k_new,
+                                          const uint4* __restrict__ v_new, uint4* __restrict__ kr_slab,
+                                          uint4* __restrict__ vr_slab, long long slab_chunks, long long first,
+                                          long long stride) {
+    const int cpr = r.head_dim / 8;                               // 16-byte chunks per (row, head)
+    const int half_d = r.head_dim / 2;
+    if (r.style == SEGKV_ROPE_INTERLEAVED) {
+        for (long long i = first; i < slab_chunks; i += stride) {
+            const int c = (int)(i % cpr);
+            const int b = (int)(i / cpr / r.kv_heads) / W;
+            const int pos = (r.plens ? r.plens[b] : r.prompt_len) + step;
+            const float* cs = r.cos + (size_t)pos * half_d + c * 4;
+            const float* sn = r.sin + (size_t)pos * half_d + c * 4;
+            float x[8];
+            unpack8(k_new[i], r.bf16, x);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float a = x[2 * e], bb = x[2 * e + 1];
+                x[2 * e] = a * cs[e] - bb * sn[e];
+                x[2 * e + 1] = bb * cs[e] + a * sn[e];
+            }
+            kr_slab[i] = pack8(x, r.bf16);
+            vr_slab[i] = v_new[i];
+        }
+    } else {
+        const int hc = cpr / 2;                                   // chunks of the low half of a row
+        for (long long j = first; j < slab_chunks / 2; j += stride) {
+            const int c = (int)(j % hc);
+            const long long rh = j / hc;                          // (row, head)
+            const int b = (int)(rh / r.kv_heads) / W;
+            const int pos = (r.plens ? r.plens[b] : r.prompt_len) + step;
+            const float* cs = r.cos + (size_t)pos * half_d + c * 8;
+            const float* sn = r.sin + (size_t)pos * half_d + c * 8;
+            const long long lo = rh * cpr + c, hi = lo + hc;
+            float xl[8], xh[8];
+            unpack8(k_new[lo], r.bf16, xl);
+            unpack8(k_new[hi], r.bf16, xh);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float a = xl[e], bb = xh[e];
+                xl[e] = a * cs[e] - bb * sn[e];
+                xh[e] = bb * cs[e] + a * sn[e];
+            }
+            kr_slab[lo] = pack8(xl, r.bf16);
+            kr_slab[hi] = pack8(xh, r.bf16);
+            vr_slab[lo] = v_new[lo];
+            vr_slab[hi] = v_new[hi];
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kBtThreads)
 append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __restrict__ beam_parent,
               const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, uint4* __restrict__ kr_slab,
               uint4* __restrict__ vr_slab, long long slab_chunks, int32_t* __restrict__ parent_row,
               const int32_t* __restrict__ anc_prev, int32_t* __restrict__ anc_cur, URow* __restrict__ ulist,
-              int32_t* __restrict__ ucount, int* __restrict__ err_word, int rebuild) {
+              int32_t* __restrict__ ucount, int* __restrict__ err_word, int rebuild, const RopeArgs rope) {
     // Programmatic dependent launch: this kernel touches nothing until the previous kernel of
     // the stream has completed, and only then lets the next one start its prologue (so a kernel
     // that starts early always finds everything older than its predecessor complete).
@@ -97,9 +184,13 @@ append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __
         // ---- copy blocks -------------------------------------------------
         const long long nb = gridDim.x - B;
         const long long first = ((long long)blockIdx.x - B) * blockDim.x + threadIdx.x;
-        for (long long i = first; i < slab_chunks; i += nb * blockDim.x) {
-            kr_slab[i] = k_new[i];
-            vr_slab[i] = v_new[i];
+        if (rope.style != 0) {
+            rope_copy(rope, W, step, k_new, v_new, kr_slab, vr_slab, slab_chunks, first, nb * blockDim.x);
+        } else {
+            for (long long i = first; i < slab_chunks; i += nb * blockDim.x) {
+                kr_slab[i] = k_new[i];
+                vr_slab[i] = v_new[i];
+            }
         }
         if (beam_parent != nullptr)
             for (long long i = first; i < rows; i += nb * blockDim.x) parent_row[i] = beam_parent[i];
@@ -191,7 +282,7 @@ append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __
 cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, const void* k_new,
                           const void* v_new, void* kr_slab_v, void* vr_slab_v, int32_t* parent_tab,
                           const int32_t* anc_prev, int32_t* anc_cur, URow* ulist, int32_t* ucount,
-                          int* err_word, int sm_count, bool pdl, cudaStream_t st) {
+                          int* err_word, int sm_count, bool pdl, cudaStream_t st, const RopeArgs* rope) {
     const long long slab_elems = (long long)d.rows * d.kv_heads * d.head_dim;
     const long long slab_chunks = slab_elems * 2 / 16;
     long long copy_blocks = (slab_chunks + kBtThreads * 4 - 1) / (kBtThreads * 4);
@@ -214,7 +305,8 @@ cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, c
     const int32_t* bp = step > 0 ? beam_parent : nullptr;
     return cudaLaunchKernelEx(&cfg, append_kernel, d.batch, d.beams, d.rows, d.max_steps, step, bp,
                               (const uint4*)k_new, (const uint4*)v_new, kr_slab, vr_slab, slab_chunks,
-                              parent_tab + (size_t)step * d.rows, anc_prev, anc_cur, ulist, ucount, err_word, 0);
+                              parent_tab + (size_t)step * d.rows, anc_prev, anc_cur, ulist, ucount, err_word, 0,
+                              rope ? *rope : RopeArgs{});
 }
 
 // The distinct-row lists of the newest step from its beam-index table alone: the table blocks of
@@ -224,7 +316,7 @@ cudaError_t launch_rebuild_lists(const Dims& d, int steps, const int32_t* anc_cu
     if (steps <= 0) return cudaSuccess;
     append_kernel<<<(unsigned)d.batch, kBtThreads, 0, st>>>(
         d.batch, d.beams, d.rows, d.max_steps, steps - 1, nullptr, nullptr, nullptr, nullptr, nullptr, 0, nullptr,
-        nullptr, const_cast<int32_t*>(anc_cur), ulist, ucount, nullptr, 1);
+        nullptr, const_cast<int32_t*>(anc_cur), ulist, ucount, nullptr, 1, RopeArgs{});
     return cudaGetLastError();
 }
 

@@ -94,6 +94,16 @@ struct segkv {
 namespace segkv_impl {
 
 // ---- kernels (each returns the cudaError_t of its launch) -----------------
+// Rotary embedding applied to the new K rows while they are appended (style 0: none).
+struct RopeArgs {
+    const float* cos;        // device [positions, D/2]
+    const float* sin;
+    const int32_t* plens;    // per-request prompt lengths or NULL
+    int prompt_len;          // the position of step t's token of request b is prompt length + t
+    int style;               // 0 none, SEGKV_ROPE_HALF, SEGKV_ROPE_INTERLEAVED
+    int head_dim, kv_heads, bf16;
+};
+
 // plens (device, [batch]) or NULL: tokens at or past a request's own length are stored as zeros
 cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v, void* kp, void* vp, const int32_t* plens,
                                      int prompt_len, cudaStream_t st);
@@ -101,7 +111,7 @@ cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v
 cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, const void* k_new,
                           const void* v_new, void* kr_slab, void* vr_slab, int32_t* parent_tab,
                           const int32_t* anc_prev, int32_t* anc_cur, URow* ulist, int32_t* ucount,
-                          int* err_word, int sm_count, bool pdl, cudaStream_t st);
+                          int* err_word, int sm_count, bool pdl, cudaStream_t st, const RopeArgs* rope = nullptr);
 // Re-derive the distinct-row lists from the current beam-index table (after fused steps).
 cudaError_t launch_rebuild_lists(const Dims& d, int steps, const int32_t* anc_cur, URow* ulist, int32_t* ucount,
                                  cudaStream_t st);

@@ -51,6 +51,7 @@ SIGNATURES = {
     "segkv_set_overlap": (_int, [_vp, _int]),
     "segkv_set_prefill_tuning": (_int, [_vp, _int]),
     "segkv_set_prompt_layout": (_int, [_vp, _int]),
+    "segkv_append_rope": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _int, _int, _vp]),
     "segkv_prefill_write_ragged": (_int, [_vp, _vp, _vp, _int, _vp, _vp]),
     "segkv_launch_count": (ctypes.c_longlong, [_vp]),
     "segkv_storage_bytes": (ctypes.c_size_t, [_int] * 7),
@@ -209,6 +210,22 @@ class SegKV:
         _check(lib().segkv_append(self._h, step, _dev(beam_parent, (self.rows,), torch.int32, "beam_parent"),
                                   _dev(k_new, shape, self.dtype, "k_new"), _dev(v_new, shape, self.dtype, "v_new"),
                                   _stream_ptr(stream)), "segkv_append")
+
+    ROPE_STYLES = {"half": 1, "interleaved": 2}
+
+    def append_rope(self, step: int, beam_parent: Optional[torch.Tensor], k_new: torch.Tensor, v_new: torch.Tensor,
+                    rope_cos: torch.Tensor, rope_sin: torch.Tensor, style="half", stream=None) -> None:
+        """append() with the rotary embedding applied to the new K rows; rope_cos / rope_sin are
+        device fp32 [positions, head_dim/2]."""
+        shape = (self.rows, self.kv_heads, self.head_dim)
+        n = int(rope_cos.shape[0])
+        tshape = (n, self.head_dim // 2)
+        code = self.ROPE_STYLES[style] if isinstance(style, str) else int(style)
+        _check(lib().segkv_append_rope(self._h, step, _dev(beam_parent, (self.rows,), torch.int32, "beam_parent"),
+                                       _dev(k_new, shape, self.dtype, "k_new"), _dev(v_new, shape, self.dtype, "v_new"),
+                                       _dev(rope_cos, tshape, torch.float32, "rope_cos"),
+                                       _dev(rope_sin, tshape, torch.float32, "rope_sin"), n, code,
+                                       _stream_ptr(stream)), "segkv_append_rope")
 
     def decode_sdpa(self, q: torch.Tensor, out: Optional[torch.Tensor] = None,
                     alibi_slopes: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:

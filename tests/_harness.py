@@ -51,6 +51,20 @@ class Run:
         self.k_steps.append(k); self.v_steps.append(v); self.q_steps.append(q)
         return t
 
+    def append_next_rope(self, cos, sin, style):
+        """Append the next step through segkv_append_rope; the oracle side gets K rows rotated by the
+        oracle's own rotary embedding (position = the request's prompt length + step)."""
+        w, t = self.w, self.h.steps
+        q, k, v = wl.make_step(w, t, self.device)
+        self.h.append_rope(t, self.parents_dev[t] if t > 0 else None, k, v, cos, sin, style)
+        plens = self.prompt_lens if self.prompt_lens is not None else [w.prompt_len] * w.batch
+        pos = np.repeat(np.asarray(plens, np.int64) + t, w.beams * w.kv_heads)          # one per (row, kv head)
+        rot = oracle.rope(w.dtype, wl.to_bits(k).reshape(-1, w.head_dim), cos.cpu().numpy()[pos],
+                          sin.cpu().numpy()[pos], style)
+        k_rot = torch.from_numpy(rot.view(np.int16).reshape(tuple(k.shape))).view(w.torch_dtype).to(self.device)
+        self.k_steps.append(k_rot); self.v_steps.append(v); self.q_steps.append(q)
+        return t
+
     def step_fused(self):
         """Append the next step and attend in one fused launch; returns (t, out, q)."""
         t = self.h.steps

@@ -270,6 +270,44 @@ def test_per_request_prompt_lengths_rowwise_and_errors():
         r.close()
 
 
+@pytest.mark.parametrize("style", ["half", "interleaved"])
+@pytest.mark.parametrize("dtype,D,ragged", [("f16", 64, False), ("bf16", 128, True), ("f16", 256, False)])
+def test_append_with_rotary_embedding(style, dtype, D, ragged):
+    # K rows rotated on their way into the response segment: the attention over them must match the
+    # oracle fed with K rows rotated by the oracle's own embedding (GQA, per-request positions when ragged)
+    w = wl.Workload("rope", 3, 3, 6, 2, D, 90, 7, dtype, "uniform", False, 80 + D // 64)
+    lens = [90, 17, 64] if ragged else None
+    cos, sin = [t.cuda() for t in wl.rope_tables(128, D)]
+    r = Run(w, prompt_lens=lens)
+    try:
+        for t in range(w.steps):
+            r.append_next_rope(cos, sin, style)
+            if t in (0, 3, w.steps - 1):
+                out, q = r.decode()
+                r.check(out, q, t, all_pairs(w))
+        assert r.h.get_error() == 0
+        assert np.array_equal(r.h.get_ancestry(), r.oracle_ancestry(w.steps - 1))
+    finally:
+        r.close()
+
+
+def test_append_with_rotary_embedding_errors():
+    w = wl.CONFIGS[0]
+    cos, sin = [t.cuda() for t in wl.rope_tables(w.prompt_len + 2, w.head_dim)]
+    r = Run(w)
+    try:
+        q, k, v = wl.make_step(w, 0, "cuda")
+        with pytest.raises(sk.SegKVError):
+            r.h.append_rope(0, None, k, v, cos, sin, 3)                 # unknown style
+        r.h.append_rope(0, None, k, v, cos, sin, "half")
+        r.h.append_rope(1, r.parents_dev[1], k, v, cos, sin, "half")
+        with pytest.raises(sk.SegKVError):
+            r.h.append_rope(2, r.parents_dev[2], k, v, cos, sin, "half")   # position prompt_len + 2 is past the tables
+        assert r.h.steps == 2
+    finally:
+        r.close()
+
+
 def test_tiled_kernel_agrees_with_rowwise_kernel():
     w = wl.Workload("cross", 2, 4, 8, 4, 128, 333, 30, "bf16", "uniform", True, 31)
     r = Run(w)
