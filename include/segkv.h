@@ -327,6 +327,25 @@ SEGKV_API int segkv_append_rope(segkv_t h, int step, const int32_t* beam_parent,
                                 int rope_positions, int style, void* stream);
 
 /*
+ * One set of beam-index tables for all layers of a model: the beam parents of
+ * a step are the same for every layer, so only one handle (the leader) needs
+ * to update the tables (Section 3.3's Indice table is kept by the beam search,
+ * once).  After segkv_share_index(h, leader) the handle h
+ *   - keeps its own prompt and response K/V, but reads the parent table, the
+ *     beam-index table and the distinct-row lists of `leader`;
+ *   - in segkv_append / segkv_append_rope stores its K/V rows only (the
+ *     beam_parent argument is ignored); the leader must already have appended
+ *     that step: ESTATE otherwise;
+ *   - in segkv_decode_sdpa needs leader and h at the same step: ESTATE otherwise;
+ *   - runs segkv_decode_step as those two launches.
+ * Both handles must be at step 0 (ESTATE) and agree in batch, beams and
+ * max_steps (EINVAL); a handle that follows cannot lead (EINVAL).
+ * leader == NULL gives h its own tables back.  Truncating or resetting is the
+ * caller's to do on every handle; destroy the followers before their leader.
+ */
+SEGKV_API int segkv_share_index(segkv_t h, segkv_t leader);
+
+/*
  * Memory layout of the prompt segment inside the handle (Section 4.1 / Fig. 6
  * of the paper compares prompt layouts for the decode kernel):
  *   SEGKV_PROMPT_HEAD_MAJOR  [batch, kv_heads, max_prompt, head_dim]  (default)

@@ -219,11 +219,16 @@ void choose_tiling(const segkv* h, int* splits, int* stages, bool* cluster) {
 
 // The attention kernel's separate form walks per-request lists of distinct rows that the append
 // kernel makes; fused steps skip them, so they are re-derived from the table when needed.
+// The handle that owns the beam-index tables h works with.
+segkv* index_of(segkv* h) { return h->leader ? h->leader : h; }
+const segkv* index_of(const segkv* h) { return h->leader ? h->leader : h; }
+
 int ensure_lists(segkv* h, cudaStream_t st) {
-    if (h->lists_valid || h->steps == 0) return SEGKV_OK;
-    SEGKV_CUDA(launch_rebuild_lists(h->d, h->steps, h->anc[(h->steps - 1) & 1], h->ulist, h->ucount, st));
+    segkv* x = index_of(h);
+    if (x->lists_valid || h->steps == 0) return SEGKV_OK;
+    SEGKV_CUDA(launch_rebuild_lists(x->d, h->steps, x->anc[(h->steps - 1) & 1], x->ulist, x->ucount, st));
     h->launches++;
-    h->lists_valid = true;
+    x->lists_valid = true;
     return SEGKV_OK;
 }
 
@@ -238,9 +243,10 @@ SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes
     a.vr = h->vr;
     a.k_chunks = (const void* const*)h->k_chunks_dev;
     a.vdelta = vdelta_of(h);
-    a.anc = h->anc[h->steps > 0 ? ((h->steps - 1) & 1) : 0];
-    a.ulist = h->ulist;
-    a.ucount = h->ucount;
+    const segkv* x = index_of(h);
+    a.anc = x->anc[h->steps > 0 ? ((h->steps - 1) & 1) : 0];
+    a.ulist = x->ulist;
+    a.ucount = x->ucount;
     a.plens = h->ragged ? h->plens : nullptr;
     a.ws = h->ws;
     a.tickets = h->tickets;
@@ -318,6 +324,7 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
     h->overlap = true;
     h->prefill_groups = 0;
     h->ragged = false;
+    h->leader = nullptr;
     d.prompt_layout = SEGKV_PROMPT_HEAD_MAJOR;
 
     int rc = SEGKV_OK;
@@ -490,6 +497,17 @@ static int append_impl(segkv_t h, int step, const int32_t* beam_parent, const vo
         int rc = ensure_chunk(h, step, (cudaStream_t)stream);
         if (rc != SEGKV_OK) return rc;
     }
+    if (h->leader) {
+        // the tables of this step have been made by the leader's call: only the K/V rows are stored
+        if (h->leader->steps != step + 1 || h->leader->truncated) return SEGKV_ESTATE;
+        SEGKV_CUDA(launch_append(h->d, step, nullptr, k_new, v_new, k_slab_of(h, step),
+                                 k_slab_of(h, step) + vdelta_of(h), nullptr, nullptr, nullptr, nullptr, nullptr,
+                                 h->err_word, h->sm_count, h->overlap && step > 0, (cudaStream_t)stream, rope, false));
+        h->launches++;
+        h->steps = step + 1;
+        h->truncated = false;
+        return SEGKV_OK;
+    }
     SEGKV_CUDA(launch_append(h->d, step, beam_parent, k_new, v_new, k_slab_of(h, step),
                              k_slab_of(h, step) + vdelta_of(h), h->parent,
                              h->anc[(step + 1) & 1], h->anc[step & 1], h->ulist, h->ucount, h->err_word,
@@ -506,6 +524,7 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
     if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SEGKV_EINVAL;
     if (h->prompt_len < 0) return SEGKV_ESTATE;
     if (h->prompt_len + h->steps <= 0) return SEGKV_ESTATE;
+    if (h->leader && h->leader->steps != h->steps) return SEGKV_ESTATE;   // the shared tables describe another step
     if (!tiled_supported(h->d)) {
         SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, 1);
         SEGKV_CUDA(launch_sdpa_rowwise(h->d, a, (cudaStream_t)stream));
@@ -570,8 +589,9 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     if (h->prompt_len < 0) return SEGKV_ESTATE;
     if (step != h->steps) return SEGKV_ESTATE;
     if (step >= h->d.max_steps) return SEGKV_ECAPACITY;
-    if (!tiled_supported(h->d)) {
-        // shapes the tiled kernel does not take: the two separate launches
+    if (!tiled_supported(h->d) || h->leader) {
+        // shapes the tiled kernel does not take, and handles that use another handle's tables
+        // (nothing to update in the attention kernel): the two separate launches
         int rc = segkv_append(h, step, beam_parent, k_new, v_new, stream);
         if (rc != SEGKV_OK) return rc;
         return segkv_decode_sdpa(h, q, out, alibi_slopes, stream);
@@ -672,7 +692,8 @@ int segkv_get_ancestry(segkv_t h, int32_t* host_out, void* stream) {
     if (h->truncated) return SEGKV_ESTATE;   // the table of the dropped step is what is stored
     if (h->steps == 0) return SEGKV_OK;
     const Dims& d = h->d;
-    const int32_t* src = h->anc[(h->steps - 1) & 1];
+    if (h->leader && h->leader->steps != h->steps) return SEGKV_ESTATE;
+    const int32_t* src = index_of(h)->anc[(h->steps - 1) & 1];
     SEGKV_CUDA(cudaMemcpy2DAsync(host_out, (size_t)h->steps * sizeof(int32_t), src,
                                  (size_t)d.max_steps * sizeof(int32_t), (size_t)h->steps * sizeof(int32_t),
                                  d.rows, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
@@ -753,6 +774,19 @@ int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, const float* 
 int segkv_set_overlap(segkv_t h, int enable) {
     if (!h) return SEGKV_EINVAL;
     h->overlap = enable != 0;
+    return SEGKV_OK;
+}
+
+int segkv_share_index(segkv_t h, segkv_t leader) {
+    if (!h || h == leader) return SEGKV_EINVAL;
+    if (h->steps != 0) return SEGKV_ESTATE;
+    if (leader) {
+        if (leader->leader) return SEGKV_EINVAL;             // a follower cannot lead
+        const Dims &a = h->d, &b = leader->d;
+        if (a.batch != b.batch || a.beams != b.beams || a.max_steps != b.max_steps) return SEGKV_EINVAL;
+        if (leader->steps != 0) return SEGKV_ESTATE;
+    }
+    h->leader = leader;
     return SEGKV_OK;
 }
 

@@ -192,6 +192,7 @@ append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __
                 vr_slab[i] = v_new[i];
             }
         }
+        if (parent_row == nullptr) return;                     // K/V rows only: the tables belong to another handle
         if (beam_parent != nullptr)
             for (long long i = first; i < rows; i += nb * blockDim.x) parent_row[i] = beam_parent[i];
         else
@@ -282,7 +283,7 @@ append_kernel(int B, int W, int rows, int max_steps, int step, const int32_t* __
 cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, const void* k_new,
                           const void* v_new, void* kr_slab_v, void* vr_slab_v, int32_t* parent_tab,
                           const int32_t* anc_prev, int32_t* anc_cur, URow* ulist, int32_t* ucount,
-                          int* err_word, int sm_count, bool pdl, cudaStream_t st, const RopeArgs* rope) {
+                          int* err_word, int sm_count, bool pdl, cudaStream_t st, const RopeArgs* rope, bool tables) {
     const long long slab_elems = (long long)d.rows * d.kv_heads * d.head_dim;
     const long long slab_chunks = slab_elems * 2 / 16;
     long long copy_blocks = (slab_chunks + kBtThreads * 4 - 1) / (kBtThreads * 4);
@@ -291,7 +292,8 @@ cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, c
     uint4* kr_slab = (uint4*)kr_slab_v;     // slab of this step inside the response segment
     uint4* vr_slab = (uint4*)vr_slab_v;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(d.batch + copy_blocks), 1, 1);
+    const int table_blocks = tables ? d.batch : 0;           // without tables every block copies rows
+    cfg.gridDim = dim3((unsigned)(table_blocks + copy_blocks), 1, 1);
     cfg.blockDim = dim3(kBtThreads, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
@@ -303,9 +305,10 @@ cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, c
         cfg.numAttrs = 1;
     }
     const int32_t* bp = step > 0 ? beam_parent : nullptr;
-    return cudaLaunchKernelEx(&cfg, append_kernel, d.batch, d.beams, d.rows, d.max_steps, step, bp,
+    return cudaLaunchKernelEx(&cfg, append_kernel, table_blocks, d.beams, d.rows, d.max_steps, step, bp,
                               (const uint4*)k_new, (const uint4*)v_new, kr_slab, vr_slab, slab_chunks,
-                              parent_tab + (size_t)step * d.rows, anc_prev, anc_cur, ulist, ucount, err_word, 0,
+                              tables ? parent_tab + (size_t)step * d.rows : (int32_t*)nullptr, anc_prev, anc_cur, ulist,
+                              ucount, err_word, 0,
                               rope ? *rope : RopeArgs{});
 }
 

@@ -72,6 +72,7 @@ struct segkv {
     int nchunks, nchunks_max;
     int32_t* parent;     // [max_steps, rows]
     int32_t* anc[2];     // [rows, max_steps], generation t lives in anc[t & 1]
+    segkv* leader;       // the handle whose beam-index tables this one uses (segkv_share_index), or NULL
     int32_t* plens;      // [batch] per-request prompt lengths (segkv_prefill_write_ragged)
     bool ragged;         // plens is in use; prompt_len is then the longest
     segkv_impl::URow* ulist;   // [batch, beams*max_steps] distinct response rows per request
@@ -111,7 +112,8 @@ cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v
 cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, const void* k_new,
                           const void* v_new, void* kr_slab, void* vr_slab, int32_t* parent_tab,
                           const int32_t* anc_prev, int32_t* anc_cur, URow* ulist, int32_t* ucount,
-                          int* err_word, int sm_count, bool pdl, cudaStream_t st, const RopeArgs* rope = nullptr);
+                          int* err_word, int sm_count, bool pdl, cudaStream_t st, const RopeArgs* rope = nullptr,
+                          bool tables = true);
 // Re-derive the distinct-row lists from the current beam-index table (after fused steps).
 cudaError_t launch_rebuild_lists(const Dims& d, int steps, const int32_t* anc_cur, URow* ulist, int32_t* ucount,
                                  cudaStream_t st);

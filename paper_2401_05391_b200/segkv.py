@@ -51,6 +51,7 @@ SIGNATURES = {
     "segkv_set_overlap": (_int, [_vp, _int]),
     "segkv_set_prefill_tuning": (_int, [_vp, _int]),
     "segkv_set_prompt_layout": (_int, [_vp, _int]),
+    "segkv_share_index": (_int, [_vp, _vp]),
     "segkv_append_rope": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _int, _int, _vp]),
     "segkv_prefill_write_ragged": (_int, [_vp, _vp, _vp, _int, _vp, _vp]),
     "segkv_launch_count": (ctypes.c_longlong, [_vp]),
@@ -318,6 +319,10 @@ class SegKV:
 
     def set_overlap(self, enable: bool) -> None:
         _check(lib().segkv_set_overlap(self._h, int(enable)), "segkv_set_overlap")
+
+    def share_index(self, leader: Optional["SegKV"]) -> None:
+        """Use `leader`'s beam-index tables (one table for all layers of a model); None undoes it."""
+        _check(lib().segkv_share_index(self._h, None if leader is None else leader._h), "segkv_share_index")
 
     PROMPT_LAYOUTS = {"head_major": 0, "token_major": 1, "seq_first": 2}
 

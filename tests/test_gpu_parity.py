@@ -308,6 +308,49 @@ def test_append_with_rotary_embedding_errors():
         r.close()
 
 
+@pytest.mark.parametrize("leader_fused", [False, True])
+def test_layers_share_one_beam_index_table(leader_fused):
+    # three "layers" with their own K/V and one set of tables: the leader updates them (by the separate
+    # append or inside the fused step), the followers store rows only and attend through the leader's tables
+    base = wl.Workload("share", 2, 4, 8, 4, 128, 130, 12, "f16", "uniform", False, 90)
+    layers = [Run(base.scaled(index=90 + 7 * i), parents=wl.make_parents(base), splits=4) for i in range(3)]
+    lead, followers = layers[0], layers[1:]
+    try:
+        for f in followers:
+            f.h.share_index(lead.h)
+        with pytest.raises(sk.SegKVError):
+            lead.h.share_index(followers[0].h)                     # a leader cannot follow its follower
+        q0, k0, v0 = wl.make_step(followers[0].w, 0, "cuda")
+        with pytest.raises(sk.SegKVError):
+            followers[0].h.append(0, None, k0, v0)                 # the leader has not made step 0 yet
+        for t in range(base.steps):
+            if leader_fused:
+                _, out, q = lead.step_fused()
+            else:
+                lead.append_next()
+                out, q = lead.decode()
+            if t in (0, 5, base.steps - 1):
+                lead.check(out, q, t, all_pairs(base))
+            for f in followers:
+                if t % 2:
+                    _, out, q = f.step_fused()                     # runs as append + attention on a follower
+                else:
+                    f.append_next()
+                    out, q = f.decode()
+                if t in (0, 5, base.steps - 1):
+                    f.check(out, q, t, all_pairs(base))
+                    assert np.array_equal(f.h.get_ancestry(), lead.oracle_ancestry(t))
+        for r in layers:
+            assert r.h.get_error() == 0
+        followers[0].h.reset()
+        followers[0].h.share_index(None)
+        with pytest.raises(sk.SegKVError):
+            followers[1].h.share_index(None)                       # not at step 0
+    finally:
+        for r in reversed(layers):
+            r.close()
+
+
 def test_tiled_kernel_agrees_with_rowwise_kernel():
     w = wl.Workload("cross", 2, 4, 8, 4, 128, 333, 30, "bf16", "uniform", True, 31)
     r = Run(w)
