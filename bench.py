@@ -464,8 +464,7 @@ def run_prefill(args):
                    "head_dim": w.head_dim, "prompt_len": n, "layers_rotated": L},
         "roofline": {"bound": "tensor", "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak,
                      "traffic": None, "peak_kind": f"of {kind} (bf16 GEMM burst; fp16 has the same nominal rate)",
-                     "kernel": ("segkv prefill attention (tcgen05, S/P/O in tensor memory, persistent CTAs)"
-                                if w.head_dim == 128 else "segkv prefill attention (mma.sync m16n8k16)")},
+                     "kernel": "segkv prefill attention (tcgen05, S/P/O in tensor memory, persistent CTAs)"},
         "gpu_launches": args.steps * L}))
 
 

@@ -35,14 +35,8 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kD = 128;        // head_dim of this kernel
 constexpr int kRows = 128;     // query rows per group (TMEM lanes)
-constexpr int kKeys = 128;     // keys per K/V tile
-constexpr int kBoxRows = 64;   // rows of one TMA box of the prompt segment's tensor map
-constexpr int kBoxBytes = kBoxRows * 128;    // one TMA box: 64 rows x 64 elements
-constexpr int kHalfTile = kKeys * 128;       // 64 of the 128 head-dim elements of all keys of a tile
-constexpr int kTileKV = 2 * kHalfTile;       // bytes of a K (or a V) tile
-constexpr int kBoxQ = kRows * 128;           // 64 of the 128 head-dim elements of a group's Q rows
+constexpr int kBoxQ = kRows * 128;           // 64 head-dim elements of a group's Q rows (one 128-byte swizzle span wide)
 constexpr int kTmemCols = 512;
 
 struct Tc5Params {
@@ -145,27 +139,40 @@ namespace {
 #define TC5_STAMP(role, kt, ev) do {} while (0)
 #endif
 
-template <int NG>
+// Shape of one instantiation: head_dim D (64, 128 or 256), KEYS keys per K/V tile, NG groups of
+// 128 query rows per CTA.  head_dim 256 leaves tensor memory for one group and 64-key tiles only.
+template <int D_, int KEYS_, int NG_>
 struct Tc5Layout {
+    static constexpr int D = D_, KEYS = KEYS_, NG = NG_;
     static constexpr int NB = NG == 1 ? 2 : 1;                   // S buffers per group
     static constexpr int kThreads = 32 * (4 * NG + 2);
+    static constexpr int kDBoxes = D / 64;                       // 64-element (128-byte) column blocks of a row
+    static constexpr int kBoxRows = D == 256 ? 32 : 64;          // rows of one TMA box of the prompt segment's tensor map
+    static constexpr int kBoxBytes = kBoxRows * 128;
+    static constexpr int kColTile = KEYS * 128;                  // one column block of all keys of a tile
+    static constexpr int kTileKV = kDBoxes * kColTile;           // bytes of a K (or a V) tile
     static constexpr int kStagesK = 3;
-    static constexpr int kStagesV = NG == 1 ? 3 : 2;
+    static constexpr int kStagesV = (NG == 1 && D <= 128) ? 3 : 2;
     static constexpr int kRingK = kStagesK * kTileKV;
     static constexpr int kRingV = kStagesV * kTileKV;
-    static constexpr int kQ = NG * 2 * kBoxQ;
+    static constexpr int kQGroup = kDBoxes * kBoxQ;              // bytes of one group's Q
+    static constexpr int kQ = NG * kQGroup;
     static constexpr int kBars = 2 * kStagesK + 2 * kStagesV + 6 * NG;   // K full/empty, V full/empty, per group: S0 S1 P O Qfull Qempty
     static constexpr size_t kBytes = 1024 + (size_t)kRingK + kRingV + kQ + 8 * kBars + 64;
+    // tensor memory: S buffers of KEYS columns first, then one O accumulator of D columns per group
+    static constexpr int kColO = NG * NB * KEYS;
+    static_assert(kColO + NG * D <= kTmemCols, "tensor memory");
+    static_assert(kBytes <= 232448, "shared memory");
 };
 
 // Row maximum of one tile's scores.  BIAS: sv[i] <- sv[i] * scale2 + slope2 * (key_i - row), the
 // maximum is in log2 units; otherwise sv keeps the raw dot products and the maximum is raw.
 // MASK: keys above the row (i > lim) are set to -inf first.
-template <bool BIAS, bool MASK>
+template <int KEYS, bool BIAS, bool MASK>
 __device__ __forceinline__ float score_max(float* sv, float scale2, float slope2, float bias0, int lim) {
     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-    for (int i = 0; i < kKeys; ++i) {
+    for (int i = 0; i < KEYS; ++i) {
         float v = sv[i];
         if (BIAS) v = fmaf(v, scale2, fmaf(slope2, (float)i, bias0));
         if (MASK) v = i > lim ? -INFINITY : v;
@@ -180,12 +187,12 @@ __device__ __forceinline__ float score_max(float* sv, float scale2, float slope2
 // next: the producer runs ahead through the K/V rings and reloads a group's Q as soon as the
 // group's last Q.K^T has been read, and the first Q.K^T of the next item executes while the
 // softmax threads are still storing the previous output.
-template <typename T, int NG>
-__global__ void __launch_bounds__(Tc5Layout<NG>::kThreads, 1)
+template <typename T, typename L>
+__global__ void __launch_bounds__(L::kThreads, 1)
 prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const Tc5Params p) {
-    using L = Tc5Layout<NG>;
-    constexpr int NB = L::NB, SK = L::kStagesK, SV = L::kStagesV;
+    constexpr int NG = L::NG, NB = L::NB, SK = L::kStagesK, SV = L::kStagesV;
+    constexpr int kD = L::D, kKeys = L::KEYS, kTileKV = L::kTileKV, kColTile = L::kColTile;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* k_ring = smem;                                       // tile: two halves [128 keys][64 elements]
@@ -215,7 +222,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     // key tiles of group g of query tile qt: up to its diagonal tile (causal); none past the prompt
     auto group_tiles = [&](int qt, int g) -> int {
         const int base = (qt * NG + g) * kRows;
-        return base < p.N ? min(nkt_all, base / kKeys + 1) : 0;
+        return base < p.N ? min(nkt_all, (base + kRows - 1) / kKeys + 1) : 0;
     };
 
     if (tid == 0) {
@@ -252,11 +259,11 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const uint32_t dst = smem_u32(dst_tile);
                 mbar_arrive_expect_tx(full, (uint32_t)kTileKV);
 #pragma unroll
-                for (int half = 0; half < 2; ++half)
+                for (int cb = 0; cb < L::kDBoxes; ++cb)
 #pragma unroll
-                    for (int rb = 0; rb < kKeys / kBoxRows; ++rb)
-                        tma_load_4d(dst + half * kHalfTile + rb * kBoxBytes, tm, half * 64, kvh,
-                                    kt * kKeys + rb * kBoxRows, b, full);
+                    for (int rb = 0; rb < kKeys / L::kBoxRows; ++rb)
+                        tma_load_4d(dst + cb * kColTile + rb * L::kBoxBytes, tm, cb * 64, kvh,
+                                    kt * kKeys + rb * L::kBoxRows, b, full);
             };
             uint32_t tp = 0;                                       // K/V tiles requested so far (ring position)
             uint32_t qi[NG];                                      // items group g has taken part in: Q barrier phases
@@ -279,10 +286,11 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     if (!ok) break;
                     ++qi[g];
                     const uint32_t qfull = gbar0 + 48 * g + 32;
-                    const uint32_t dst = smem_u32(q_smem) + (uint32_t)g * 2 * kBoxQ;
-                    mbar_arrive_expect_tx(qfull, 2u * kBoxQ);
-                    tma_load_4d(dst, &tm_q, 0, h, (qt * NG + g) * kRows, b, qfull);
-                    tma_load_4d(dst + kBoxQ, &tm_q, 64, h, (qt * NG + g) * kRows, b, qfull);
+                    const uint32_t dst = smem_u32(q_smem) + (uint32_t)g * L::kQGroup;
+                    mbar_arrive_expect_tx(qfull, (uint32_t)L::kQGroup);
+#pragma unroll
+                    for (int cb = 0; cb < L::kDBoxes; ++cb)
+                        tma_load_4d(dst + cb * kBoxQ, &tm_q, cb * 64, h, (qt * NG + g) * kRows, b, qfull);
                 }
                 for (int kt = 0; kt < nkt && ok; ++kt, ++tp) {
                     const uint32_t sk = tp % SK, sv = tp % SV;
@@ -316,14 +324,14 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
                 // S_g[buf] = Q_g . K^T for the group's tile kt; after its last one the group's Q may be replaced
                 auto issue_qk = [&](int g, int kt, int buf) {
-                    const uint32_t q_addr = smem_u32(q_smem) + (uint32_t)g * 2 * kBoxQ;
+                    const uint32_t q_addr = smem_u32(q_smem) + (uint32_t)g * L::kQGroup;
                     const uint32_t k_addr = smem_u32(k_ring + (size_t)((tp + kt) % SK) * kTileKV);
 #pragma unroll
                     for (int ks = 0; ks < kD / 16; ++ks) {
                         const uint32_t off = (uint32_t)(ks & 3) * 32;
-                        tc_mma_ss(tmem + 128u * (uint32_t)(g + buf),
+                        tc_mma_ss(tmem + (uint32_t)(kKeys * (g * NB + buf)),
                                   smem_desc(q_addr + (ks >> 2) * kBoxQ + off, 16, 1024),
-                                  smem_desc(k_addr + (ks >> 2) * kHalfTile + off, 16, 1024), p.idesc_qk, ks > 0);
+                                  smem_desc(k_addr + (ks >> 2) * kColTile + off, 16, 1024), p.idesc_qk, ks > 0);
                     }
                     tc_commit(gbar0 + 48 * g + 8 * buf);
                     if (kt + 1 == gt[g]) tc_commit(gbar0 + 48 * g + 40);
@@ -364,11 +372,11 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         if (!ok) break;
                         TC5_STAMP(2, kt, 1 + 3 * g);
                         tc_fence_after();
-                        const uint32_t p_tmem = tmem + 128u * (uint32_t)(g + (NB == 2 ? (int)(n[g] & 1) : 0));
+                        const uint32_t p_tmem = tmem + (uint32_t)(kKeys * (g * NB + (NB == 2 ? (int)(n[g] & 1) : 0)));
 #pragma unroll
                         for (int kk = 0; kk < kKeys / 16; ++kk)   // O_g += P_g[:, 16 keys] . V[16 keys, :]
-                            tc_mma_ts(tmem + 256u + 128u * (uint32_t)g, p_tmem + kk * 8,
-                                      smem_desc(v_addr + kk * 2048, kHalfTile, 1024), p.idesc_pv, (kt > 0 || kk > 0));
+                            tc_mma_ts(tmem + (uint32_t)(L::kColO + kD * g), p_tmem + kk * 8,
+                                      smem_desc(v_addr + kk * 2048, kColTile, 1024), p.idesc_pv, (kt > 0 || kk > 0));
                         tc_commit(gbar0 + 48 * g + 24);
 #if defined(SEGKV_TC5_TIMELINE) && SEGKV_TC5_TIMELINE == 3
                         mbar_wait_hot(gbar0 + 48 * g + 24, n[g] & 1);   // measurement only: serialise on P.V
@@ -401,7 +409,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const int g = warp >> 2, r = tid & (kRows - 1);
         const uint32_t bar_s0 = gbar0 + 48 * g, bar_p = bar_s0 + 16, bar_o = bar_s0 + 24;
         const uint32_t tm_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);     // this warp's TMEM lanes
-        const uint32_t tm_o = tm_lane + 256u + 128u * (uint32_t)g;
+        const uint32_t tm_o = tm_lane + (uint32_t)(L::kColO + kD * g);
         const bool stamp = lane == 0 && (warp & 3) == 0;
         const size_t qstride = (size_t)p.H * kD;
         uint32_t n = 0;                                           // tiles of this group so far: barrier phases
@@ -417,7 +425,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             float m_ref = -INFINITY, l_run = 0.f;
             for (int kt = 0; kt < my_tiles; ++kt, ++n) {
                 const int buf = NB == 2 ? (int)(n & 1) : 0;
-                const uint32_t tm_s = tm_lane + 128u * (uint32_t)(g + buf);
+                const uint32_t tm_s = tm_lane + (uint32_t)(kKeys * (g * NB + buf));
                 ok = mbar_wait_hot(bar_s0 + 8 * buf, (NB == 2 ? (n >> 1) : n) & 1);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
@@ -430,17 +438,17 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 if (stamp) TC5_STAMP(g, kt, 1);
                 float* sv = reinterpret_cast<float*>(sr);
                 const int key0 = kt * kKeys;
-                const bool diag = key0 + kKeys - 1 > row0;         // the group's diagonal tile
+                const bool diag = key0 + kKeys - 1 > row0;         // a tile that reaches past the group's first row
                 // scores in log2 units: s * scale2 (+ ALiBi bias); the scale is folded into the exponent's
                 // FMA unless a bias has to be added first; keys above the row (diagonal tile) become -inf
                 const bool biased = p.slopes != nullptr;
                 const int lim = row - key0;                        // key index i of this tile is visible iff i <= lim
                 const float bias0 = slope2 * (float)(key0 - row);
                 float tmax;
-                if (biased) tmax = diag ? score_max<true, true>(sv, p.scale2, slope2, bias0, lim)
-                                        : score_max<true, false>(sv, p.scale2, slope2, bias0, lim);
-                else tmax = (diag ? score_max<false, true>(sv, p.scale2, slope2, bias0, lim)
-                                  : score_max<false, false>(sv, p.scale2, slope2, bias0, lim)) * p.scale2;
+                if (biased) tmax = diag ? score_max<kKeys, true, true>(sv, p.scale2, slope2, bias0, lim)
+                                        : score_max<kKeys, true, false>(sv, p.scale2, slope2, bias0, lim);
+                else tmax = (diag ? score_max<kKeys, false, true>(sv, p.scale2, slope2, bias0, lim)
+                                  : score_max<kKeys, false, false>(sv, p.scale2, slope2, bias0, lim)) * p.scale2;
                 // a new reference only when the maximum has grown by more than 2^8: exponentials stay
                 // below 2^8 of the reference, the sum and O use the same reference
                 const bool need = tmax > m_ref + 8.f;
@@ -460,11 +468,19 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
                 l_run = l_run * alpha + ((ls[0] + ls[1]) + (ls[2] + ls[3]));
                 if (stamp) TC5_STAMP(g, kt, 2);
-                if (kt > 0 && __any_sync(0xffffffffu, need)) {
-                    ok = mbar_wait_hot(bar_o, (n - 1) & 1);        // P.V of the previous tile done: O stable
+                // O may be touched once P.V of the previous tile is done.  A parity wait is only
+                // meaningful on the barrier's current or previous phase, so with two S buffers,
+                // where nothing else ties this thread to the P.V before last, every phase of the O
+                // barrier is waited for in turn (with one S buffer the scores of this tile were
+                // produced behind that P.V in the pipe, and waiting here is only needed to rescale).
+                const bool rescale = kt > 0 && __any_sync(0xffffffffu, need);
+                if (kt > 0 && (NB == 2 || rescale)) {
+                    ok = mbar_wait_hot(bar_o, (n - 1) & 1);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after();
+                }
+                if (rescale) {
 #pragma unroll
                     for (int c = 0; c < kD / 32; ++c) {
                         uint32_t orr[32];
@@ -521,53 +537,69 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     }
 }
 
-template <typename T, int NG>
-cudaError_t launch_tc5(const Dims& d, const PrefillArgs& a, const Tc5Params& p, int sms, cudaStream_t st) {
-    using L = Tc5Layout<NG>;
-    auto kern = prefill_tc5_kernel<T, NG>;
+template <typename T, typename L>
+cudaError_t launch_tc5(const Dims& d, const PrefillArgs& a, Tc5Params p, int sms, cudaStream_t st) {
+    constexpr int NG = L::NG;
+    auto kern = prefill_tc5_kernel<T, L>;
+    // Never two CTAs on one SM: each allocates all of tensor memory and keeps it while it walks
+    // its items, so a second one would wait for it inside tcgen05.alloc.
+    constexpr size_t smem = L::kBytes > 120 * 1024 ? L::kBytes : 120 * 1024;
     static bool configured[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
+    // instruction descriptors: fp32 accumulate, A/B format, operand majors, N >> 3, M >> 4
+    const uint32_t fmt = d.dtype == SEGKV_BF16 ? 1u : 0u;
+    const uint32_t common = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kRows >> 4) << 24);
+    p.idesc_qk = common | ((uint32_t)(L::KEYS >> 3) << 17);               // A, B both K-major; N = keys of a tile
+    p.idesc_pv = common | (1u << 16) | ((uint32_t)(L::D >> 3) << 17);     // B (= V) MN-major; N = head_dim
+    p.scale2 = 1.4426950408889634f / sqrtf((float)L::D);
     const long items = (long)((a.prompt_len + kRows * NG - 1) / (kRows * NG)) * d.heads * d.batch;
-    const unsigned grid = (unsigned)(items < sms ? items : sms);  // one CTA per SM: the shared memory allows no more
-    Tc5Params pp = p;
-    pp.snake = items < 8L * sms;
-    kern<<<grid, L::kThreads, L::kBytes, st>>>(*a.tm_q, *a.tm_k, *a.tm_v, pp);
+    const unsigned grid = (unsigned)(items < sms ? items : sms);  // one CTA per SM
+    p.snake = items < 8L * sms;
+    kern<<<grid, L::kThreads, smem, st>>>(*a.tm_q, *a.tm_k, *a.tm_v, p);
     return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t dispatch_tc5(const Dims& d, const PrefillArgs& a, const Tc5Params& p, int sms, cudaStream_t st) {
+    // two row groups per CTA once there are enough 256-row items to fill the machine a few times over
+    const long items2 = (long)((a.prompt_len + 2 * kRows - 1) / (2 * kRows)) * d.heads * d.batch;
+    const bool two = a.row_groups ? a.row_groups == 2 : items2 >= 2L * sms;
+    switch (d.head_dim) {
+        case 64:
+            return two ? launch_tc5<T, Tc5Layout<64, 128, 2>>(d, a, p, sms, st)
+                       : launch_tc5<T, Tc5Layout<64, 128, 1>>(d, a, p, sms, st);
+        case 128:
+            return two ? launch_tc5<T, Tc5Layout<128, 128, 2>>(d, a, p, sms, st)
+                       : launch_tc5<T, Tc5Layout<128, 128, 1>>(d, a, p, sms, st);
+        case 256:   // O alone takes 256 of the 512 columns: one group, 64-key tiles, S double-buffered
+            return launch_tc5<T, Tc5Layout<256, 64, 1>>(d, a, p, sms, st);
+        default: return cudaErrorInvalidValue;
+    }
 }
 
 }  // namespace
 
-bool prefill_tc5_supported(const Dims& d) { return d.head_dim == kD; }
+bool prefill_tc5_supported(const Dims& d) { return d.head_dim == 64 || d.head_dim == 128 || d.head_dim == 256; }
 
 cudaError_t launch_prefill_tc5(const Dims& d, const PrefillArgs& a, cudaStream_t st) {
-    if (d.head_dim != kD) return cudaErrorInvalidValue;
-    const bool bf = d.dtype == SEGKV_BF16;
+    if (!prefill_tc5_supported(d) || !a.tm_q) return cudaErrorInvalidValue;
     Tc5Params p;
     p.q = a.q; p.out = a.out; p.slopes = a.slopes; p.err_word = a.err_word;
     p.N = a.prompt_len; p.H = d.heads; p.Hkv = d.kv_heads; p.G = d.group; p.B = d.batch;
-    p.scale2 = 1.4426950408889634f / sqrtf((float)kD);
-    // instruction descriptor: fp32 accumulate, A/B format, operand majors, N >> 3, M >> 4
-    const uint32_t fmt = bf ? 1u : 0u;
-    const uint32_t common = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kRows >> 4) << 24);
-    p.idesc_qk = common | ((uint32_t)(kKeys >> 3) << 17);                 // A, B both K-major
-    p.idesc_pv = common | (1u << 16) | ((uint32_t)(kD >> 3) << 17);       // B (= V) MN-major
-    // two row groups per CTA once there are enough 256-row CTAs to fill the machine a few times over
+    p.scale2 = 0.f; p.idesc_qk = p.idesc_pv = 0; p.snake = 0;
     int sms = 148;
     {
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     }
-    const long ctas2 = (long)((a.prompt_len + 2 * kRows - 1) / (2 * kRows)) * d.heads * d.batch;
-    const bool two = a.row_groups ? a.row_groups == 2 : ctas2 >= 2L * sms;
-    if (two) return bf ? launch_tc5<__nv_bfloat16, 2>(d, a, p, sms, st) : launch_tc5<__half, 2>(d, a, p, sms, st);
-    return bf ? launch_tc5<__nv_bfloat16, 1>(d, a, p, sms, st) : launch_tc5<__half, 1>(d, a, p, sms, st);
+    return d.dtype == SEGKV_BF16 ? dispatch_tc5<__nv_bfloat16>(d, a, p, sms, st) : dispatch_tc5<__half>(d, a, p, sms, st);
 }
 
 }  // namespace segkv_impl

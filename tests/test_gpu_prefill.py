@@ -93,6 +93,16 @@ def test_prefill_prompt_layouts(layout, D, P):
     h.destroy()
 
 
+@pytest.mark.parametrize("D,row_groups", [(256, 0), (128, 1), (64, 1), (64, 2)])
+def test_prefill_many_items_per_cta(D, row_groups):
+    # 768 or more work items on 148 persistent CTAs, tile counts 5 / 4 / 2 per item: every CTA walks
+    # several items back to back (barrier phases, ring positions and tensor-memory buffers carry over)
+    w = wl.Workload("pf", 16, 2, 16, 16, D, 300, 2, "f16", "uniform", False, 97)
+    for _ in range(2):
+        h = run_prefill(w, lambda w: sampled_rows(w, 300), row_groups)[0]
+        h.destroy()
+
+
 def test_prefill_llama2_7b_shape_sampled():
     h = run_prefill(wl.CONFIGS[1], lambda w: sampled_rows(w, 256))[0]
     h.destroy()
