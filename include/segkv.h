@@ -120,9 +120,9 @@ SEGKV_API int segkv_prefill_write(segkv_t h, const void* k, const void* v, int p
  * length: the decode attention and the fused step attend to its prompt_lens[b]
  * prompt tokens followed by the response steps, ALiBi positions count from its
  * own length.  The padding is stored as zeros.  segkv_prompt_len returns
- * padded_len.  segkv_prefill_sdpa still computes all padded_len rows of every
- * request; rows at or past a request's length attend to zeros and are to be
- * ignored.  A later segkv_prefill_write returns the handle to one length.
+ * padded_len.  segkv_prefill_sdpa takes q and out in the padded shape, computes
+ * rows [0, prompt_lens[b]) of request b and leaves the rows behind them in out
+ * untouched.  A later segkv_prefill_write returns the handle to one length.
  * Errors: EINVAL (NULL, a length out of range), ECAPACITY, ECUDA.
  */
 SEGKV_API int segkv_prefill_write_ragged(segkv_t h, const void* k, const void* v, int padded_len,

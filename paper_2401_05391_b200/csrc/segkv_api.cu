@@ -443,6 +443,7 @@ int segkv_prefill_sdpa(segkv_t h, const void* q, void* out, const float* alibi_s
     a.q = q; a.out = out; a.slopes = alibi_slopes; a.err_word = h->err_word;
     a.prompt_len = h->prompt_len; a.tm_k = &h->tm_kp; a.tm_v = &h->tm_vp;
     a.row_groups = h->prefill_groups;
+    a.plens = h->ragged ? h->plens : nullptr;
     CUtensorMap tm_q;
     a.tm_q = nullptr;
     if (prefill_tc5_supported(h->d)) {

@@ -176,6 +176,7 @@ struct PrefillArgs {
     int prompt_len;
     const CUtensorMap* tm_k;
     const CUtensorMap* tm_v;
+    const int32_t* plens;      // device [batch] prompt lengths when they differ per request, else NULL
     const CUtensorMap* tm_q;   // over q as [batch][prompt_len][heads][D], box 64 elements x 128 tokens; NULL if unused
     int row_groups;      // 0 = automatic
 };

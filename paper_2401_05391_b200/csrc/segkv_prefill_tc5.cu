@@ -44,6 +44,7 @@ struct Tc5Params {
     void* out;
     const float* slopes;
     int* err_word;
+    const int32_t* plens;    // per-request prompt lengths (rows and keys past them are skipped), or NULL
     int N, H, Hkv, G, B, snake;
     float scale2;
     uint32_t idesc_qk, idesc_pv;
@@ -206,7 +207,6 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int nkt_all = (p.N + kKeys - 1) / kKeys;
     const int nqt = (p.N + kRows * NG - 1) / (kRows * NG);
     const int hb_count = p.H * p.B;
     const int n_items = nqt * hb_count;
@@ -220,9 +220,12 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     // item w -> query tile (longest first), head, request
     auto item_qt = [&](int w) { return nqt - 1 - w / hb_count; };
     // key tiles of group g of query tile qt: up to its diagonal tile (causal); none past the prompt
-    auto group_tiles = [&](int qt, int g) -> int {
+    // nb = the request's own prompt length: with ragged prompts the items are still laid out for the
+    // longest one, and a shorter request leaves its later items (and the tail of one) without work
+    auto request_len = [&](int b) -> int { return p.plens ? __ldg(p.plens + b) : p.N; };
+    auto group_tiles = [&](int qt, int g, int nb) -> int {
         const int base = (qt * NG + g) * kRows;
-        return base < p.N ? min(nkt_all, (base + kRows - 1) / kKeys + 1) : 0;
+        return base < nb ? min((nb + kKeys - 1) / kKeys, (base + kRows - 1) / kKeys + 1) : 0;
     };
 
     if (tid == 0) {
@@ -278,7 +281,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 int nkt = 0;
 #pragma unroll
                 for (int g = 0; g < NG; ++g) {
-                    const int gt = group_tiles(qt, g);
+                    const int gt = group_tiles(qt, g, request_len(b));
                     nkt = max(nkt, gt);
                     if (gt == 0) continue;
                     // the group's Q rows (past the prompt: zeros), once its previous Q is no longer read
@@ -315,13 +318,14 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             for (int j = 0; j * (int)gridDim.x < n_items && ok; ++j) {
                 const int w = round_item(j);
                 if (w >= n_items) continue;
-                const int qt = item_qt(w);
+                const int qt = item_qt(w), nb = request_len((w % hb_count) / p.H);
                 int gt[NG], nkt = 0;
 #pragma unroll
                 for (int g = 0; g < NG; ++g) {
-                    gt[g] = group_tiles(qt, g);
+                    gt[g] = group_tiles(qt, g, nb);
                     nkt = max(nkt, gt[g]);
                 }
+                if (nkt == 0) continue;                           // the request ends before this item's rows
                 // S_g[buf] = Q_g . K^T for the group's tile kt; after its last one the group's Q may be replaced
                 auto issue_qk = [&](int g, int kt, int buf) {
                     const uint32_t q_addr = smem_u32(q_smem) + (uint32_t)g * L::kQGroup;
@@ -418,7 +422,8 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const int w = round_item(j);
             if (w >= n_items) continue;
             const int qt = item_qt(w), hb = w % hb_count, h = hb % p.H, b = hb / p.H;
-            const int my_tiles = group_tiles(qt, g);
+            const int nb = request_len(b);
+            const int my_tiles = group_tiles(qt, g, nb);
             if (my_tiles == 0) continue;
             const int row0 = (qt * NG + g) * kRows, row = row0 + r;
             const float slope2 = p.slopes ? p.slopes[h] * 1.4426950408889634f : 0.f;
@@ -515,7 +520,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 uint32_t orr[32];
                 tc_ld32(tm_o + c * 32, orr);
                 tc_wait_ld();
-                if (row < p.N) {
+                if (row < nb) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
                         *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = make_uint4(
@@ -591,6 +596,7 @@ cudaError_t launch_prefill_tc5(const Dims& d, const PrefillArgs& a, cudaStream_t
     if (!prefill_tc5_supported(d) || !a.tm_q) return cudaErrorInvalidValue;
     Tc5Params p;
     p.q = a.q; p.out = a.out; p.slopes = a.slopes; p.err_word = a.err_word;
+    p.plens = a.plens;
     p.N = a.prompt_len; p.H = d.heads; p.Hkv = d.kv_heads; p.G = d.group; p.B = d.batch;
     p.scale2 = 0.f; p.idesc_qk = p.idesc_pv = 0; p.snake = 0;
     int sms = 148;

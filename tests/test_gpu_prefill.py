@@ -103,6 +103,39 @@ def test_prefill_many_items_per_cta(D, row_groups):
         h.destroy()
 
 
+@pytest.mark.parametrize("dtype,D", [("f16", 128), ("bf16", 128), ("f16", 256), ("f16", 64)])
+def test_prefill_per_request_prompt_lengths(dtype, D):
+    # ragged prompts: each request is computed up to its own length (against the oracle run on that
+    # request alone), the poisoned padding never leaks in, and the rows behind a request's length stay untouched
+    lens = [300, 1, 129, 64, 257]
+    w = wl.Workload("pf", len(lens), 2, 4, 2, D, 300, 2, dtype, "uniform", dtype == "bf16", 98)
+    h = sk.SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, w.steps, w.torch_dtype)
+    try:
+        kp, vp = wl.make_prompt(w, "cuda")
+        q = wl.make_prefill_query(w, "cuda")
+        for b, n in enumerate(lens):
+            kp[b, n:] = float("nan")
+            vp[b, n:] = float("inf")
+        slopes = wl.alibi_slopes(w.heads).cuda() if w.alibi else None
+        for groups in (1, 2):
+            if D == 256 and groups == 2:
+                continue
+            h.set_prefill_tuning(groups)
+            h.prefill_write_ragged(kp, vp, lens)
+            out = torch.full_like(q, 512.0)
+            h.prefill_sdpa(q, out, slopes)
+            torch.cuda.synchronize()
+            assert h.get_error() == 0
+            for b, n in enumerate(lens):
+                assert bool((out[b, n:].float() == 512.0).all()), "rows behind the request's length were written"
+                w1 = w.scaled(batch=1, prompt_len=n)
+                rows = [(0, i, hd) for i in sorted({0, n - 1, n // 2, min(n - 1, 63), min(n - 1, 128)}) for hd in range(w.heads)]
+                check_rows(w1, q[b:b + 1, :n].contiguous(), kp[b:b + 1, :n].contiguous(), vp[b:b + 1, :n].contiguous(),
+                           out[b:b + 1, :n].contiguous(), slopes, rows)
+    finally:
+        h.destroy()
+
+
 def test_prefill_llama2_7b_shape_sampled():
     h = run_prefill(wl.CONFIGS[1], lambda w: sampled_rows(w, 256))[0]
     h.destroy()
