@@ -8,7 +8,10 @@ rows); this file compiles it with the host compiler and marshals numpy arrays.
 Parity status: the attention context has no printed value in the paper, so it
 is pinned by special cases, closed forms, invariants and a copied-cache brute
 force (``tests/test_oracle_pins.py``); the cache-size formulas are pinned to
-the values the paper prints for GPT-J-6B (Section 3.2).
+the values the paper prints for GPT-J-6B (Section 3.2); the rotary embedding
+of key rows (``rope``, numpy float64) is pinned to complex multiplication, the
+identity at position 0, the exact quarter turn, norm preservation and the
+relative-position property, and ``narrow`` to torch's conversions.
 """
 from __future__ import annotations
 
