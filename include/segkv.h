@@ -138,7 +138,13 @@ SEGKV_API int segkv_prefill_write_ragged(segkv_t h, const void* k, const void* v
  *   q, out: device [batch, prompt_len, heads, head_dim] (token-major, like k and v of the write);
  *   alibi_slopes: device float [heads] or NULL; bias = slope[hd] * (j - i).
  * fp16/bf16 operands, fp32 scores/softmax/accumulation, output rounded to nearest-even.
- * Errors: EINVAL, ESTATE (no prompt stored), ECUDA.  segkv_prefill is segkv_prefill_write followed by segkv_prefill_sdpa.
+ * Errors: EINVAL, ESTATE (no prompt stored), ECUDA.
+ *
+ * segkv_prefill does what segkv_prefill_write followed by segkv_prefill_sdpa does, in ONE launch:
+ * the attention kernel reads K/V from the caller's k and v (as given to segkv_prefill_write) and
+ * stores every tile into the prompt segment on its way through shared memory, each tile by exactly
+ * one CTA, so no separate copy of the prompt is made first.  The segment and the output agree bit
+ * for bit with the two-call form.  Errors: those of the two calls.
  */
 SEGKV_API int segkv_prefill_sdpa(segkv_t h, const void* q, void* out, const float* alibi_slopes, void* stream);
 SEGKV_API int segkv_prefill(segkv_t h, const void* k, const void* v, const void* q, void* out, int prompt_len,

@@ -107,6 +107,31 @@ int make_query_map(const segkv* h, const void* q, int prompt_len, CUtensorMap* o
     return SEGKV_OK;
 }
 
+// Tensor map over the caller's prefill K or V, token-major [batch][prompt_len][kv_heads][D], in
+// the coordinates of the prompt-segment maps (d, kv head, token, request) and with their box.
+int make_kv_source_map(const segkv* h, const void* base, int prompt_len, CUtensorMap* out) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled entry point not available");
+        return SEGKV_ECUDA;
+    }
+    const Dims& d = h->d;
+    const cuuint64_t row = (cuuint64_t)d.head_dim * 2;
+    cuuint64_t dims[4] = {(cuuint64_t)d.head_dim, (cuuint64_t)d.kv_heads, (cuuint64_t)prompt_len, (cuuint64_t)d.batch};
+    cuuint64_t strides[3] = {row, row * d.kv_heads, row * d.kv_heads * prompt_len};
+    cuuint32_t box[4] = {64, 1, (cuuint32_t)tiled_tile_keys(d.head_dim), 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUtensorMapDataType dt = d.dtype == SEGKV_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    CUresult r = fn(out, dt, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled (prefill K/V) failed with CUresult %d", (int)r);
+        return SEGKV_ECUDA;
+    }
+    return SEGKV_OK;
+}
+
 void free_all(segkv* h) {
     void* ptrs[] = {h->kp, h->vp, h->kr, h->k_chunks_dev, h->parent, h->anc[0], h->anc[1], h->ulist, h->ucount, h->plens,
                     h->err_word, h->ws, h->tickets, h->st_q, h->st_out, h->st_k, h->st_v, h->st_parent,
@@ -444,6 +469,7 @@ int segkv_prefill_sdpa(segkv_t h, const void* q, void* out, const float* alibi_s
     a.prompt_len = h->prompt_len; a.tm_k = &h->tm_kp; a.tm_v = &h->tm_vp;
     a.row_groups = h->prefill_groups;
     a.plens = h->ragged ? h->plens : nullptr;
+    a.tm_k_src = a.tm_v_src = nullptr;
     CUtensorMap tm_q;
     a.tm_q = nullptr;
     if (prefill_tc5_supported(h->d)) {
@@ -458,9 +484,41 @@ int segkv_prefill_sdpa(segkv_t h, const void* q, void* out, const float* alibi_s
 
 int segkv_prefill(segkv_t h, const void* k, const void* v, const void* q, void* out, int prompt_len,
                   const float* alibi_slopes, void* stream) {
-    int rc = segkv_prefill_write(h, k, v, prompt_len, stream);
+    if (!h) return SEGKV_EINVAL;
+    if (prompt_len <= 0 || !prefill_tc5_supported(h->d)) {
+        int rc = segkv_prefill_write(h, k, v, prompt_len, stream);
+        if (rc != SEGKV_OK) return rc;
+        return segkv_prefill_sdpa(h, q, out, alibi_slopes, stream);
+    }
+    // One launch: the attention kernel reads K/V from the caller's arrays and stores every tile
+    // into the prompt segment on the way (each tile by exactly one CTA), instead of a copy kernel
+    // first and the attention over the copy after it.
+    if (!k || !v || !q || !out || !aligned16(k) || !aligned16(v) || !aligned16(q) || !aligned16(out)) return SEGKV_EINVAL;
+    if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SEGKV_EINVAL;
+    if (prompt_len > h->d.max_prompt) return SEGKV_ECAPACITY;
+    h->tm_valid = false;
+    int rc = make_prompt_map(h, h->kp, prompt_len, &h->tm_kp);
+    if (rc == SEGKV_OK) rc = make_prompt_map(h, h->vp, prompt_len, &h->tm_vp);
+    CUtensorMap tm_q, tm_ks, tm_vs;
+    if (rc == SEGKV_OK) rc = make_kv_source_map(h, k, prompt_len, &tm_ks);
+    if (rc == SEGKV_OK) rc = make_kv_source_map(h, v, prompt_len, &tm_vs);
+    if (rc == SEGKV_OK) rc = make_query_map(h, q, prompt_len, &tm_q);
     if (rc != SEGKV_OK) return rc;
-    return segkv_prefill_sdpa(h, q, out, alibi_slopes, stream);
+    PrefillArgs a;
+    a.q = q; a.out = out; a.slopes = alibi_slopes; a.err_word = h->err_word;
+    a.prompt_len = prompt_len; a.tm_k = &h->tm_kp; a.tm_v = &h->tm_vp;
+    a.row_groups = h->prefill_groups;
+    a.plens = nullptr;
+    a.tm_k_src = &tm_ks; a.tm_v_src = &tm_vs; a.tm_q = &tm_q;
+    h->prompt_len = -1;                                       // nothing valid is stored if the launch fails
+    SEGKV_CUDA(launch_prefill_sdpa(h->d, a, (cudaStream_t)stream));
+    h->launches++;
+    h->tm_valid = true;
+    h->prompt_len = prompt_len;
+    h->steps = 0;
+    h->truncated = false;
+    h->ragged = false;
+    return SEGKV_OK;
 }
 
 static int append_impl(segkv_t h, int step, const int32_t* beam_parent, const void* k_new, const void* v_new,

@@ -177,6 +177,10 @@ struct PrefillArgs {
     const CUtensorMap* tm_k;
     const CUtensorMap* tm_v;
     const int32_t* plens;      // device [batch] prompt lengths when they differ per request, else NULL
+    // fused prefill: K/V tiles are read from the caller's token-major arrays through these maps and
+    // every tile is also stored into the prompt segment (tm_k / tm_v) by one CTA; NULL: read the segment
+    const CUtensorMap* tm_k_src;
+    const CUtensorMap* tm_v_src;
     const CUtensorMap* tm_q;   // over q as [batch][prompt_len][heads][D], box 64 elements x 128 tokens; NULL if unused
     int row_groups;      // 0 = automatic
 };

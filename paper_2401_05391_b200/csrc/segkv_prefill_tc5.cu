@@ -46,6 +46,7 @@ struct Tc5Params {
     int* err_word;
     const int32_t* plens;    // per-request prompt lengths (rows and keys past them are skipped), or NULL
     int N, H, Hkv, G, B, snake;
+    int store_kv;            // 1: every K/V tile is also written to the prompt segment, by the item that owns it
     float scale2;
     uint32_t idesc_qk, idesc_pv;
 };
@@ -188,11 +189,16 @@ __device__ __forceinline__ float score_max(float* sv, float scale2, float slope2
 // next: the producer runs ahead through the K/V rings and reloads a group's Q as soon as the
 // group's last Q.K^T has been read, and the first Q.K^T of the next item executes while the
 // softmax threads are still storing the previous output.
-template <typename T, typename L>
+// MODE 0: K/V from the prompt segment, one prompt length; 1: fused prefill (K/V from the caller's arrays,
+// every tile stored into the segment); 2: per-request prompt lengths (kept out of the other two: the
+// lengths as run-time values cost registers that the softmax threads of the two-group shape do not have).
+template <typename T, typename L, int MODE>
 __global__ void __launch_bounds__(L::kThreads, 1)
 prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                   const __grid_constant__ CUtensorMap tm_v, const Tc5Params p) {
+                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k_seg,
+                   const __grid_constant__ CUtensorMap tm_v_seg, const Tc5Params p) {
     constexpr int NG = L::NG, NB = L::NB, SK = L::kStagesK, SV = L::kStagesV;
+    constexpr bool STORE = MODE == 1, RAGGED = MODE == 2;
     constexpr int kD = L::D, kKeys = L::KEYS, kTileKV = L::kTileKV, kColTile = L::kColTile;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -222,14 +228,22 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     // key tiles of group g of query tile qt: up to its diagonal tile (causal); none past the prompt
     // nb = the request's own prompt length: with ragged prompts the items are still laid out for the
     // longest one, and a shorter request leaves its later items (and the tail of one) without work
-    auto request_len = [&](int b) -> int { return p.plens ? __ldg(p.plens + b) : p.N; };
+    auto request_len = [&](int b) -> int { return RAGGED ? __ldg(p.plens + b) : p.N; };
     auto group_tiles = [&](int qt, int g, int nb) -> int {
         const int base = (qt * NG + g) * kRows;
         return base < nb ? min((nb + kKeys - 1) / kKeys, (base + kRows - 1) / kKeys + 1) : 0;
     };
 
     if (tid == 0) {
-        for (int s = 0; s < 2 * SK + 2 * SV; ++s) mbar_init(kfull0 + 8 * s, 1);
+        // a stage is released by the MMAs that read it and, when tiles are stored on, by the store thread
+        for (int s = 0; s < SK; ++s) {
+            mbar_init(kfull0 + 8 * s, 1);
+            mbar_init(kempty0 + 8 * s, STORE ? 2 : 1);
+        }
+        for (int s = 0; s < SV; ++s) {
+            mbar_init(vfull0 + 8 * s, 1);
+            mbar_init(vempty0 + 8 * s, STORE ? 2 : 1);
+        }
         for (int g = 0; g < NG; ++g) {
             mbar_init(gbar0 + 48 * g, 1);
             mbar_init(gbar0 + 48 * g + 8, 1);
@@ -305,6 +319,51 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     load_tile(&tm_v, v_ring + (size_t)sv * kTileKV, kt, kvh, b, vfull0 + 8 * sv);
                 }
             }
+            if (!ok) s_abort = 1;
+        } else if (STORE && lane == 1) {
+            // ---- fused prefill: the tiles just read from the caller's K/V also become the prompt segment
+            // (paper Section 3.2: the prompt is kept once per request).  Tile kt of a kv head is stored by
+            // exactly one item: the first query head of the group, at the query tile whose rows start the
+            // tile's keys.  The thread follows the producer's tile sequence, waits for a tile to land,
+            // stores it if this item owns it (TMA store from the same swizzled tile), and adds its
+            // release of the stage to the MMAs' once the store has read shared memory.
+            prefetch_tmap(&tm_k_seg);
+            prefetch_tmap(&tm_v_seg);
+            auto store_tile = [&](const CUtensorMap* tm, uint8_t* src_tile, int kt, int kvh, int b) {
+                const uint32_t src = smem_u32(src_tile);
+#pragma unroll
+                for (int cb = 0; cb < L::kDBoxes; ++cb)
+#pragma unroll
+                    for (int rb = 0; rb < kKeys / L::kBoxRows; ++rb)
+                        tma_store_4d(tm, src + cb * kColTile + rb * L::kBoxBytes, cb * 64, kvh,
+                                     kt * kKeys + rb * L::kBoxRows, b);
+                bulk_commit_group();
+                bulk_wait_read_all();
+            };
+            uint32_t tp = 0;
+            bool ok = true;
+            for (int j = 0; j * (int)gridDim.x < n_items && ok; ++j) {
+                const int w = round_item(j);
+                if (w >= n_items) continue;
+                const int qt = item_qt(w), hb = w % hb_count, h = hb % p.H, b = hb / p.H;
+                const int kvh = h / p.G;
+                int nkt = 0;
+#pragma unroll
+                for (int g = 0; g < NG; ++g) nkt = max(nkt, group_tiles(qt, g, request_len(b)));
+                for (int kt = 0; kt < nkt && ok; ++kt, ++tp) {
+                    const bool mine = (h % p.G) == 0 && (kt * kKeys) / (kRows * NG) == qt;
+                    const uint32_t sk = tp % SK, sv = tp % SV;
+                    ok = mbar_wait(kfull0 + 8 * sk, (tp / SK) & 1);
+                    if (!ok) break;
+                    if (mine) store_tile(&tm_k_seg, k_ring + (size_t)sk * kTileKV, kt, kvh, b);
+                    mbar_arrive(kempty0 + 8 * sk);
+                    ok = mbar_wait(vfull0 + 8 * sv, (tp / SV) & 1);
+                    if (!ok) break;
+                    if (mine) store_tile(&tm_v_seg, v_ring + (size_t)sv * kTileKV, kt, kvh, b);
+                    mbar_arrive(vempty0 + 8 * sv);
+                }
+            }
+            bulk_wait_all();                                      // the stores themselves, before the CTA may exit
             if (!ok) s_abort = 1;
         }
     } else if (warp == 4 * NG + 1) {
@@ -422,8 +481,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const int w = round_item(j);
             if (w >= n_items) continue;
             const int qt = item_qt(w), hb = w % hb_count, h = hb % p.H, b = hb / p.H;
-            const int nb = request_len(b);
-            const int my_tiles = group_tiles(qt, g, nb);
+            const int my_tiles = group_tiles(qt, g, request_len(b));
             if (my_tiles == 0) continue;
             const int row0 = (qt * NG + g) * kRows, row = row0 + r;
             const float slope2 = p.slopes ? p.slopes[h] * 1.4426950408889634f : 0.f;
@@ -520,7 +578,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 uint32_t orr[32];
                 tc_ld32(tm_o + c * 32, orr);
                 tc_wait_ld();
-                if (row < nb) {
+                if (row < request_len(b)) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
                         *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = make_uint4(
@@ -545,7 +603,6 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 template <typename T, typename L>
 cudaError_t launch_tc5(const Dims& d, const PrefillArgs& a, Tc5Params p, int sms, cudaStream_t st) {
     constexpr int NG = L::NG;
-    auto kern = prefill_tc5_kernel<T, L>;
     // Never two CTAs on one SM: each allocates all of tensor memory and keeps it while it walks
     // its items, so a second one would wait for it inside tcgen05.alloc.
     constexpr size_t smem = L::kBytes > 120 * 1024 ? L::kBytes : 120 * 1024;
@@ -553,7 +610,11 @@ cudaError_t launch_tc5(const Dims& d, const PrefillArgs& a, Tc5Params p, int sms
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(prefill_tc5_kernel<T, L, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(prefill_tc5_kernel<T, L, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(prefill_tc5_kernel<T, L, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -566,7 +627,12 @@ cudaError_t launch_tc5(const Dims& d, const PrefillArgs& a, Tc5Params p, int sms
     const long items = (long)((a.prompt_len + kRows * NG - 1) / (kRows * NG)) * d.heads * d.batch;
     const unsigned grid = (unsigned)(items < sms ? items : sms);  // one CTA per SM
     p.snake = items < 8L * sms;
-    kern<<<grid, L::kThreads, smem, st>>>(*a.tm_q, *a.tm_k, *a.tm_v, p);
+    // fused prefill: load through the maps over the caller's arrays, store through the segment's
+    const bool store = a.tm_k_src && a.tm_v_src;
+    p.store_kv = store ? 1 : 0;
+    if (store) prefill_tc5_kernel<T, L, 1><<<grid, L::kThreads, smem, st>>>(*a.tm_q, *a.tm_k_src, *a.tm_v_src, *a.tm_k, *a.tm_v, p);
+    else if (p.plens) prefill_tc5_kernel<T, L, 2><<<grid, L::kThreads, smem, st>>>(*a.tm_q, *a.tm_k, *a.tm_v, *a.tm_k, *a.tm_v, p);
+    else prefill_tc5_kernel<T, L, 0><<<grid, L::kThreads, smem, st>>>(*a.tm_q, *a.tm_k, *a.tm_v, *a.tm_k, *a.tm_v, p);
     return cudaGetLastError();
 }
 

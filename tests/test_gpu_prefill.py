@@ -136,6 +136,42 @@ def test_prefill_per_request_prompt_lengths(dtype, D):
         h.destroy()
 
 
+@pytest.mark.parametrize("layout", [None, "token_major", "seq_first"])
+@pytest.mark.parametrize("dtype,D,heads,kv_heads,P", [("f16", 128, 8, 2, 300), ("bf16", 128, 4, 4, 129), ("f16", 256, 4, 2, 150),
+                                                      ("f16", 64, 6, 3, 520)])
+def test_fused_prefill_stores_the_same_segment_and_output_as_the_two_calls(layout, dtype, D, heads, kv_heads, P):
+    # segkv_prefill (one launch: attention + prompt store) against segkv_prefill_write + segkv_prefill_sdpa:
+    # same output bit for bit, and the decode attention over the stored segment agrees bit for bit too
+    w = wl.Workload("pf", 3, 2, heads, kv_heads, D, P, 3, dtype, "uniform", dtype == "bf16", 99)
+    kp, vp = wl.make_prompt(w, "cuda")
+    q = wl.make_prefill_query(w, "cuda")
+    slopes = wl.alibi_slopes(w.heads).cuda() if w.alibi else None
+    qd, kd, vd = wl.make_step(w, 0, "cuda")
+    results = []
+    for fused in (False, True):
+        h = sk.SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len + 40, w.steps, w.torch_dtype)
+        try:
+            if layout is not None:
+                h.set_prompt_layout(layout)
+            out = torch.full_like(q, 512.0)
+            if fused:
+                h.prefill(kp, vp, q, out, slopes)
+            else:
+                h.prefill_write(kp, vp)
+                h.prefill_sdpa(q, out, slopes)
+            dec0 = h.decode_sdpa(qd, None, slopes)                 # prompt only
+            h.append(0, None, kd, vd)
+            dec1 = h.decode_sdpa(qd, None, slopes)
+            torch.cuda.synchronize()
+            assert h.get_error() == 0
+            results.append((out.clone(), dec0.clone(), dec1.clone()))
+        finally:
+            h.destroy()
+    for a, b in zip(*results):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    check_rows(w, q, kp, vp, results[1][0], slopes, sampled_rows(w, 96))
+
+
 def test_prefill_llama2_7b_shape_sampled():
     h = run_prefill(wl.CONFIGS[1], lambda w: sampled_rows(w, 256))[0]
     h.destroy()
