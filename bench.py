@@ -343,15 +343,27 @@ def run_ours(args):
     # ---- end to end from host memory through segkv_step_host
     e2e = None
     if not args.no_e2e:
-        hq = [tuple(x.cpu().pin_memory() for x in (q, k, v)) + (torch.empty_like(q, device="cpu").pin_memory(),)
-              for _, q, k, v, _ in handles]
-        hp = parents[t].cpu().pin_memory() if t > 0 else None
-        hs = slopes.cpu().pin_memory() if slopes is not None else None
+        # every layer's step inputs packed into one pinned host block (one copy in, one launch, one copy out)
+        total, off = handles[0][0].host_pack_layout()
+        hs = slopes is not None
+        hq = []
+        for _, q, k, v, _ in handles:
+            blk = torch.zeros(total, dtype=torch.uint8).pin_memory()
+
+            def put(o, x):
+                raw = x.contiguous().cpu().view(torch.uint8).reshape(-1)
+                blk[o:o + raw.numel()] = raw
+            if t > 0:
+                put(off[0], parents[t])
+            if hs:
+                put(off[1], slopes)
+            put(off[2], k); put(off[3], v); put(off[4], q)
+            hq.append((blk, torch.empty_like(q, device="cpu").pin_memory()))
 
         def host_step():
-            for (h, *_), (q, k, v, o) in zip(handles, hq):
+            for (h, *_), (blk, o) in zip(handles, hq):
                 h.truncate_last()
-                h.step_host(t, hp, k, v, q, o, hs, stream=stream)
+                h.step_host_packed(t, blk, o, has_slopes=hs, stream=stream)
         n_e2e = max(3, min(args.steps, 20))
         for _ in range(3):
             host_step()
@@ -365,7 +377,7 @@ def run_ours(args):
         sec = (time.perf_counter() - t0) / n_e2e
         sec = sharding.max_over_ranks(sec, dev)
         q, k = handles[0][1], handles[0][2]
-        h2d = L * (q.numel() * 2 + 2 * k.numel() * 2 + (w.rows * 4 if t > 0 else 0) + (w.heads * 4 if hs is not None else 0))
+        h2d = L * total                      # the packed block: parents, slopes, k, v, q and their padding
         d2h = L * q.numel() * 2
         e2e = {"value": sharding.whole_job_rate(L * ubytes, world, sec) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "us_per_step_per_layer": sec * 1e6 / L}

@@ -249,6 +249,23 @@ SEGKV_API int segkv_step_host(segkv_t h, int step, const int32_t* beam_parent, c
                     const void* v_new, const void* q, void* out, const float* alibi_slopes,
                     void* stream);
 
+/*
+ * segkv_step_host with the step's inputs packed into ONE host block, so that a step
+ * costs one copy in, one launch and one copy out (each cudaMemcpyAsync costs
+ * several microseconds, more than the kernel at small shapes).
+ * segkv_host_pack_bytes returns the size of the block and, if `offsets` is not
+ * NULL, the byte offsets of its five sections in offsets[0..4]: beam_parent
+ * (int32 [rows]), alibi slopes (float [heads]), k_new, v_new, q (layouts as in
+ * segkv_decode_step); every section starts on a 256-byte boundary.  host_in is
+ * that block (the parent section is ignored at step 0, the slopes section when
+ * has_slopes == 0), host_out receives `out`.  Both are host pointers, pinned
+ * for asynchronous copies.  Errors: as segkv_step_host.
+ */
+SEGKV_API size_t segkv_host_pack_bytes(segkv_t h, size_t* offsets);
+SEGKV_API int segkv_step_host_packed(segkv_t h, int step, const void* host_in, void* host_out, int has_slopes,
+                                     void* stream);
+
+
 /* ---- test and benchmark aids ------------------------------------------- */
 
 /* Forget all appended steps; keep_prompt == 0 also forgets the prompt. */

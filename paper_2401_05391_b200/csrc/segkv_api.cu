@@ -134,7 +134,7 @@ int make_kv_source_map(const segkv* h, const void* base, int prompt_len, CUtenso
 
 void free_all(segkv* h) {
     void* ptrs[] = {h->kp, h->vp, h->kr, h->k_chunks_dev, h->parent, h->anc[0], h->anc[1], h->ulist, h->ucount, h->plens,
-                    h->err_word, h->ws, h->tickets, h->st_q, h->st_out, h->st_k, h->st_v, h->st_parent,
+                    h->err_word, h->ws, h->tickets, h->st_q, h->st_out, h->st_k, h->st_v, h->st_parent, h->st_pack,
                     h->st_slopes};
     for (void* p : ptrs)
         if (p) cudaFree(p);
@@ -398,6 +398,7 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
     SEGKV_TRY(dmalloc(&h->st_v, kvbytes));
     SEGKV_TRY(dmalloc(&h->st_parent, (size_t)d.rows * sizeof(int32_t)));
     SEGKV_TRY(dmalloc(&h->st_slopes, (size_t)heads * sizeof(float)));
+    SEGKV_TRY(dmalloc(&h->st_pack, segkv_host_pack_bytes(h, nullptr)));
 #undef SEGKV_TRY
     rc = alloc_workspace(h, 1);
     if (rc != SEGKV_OK) return fail(rc);
@@ -723,6 +724,40 @@ int segkv_step_host(segkv_t h, int step, const int32_t* beam_parent, const void*
                                alibi_slopes ? h->st_slopes : nullptr, stream);
     if (rc != SEGKV_OK) return rc;
     SEGKV_CUDA(cudaMemcpyAsync(out, h->st_out, qbytes, cudaMemcpyDeviceToHost, st));
+    SEGKV_CUDA(cudaStreamSynchronize(st));
+    return SEGKV_OK;
+}
+
+size_t segkv_host_pack_bytes(segkv_t h, size_t* offsets) {
+    if (!h) return 0;
+    const Dims& d = h->d;
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const size_t qbytes = (size_t)d.rows * d.heads * d.head_dim * 2;
+    const size_t kvbytes = (size_t)d.rows * d.kv_heads * d.head_dim * 2;
+    size_t off[5];
+    off[0] = 0;                                            // beam_parent  int32 [rows]
+    off[1] = off[0] + up((size_t)d.rows * sizeof(int32_t));   // alibi slopes float [heads]
+    off[2] = off[1] + up((size_t)d.heads * sizeof(float));    // k_new
+    off[3] = off[2] + up(kvbytes);                            // v_new
+    off[4] = off[3] + up(kvbytes);                            // q
+    if (offsets)
+        for (int i = 0; i < 5; ++i) offsets[i] = off[i];
+    return off[4] + up(qbytes);
+}
+
+int segkv_step_host_packed(segkv_t h, int step, const void* host_in, void* host_out, int has_slopes, void* stream) {
+    if (!h || !host_in || !host_out) return SEGKV_EINVAL;
+    const Dims& d = h->d;
+    cudaStream_t st = (cudaStream_t)stream;
+    size_t off[5];
+    const size_t total = segkv_host_pack_bytes(h, off);
+    const size_t qbytes = (size_t)d.rows * d.heads * d.head_dim * 2;
+    SEGKV_CUDA(cudaMemcpyAsync(h->st_pack, host_in, total, cudaMemcpyHostToDevice, st));
+    char* base = (char*)h->st_pack;
+    int rc = segkv_decode_step(h, step, step > 0 ? (const int32_t*)(base + off[0]) : nullptr, base + off[2], base + off[3],
+                               base + off[4], h->st_out, has_slopes ? (const float*)(base + off[1]) : nullptr, stream);
+    if (rc != SEGKV_OK) return rc;
+    SEGKV_CUDA(cudaMemcpyAsync(host_out, h->st_out, qbytes, cudaMemcpyDeviceToHost, st));
     SEGKV_CUDA(cudaStreamSynchronize(st));
     return SEGKV_OK;
 }

@@ -73,6 +73,7 @@ struct segkv {
     int32_t* parent;     // [max_steps, rows]
     int32_t* anc[2];     // [rows, max_steps], generation t lives in anc[t & 1]
     segkv* leader;       // the handle whose beam-index tables this one uses (segkv_share_index), or NULL
+    void* st_pack;       // staging for segkv_step_host_packed: parent | slopes | k | v | q in one block
     int32_t* plens;      // [batch] per-request prompt lengths (segkv_prefill_write_ragged)
     bool ragged;         // plens is in use; prompt_len is then the longest
     segkv_impl::URow* ulist;   // [batch, beams*max_steps] distinct response rows per request

@@ -38,6 +38,8 @@ SIGNATURES = {
     "segkv_decode_step": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "segkv_decode_sdpa_static": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "segkv_step_host": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "segkv_host_pack_bytes": (ctypes.c_size_t, [_vp, _vp]),
+    "segkv_step_host_packed": (_int, [_vp, _int, _vp, _vp, _int, _vp]),
     "segkv_reset": (_int, [_vp, _int]),
     "segkv_truncate_last": (_int, [_vp]),
     "segkv_get_ancestry": (_int, [_vp, _vp, _vp]),
@@ -271,6 +273,22 @@ class SegKV:
                                      _host(q, qs, self.dtype, "q"), _host(out, qs, self.dtype, "out"),
                                      _host(alibi_slopes, (self.heads,), torch.float32, "alibi_slopes"),
                                      _stream_ptr(stream)), "segkv_step_host")
+        return out
+
+    def host_pack_layout(self):
+        """(total bytes, offsets of beam_parent / slopes / k_new / v_new / q) of the packed host block."""
+        off = (ctypes.c_size_t * 5)()
+        total = int(lib().segkv_host_pack_bytes(self._h, ctypes.cast(off, ctypes.c_void_p)))
+        return total, [int(x) for x in off]
+
+    def step_host_packed(self, step: int, packed: torch.Tensor, out: torch.Tensor, has_slopes: bool = False,
+                         stream=None) -> torch.Tensor:
+        """One step from one packed host block (a uint8 tensor laid out as host_pack_layout says)."""
+        total, _ = self.host_pack_layout()
+        qs = (self.rows, self.heads, self.head_dim)
+        _check(lib().segkv_step_host_packed(self._h, step, _host(packed, (total,), torch.uint8, "packed"),
+                                            _host(out, qs, self.dtype, "out"), int(has_slopes), _stream_ptr(stream)),
+               "segkv_step_host_packed")
         return out
 
     # ------------------------------------------------------------------ aids

@@ -484,6 +484,35 @@ def test_step_host_matches_device_calls():
         r.close(); r2.close()
 
 
+def test_step_host_packed_matches_device_calls():
+    # one packed host block in, one copy out: same bits as the device-pointer calls (ALiBi slopes in the block too)
+    w = wl.Workload("packed", 2, 4, 8, 4, 128, 150, 6, "bf16", "uniform", True, 123)
+    r = Run(w)
+    r2 = Run(w)
+    try:
+        total, off = r2.h.host_pack_layout()
+        assert all(o % 256 == 0 for o in off) and total > off[4]
+        blk = torch.zeros(total, dtype=torch.uint8).pin_memory()
+        oh = torch.empty((w.rows, w.heads, w.head_dim), dtype=w.torch_dtype).pin_memory()
+
+        def put(o, t):
+            raw = t.contiguous().cpu().view(torch.uint8).reshape(-1)
+            blk[o:o + raw.numel()] = raw
+        put(off[1], r.slopes)
+        for t in range(w.steps):
+            r.append_next()
+            out, q = r.decode()
+            if t > 0:
+                put(off[0], torch.from_numpy(r.parents[t]))
+            put(off[2], r.k_steps[t]); put(off[3], r.v_steps[t]); put(off[4], q)
+            r2.h.step_host_packed(t, blk, oh, has_slopes=True)
+            assert torch.allclose(oh.float(), out.cpu().float(), atol=4e-3, rtol=2e-2)
+        assert np.array_equal(r2.h.get_ancestry(), r.h.get_ancestry())
+        assert r2.h.get_error() == 0
+    finally:
+        r.close(); r2.close()
+
+
 def test_argument_and_state_errors():
     h = sk.SegKV(1, 2, 2, 2, 64, 16, 4, torch.float16)
     dev = "cuda"
