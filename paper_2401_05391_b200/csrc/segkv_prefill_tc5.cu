@@ -370,6 +370,9 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         // -------------------------------- MMA issuer --------------------------------
         if (lane == 0) {
             uint32_t tp = 0;                                       // ring position of the item's first K/V tile
+            const uint64_t q_desc0 = smem_desc(smem_u32(q_smem), 16, 1024);
+            const uint64_t k_desc0 = smem_desc(smem_u32(k_ring), 16, 1024);
+            const uint64_t v_desc0 = smem_desc(smem_u32(v_ring), kColTile, 1024);
             uint32_t n[NG], qi[NG];                               // tiles / items of group g so far: barrier phases
 #pragma unroll
             for (int g = 0; g < NG; ++g) n[g] = qi[g] = 0;
@@ -387,15 +390,16 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 if (nkt == 0) continue;                           // the request ends before this item's rows
                 // S_g[buf] = Q_g . K^T for the group's tile kt; after its last one the group's Q may be replaced
                 auto issue_qk = [&](int g, int kt, int buf) {
-                    const uint32_t q_addr = smem_u32(q_smem) + (uint32_t)g * L::kQGroup;
-                    const uint32_t k_addr = smem_u32(k_ring + (size_t)((tp + kt) % SK) * kTileKV);
+                    // One descriptor per operand and tile; a K-step only moves the start address, which
+                    // sits in the descriptor's low bits in units of 16 bytes: the issuing thread is a
+                    // single lane, and every instruction it spends per MMA is time the tensor pipe waits.
+                    const uint64_t qd = q_desc0 + (uint64_t)(((uint32_t)g * L::kQGroup) >> 4);
+                    const uint64_t kd = k_desc0 + (uint64_t)((((tp + kt) % SK) * (uint32_t)kTileKV) >> 4);
+                    const uint32_t d_tmem = tmem + (uint32_t)(kKeys * (g * NB + buf));
 #pragma unroll
-                    for (int ks = 0; ks < kD / 16; ++ks) {
-                        const uint32_t off = (uint32_t)(ks & 3) * 32;
-                        tc_mma_ss(tmem + (uint32_t)(kKeys * (g * NB + buf)),
-                                  smem_desc(q_addr + (ks >> 2) * kBoxQ + off, 16, 1024),
-                                  smem_desc(k_addr + (ks >> 2) * kColTile + off, 16, 1024), p.idesc_qk, ks > 0);
-                    }
+                    for (int ks = 0; ks < kD / 16; ++ks)
+                        tc_mma_ss(d_tmem, qd + (uint64_t)(((ks >> 2) * kBoxQ + (ks & 3) * 32) >> 4),
+                                  kd + (uint64_t)(((ks >> 2) * kColTile + (ks & 3) * 32) >> 4), p.idesc_qk, ks > 0);
                     tc_commit(gbar0 + 48 * g + 8 * buf);
                     if (kt + 1 == gt[g]) tc_commit(gbar0 + 48 * g + 40);
                 };
@@ -424,7 +428,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         tc_commit(kempty0 + 8 * ((tp + kt + 1) % SK));
                     }
                     const uint32_t sv = (tp + kt) % SV;
-                    const uint32_t v_addr = smem_u32(v_ring + (size_t)sv * kTileKV);
+                    const uint64_t vd = v_desc0 + (uint64_t)((sv * (uint32_t)kTileKV) >> 4);
                     ok = mbar_wait_hot(vfull0 + 8 * sv, ((tp + kt) / SV) & 1);
                     if (!ok) break;
                     bool k_next = false;
@@ -439,7 +443,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
                         for (int kk = 0; kk < kKeys / 16; ++kk)   // O_g += P_g[:, 16 keys] . V[16 keys, :]
                             tc_mma_ts(tmem + (uint32_t)(L::kColO + kD * g), p_tmem + kk * 8,
-                                      smem_desc(v_addr + kk * 2048, kColTile, 1024), p.idesc_pv, (kt > 0 || kk > 0));
+                                      vd + (uint64_t)((kk * 2048) >> 4), p.idesc_pv, (kt > 0 || kk > 0));
                         tc_commit(gbar0 + 48 * g + 24);
 #if defined(SEGKV_TC5_TIMELINE) && SEGKV_TC5_TIMELINE == 3
                         mbar_wait_hot(gbar0 + 48 * g + 24, n[g] & 1);   // measurement only: serialise on P.V
