@@ -55,81 +55,53 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// Tensor map over one prompt array seen as [batch][prompt_len][kv_heads][D] in coordinates
-// (d, head, token, request), with the strides of the handle's prompt layout: tokens >=
-// prompt_len read as zero, a box holds one (request, head).
-// Box = 64 elements (128 bytes, one swizzle span) x one tile of tokens.
-int make_prompt_map(const segkv* h, void* base, int prompt_len, CUtensorMap* out) {
+// A 4-D tensor map in coordinates (d, head, token, request) over 16-bit elements: `heads` heads,
+// `tokens` tokens (those past the extent read as zero), element strides of a head / token /
+// request as given, box = 64 elements (128 bytes, one swizzle span) x box_tokens tokens of one
+// (request, head), 128-byte swizzle.  `what` names the array in the error text.
+int encode_map_4d(const segkv* h, const void* base, int heads, int tokens, long long stride_h, long long stride_p,
+                  long long stride_b, int box_tokens, const char* what, CUtensorMap* out) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) {
         snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled entry point not available");
         return SEGKV_ECUDA;
     }
     const Dims& d = h->d;
-    const PromptStrides ps = prompt_strides(d);
-    cuuint64_t dims[4] = {(cuuint64_t)d.head_dim, (cuuint64_t)d.kv_heads, (cuuint64_t)prompt_len, (cuuint64_t)d.batch};
-    cuuint64_t strides[3] = {(cuuint64_t)ps.h * 2, (cuuint64_t)ps.p * 2, (cuuint64_t)ps.b * 2};
-    cuuint32_t box[4] = {64, 1, (cuuint32_t)tiled_tile_keys(d.head_dim), 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUtensorMapDataType dt = d.dtype == SEGKV_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
-    CUresult r = fn(out, dt, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
-        return SEGKV_ECUDA;
-    }
-    return SEGKV_OK;
-}
-
-// Tensor map over the prefill query [batch][prompt_len][heads][D] (token-major): one box is 64
-// elements of one head for 128 consecutive tokens; tokens >= prompt_len read as zero.
-int make_query_map(const segkv* h, const void* q, int prompt_len, CUtensorMap* out) {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) {
-        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled entry point not available");
-        return SEGKV_ECUDA;
-    }
-    const Dims& d = h->d;
-    const cuuint64_t row = (cuuint64_t)d.head_dim * 2;
-    cuuint64_t dims[4] = {(cuuint64_t)d.head_dim, (cuuint64_t)d.heads, (cuuint64_t)prompt_len, (cuuint64_t)d.batch};
-    cuuint64_t strides[3] = {row, row * d.heads, row * d.heads * prompt_len};
-    cuuint32_t box[4] = {64, 1, 128, 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUtensorMapDataType dt = d.dtype == SEGKV_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
-    CUresult r = fn(out, dt, 4, const_cast<void*>(q), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled (query) failed with CUresult %d", (int)r);
-        return SEGKV_ECUDA;
-    }
-    return SEGKV_OK;
-}
-
-// Tensor map over the caller's prefill K or V, token-major [batch][prompt_len][kv_heads][D], in
-// the coordinates of the prompt-segment maps (d, kv head, token, request) and with their box.
-int make_kv_source_map(const segkv* h, const void* base, int prompt_len, CUtensorMap* out) {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) {
-        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled entry point not available");
-        return SEGKV_ECUDA;
-    }
-    const Dims& d = h->d;
-    const cuuint64_t row = (cuuint64_t)d.head_dim * 2;
-    cuuint64_t dims[4] = {(cuuint64_t)d.head_dim, (cuuint64_t)d.kv_heads, (cuuint64_t)prompt_len, (cuuint64_t)d.batch};
-    cuuint64_t strides[3] = {row, row * d.kv_heads, row * d.kv_heads * prompt_len};
-    cuuint32_t box[4] = {64, 1, (cuuint32_t)tiled_tile_keys(d.head_dim), 1};
+    cuuint64_t dims[4] = {(cuuint64_t)d.head_dim, (cuuint64_t)heads, (cuuint64_t)tokens, (cuuint64_t)d.batch};
+    cuuint64_t strides[3] = {(cuuint64_t)stride_h * 2, (cuuint64_t)stride_p * 2, (cuuint64_t)stride_b * 2};
+    cuuint32_t box[4] = {64, 1, (cuuint32_t)box_tokens, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUtensorMapDataType dt = d.dtype == SEGKV_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
     CUresult r = fn(out, dt, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
-        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled (prefill K/V) failed with CUresult %d", (int)r);
+        snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled (%s) failed with CUresult %d", what, (int)r);
         return SEGKV_ECUDA;
     }
     return SEGKV_OK;
+}
+
+// One prompt array of the handle, [batch][prompt_len][kv_heads][D] logically, with the strides
+// of the handle's prompt layout; a box is one tile of tokens.
+int make_prompt_map(const segkv* h, void* base, int prompt_len, CUtensorMap* out) {
+    const PromptStrides ps = prompt_strides(h->d);
+    return encode_map_4d(h, base, h->d.kv_heads, prompt_len, ps.h, ps.p, ps.b, tiled_tile_keys(h->d.head_dim),
+                         "prompt segment", out);
+}
+
+// The prefill query [batch][prompt_len][heads][D] (token-major): a box is 128 consecutive tokens.
+int make_query_map(const segkv* h, const void* q, int prompt_len, CUtensorMap* out) {
+    const long long D = h->d.head_dim, H = h->d.heads;
+    return encode_map_4d(h, q, h->d.heads, prompt_len, D, D * H, D * H * prompt_len, 128, "prefill query", out);
+}
+
+// The caller's prefill K or V, token-major [batch][prompt_len][kv_heads][D], with the box of the
+// prompt-segment maps.
+int make_kv_source_map(const segkv* h, const void* base, int prompt_len, CUtensorMap* out) {
+    const long long D = h->d.head_dim, Hkv = h->d.kv_heads;
+    return encode_map_4d(h, base, h->d.kv_heads, prompt_len, D, D * Hkv, D * Hkv * prompt_len,
+                         tiled_tile_keys(h->d.head_dim), "prefill K/V", out);
 }
 
 void free_all(segkv* h) {
