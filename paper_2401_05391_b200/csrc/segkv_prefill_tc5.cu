@@ -1,31 +1,34 @@
-// Prefill attention on the fifth-generation tensor cores (tcgen05 + tensor memory), head_dim 128.
+// Prefill attention on the fifth-generation tensor cores (tcgen05 + tensor memory), head_dim 64,
+// 128 or 256 (paper Section 3.1 / 3.3: the prefill kernel is the special case of the customised
+// SDPA kernel that sees only the query and the prompt key/value, batch-first in and out):
+//     out[b,i,h,:] = softmax_{j<=i}( q[b,i,h,:] . K[b,j,:] / sqrt(D) + bias ) . V[b,j,:].
 //
-// Same operation as segkv_prefill_sdpa.cu (paper Section 3.1 / 3.3: causal attention of the
-// prompt, batch-first in and out, K/V from the prompt segment), laid out for tcgen05:
-//
-//   * a CTA owns one or two groups of 128 query rows of one (request, head): one row per TMEM
-//     lane and per softmax thread;
-//   * Q [128 x 128] of each group is staged once in shared memory in the 128-byte-swizzled
-//     K-major layout; K and V tiles of 128 keys arrive by TMA in the same layout (the prompt
-//     segment's tensor maps), through separate rings: a K tile is needed one step before the V
-//     tile of the same keys;
-//   * one elected thread issues the MMAs: S = Q.K^T (M 128, N 128, eight K-steps of 16) into a
-//     128-column TMEM buffer and O += P.V (M 128, N 128, eight K-steps) into a 128-column TMEM
-//     accumulator.  P never touches shared memory: the softmax threads write it, rounded to the
-//     16-bit type, over the first 64 columns of the S buffer it came from, and the MMA takes its
-//     A operand from tensor memory.  V is consumed as an MN-major B operand straight from its
-//     row-major tile.  Both operands in shared memory would make every MMA wait for 8 KB of
-//     shared-memory reads; with P in tensor memory P.V reads only V;
+//   * one persistent CTA per SM walks a static list of work items (one or two groups of 128
+//     query rows of one (request, head)), longest first; a group's rows are one per TMEM lane and
+//     per softmax thread;
+//   * Q of each group arrives by TMA (a per-call tensor map over [B, N, H, D]) in the
+//     128-byte-swizzled K-major layout; K and V tiles (128 keys; 64 at head_dim 256) arrive by TMA
+//     in the same layout through separate rings: a K tile is needed one step before the V tile
+//     of the same keys.  They come from the prompt segment, or (fused prefill) from the caller's
+//     arrays, and are then also stored on into the segment, each tile by one CTA;
+//   * one elected thread issues the MMAs: S = Q.K^T (M 128, N = keys of a tile, K-steps of 16)
+//     into a TMEM buffer and O += P.V (M 128, N = head_dim) into a TMEM accumulator.  P never
+//     touches shared memory: the softmax threads write it, rounded to the 16-bit type, over the
+//     first half of the columns of the S buffer it came from, and the MMA takes its A operand
+//     from tensor memory.  V is consumed as an MN-major B operand straight from its row-major
+//     tile;
 //   * the softmax threads read S with tcgen05.ld (no shuffles for the row max / sum) and
 //     rescale O in tensor memory only when a row's maximum has grown by more than 2^8 since the
 //     reference it is using (the sum uses the same reference, so the result is exact);
 //   * with two groups per CTA each has one S buffer and the tensor cores work for one group
 //     while the other is in its softmax; with one group S is double-buffered so that Q.K^T of
-//     tile j+1 runs under the softmax of tile j.
+//     tile j+1 runs under the softmax of tile j.  The tail of one item overlaps the head of the
+//     next (loads, and the first Q.K^T while the previous output is stored).
 //
-// Tensor memory (512 columns): S buffers at 0 and 128, O accumulators at 256 (+128 for the
-// second group).  Every mbarrier wait is bounded; on expiry the kernel flags
-// SEGKV_DEV_WAIT_LIMIT, skips the output and still releases its tensor memory.
+// Tensor memory (all 512 columns are allocated): S buffers first, then one O accumulator per
+// group.  Every mbarrier is waited on phase by phase (a parity wait cannot tell phases two
+// apart) and every wait is bounded; on expiry the kernel flags SEGKV_DEV_WAIT_LIMIT, skips
+// the output and still releases its tensor memory.
 #include "segkv_internal.h"
 #include "segkv_ptx.cuh"
 
