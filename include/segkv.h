@@ -97,7 +97,9 @@ SEGKV_API int segkv_create_growing(segkv_t* out, int batch, int beams, int heads
  * (Eq. 3 for one layer; "steps held" is max_steps, or the chunks opened so far). */
 SEGKV_API long long segkv_allocated_kv_bytes(segkv_t h);
 
-/* Free everything the handle owns.  Synchronises the device.  NULL is allowed. */
+/* Free everything the handle owns.  Synchronises the device.  NULL is allowed.
+ * ESTATE (and nothing freed) while other handles use this one's tables
+ * (segkv_share_index). */
 SEGKV_API int segkv_destroy(segkv_t h);
 
 /*
@@ -364,7 +366,9 @@ SEGKV_API int segkv_append_rope(segkv_t h, int step, const int32_t* beam_parent,
  * Both handles must be at step 0 (ESTATE) and agree in batch, beams and
  * max_steps (EINVAL); a handle that follows cannot lead (EINVAL).
  * leader == NULL gives h its own tables back.  Truncating or resetting is the
- * caller's to do on every handle; destroy the followers before their leader.
+ * caller's to do on every handle.  segkv_destroy of a handle that others still
+ * follow returns ESTATE and destroys nothing: destroy the followers (or give
+ * them their own tables back) first.
  */
 SEGKV_API int segkv_share_index(segkv_t h, segkv_t leader);
 

@@ -322,6 +322,7 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
     h->prefill_groups = 0;
     h->ragged = false;
     h->leader = nullptr;
+    h->followers = 0;
     d.prompt_layout = SEGKV_PROMPT_HEAD_MAJOR;
 
     int rc = SEGKV_OK;
@@ -380,6 +381,8 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
 
 int segkv_destroy(segkv_t h) {
     if (!h) return SEGKV_OK;
+    if (h->followers > 0) return SEGKV_ESTATE;        // other handles still read this one's tables
+    if (h->leader) h->leader->followers--;
     cudaDeviceSynchronize();
     free_all(h);
     delete h;
@@ -851,7 +854,10 @@ int segkv_share_index(segkv_t h, segkv_t leader) {
         const Dims &a = h->d, &b = leader->d;
         if (a.batch != b.batch || a.beams != b.beams || a.max_steps != b.max_steps) return SEGKV_EINVAL;
         if (leader->steps != 0) return SEGKV_ESTATE;
+        if (h->followers > 0) return SEGKV_EINVAL;           // a handle that leads cannot follow
     }
+    if (h->leader) h->leader->followers--;
+    if (leader) leader->followers++;
     h->leader = leader;
     return SEGKV_OK;
 }

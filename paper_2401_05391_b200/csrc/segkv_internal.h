@@ -73,6 +73,7 @@ struct segkv {
     int32_t* parent;     // [max_steps, rows]
     int32_t* anc[2];     // [rows, max_steps], generation t lives in anc[t & 1]
     segkv* leader;       // the handle whose beam-index tables this one uses (segkv_share_index), or NULL
+    int followers;       // handles that use THIS one's tables; it cannot be destroyed while there are any
     void* st_pack;       // staging for segkv_step_host_packed: parent | slopes | k | v | q in one block
     int32_t* plens;      // [batch] per-request prompt lengths (segkv_prefill_write_ragged)
     bool ragged;         // plens is in use; prompt_len is then the longest

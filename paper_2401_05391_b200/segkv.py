@@ -150,7 +150,7 @@ class SegKV:
     # ------------------------------------------------------------ life cycle
     def destroy(self) -> None:
         if getattr(self, "_h", None) is not None and self._h:
-            lib().segkv_destroy(self._h)
+            _check(lib().segkv_destroy(self._h), "segkv_destroy")     # refused while other handles follow this one
             self._h = None
 
     def __del__(self):

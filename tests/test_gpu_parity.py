@@ -342,6 +342,7 @@ def test_layers_share_one_beam_index_table(leader_fused):
                     assert np.array_equal(f.h.get_ancestry(), lead.oracle_ancestry(t))
         for r in layers:
             assert r.h.get_error() == 0
+        assert sk.lib().segkv_destroy(lead.h._h) == -2           # ESTATE: two handles still follow it
         followers[0].h.reset()
         followers[0].h.share_index(None)
         with pytest.raises(sk.SegKVError):
