@@ -200,6 +200,14 @@ def test_prefill_is_bit_reproducible_across_runs(D, H, Hkv, P, groups):
         h.destroy()
 
 
+@pytest.mark.parametrize("D,H,Hkv,P", [(128, 8, 8, 4096), (256, 8, 2, 3000)])
+def test_prefill_long_prompt_sampled(D, H, Hkv, P):
+    # 32 or more key tiles per row group, items of very different lengths on every CTA
+    w = wl.Workload("pf", 1, 2, H, Hkv, D, P, 2, "f16", "uniform", False, 94)
+    h = run_prefill(w, lambda w: sampled_rows(w, 96))[0]
+    h.destroy()
+
+
 def test_prefill_llama2_7b_shape_sampled():
     h = run_prefill(wl.CONFIGS[1], lambda w: sampled_rows(w, 256))[0]
     h.destroy()
