@@ -52,6 +52,7 @@ def parse():
     ap.add_argument("--prompt-layout", default="head_major", choices=["head_major", "token_major", "seq_first"],
                     help="memory layout of the prompt segment (the paper's Fig. 6 compares layouts)")
     ap.add_argument("--beams", type=int, default=0, help="override the workload's beam width")
+    ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length")
     ap.add_argument("--prefill", action="store_true", help="time the prefill attention instead of the decode step")
     ap.add_argument("--prefill-groups", type=int, default=0,
                     help="128-row groups per CTA of the head_dim-128 prefill kernel (1 or 2; 0 = automatic)")
@@ -223,6 +224,8 @@ def run_ours(args):
         w = w.scaled(batch=args.batch, name=f"{w.name}[batch={args.batch}]")
     if args.beams:
         w = w.scaled(beams=args.beams, name=f"{w.name}[beams={args.beams}]")
+    if args.prompt_len:
+        w = w.scaled(prompt_len=args.prompt_len, name=f"{w.name}[prompt={args.prompt_len}]")
     L = args.layers or DEFAULT_LAYERS.get(w.name.split("[")[0], 1)
     T = args.at_step or w.steps
     t = T - 1
@@ -454,6 +457,8 @@ def run_prefill(args):
         w = w.scaled(batch=args.batch, name=f"{w.name}[batch={args.batch}]")
     if args.beams:
         w = w.scaled(beams=args.beams, name=f"{w.name}[beams={args.beams}]")
+    if args.prompt_len:
+        w = w.scaled(prompt_len=args.prompt_len, name=f"{w.name}[prompt={args.prompt_len}]")
     L = args.layers or DEFAULT_LAYERS.get(w.name.split("[")[0], 1)
     handles = []
     for layer in range(L):
