@@ -637,7 +637,12 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     bool cluster;
     choose_tiling(h, &splits, &stages, &cluster);
     h->steps = step;
-    if (splits == 1 && !h->fuse_always) {
+    // rows a CTA's share of the steps can reach: beyond a tile and a half of them, deriving the rows
+    // in the kernel costs more than the separate append launch (measured at prompts of 128 to 512
+    // tokens with 128 steps: 10.0-10.6 us as two launches against 10.8-12.9 us fused)
+    const long long rows_per_cta = (long long)((step + 1 + splits - 1) / splits) * d.beams;
+    const bool long_tail = h->splits_forced <= 0 && 2 * rows_per_cta > 3 * tiled_tile_keys(d.head_dim);   // a forced split count keeps the fused kernel
+    if ((splits == 1 || long_tail) && !h->fuse_always) {
         // Work groups that fill the GPU on their own are bandwidth-bound: the separate append is
         // then ~1 % of the step and the list it makes keeps the response tiles dense and cheap
         // to build, so the two launches are the faster form.
