@@ -121,6 +121,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     return ((uint64_t)hi << 32) | lo;
 }
 
+template <bool B> struct BoolC { static constexpr bool value = B; };
+template <typename T> struct SplitP { typedef char yes; static constexpr bool value = false; };
+template <> struct SplitP<__nv_bfloat16> { typedef char yes; static constexpr bool value = true; };
+
 // Critical-path wait: poll without sleeping first (the hardware suspends the thread inside
 // try_wait for a while), then fall back to the bounded, sleeping wait.
 __device__ __forceinline__ bool mbar_wait_hot(uint32_t bar, uint32_t parity) {
@@ -187,6 +191,22 @@ __device__ __forceinline__ float score_max(float* sv, float scale2, float slope2
     return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
 }
 
+// bf16 keeps 8 significant bits of a softmax weight.  Where a few keys carry a row's whole weight
+// and their values cancel, that rounding alone exceeds the path's tolerance, so where it can
+// happen the weights go to the tensor cores as TWO bf16 parts, p = hi + lo (hi = p cut to bf16,
+// lo = bf16(p - hi): 16 significant bits together), lo in the second half of the S buffer's
+// columns, and O takes a second P.V MMA for those keys.  Which keys is known from the launch
+// shape: the first key tile of the rows that start the prompt (a handful of keys in all), and,
+// under an ALiBi slope steep enough to put a row's weight on its nearest neighbours, the keys
+// within kSplitWindow of the group's rows.  fp16 weights (11 bits) never need it.
+constexpr float kSplitSlope = 0.0625f;   // weights fall by e^-slope per key: below this, dozens of keys share a row's weight
+constexpr int kSplitWindow = 64;
+// Do the `nkeys` keys from `key0` on get two-part weights, for the group whose first row is row0?
+__device__ __forceinline__ bool split_p_keys(int row0, int key0, int nkeys, float slope) {
+    if (row0 == 0 && key0 < kRows) return true;
+    return slope >= kSplitSlope && key0 + nkeys - 1 >= row0 - kSplitWindow;
+}
+
 // One CTA per SM walks a static list of work items (128*NG query rows of one (request, head)),
 // longest first and dealt round-robin, so that the tail of one item overlaps the head of the
 // next: the producer runs ahead through the K/V rings and reloads a group's Q as soon as the
@@ -202,6 +222,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                    const __grid_constant__ CUtensorMap tm_v_seg, const Tc5Params p) {
     constexpr int NG = L::NG, NB = L::NB, SK = L::kStagesK, SV = L::kStagesV;
     constexpr bool STORE = MODE == 1, RAGGED = MODE == 2;
+    constexpr bool kSplitP = sizeof(typename SplitP<T>::yes) != 0 && SplitP<T>::value;
     constexpr int kD = L::D, kKeys = L::KEYS, kTileKV = L::kTileKV, kColTile = L::kColTile;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -384,6 +405,8 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const int w = round_item(j);
                 if (w >= n_items) continue;
                 const int qt = item_qt(w), nb = request_len((w % hb_count) / p.H);
+                // requested here, used after the first waits of the item
+                const float slope = (kSplitP && p.slopes) ? __ldg(p.slopes + (w % hb_count) % p.H) : 0.f;
                 int gt[NG], nkt = 0;
 #pragma unroll
                 for (int g = 0; g < NG; ++g) {
@@ -447,6 +470,13 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         for (int kk = 0; kk < kKeys / 16; ++kk)   // O_g += P_g[:, 16 keys] . V[16 keys, :]
                             tc_mma_ts(tmem + (uint32_t)(L::kColO + kD * g), p_tmem + kk * 8,
                                       vd + (uint64_t)((kk * 2048) >> 4), p.idesc_pv, (kt > 0 || kk > 0));
+                        if (kSplitP && split_p_keys((qt * NG + g) * kRows, kt * kKeys, kKeys, slope)) {
+#pragma unroll
+                            for (int kk = 0; kk < kKeys / 16; ++kk)   // ... and the low parts of the weights that have one
+                                if (split_p_keys((qt * NG + g) * kRows, kt * kKeys + 16 * kk, 16, slope))
+                                    tc_mma_ts(tmem + (uint32_t)(L::kColO + kD * g), p_tmem + kKeys / 2 + kk * 8,
+                                              vd + (uint64_t)((kk * 2048) >> 4), p.idesc_pv, 1u);
+                        }
                         tc_commit(gbar0 + 48 * g + 24);
 #if defined(SEGKV_TC5_TIMELINE) && SEGKV_TC5_TIMELINE == 3
                         mbar_wait_hot(gbar0 + 48 * g + 24, n[g] & 1);   // measurement only: serialise on P.V
@@ -491,7 +521,8 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const int my_tiles = group_tiles(qt, g, request_len(b));
             if (my_tiles == 0) continue;
             const int row0 = (qt * NG + g) * kRows, row = row0 + r;
-            const float slope2 = p.slopes ? p.slopes[h] * 1.4426950408889634f : 0.f;
+            const float slope_nat = p.slopes ? p.slopes[h] : 0.f;
+            const float slope2 = slope_nat * 1.4426950408889634f;
             float m_ref = -INFINITY, l_run = 0.f;
             for (int kt = 0; kt < my_tiles; ++kt, ++n) {
                 const int buf = NB == 2 ? (int)(n & 1) : 0;
@@ -500,76 +531,108 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (stamp) TC5_STAMP(g, kt, 0);
-                tc_fence_after();
-                uint32_t sr[kKeys];
-#pragma unroll
-                for (int c = 0; c < kKeys / 32; ++c) tc_ld32(tm_s + 32 * c, sr + 32 * c);
-                tc_wait_ld();
-                if (stamp) TC5_STAMP(g, kt, 1);
-                float* sv = reinterpret_cast<float*>(sr);
-                const int key0 = kt * kKeys;
-                const bool diag = key0 + kKeys - 1 > row0;         // a tile that reaches past the group's first row
-                // scores in log2 units: s * scale2 (+ ALiBi bias); the scale is folded into the exponent's
-                // FMA unless a bias has to be added first; keys above the row (diagonal tile) become -inf
-                const bool biased = p.slopes != nullptr;
-                const int lim = row - key0;                        // key index i of this tile is visible iff i <= lim
-                const float bias0 = slope2 * (float)(key0 - row);
-                float tmax;
-                if (biased) tmax = diag ? score_max<kKeys, true, true>(sv, p.scale2, slope2, bias0, lim)
-                                        : score_max<kKeys, true, false>(sv, p.scale2, slope2, bias0, lim);
-                else tmax = (diag ? score_max<kKeys, false, true>(sv, p.scale2, slope2, bias0, lim)
-                                  : score_max<kKeys, false, false>(sv, p.scale2, slope2, bias0, lim)) * p.scale2;
-                // a new reference only when the maximum has grown by more than 2^8: exponentials stay
-                // below 2^8 of the reference, the sum and O use the same reference
-                const bool need = tmax > m_ref + 8.f;
-                float alpha = 1.f;
-                if (need) {
-                    alpha = exp2f(m_ref - tmax);                   // 0 on the first tile
-                    m_ref = tmax;
-                }
-                float ls[4] = {0.f, 0.f, 0.f, 0.f};
-                uint32_t pk[kKeys / 2];
-                const float sc = biased ? 1.f : p.scale2, nm = -m_ref;
-#pragma unroll
-                for (int i = 0; i < kKeys; i += 2) {
-                    const float e0 = exp2f(fmaf(sv[i], sc, nm)), e1 = exp2f(fmaf(sv[i + 1], sc, nm));
-                    ls[(i >> 1) & 3] += e0 + e1;
-                    pk[i >> 1] = Mma<T>::pack(e0, e1);
-                }
-                l_run = l_run * alpha + ((ls[0] + ls[1]) + (ls[2] + ls[3]));
-                if (stamp) TC5_STAMP(g, kt, 2);
-                // O may be touched once P.V of the previous tile is done.  A parity wait is only
-                // meaningful on the barrier's current or previous phase, so with two S buffers,
-                // where nothing else ties this thread to the P.V before last, every phase of the O
-                // barrier is waited for in turn (with one S buffer the scores of this tile were
-                // produced behind that P.V in the pipe, and waiting here is only needed to rescale).
-                const bool rescale = kt > 0 && __any_sync(0xffffffffu, need);
-                if (kt > 0 && (NB == 2 || rescale)) {
-                    ok = mbar_wait_hot(bar_o, (n - 1) & 1);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
+                // One tile of the group, from the scores in tensor memory to the weights handed to the
+                // MMA thread.  Two instances (weights in one part / in two parts) rather than a branch
+                // in the middle: the 128 scores live in registers, and a fork with all of them live
+                // costs the two-group shape hundreds of bytes of spills.
+                auto tile = [&](auto two_parts) -> bool {
+                    constexpr bool split = decltype(two_parts)::value;
                     tc_fence_after();
-                }
-                if (rescale) {
+                    uint32_t sr[kKeys];
 #pragma unroll
-                    for (int c = 0; c < kD / 32; ++c) {
-                        uint32_t orr[32];
-                        tc_ld32(tm_o + c * 32, orr);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
-                        tc_st32(tm_o + c * 32, orr);
+                    for (int c = 0; c < kKeys / 32; ++c) tc_ld32(tm_s + 32 * c, sr + 32 * c);
+                    tc_wait_ld();
+                    if (stamp) TC5_STAMP(g, kt, 1);
+                    float* sv = reinterpret_cast<float*>(sr);
+                    const int key0 = kt * kKeys;
+                    const bool diag = key0 + kKeys - 1 > row0;         // a tile that reaches past the group's first row
+                    // scores in log2 units: s * scale2 (+ ALiBi bias); the scale is folded into the exponent's
+                    // FMA unless a bias has to be added first; keys above the row (diagonal tile) become -inf
+                    const bool biased = p.slopes != nullptr;
+                    const int lim = row - key0;                        // key index i of this tile is visible iff i <= lim
+                    const float bias0 = slope2 * (float)(key0 - row);
+                    float tmax;
+                    if (biased) tmax = diag ? score_max<kKeys, true, true>(sv, p.scale2, slope2, bias0, lim)
+                                            : score_max<kKeys, true, false>(sv, p.scale2, slope2, bias0, lim);
+                    else tmax = (diag ? score_max<kKeys, false, true>(sv, p.scale2, slope2, bias0, lim)
+                                      : score_max<kKeys, false, false>(sv, p.scale2, slope2, bias0, lim)) * p.scale2;
+                    // a new reference only when the maximum has grown by more than 2^8: exponentials stay
+                    // below 2^8 of the reference, the sum and O use the same reference
+                    const bool need = tmax > m_ref + 8.f;
+                    float alpha = 1.f;
+                    if (need) {
+                        alpha = exp2f(m_ref - tmax);                   // 0 on the first tile
+                        m_ref = tmax;
                     }
-                    if (stamp) TC5_STAMP(g, kt, 3);
-                }
-                // P over the first 64 columns of the S buffer: two 16-bit weights per column, the A
-                // operand layout of the MMA that follows.  S has been read completely above.
+                    float ls[4] = {0.f, 0.f, 0.f, 0.f};
+                    uint32_t pk[kKeys / 2];
+                    const float sc = biased ? 1.f : p.scale2, nm = -m_ref;
+                    if (!split) {
 #pragma unroll
-                for (int c = 0; c < kKeys / 32; ++c) tc_st16(tm_s + 16 * c, pk + 16 * c);
-                tc_wait_st();
-                tc_fence_before();
-                mbar_arrive(bar_p);
-                if (stamp) TC5_STAMP(g, kt, 4);
+                        for (int i = 0; i < kKeys; i += 2) {
+                            const float e0 = exp2f(fmaf(sv[i], sc, nm)), e1 = exp2f(fmaf(sv[i + 1], sc, nm));
+                            ls[(i >> 1) & 3] += e0 + e1;
+                            pk[i >> 1] = Mma<T>::pack(e0, e1);
+                        }
+                    } else {
+                        // weights as two bf16 parts: the high parts over the first half of the S buffer's
+                        // columns, the low parts over the second half, 32 keys at a time (S is in registers
+                        // and the MMAs that read the buffer's previous contents have completed)
+#pragma unroll
+                        for (int c = 0; c < kKeys / 32; ++c) {
+                            uint32_t ph[16], pl[16];
+#pragma unroll
+                            for (int i = 0; i < 32; i += 2) {
+                                const float e0 = exp2f(fmaf(sv[32 * c + i], sc, nm)), e1 = exp2f(fmaf(sv[32 * c + i + 1], sc, nm));
+                                ls[(i >> 1) & 3] += e0 + e1;
+                                const uint32_t b0 = __float_as_uint(e0), b1 = __float_as_uint(e1);
+                                ph[i >> 1] = __byte_perm(b0, b1, 0x7632);
+                                pl[i >> 1] = Mma<T>::pack(e0 - __uint_as_float(b0 & 0xFFFF0000u), e1 - __uint_as_float(b1 & 0xFFFF0000u));
+                            }
+                            tc_st16(tm_s + 16 * c, ph);
+                            tc_st16(tm_s + kKeys / 2 + 16 * c, pl);
+                        }
+                    }
+                    l_run = l_run * alpha + ((ls[0] + ls[1]) + (ls[2] + ls[3]));
+                    if (stamp) TC5_STAMP(g, kt, 2);
+                    // O may be touched once P.V of the previous tile is done.  A parity wait is only
+                    // meaningful on the barrier's current or previous phase, so with two S buffers,
+                    // where nothing else ties this thread to the P.V before last, every phase of the O
+                    // barrier is waited for in turn (with one S buffer the scores of this tile were
+                    // produced behind that P.V in the pipe, and waiting here is only needed to rescale).
+                    const bool rescale = kt > 0 && __any_sync(0xffffffffu, need);
+                    if (kt > 0 && (NB == 2 || rescale)) {
+                        bool arrived = mbar_wait_hot(bar_o, (n - 1) & 1);
+                        arrived = __all_sync(0xffffffffu, arrived);
+                        if (!arrived) return false;
+                        tc_fence_after();
+                    }
+                    if (rescale) {
+#pragma unroll
+                        for (int c = 0; c < kD / 32; ++c) {
+                            uint32_t orr[32];
+                            tc_ld32(tm_o + c * 32, orr);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+                            tc_st32(tm_o + c * 32, orr);
+                        }
+                        if (stamp) TC5_STAMP(g, kt, 3);
+                    }
+                    // P over the first 64 columns of the S buffer: two 16-bit weights per column, the A
+                    // operand layout of the MMA that follows.  S has been read completely above.
+                    if (!split) {
+#pragma unroll
+                        for (int c = 0; c < kKeys / 32; ++c) tc_st16(tm_s + 16 * c, pk + 16 * c);
+                    }
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(bar_p);
+                    if (stamp) TC5_STAMP(g, kt, 4);
+                    return true;
+                };
+                ok = (kSplitP && split_p_keys(row0, kt * kKeys, kKeys, slope_nat)) ? tile(BoolC<kSplitP>{}) : tile(BoolC<false>{});
+                if (!ok) break;
             }
             if (!ok) break;
             // the item's output: O / l, once the last P.V has landed.  The next item's first P.V
@@ -625,7 +688,8 @@ cudaError_t launch_tc5(const Dims& d, const PrefillArgs& a, Tc5Params p, int sms
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-    // instruction descriptors: fp32 accumulate, A/B format, operand majors, N >> 3, M >> 4
+    // instruction descriptors: fp32 accumulate, A/B format (the same for both operands: a P in fp16
+    // against a V in bf16 is not a pair the f16 kind takes), operand majors, N >> 3, M >> 4
     const uint32_t fmt = d.dtype == SEGKV_BF16 ? 1u : 0u;
     const uint32_t common = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kRows >> 4) << 24);
     p.idesc_qk = common | ((uint32_t)(L::KEYS >> 3) << 17);               // A, B both K-major; N = keys of a tile
