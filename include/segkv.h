@@ -209,8 +209,9 @@ SEGKV_API int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent,
  * segkv_decode_sdpa for callers that must not allocate device memory.  (The
  * paper has no counterpart: this is a deployment variant of the same kernel.)
  *
- * Who needs it: segkv_decode_sdpa may grow its split workspace with cudaMalloc
- * when the launch shape changes.  A caller inside a serving loop whose memory
+ * Who needs it: segkv_decode_sdpa keeps its split workspace in memory the handle
+ * allocates with cudaMalloc (at create time, and again when segkv_set_tuning
+ * asks for more splits than that covers).  A caller inside a serving loop whose memory
  * pool owns the whole device, a caller whose next request must not stall
  * behind the device-wide synchronisation an allocation implies, or a caller
  * that is not allowed to call the CUDA allocator at all (a plug-in running
@@ -231,7 +232,8 @@ SEGKV_API int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent,
  *     query columns per kv head, which the tiled kernel does not take;
  *   - the first call on each device looks the array's device address up
  *     (cudaGetSymbolAddress, with the handle's device current).  Make that
- *     first call before any stream capture begins;
+ *     first call before any stream capture begins, and from one host thread
+ *     (later calls only read the stored address);
  *   - all handles and all calls share the one array, and it keeps what the
  *     last call left: the counters are cleared on the stream at the start of
  *     every call, and two calls that overlap on the GPU (different streams, or
@@ -396,6 +398,23 @@ SEGKV_API int segkv_set_prompt_layout(segkv_t h, int layout);
  * ignore it.  A launch-shape knob: the paper has no counterpart.
  */
 SEGKV_API int segkv_set_prefill_tuning(segkv_t h, int row_groups);
+
+/*
+ * Test aid for the kernels' bounded waits (no counterpart in the paper).  Every
+ * wait inside the attention kernels gives up after about two seconds, sets
+ * SEGKV_DEV_WAIT_LIMIT in the device error word, lets copies in flight land,
+ * releases what the kernel holds and returns without writing the output; the
+ * call that launched it still returns SEGKV_OK and segkv_get_error() reports
+ * the flag.  Nothing on a healthy device makes a wait run out, so a test asks
+ * for it: the handle's NEXT attention launch (segkv_decode_sdpa,
+ * segkv_decode_step's fused form, segkv_decode_sdpa_static or
+ * segkv_prefill_sdpa) uses `wait_limit_ns` (0 = default) as the limit of its
+ * waits and, if `skip_arrival` is non-zero, leaves out one plain mbarrier
+ * arrival of one role (never a copy), so that the role waiting for it runs
+ * into the limit.  The kernel returns by itself; later launches are normal.
+ * Errors: EINVAL (NULL handle, negative limit).
+ */
+SEGKV_API int segkv_debug_inject(segkv_t h, long long wait_limit_ns, int skip_arrival);
 
 /* Kernels launched by the handle since creation (each launch counted once). */
 SEGKV_API long long segkv_launch_count(segkv_t h);

@@ -255,6 +255,8 @@ SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes
     a.pdl = false;
     a.prompt_immutable = h->steps > 0;     // the first append after a prefill is a fully serialised launch
     a.fused = false;
+    a.wait_ns = h->dbg_wait_ns;
+    a.dbg_skip = h->dbg_skip;
     a.parent = nullptr;
     a.k_new = a.v_new = nullptr;
     a.kr_new_slab = a.vr_new_slab = nullptr;
@@ -373,7 +375,15 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
     SEGKV_TRY(dmalloc(&h->st_slopes, (size_t)heads * sizeof(float)));
     SEGKV_TRY(dmalloc(&h->st_pack, segkv_host_pack_bytes(h, nullptr)));
 #undef SEGKV_TRY
-    rc = alloc_workspace(h, 1);
+    // The split workspace for the largest split count the automatic choice can make (one wave of
+    // CTA slots shared among the work groups), so that the decode loop never allocates.
+    {
+        const long long slabs = (long long)batch * kv_heads, slots = (long long)h->sm_count * 2;
+        long long most = slots / slabs;
+        if (most < 1) most = 1;
+        if (most > kMaxSplits) most = kMaxSplits;
+        rc = alloc_workspace(h, (int)most);
+    }
     if (rc != SEGKV_OK) return fail(rc);
     *out = h;
     return SEGKV_OK;
@@ -422,7 +432,7 @@ static int prefill_write_impl(segkv_t h, const void* k, const void* v, int promp
     cudaStream_t st = (cudaStream_t)stream;
     h->tm_valid = false;
     if (prompt_len > 0) {
-        SEGKV_CUDA(launch_prefill_transpose(h->d, k, v, h->kp, h->vp, plens_dev, prompt_len, st));
+        SEGKV_CUDA(launch_prefill_transpose(h->d, k, v, h->kp, h->vp, plens_dev, prompt_len, h->sm_count, st));
         h->launches++;
         int rc = make_prompt_map(h, h->kp, prompt_len, &h->tm_kp);
         if (rc == SEGKV_OK) rc = make_prompt_map(h, h->vp, prompt_len, &h->tm_vp);
@@ -439,11 +449,15 @@ int segkv_prefill_sdpa(segkv_t h, const void* q, void* out, const float* alibi_s
     if (!h || !q || !out || !aligned16(q) || !aligned16(out)) return SEGKV_EINVAL;
     if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SEGKV_EINVAL;
     if (h->prompt_len <= 0 || !h->tm_valid) return SEGKV_ESTATE;
-    if (!prefill_sdpa_supported(h->d)) return SEGKV_EINVAL;
+    if (!prefill_tc5_supported(h->d)) return SEGKV_EINVAL;
     PrefillArgs a;
     a.q = q; a.out = out; a.slopes = alibi_slopes; a.err_word = h->err_word;
     a.prompt_len = h->prompt_len; a.tm_k = &h->tm_kp; a.tm_v = &h->tm_vp;
     a.row_groups = h->prefill_groups;
+    a.wait_ns = h->dbg_wait_ns;
+    a.dbg_skip = h->dbg_skip;
+    h->dbg_wait_ns = 0;
+    h->dbg_skip = false;
     a.plens = h->ragged ? h->plens : nullptr;
     a.tm_k_src = a.tm_v_src = nullptr;
     CUtensorMap tm_q;
@@ -453,7 +467,7 @@ int segkv_prefill_sdpa(segkv_t h, const void* q, void* out, const float* alibi_s
         if (rc != SEGKV_OK) return rc;
         a.tm_q = &tm_q;
     }
-    SEGKV_CUDA(launch_prefill_sdpa(h->d, a, (cudaStream_t)stream));
+    SEGKV_CUDA(launch_prefill_tc5(h->d, a, (cudaStream_t)stream));
     h->launches++;
     return SEGKV_OK;
 }
@@ -484,10 +498,12 @@ int segkv_prefill(segkv_t h, const void* k, const void* v, const void* q, void* 
     a.q = q; a.out = out; a.slopes = alibi_slopes; a.err_word = h->err_word;
     a.prompt_len = prompt_len; a.tm_k = &h->tm_kp; a.tm_v = &h->tm_vp;
     a.row_groups = h->prefill_groups;
+    a.wait_ns = 0;
+    a.dbg_skip = false;
     a.plens = nullptr;
     a.tm_k_src = &tm_ks; a.tm_v_src = &tm_vs; a.tm_q = &tm_q;
     h->prompt_len = -1;                                       // nothing valid is stored if the launch fails
-    SEGKV_CUDA(launch_prefill_sdpa(h->d, a, (cudaStream_t)stream));
+    SEGKV_CUDA(launch_prefill_tc5(h->d, a, (cudaStream_t)stream));
     h->launches++;
     h->tm_valid = true;
     h->prompt_len = prompt_len;
@@ -583,6 +599,8 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
     SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, splits);
     a.cluster = cluster;
     a.pdl = h->overlap;
+    h->dbg_wait_ns = 0;                  // an injected fault applies to one launch
+    h->dbg_skip = false;
     SEGKV_CUDA(launch_sdpa_tiled(h->d, a, h->tm_kp, h->tm_vp, stages, (cudaStream_t)stream));
     h->launches++;
     return SEGKV_OK;
@@ -593,6 +611,7 @@ int segkv_decode_sdpa_static(segkv_t h, const void* q, void* out, const float* a
     if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SEGKV_EINVAL;
     if (h->prompt_len < 0) return SEGKV_ESTATE;
     if (h->prompt_len + h->steps <= 0) return SEGKV_ESTATE;
+    if (h->leader && h->leader->steps != h->steps) return SEGKV_ESTATE;   // the shared tables describe another step
     if (!tiled_supported(h->d)) return SEGKV_EINVAL;
     {
         int rc = ensure_lists(h, (cudaStream_t)stream);     // a kernel launch at most, never an allocation
@@ -604,6 +623,8 @@ int segkv_decode_sdpa_static(segkv_t h, const void* q, void* out, const float* a
     SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, splits);
     a.pdl = h->overlap;
     int too_big = 0;
+    h->dbg_wait_ns = 0;
+    h->dbg_skip = false;
     SEGKV_CUDA(launch_sdpa_tiled_static(h->d, a, h->tm_kp, h->tm_vp, stages, (cudaStream_t)stream, &too_big));
     if (too_big) {
         snprintf(g_cuda_err, sizeof g_cuda_err,
@@ -675,6 +696,8 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     a.vr_new_slab = k_slab_of(h, step) + vdelta_of(h);
     a.anc_dst = h->anc[step & 1];
     a.parent_row = h->parent + (size_t)step * d.rows;
+    h->dbg_wait_ns = 0;
+    h->dbg_skip = false;
     SEGKV_CUDA(launch_sdpa_tiled(d, a, h->tm_kp, h->tm_vp, stages, (cudaStream_t)stream));
     h->launches++;
     h->steps = step + 1;
@@ -818,6 +841,12 @@ int segkv_set_tuning(segkv_t h, int splits, int stages, int combine) {
     if (!h || splits < 0 || splits > kMaxSplits || stages < 0 || stages > 16) return SEGKV_EINVAL;
     if (combine < 0 || combine > 2) return SEGKV_EINVAL;
     if (stages > 0 && tiled_smem_bytes(h->d, stages) > h->smem_optin) return SEGKV_EINVAL;
+    if (splits > h->ws_splits) {
+        // a forced split count beyond what the handle was sized for: grow the workspace here, not in the decode loop
+        SEGKV_CUDA(cudaDeviceSynchronize());
+        int rc = alloc_workspace(h, splits);
+        if (rc != SEGKV_OK) return rc;
+    }
     h->splits_forced = splits;
     h->stages_forced = stages;
     h->combine_forced = combine;
@@ -877,6 +906,13 @@ int segkv_set_prompt_layout(segkv_t h, int layout) {
 int segkv_set_prefill_tuning(segkv_t h, int row_groups) {
     if (!h || row_groups < 0 || row_groups > 2) return SEGKV_EINVAL;
     h->prefill_groups = row_groups;
+    return SEGKV_OK;
+}
+
+int segkv_debug_inject(segkv_t h, long long wait_limit_ns, int skip_arrival) {
+    if (!h || wait_limit_ns < 0) return SEGKV_EINVAL;
+    h->dbg_wait_ns = (unsigned long long)wait_limit_ns;
+    h->dbg_skip = skip_arrival != 0;
     return SEGKV_OK;
 }
 

@@ -39,14 +39,14 @@ __global__ void prefill_transpose_kernel(const uint4* __restrict__ k, const uint
 }
 
 cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v, void* kp, void* vp, const int32_t* plens,
-                                     int prompt_len, cudaStream_t st) {
+                                     int prompt_len, int sm_count, cudaStream_t st) {
     const int chunks = d.head_dim * 2 / 16;
     const PromptStrides ps = prompt_strides(d);
     long long total = (long long)d.batch * prompt_len * d.kv_heads * chunks;
     if (total == 0) return cudaSuccess;
     int threads = 256;
     long long blocks = (total + threads - 1) / threads;
-    if (blocks > 148 * 32) blocks = 148 * 32;
+    if (blocks > (long long)sm_count * 32) blocks = (long long)sm_count * 32;
     prefill_transpose_kernel<<<(unsigned)blocks, threads, 0, st>>>(
         (const uint4*)k, (const uint4*)v, (uint4*)kp, (uint4*)vp, d.batch, prompt_len, d.kv_heads, chunks,
         ps.b / 8, ps.h / 8, ps.p / 8, plens);

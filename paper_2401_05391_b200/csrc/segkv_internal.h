@@ -60,6 +60,8 @@ struct segkv {
     bool overlap;        // programmatic dependent launch between consecutive kernels
     int prefill_groups;  // 0 = automatic; 1 or 2 row groups per CTA of the tcgen05 prefill kernel
     bool fuse_always;    // segkv_decode_step uses the fused kernel even for a single split
+    unsigned long long dbg_wait_ns;   // segkv_debug_inject: applies to the next attention launch, then clears
+    bool dbg_skip;
     long long launches;
     // device storage (owned)
     void* kp;            // [batch, kv_heads, max_prompt, D] (or the layout chosen by segkv_set_prompt_layout)
@@ -109,7 +111,7 @@ struct RopeArgs {
 
 // plens (device, [batch]) or NULL: tokens at or past a request's own length are stored as zeros
 cudaError_t launch_prefill_transpose(const Dims& d, const void* k, const void* v, void* kp, void* vp, const int32_t* plens,
-                                     int prompt_len, cudaStream_t st);
+                                     int prompt_len, int sm_count, cudaStream_t st);
 
 cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, const void* k_new,
                           const void* v_new, void* kr_slab, void* vr_slab, int32_t* parent_tab,
@@ -142,6 +144,10 @@ struct SdpaArgs {
     bool pdl;                // launch with programmatic stream serialisation
     bool prompt_immutable;   // a fully serialised launch has followed the last prompt store
     // fused decode step (append + beam-index update + attention in one launch)
+    // test aid (segkv_debug_inject): limit of the kernel's bounded waits (0 = default) and one
+    // barrier arrival left out so that a wait runs out
+    unsigned long long wait_ns;
+    bool dbg_skip;
     bool fused;
     const int32_t* parent;   // [rows] device, NULL at step 0
     const void* k_new;
@@ -169,7 +175,7 @@ size_t tiled_static_scratch_bytes();
 cudaError_t launch_sdpa_tiled_static(const Dims& d, SdpaArgs a, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                      int stages, cudaStream_t st, int* too_big);
 
-// Causal prefill attention over the prompt segment (tile rows must be 64: head_dim 64 or 128).
+// Causal prefill attention over the prompt segment.
 struct PrefillArgs {
     const void* q;
     void* out;
@@ -185,10 +191,10 @@ struct PrefillArgs {
     const CUtensorMap* tm_v_src;
     const CUtensorMap* tm_q;   // over q as [batch][prompt_len][heads][D], box 64 elements x 128 tokens; NULL if unused
     int row_groups;      // 0 = automatic
+    unsigned long long wait_ns;   // test aid, as in SdpaArgs
+    bool dbg_skip;
 };
-bool prefill_sdpa_supported(const Dims& d);
-cudaError_t launch_prefill_sdpa(const Dims& d, const PrefillArgs& a, cudaStream_t st);
-// the same operation on tcgen05 tensor cores with TMEM accumulators (head_dim 128)
+// tcgen05 tensor cores with TMEM accumulators; head_dim 64, 128 or 256
 bool prefill_tc5_supported(const Dims& d);
 cudaError_t launch_prefill_tc5(const Dims& d, const PrefillArgs& a, cudaStream_t st);
 

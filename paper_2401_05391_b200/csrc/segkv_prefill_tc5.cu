@@ -52,6 +52,8 @@ struct Tc5Params {
     int store_kv;            // 1: every K/V tile is also written to the prompt segment, by the item that owns it
     float scale2;
     uint32_t idesc_qk, idesc_pv;
+    int dbg_skip;            // test aid: one softmax thread leaves out one barrier arrival, so that a wait runs out
+    unsigned long long wait_ns;   // limit of every bounded wait
 };
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -127,11 +129,11 @@ template <> struct SplitP<__nv_bfloat16> { typedef char yes; static constexpr bo
 
 // Critical-path wait: poll without sleeping first (the hardware suspends the thread inside
 // try_wait for a while), then fall back to the bounded, sleeping wait.
-__device__ __forceinline__ bool mbar_wait_hot(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_hot(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
 #pragma unroll 1
     for (int i = 0; i < 4096; ++i)
         if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait(bar, parity);
+    return mbar_wait(bar, parity, limit_ns);
 }
 
 #ifdef SEGKV_TC5_TIMELINE
@@ -323,7 +325,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     nkt = max(nkt, gt);
                     if (gt == 0) continue;
                     // the group's Q rows (past the prompt: zeros), once its previous Q is no longer read
-                    ok = mbar_wait(gbar0 + 48 * g + 40, (qi[g] & 1) ^ 1);
+                    ok = mbar_wait(gbar0 + 48 * g + 40, (qi[g] & 1) ^ 1, p.wait_ns);
                     if (!ok) break;
                     ++qi[g];
                     const uint32_t qfull = gbar0 + 48 * g + 32;
@@ -335,10 +337,10 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
                 for (int kt = 0; kt < nkt && ok; ++kt, ++tp) {
                     const uint32_t sk = tp % SK, sv = tp % SV;
-                    ok = mbar_wait(kempty0 + 8 * sk, ((tp / SK) & 1) ^ 1);
+                    ok = mbar_wait(kempty0 + 8 * sk, ((tp / SK) & 1) ^ 1, p.wait_ns);
                     if (!ok) break;
                     load_tile(&tm_k, k_ring + (size_t)sk * kTileKV, kt, kvh, b, kfull0 + 8 * sk);
-                    ok = mbar_wait(vempty0 + 8 * sv, ((tp / SV) & 1) ^ 1);
+                    ok = mbar_wait(vempty0 + 8 * sv, ((tp / SV) & 1) ^ 1, p.wait_ns);
                     if (!ok) break;
                     load_tile(&tm_v, v_ring + (size_t)sv * kTileKV, kt, kvh, b, vfull0 + 8 * sv);
                 }
@@ -377,11 +379,11 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 for (int kt = 0; kt < nkt && ok; ++kt, ++tp) {
                     const bool mine = (h % p.G) == 0 && (kt * kKeys) / (kRows * NG) == qt;
                     const uint32_t sk = tp % SK, sv = tp % SV;
-                    ok = mbar_wait(kfull0 + 8 * sk, (tp / SK) & 1);
+                    ok = mbar_wait(kfull0 + 8 * sk, (tp / SK) & 1, p.wait_ns);
                     if (!ok) break;
                     if (mine) store_tile(&tm_k_seg, k_ring + (size_t)sk * kTileKV, kt, kvh, b);
                     mbar_arrive(kempty0 + 8 * sk);
-                    ok = mbar_wait(vfull0 + 8 * sv, (tp / SV) & 1);
+                    ok = mbar_wait(vfull0 + 8 * sv, (tp / SV) & 1, p.wait_ns);
                     if (!ok) break;
                     if (mine) store_tile(&tm_v_seg, v_ring + (size_t)sv * kTileKV, kt, kvh, b);
                     mbar_arrive(vempty0 + 8 * sv);
@@ -430,13 +432,13 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     if (kt + 1 == gt[g]) tc_commit(gbar0 + 48 * g + 40);
                 };
                 auto wait_k = [&](int kt) -> bool {
-                    const bool r = mbar_wait_hot(kfull0 + 8 * ((tp + kt) % SK), ((tp + kt) / SK) & 1);
+                    const bool r = mbar_wait_hot(kfull0 + 8 * ((tp + kt) % SK), ((tp + kt) / SK) & 1, p.wait_ns);
                     tc_fence_after();
                     return r;
                 };
 #pragma unroll
                 for (int g = 0; g < NG; ++g)
-                    if (gt[g] > 0 && ok) ok = mbar_wait_hot(gbar0 + 48 * g + 32, qi[g]++ & 1);   // Q_g landed
+                    if (gt[g] > 0 && ok) ok = mbar_wait_hot(gbar0 + 48 * g + 32, qi[g]++ & 1, p.wait_ns);   // Q_g landed
                 if (ok) ok = wait_k(0);
                 if (!ok) break;
 #pragma unroll
@@ -455,13 +457,13 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     }
                     const uint32_t sv = (tp + kt) % SV;
                     const uint64_t vd = v_desc0 + (uint64_t)((sv * (uint32_t)kTileKV) >> 4);
-                    ok = mbar_wait_hot(vfull0 + 8 * sv, ((tp + kt) / SV) & 1);
+                    ok = mbar_wait_hot(vfull0 + 8 * sv, ((tp + kt) / SV) & 1, p.wait_ns);
                     if (!ok) break;
                     bool k_next = false;
 #pragma unroll
                     for (int g = 0; g < NG; ++g) {
                         if (kt >= gt[g]) continue;
-                        ok = mbar_wait_hot(gbar0 + 48 * g + 16, n[g] & 1);   // P_g written over its S buffer
+                        ok = mbar_wait_hot(gbar0 + 48 * g + 16, n[g] & 1, p.wait_ns);   // P_g written over its S buffer
                         if (!ok) break;
                         TC5_STAMP(2, kt, 1 + 3 * g);
                         tc_fence_after();
@@ -479,7 +481,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         }
                         tc_commit(gbar0 + 48 * g + 24);
 #if defined(SEGKV_TC5_TIMELINE) && SEGKV_TC5_TIMELINE == 3
-                        mbar_wait_hot(gbar0 + 48 * g + 24, n[g] & 1);   // measurement only: serialise on P.V
+                        mbar_wait_hot(gbar0 + 48 * g + 24, n[g] & 1, p.wait_ns);   // measurement only: serialise on P.V
                         TC5_STAMP(2, kt, 2 + 3 * g);
 #endif
                         ++n[g];
@@ -491,7 +493,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             }
                             issue_qk(g, kt + 1, 0);
 #if defined(SEGKV_TC5_TIMELINE) && SEGKV_TC5_TIMELINE == 3
-                            mbar_wait_hot(gbar0 + 48 * g, n[g] & 1);    // measurement only: serialise on Q.K^T
+                            mbar_wait_hot(gbar0 + 48 * g, n[g] & 1, p.wait_ns);    // measurement only: serialise on Q.K^T
                             TC5_STAMP(2, kt, 3 + 3 * g);
 #endif
                         }
@@ -527,7 +529,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             for (int kt = 0; kt < my_tiles; ++kt, ++n) {
                 const int buf = NB == 2 ? (int)(n & 1) : 0;
                 const uint32_t tm_s = tm_lane + (uint32_t)(kKeys * (g * NB + buf));
-                ok = mbar_wait_hot(bar_s0 + 8 * buf, (NB == 2 ? (n >> 1) : n) & 1);
+                ok = mbar_wait_hot(bar_s0 + 8 * buf, (NB == 2 ? (n >> 1) : n) & 1, p.wait_ns);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (stamp) TC5_STAMP(g, kt, 0);
@@ -602,7 +604,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     // produced behind that P.V in the pipe, and waiting here is only needed to rescale).
                     const bool rescale = kt > 0 && __any_sync(0xffffffffu, need);
                     if (kt > 0 && (NB == 2 || rescale)) {
-                        bool arrived = mbar_wait_hot(bar_o, (n - 1) & 1);
+                        bool arrived = mbar_wait_hot(bar_o, (n - 1) & 1, p.wait_ns);
                         arrived = __all_sync(0xffffffffu, arrived);
                         if (!arrived) return false;
                         tc_fence_after();
@@ -627,7 +629,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     }
                     tc_wait_st();
                     tc_fence_before();
-                    mbar_arrive(bar_p);
+                    if (!(p.dbg_skip && tid == 0 && n == 0)) mbar_arrive(bar_p);
                     if (stamp) TC5_STAMP(g, kt, 4);
                     return true;
                 };
@@ -637,7 +639,7 @@ prefill_tc5_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             if (!ok) break;
             // the item's output: O / l, once the last P.V has landed.  The next item's first P.V
             // cannot overwrite O before these loads: it waits for this thread's next P arrival.
-            ok = mbar_wait_hot(bar_o, (n - 1) & 1);
+            ok = mbar_wait_hot(bar_o, (n - 1) & 1, p.wait_ns);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -736,6 +738,8 @@ cudaError_t launch_prefill_tc5(const Dims& d, const PrefillArgs& a, cudaStream_t
     p.plens = a.plens;
     p.N = a.prompt_len; p.H = d.heads; p.Hkv = d.kv_heads; p.G = d.group; p.B = d.batch;
     p.scale2 = 0.f; p.idesc_qk = p.idesc_pv = 0; p.snake = 0;
+    p.dbg_skip = a.dbg_skip ? 1 : 0;
+    p.wait_ns = a.wait_ns ? a.wait_ns : kWaitLimitNs;
     int sms = 148;
     {
         int dev = 0;

@@ -37,10 +37,11 @@ __device__ __forceinline__ uint64_t global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait (about two seconds): false when it gave up.  Between polls the warp sleeps a
-// few tens of nanoseconds so that waiting warps do not crowd the load/store pipe that the
-// producer warps need for their copies.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait: false when it gave up after limit_ns (kWaitLimitNs, about two seconds, unless a
+// test shortens it).  Between polls the warp sleeps a few tens of nanoseconds so that waiting
+// warps do not crowd the load/store pipe that the producer warps need for their copies.
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_ns();
     for (;;) {
@@ -49,7 +50,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
             __nanosleep(32);
             if (mbar_try_wait(bar, parity)) return true;
         }
-        if (global_ns() - t0 > 2000000000ull) return false;
+        if (global_ns() - t0 > limit_ns) return false;
     }
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

@@ -7,8 +7,8 @@
 //
 //  * grid = (request, kv head, split).  A CTA owns ALL beams (and all query
 //    heads of the kv head's group) of its work group, so a K/V byte staged in
-//    shared memory is used by every beam: prompt bytes cross HBM once, not BW
-//    times (Section 4.2.1: "accesses only 1/BW amount data in HBM").
+//    shared memory is used by every beam: prompt bytes cross HBM once per
+//    request, not once per beam (the saving Section 4.2.1 describes).
 //  * two producer warps feed a ring of shared-memory stages.  The TMA warp
 //    fetches prompt tiles (cp.async.bulk.tensor, 128-byte swizzle) from the
 //    head-major prompt segment; it sets the mbarriers up itself and issues the
@@ -107,6 +107,10 @@ namespace {
 #define SEGKV_STAMP(ev) do {} while (0)
 #endif
 
+// A CTA whose bounded wait ran out adds this to its work group's arrival counter on top of its
+// ticket (splits are at most kMaxSplits, far below it).
+constexpr int kTicketAborted = 1 << 16;
+
 struct TiledParams {
     const void* q;
     void* out;
@@ -137,6 +141,8 @@ struct TiledParams {
     int quota;      // distinct response rows per split (the last split also takes any excess)
     int cluster;    // 1: the S CTAs of a work group form a thread-block cluster
     int early_prompt;  // 1: prompt tiles may be fetched before the previous kernel has completed
+    int dbg_skip;      // test aid: the gather warp leaves out one plain barrier arrival, so that a wait runs out
+    unsigned long long wait_ns;   // limit of every bounded wait
 #ifdef SEGKV_TIMELINE
     int dbg_launch;
 #endif
@@ -285,7 +291,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         // ============================ prompt tiles beyond the first round ============================
         bool ok = true;
         for (int k = tma_issued; k < npt; ++k) {
-            ok = mbar_wait(empty0 + 8 * (k % stages), (((uint32_t)(k / stages)) & 1) ^ 1);
+            ok = mbar_wait(empty0 + 8 * (k % stages), (((uint32_t)(k / stages)) & 1) ^ 1, p.wait_ns);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             issue_prompt_tile(k);
@@ -359,7 +365,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             }
             if (lane == 0) tile_hdr[st] = make_int2(cnt, last ? 1 : 0);
             __syncwarp();
-            if (lane == 0) mbar_arrive(full0 + 8 * st);
+            if (lane == 0 && !p.dbg_skip) mbar_arrive(full0 + 8 * st);
         };
         auto publish_tile = [&](int st, int cnt, bool last) {
             copy_rows(st, cnt);
@@ -385,7 +391,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             const int nrt = (e1 - e0 + TILE - 1) / TILE;
             SEGKV_STAMP(4);
             if (nrt > 0) {
-                ok = mbar_wait(hand, 0);
+                ok = mbar_wait(hand, 0, p.wait_ns);
                 ok = __all_sync(0xffffffffu, ok);
             }
             for (int r = 0; r < nrt && ok; ++r) {
@@ -401,7 +407,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                                     : make_uint2(0u, 0u);
                 }
                 const int st = k % stages;
-                ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1);
+                ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1, p.wait_ns);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 URow* meta_st = meta + (size_t)st * TILE;
@@ -456,7 +462,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             }
             SEGKV_STAMP(4);
             if (rs1 > rs0) {
-                ok = mbar_wait(hand, 0);
+                ok = mbar_wait(hand, 0, p.wait_ns);
                 ok = __all_sync(0xffffffffu, ok);
             }
             // Windows of spw steps at fixed positions; the table entries of four windows are
@@ -500,7 +506,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     }
                     if (!open) {
                         st = k % stages;
-                        ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1);
+                        ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1, p.wait_ns);
                         ok = __all_sync(0xffffffffu, ok);
                         if (!ok) break;
                         open = true;
@@ -686,7 +692,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         int k = 0;
         for (; k < npt; ++k) {
             const int st = k % stages;
-            ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1);
+            ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1, p.wait_ns);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const int pos0 = (pt0 + k) * TILE;
@@ -701,7 +707,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             const int nrt = (e1 - e0 + TILE - 1) / TILE;
             for (int r = 0; r < nrt; ++r, ++k) {
                 const int st = k % stages;
-                ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1);
+                ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1, p.wait_ns);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 consume(st, true, min(TILE, e1 - (e0 + r * TILE)), 0);
@@ -713,7 +719,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             // warp knows; it says so in the tile's header
             for (;;) {
                 const int st = k % stages;
-                ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1);
+                ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1, p.wait_ns);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 const int2 hd = tile_hdr[st];
@@ -740,7 +746,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         // before the shared memory is released; the output is left untouched.
         if (warp == TMA_WARP)
             for (int k = max(0, tma_issued - stages); k < tma_issued; ++k)
-                (void)mbar_wait(full0 + 8 * (k % stages), (uint32_t)(k / stages) & 1);
+                (void)mbar_wait(full0 + 8 * (k % stages), (uint32_t)(k / stages) & 1, p.wait_ns);
         if (warp == GATHER_WARP) cp_async_wait_all();
     }
 
@@ -846,7 +852,16 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         if (tid == 0) SEGKV_STAMP(13);
         return;
     }
-    if (aborted) return;
+    if (aborted) {
+        // The work group's arrival counter must still come back to zero for the next launch: take the
+        // ticket, marked, so that the last CTA to arrive skips the merge (the output stays untouched).
+        if (S > 1 && tid == 0) {
+            int ticket;
+            asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(ticket) : "l"(p.tickets + slab), "r"(kTicketAborted + 1) : "memory");
+            if ((ticket & (kTicketAborted - 1)) == S - 1) p.tickets[slab] = 0;
+        }
+        return;
+    }
 
     float* wso_cta = p.ws_o + ((size_t)slab * S + split) * ncols * D;
     float* wsml_cta = p.ws_ml + ((size_t)slab * S + split) * ncols * 2;
@@ -874,11 +889,12 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         // ticket; acquire: the last arriver sees every other CTA's partials
         int ticket;
         asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(ticket) : "l"(p.tickets + slab) : "memory");
-        s_last = (ticket == S - 1);
+        s_last = (ticket & (kTicketAborted - 1)) == S - 1 ? 1 + (ticket >= kTicketAborted ? 1 : 0) : 0;
+        if (s_last == 2) p.tickets[slab] = 0;     // a CTA of the group gave up: no merge, counter ready for the next launch
     }
     __syncthreads();
     if (tid == 0) SEGKV_STAMP(12);
-    if (!s_last) return;
+    if (s_last != 1) return;
 
     // One pass: each thread owns a float4 of one column and folds the splits in, eight at a
     // time (their partial outputs and max/sum pairs are all requested before any is used).
@@ -951,6 +967,8 @@ cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk,
     if (p.quota < 1) p.quota = 1;
     p.cluster = a.cluster ? 1 : 0;
     p.early_prompt = (a.pdl && a.prompt_immutable) ? 1 : 0;
+    p.dbg_skip = a.dbg_skip ? 1 : 0;
+    p.wait_ns = a.wait_ns ? a.wait_ns : kWaitLimitNs;
 #ifdef SEGKV_TIMELINE
     static int launch_id = 0;
     p.dbg_launch = launch_id++;

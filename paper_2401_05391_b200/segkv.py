@@ -56,6 +56,7 @@ SIGNATURES = {
     "segkv_share_index": (_int, [_vp, _vp]),
     "segkv_append_rope": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _int, _int, _vp]),
     "segkv_prefill_write_ragged": (_int, [_vp, _vp, _vp, _int, _vp, _vp]),
+    "segkv_debug_inject": (_int, [_vp, ctypes.c_longlong, _int]),
     "segkv_launch_count": (ctypes.c_longlong, [_vp]),
     "segkv_storage_bytes": (ctypes.c_size_t, [_int] * 7),
     "segkv_strerror": (ctypes.c_char_p, [_int]),
@@ -320,6 +321,9 @@ class SegKV:
         flags = _int(0)
         _check(lib().segkv_get_error(self._h, ctypes.byref(flags)), "segkv_get_error")
         return flags.value
+
+    def debug_inject(self, wait_limit_ns: int = 0, skip_arrival: bool = False) -> None:
+        _check(lib().segkv_debug_inject(self._h, int(wait_limit_ns), int(bool(skip_arrival))), "segkv_debug_inject")
 
     def set_tuning(self, splits: int = 0, stages: int = 0, combine: int = 0) -> None:
         _check(lib().segkv_set_tuning(self._h, splits, stages, combine), "segkv_set_tuning")

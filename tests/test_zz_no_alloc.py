@@ -17,7 +17,7 @@ import torch
 from paper_2401_05391_b200 import segkv as sk
 from paper_2401_05391_b200 import workloads as wl
 
-from _harness import ATOL, RTOL, Run
+from _harness import ATOL, RTOL, Run, all_pairs
 
 pytestmark = pytest.mark.gpu
 
@@ -44,6 +44,7 @@ def test_static_scratch_entry_point_matches_regular_one_twice_in_a_row():
             torch.cuda.synchronize()
             assert not torch.isnan(out.float()).any(), f"call {call}: unwritten outputs"
             assert _close(out, ref), f"call {call}: differs from segkv_decode_sdpa beyond the tolerance"
+            r.check(out, q, w.steps - 1, all_pairs(w))             # and against the CPU oracle itself
         # a different split count right after: other ticket/partial footprint in the same array
         r.h.set_tuning(3, 0, 0)
         out = torch.full_like(ref, float("nan"))
@@ -73,3 +74,26 @@ def test_static_scratch_entry_point_rejects_what_does_not_fit():
         torch.cuda.synchronize()
     finally:
         h.destroy()
+
+
+def test_static_scratch_entry_point_checks_the_shared_index_tables_step():
+    # a handle that reads another handle's beam-index tables must be at the leader's step, as for
+    # segkv_decode_sdpa: after the leader has moved on, its tables describe another step
+    w = wl.Workload("follow", 1, 4, 4, 4, 128, 64, 4, "f16", "uniform", False, 52)
+    lead = Run(w)
+    foll = Run(w.scaled(index=53), parents=lead.parents)
+    try:
+        foll.h.share_index(lead.h)
+        for _ in range(2):
+            lead.append_next(); foll.append_next()
+        q = foll.q_steps[-1]
+        out = torch.full((w.rows, w.heads, w.head_dim), float("nan"), dtype=w.torch_dtype, device="cuda")
+        foll.h.decode_sdpa_static(q, out)                       # same step: fine
+        torch.cuda.synchronize()
+        foll.check(out, q, 1, all_pairs(w))
+        lead.append_next()                                      # the leader moves on alone
+        with pytest.raises(sk.SegKVError) as e:
+            foll.h.decode_sdpa_static(q, out)
+        assert e.value.code == sk.SEGKV_ESTATE
+    finally:
+        foll.close(); lead.close()
