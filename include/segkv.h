@@ -310,6 +310,19 @@ SEGKV_API int segkv_prompt_len(segkv_t h);
  * segkv_get_splits returns the split count the next segkv_decode_sdpa will use.
  */
 SEGKV_API int segkv_set_tuning(segkv_t h, int splits, int stages, int combine);
+
+/*
+ * Pick the form of the decode attention kernel (a launch-shape knob: the paper
+ * has no counterpart).  tile_keys = 64: tiles of 64 keys, four consumer warps,
+ * two CTAs per SM (32 keys, two warps at head_dim 256): the form for launches
+ * of several waves.  tile_keys = 32: tiles of 32 keys, two consumer warps, CTAs
+ * of a quarter of an SM, so that the CTAs of two consecutive launches fit side
+ * by side and the later one fetches its keys while the earlier one still
+ * computes; only for head_dim <= 128 and beams*(heads/kv_heads) <= 8.
+ * 0 = automatic (the default).  Errors: EINVAL (other values, or 32 for a shape
+ * that has no such form).
+ */
+SEGKV_API int segkv_set_tile(segkv_t h, int tile_keys);
 SEGKV_API int segkv_get_splits(segkv_t h);
 
 /*

@@ -84,10 +84,20 @@ int encode_map_4d(const segkv* h, const void* base, int heads, int tokens, long 
 
 // One prompt array of the handle, [batch][prompt_len][kv_heads][D] logically, with the strides
 // of the handle's prompt layout; a box is one tile of tokens.
-int make_prompt_map(const segkv* h, void* base, int prompt_len, CUtensorMap* out) {
+int make_prompt_map(const segkv* h, void* base, int prompt_len, int box_tokens, CUtensorMap* out) {
     const PromptStrides ps = prompt_strides(h->d);
-    return encode_map_4d(h, base, h->d.kv_heads, prompt_len, ps.h, ps.p, ps.b, tiled_tile_keys(h->d.head_dim),
-                         "prompt segment", out);
+    return encode_map_4d(h, base, h->d.kv_heads, prompt_len, ps.h, ps.p, ps.b, box_tokens, "prompt segment", out);
+}
+
+// The handle's maps of its prompt segment: boxes of one regular tile (which the prefill kernel
+// shares) and boxes of 32 tokens for the small-CTA form of the decode kernel.
+int make_prompt_maps(segkv* h, int prompt_len) {
+    const int box = tiled_tile_keys(h->d.head_dim, false);
+    int rc = make_prompt_map(h, h->kp, prompt_len, box, &h->tm_kp);
+    if (rc == SEGKV_OK) rc = make_prompt_map(h, h->vp, prompt_len, box, &h->tm_vp);
+    if (rc == SEGKV_OK) rc = make_prompt_map(h, h->kp, prompt_len, 32, &h->tm_kp32);
+    if (rc == SEGKV_OK) rc = make_prompt_map(h, h->vp, prompt_len, 32, &h->tm_vp32);
+    return rc;
 }
 
 // The prefill query [batch][prompt_len][heads][D] (token-major): a box is 128 consecutive tokens.
@@ -101,7 +111,7 @@ int make_query_map(const segkv* h, const void* q, int prompt_len, CUtensorMap* o
 int make_kv_source_map(const segkv* h, const void* base, int prompt_len, CUtensorMap* out) {
     const long long D = h->d.head_dim, Hkv = h->d.kv_heads;
     return encode_map_4d(h, base, h->d.kv_heads, prompt_len, D, D * Hkv, D * Hkv * prompt_len,
-                         tiled_tile_keys(h->d.head_dim), "prefill K/V", out);
+                         tiled_tile_keys(h->d.head_dim, false), "prefill K/V", out);
 }
 
 void free_all(segkv* h) {
@@ -166,17 +176,37 @@ int alloc_workspace(segkv* h, int splits) {
     return SEGKV_OK;
 }
 
-// Launch shape of the tiled kernel.  Stages: as many as keep two CTAs resident per SM.
-// Splits: none when the work groups alone fill the GPU twice over, else enough to give
-// every CTA slot of one wave a share (never less than one tile each).
-void choose_tiling(const segkv* h, int* splits, int* stages, bool* cluster) {
+// Launch shape of the tiled kernel.
+struct Tiling {
+    int splits, stages;
+    bool cluster;     // the splits of a work group merge inside a thread-block cluster
+    bool small;       // 32-key tiles, quarter-SM CTAs
+};
+
+// CTAs of the chosen form that one SM holds at once.
+int ctas_per_sm(bool small) { return small ? 4 : 2; }
+
+// Most splits the automatic choice makes for this handle (what the split workspace is sized for).
+int max_auto_splits(const segkv* h) {
+    const long long slabs = (long long)h->d.batch * h->d.kv_heads;
+    long long most = (long long)h->sm_count * 4 / slabs;
+    if (most < 1) most = 1;
+    return (int)(most > kMaxSplits ? kMaxSplits : most);
+}
+
+// Stages: as many as keep the form's CTAs per SM resident.  Splits: none when the work groups
+// alone fill the GPU twice over, else enough to give every CTA slot of one wave a share (never
+// less than one tile each).
+Tiling choose_tiling(const segkv* h) {
     const Dims& d = h->d;
-    const int tile = tiled_tile_keys(d.head_dim);
+    Tiling t;
+    t.small = h->tile_forced == 32 && tiled_small_ok(d);
+    const int tile = tiled_tile_keys(d.head_dim, t.small);
     const int P = h->prompt_len > 0 ? h->prompt_len : 0;
     const long long ntp = (P + tile - 1) / tile;
     const long long ntr = (h->steps + 2 * d.beams + tile - 1) / tile;      // estimate, rows are mostly shared
     const long long slabs = (long long)d.batch * d.kv_heads;
-    const long long slots = (long long)h->sm_count * 2;
+    const long long slots = (long long)h->sm_count * ctas_per_sm(t.small);
     int sp = h->splits_forced;
     if (sp <= 0) {
         sp = 1;
@@ -194,24 +224,25 @@ void choose_tiling(const segkv* h, int* splits, int* stages, bool* cluster) {
     if (sp > kMaxSplits) sp = kMaxSplits;
     int st = h->stages_forced;
     if (st <= 0) {
-        // as deep a ring as still lets two CTAs share an SM ...
+        // as deep a ring as still lets the form's CTAs share an SM ...
         st = 2;
-        const size_t budget = (h->smem_optin + 1024) / 2 - 1024 - 2048;
-        while (st < 8 && tiled_smem_bytes(d, st + 1) <= budget) ++st;
+        const size_t budget = (h->smem_optin + 1024) / ctas_per_sm(t.small) - 1024 - (t.small ? 0 : 2048);
+        while (st < 8 && tiled_smem_bytes(d, st + 1, t.small) <= budget) ++st;
         // ... or, when the whole launch is one wave, deep enough to hold a CTA's whole share
         const long long per_cta = (ntp + sp - 1) / sp + (ntr + sp - 1) / sp;
-        if (slabs * sp <= h->sm_count && per_cta > st) {
-            while (st < per_cta && st < 8 && tiled_smem_bytes(d, st + 1) <= h->smem_optin) ++st;
+        if (!t.small && slabs * sp <= h->sm_count && per_cta > st) {
+            while (st < per_cta && st < 8 && tiled_smem_bytes(d, st + 1, t.small) <= h->smem_optin) ++st;
         }
     }
-    while (st > 1 && tiled_smem_bytes(d, st) > h->smem_optin) --st;
-    *splits = sp;
-    *stages = st;
+    while (st > 1 && tiled_smem_bytes(d, st, t.small) > h->smem_optin) --st;
+    t.splits = sp;
+    t.stages = st;
     // The workspace merge is the default: launches that merge inside a cluster were measured
     // not to start early under programmatic dependent launch, which costs more than the
     // cluster merge saves.  With overlap off the cluster merge is the faster one.
     const bool want_cluster = h->combine_forced == 2 || (h->combine_forced == 0 && !h->overlap);
-    *cluster = sp > 1 && want_cluster && tiled_cluster_ok(d, sp);
+    t.cluster = sp > 1 && want_cluster && tiled_cluster_ok(d, sp);
+    return t;
 }
 
 // The attention kernel's separate form walks per-request lists of distinct rows that the append
@@ -252,6 +283,7 @@ SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes
     a.steps = h->steps;
     a.splits = splits;
     a.cluster = false;
+    a.small = false;
     a.pdl = false;
     a.prompt_immutable = h->steps > 0;     // the first append after a prefill is a fully serialised launch
     a.fused = false;
@@ -377,13 +409,7 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
 #undef SEGKV_TRY
     // The split workspace for the largest split count the automatic choice can make (one wave of
     // CTA slots shared among the work groups), so that the decode loop never allocates.
-    {
-        const long long slabs = (long long)batch * kv_heads, slots = (long long)h->sm_count * 2;
-        long long most = slots / slabs;
-        if (most < 1) most = 1;
-        if (most > kMaxSplits) most = kMaxSplits;
-        rc = alloc_workspace(h, (int)most);
-    }
+    rc = alloc_workspace(h, max_auto_splits(h));
     if (rc != SEGKV_OK) return fail(rc);
     *out = h;
     return SEGKV_OK;
@@ -434,8 +460,7 @@ static int prefill_write_impl(segkv_t h, const void* k, const void* v, int promp
     if (prompt_len > 0) {
         SEGKV_CUDA(launch_prefill_transpose(h->d, k, v, h->kp, h->vp, plens_dev, prompt_len, h->sm_count, st));
         h->launches++;
-        int rc = make_prompt_map(h, h->kp, prompt_len, &h->tm_kp);
-        if (rc == SEGKV_OK) rc = make_prompt_map(h, h->vp, prompt_len, &h->tm_vp);
+        int rc = make_prompt_maps(h, prompt_len);
         if (rc != SEGKV_OK) return rc;
         h->tm_valid = true;
     }
@@ -487,8 +512,7 @@ int segkv_prefill(segkv_t h, const void* k, const void* v, const void* q, void* 
     if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SEGKV_EINVAL;
     if (prompt_len > h->d.max_prompt) return SEGKV_ECAPACITY;
     h->tm_valid = false;
-    int rc = make_prompt_map(h, h->kp, prompt_len, &h->tm_kp);
-    if (rc == SEGKV_OK) rc = make_prompt_map(h, h->vp, prompt_len, &h->tm_vp);
+    int rc = make_prompt_maps(h, prompt_len);
     CUtensorMap tm_q, tm_ks, tm_vs;
     if (rc == SEGKV_OK) rc = make_kv_source_map(h, k, prompt_len, &tm_ks);
     if (rc == SEGKV_OK) rc = make_kv_source_map(h, v, prompt_len, &tm_vs);
@@ -586,22 +610,23 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
         int rc = ensure_lists(h, (cudaStream_t)stream);
         if (rc != SEGKV_OK) return rc;
     }
-    int splits, stages;
-    bool cluster;
-    choose_tiling(h, &splits, &stages, &cluster);
-    if (h->combine_forced == 2 && splits > 1 && !cluster) return SEGKV_EINVAL;
-    if (!cluster && splits > h->ws_splits) {
+    const Tiling tl = choose_tiling(h);
+    const int splits = tl.splits;
+    if (h->combine_forced == 2 && splits > 1 && !tl.cluster) return SEGKV_EINVAL;
+    if (!tl.cluster && splits > h->ws_splits) {
         // growing the workspace must not race with work still using the old one
         SEGKV_CUDA(cudaDeviceSynchronize());
         int rc = alloc_workspace(h, splits);
         if (rc != SEGKV_OK) return rc;
     }
     SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, splits);
-    a.cluster = cluster;
+    a.cluster = tl.cluster;
+    a.small = tl.small;
     a.pdl = h->overlap;
     h->dbg_wait_ns = 0;                  // an injected fault applies to one launch
     h->dbg_skip = false;
-    SEGKV_CUDA(launch_sdpa_tiled(h->d, a, h->tm_kp, h->tm_vp, stages, (cudaStream_t)stream));
+    SEGKV_CUDA(launch_sdpa_tiled(h->d, a, tl.small ? h->tm_kp32 : h->tm_kp, tl.small ? h->tm_vp32 : h->tm_vp, tl.stages,
+                                 (cudaStream_t)stream));
     h->launches++;
     return SEGKV_OK;
 }
@@ -617,15 +642,16 @@ int segkv_decode_sdpa_static(segkv_t h, const void* q, void* out, const float* a
         int rc = ensure_lists(h, (cudaStream_t)stream);     // a kernel launch at most, never an allocation
         if (rc != SEGKV_OK) return rc;
     }
-    int splits, stages;
-    bool cluster;
-    choose_tiling(h, &splits, &stages, &cluster);
+    const Tiling tl = choose_tiling(h);
+    const int splits = tl.splits;
     SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, splits);
     a.pdl = h->overlap;
+    a.small = tl.small;
     int too_big = 0;
     h->dbg_wait_ns = 0;
     h->dbg_skip = false;
-    SEGKV_CUDA(launch_sdpa_tiled_static(h->d, a, h->tm_kp, h->tm_vp, stages, (cudaStream_t)stream, &too_big));
+    SEGKV_CUDA(launch_sdpa_tiled_static(h->d, a, tl.small ? h->tm_kp32 : h->tm_kp, tl.small ? h->tm_vp32 : h->tm_vp,
+                                        tl.stages, (cudaStream_t)stream, &too_big));
     if (too_big) {
         snprintf(g_cuda_err, sizeof g_cuda_err,
                  "segkv_decode_sdpa_static: %d splits of this shape need more than the %zu bytes of built-in scratch",
@@ -654,15 +680,15 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     }
     const Dims& d = h->d;
     h->steps = step + 1;                 // the launch shape is chosen for the step being added
-    int splits, stages;
-    bool cluster;
-    choose_tiling(h, &splits, &stages, &cluster);
+    const Tiling tl = choose_tiling(h);
+    const int splits = tl.splits;
+    const bool cluster = tl.cluster;
     h->steps = step;
     // rows a CTA's share of the steps can reach: beyond a tile and a half of them, deriving the rows
     // in the kernel costs more than the separate append launch (measured at prompts of 128 to 512
     // tokens with 128 steps: 10.0-10.6 us as two launches against 10.8-12.9 us fused)
     const long long rows_per_cta = (long long)((step + 1 + splits - 1) / splits) * d.beams;
-    const bool long_tail = h->splits_forced <= 0 && 2 * rows_per_cta > 3 * tiled_tile_keys(d.head_dim);   // a forced split count keeps the fused kernel
+    const bool long_tail = h->splits_forced <= 0 && 2 * rows_per_cta > 3 * tiled_tile_keys(d.head_dim, tl.small);   // a forced split count keeps the fused kernel
     if ((splits == 1 || long_tail) && !h->fuse_always) {
         // Work groups that fill the GPU on their own are bandwidth-bound: the separate append is
         // then ~1 % of the step and the list it makes keeps the response tiles dense and cheap
@@ -685,6 +711,7 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     a.steps = step + 1;
     a.anc = h->anc[(step + 1) & 1];      // table of step-1 (unused at step 0)
     a.cluster = cluster;
+    a.small = tl.small;
     // the first step after a prefill is fully serialised; from then on the prompt cannot change
     a.pdl = h->overlap && step > 0;
     a.prompt_immutable = step > 0;
@@ -698,7 +725,8 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     a.parent_row = h->parent + (size_t)step * d.rows;
     h->dbg_wait_ns = 0;
     h->dbg_skip = false;
-    SEGKV_CUDA(launch_sdpa_tiled(d, a, h->tm_kp, h->tm_vp, stages, (cudaStream_t)stream));
+    SEGKV_CUDA(launch_sdpa_tiled(d, a, tl.small ? h->tm_kp32 : h->tm_kp, tl.small ? h->tm_vp32 : h->tm_vp, tl.stages,
+                                 (cudaStream_t)stream));
     h->launches++;
     h->steps = step + 1;
     h->truncated = false;
@@ -840,7 +868,7 @@ int segkv_prompt_len(segkv_t h) { return h ? h->prompt_len : SEGKV_EINVAL; }
 int segkv_set_tuning(segkv_t h, int splits, int stages, int combine) {
     if (!h || splits < 0 || splits > kMaxSplits || stages < 0 || stages > 16) return SEGKV_EINVAL;
     if (combine < 0 || combine > 2) return SEGKV_EINVAL;
-    if (stages > 0 && tiled_smem_bytes(h->d, stages) > h->smem_optin) return SEGKV_EINVAL;
+    if (stages > 0 && tiled_smem_bytes(h->d, stages, h->tile_forced == 32) > h->smem_optin) return SEGKV_EINVAL;
     if (splits > h->ws_splits) {
         // a forced split count beyond what the handle was sized for: grow the workspace here, not in the decode loop
         SEGKV_CUDA(cudaDeviceSynchronize());
@@ -857,10 +885,7 @@ int segkv_set_tuning(segkv_t h, int splits, int stages, int combine) {
 int segkv_get_splits(segkv_t h) {
     if (!h) return SEGKV_EINVAL;
     if (!tiled_supported(h->d)) return 1;
-    int splits, stages;
-    bool cluster;
-    choose_tiling(h, &splits, &stages, &cluster);
-    return splits;
+    return choose_tiling(h).splits;
 }
 
 int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, const float* alibi_slopes, void* stream) {
@@ -906,6 +931,13 @@ int segkv_set_prompt_layout(segkv_t h, int layout) {
 int segkv_set_prefill_tuning(segkv_t h, int row_groups) {
     if (!h || row_groups < 0 || row_groups > 2) return SEGKV_EINVAL;
     h->prefill_groups = row_groups;
+    return SEGKV_OK;
+}
+
+int segkv_set_tile(segkv_t h, int tile_keys) {
+    if (!h || (tile_keys != 0 && tile_keys != 32 && tile_keys != 64)) return SEGKV_EINVAL;
+    if (tile_keys == 32 && !tiled_small_ok(h->d)) return SEGKV_EINVAL;
+    h->tile_forced = tile_keys;
     return SEGKV_OK;
 }
 

@@ -57,6 +57,7 @@ struct segkv {
     int splits_forced;   // 0 = automatic
     int stages_forced;   // 0 = automatic
     int combine_forced;  // 0 = automatic, 1 = global workspace + ticket, 2 = cluster
+    int tile_forced;     // 0 = automatic, 32 or 64 keys per tile of the decode kernel
     bool overlap;        // programmatic dependent launch between consecutive kernels
     int prefill_groups;  // 0 = automatic; 1 or 2 row groups per CTA of the tcgen05 prefill kernel
     bool fuse_always;    // segkv_decode_step uses the fused kernel even for a single split
@@ -93,6 +94,7 @@ struct segkv {
     float* st_slopes;
     // tensor maps of the prompt segment (valid once prompt_len > 0)
     CUtensorMap tm_kp, tm_vp;
+    CUtensorMap tm_kp32, tm_vp32;   // the same arrays in boxes of 32 tokens, for the small-CTA form of the decode kernel
     bool tm_valid;
 };
 
@@ -140,6 +142,7 @@ struct SdpaArgs {
     int* tickets;
     int* err_word;
     int prompt_len, steps, splits;
+    bool small;              // 32-key tiles and two consumer warps (tensor maps with 32-row boxes)
     bool cluster;            // merge the splits inside a thread-block cluster
     bool pdl;                // launch with programmatic stream serialisation
     bool prompt_immutable;   // a fully serialised launch has followed the last prompt store
@@ -165,8 +168,9 @@ cudaError_t launch_sdpa_rowwise(const Dims& d, const SdpaArgs& a, cudaStream_t s
 // Tiled split-KV kernel (TMA-staged prompt tiles, gathered response rows, tensor-core tiles).
 bool tiled_supported(const Dims& d);
 bool tiled_cluster_ok(const Dims& d, int splits);        // can `splits` CTAs merge as one cluster?
-int tiled_tile_keys(int head_dim);                       // rows of one shared-memory tile
-size_t tiled_smem_bytes(const Dims& d, int stages);      // dynamic shared memory of one CTA
+bool tiled_small_ok(const Dims& d);                      // is there a 32-key-tile form (quarter-SM CTAs) for this shape?
+int tiled_tile_keys(int head_dim, bool small);           // rows of one shared-memory tile
+size_t tiled_smem_bytes(const Dims& d, int stages, bool small);   // dynamic shared memory of one CTA
 cudaError_t launch_sdpa_tiled(const Dims& d, const SdpaArgs& a, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                               int stages, cudaStream_t st);
 

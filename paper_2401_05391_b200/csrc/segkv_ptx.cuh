@@ -108,6 +108,7 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
 
 template <typename T> struct Mma;
 template <> struct Mma<__half> {
+    static constexpr bool kWeights11Bits = true;
     static __device__ __forceinline__ void run(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
         asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
@@ -120,6 +121,7 @@ template <> struct Mma<__half> {
     static __device__ __forceinline__ __half down(float f) { return __float2half_rn(f); }
 };
 template <> struct Mma<__nv_bfloat16> {
+    static constexpr bool kWeights11Bits = false;
     static __device__ __forceinline__ void run(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
         asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])

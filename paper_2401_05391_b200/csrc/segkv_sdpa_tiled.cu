@@ -183,7 +183,7 @@ struct Layout {
 };
 
 template <typename T, int D, int NT, int CW, bool FUSED>
-__global__ void __launch_bounds__(32 * (CW + 2), NT > 1 ? 1 : 2)
+__global__ void __launch_bounds__(32 * (CW + 2), NT > 1 ? 1 : (CW == 2 && D <= 128 ? 4 : 2))
 sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                   const TiledParams p) {
     using L = Layout<D, CW>;
@@ -628,7 +628,12 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     kpos[r] = (float)(pos0 + key - qpos);
                 }
             }
-            uint32_t pfrag[NT][2];
+            // P^T fragments.  bf16 keeps 8 significant bits of a weight, which is not enough where a few
+            // keys carry a column's whole weight (a steep ALiBi slope) and their values cancel, so bf16
+            // weights go to the tensor cores in two parts, p = hi + lo (16 bits together): the kernel
+            // is bound by HBM and the second set of MMAs is free.  fp16 weights (11 bits) go as they are.
+            constexpr bool kTwoPart = sizeof(T) == 2 && !Mma<T>::kWeights11Bits;
+            uint32_t pfrag[NT][2], pfrag_lo[NT][2];
             bool rescale = false;
             float alpha[NT][2];
 #pragma unroll
@@ -660,8 +665,13 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     l_run[nt][c] = l_run[nt][c] * a + p0 + p1;
                 }
                 // P^T as the B operand of O^T += V^T . P^T
-                pfrag[nt][0] = movmatrix_trans(Mma<T>::pack(s[0][0], s[0][1]));
-                pfrag[nt][1] = movmatrix_trans(Mma<T>::pack(s[1][0], s[1][1]));
+                const uint32_t h0 = Mma<T>::pack(s[0][0], s[0][1]), h1 = Mma<T>::pack(s[1][0], s[1][1]);
+                pfrag[nt][0] = movmatrix_trans(h0);
+                pfrag[nt][1] = movmatrix_trans(h1);
+                if constexpr (kTwoPart) {
+                    pfrag_lo[nt][0] = movmatrix_trans(Mma<T>::pack(s[0][0] - __uint_as_float(h0 << 16), s[0][1] - __uint_as_float(h0 & 0xFFFF0000u)));
+                    pfrag_lo[nt][1] = movmatrix_trans(Mma<T>::pack(s[1][0] - __uint_as_float(h1 << 16), s[1][1] - __uint_as_float(h1 & 0xFFFF0000u)));
+                }
             }
             if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll
@@ -683,7 +693,10 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     uint32_t a[4];
                     ldmatrix_x4_trans(a, chunk_addr(v_src, key, ch, resp));
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) Mma<T>::run(o_acc[nt][mt], a, pfrag[nt][0], pfrag[nt][1]);
+                    for (int nt = 0; nt < NT; ++nt) {
+                        Mma<T>::run(o_acc[nt][mt], a, pfrag[nt][0], pfrag[nt][1]);
+                        if constexpr (kTwoPart) Mma<T>::run(o_acc[nt][mt], a, pfrag_lo[nt][0], pfrag_lo[nt][1]);
+                    }
                 }
             }
         };
@@ -696,7 +709,9 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const int pos0 = (pt0 + k) * TILE;
+            if (warp == 0 && k == 0) SEGKV_STAMP(7);
             consume(st, false, min(TILE, P - pos0), pos0);
+            if (warp == 0 && k == 0) SEGKV_STAMP(6);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + 8 * st);
         }
@@ -1007,6 +1022,13 @@ cudaError_t dispatch(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk, c
     const int nt = (d.beams * d.group + 7) / 8;
     if (a.splits < 1 || a.splits > kMaxSplits) return cudaErrorInvalidValue;
     if (a.cluster && !tiled_cluster_ok(d, a.splits)) return cudaErrorInvalidValue;
+    if (nt == 1 && a.small && d.head_dim <= 128) {
+        // 32-key tiles, two consumer warps: a CTA of a quarter of an SM, for launches of at most one wave
+        if (d.head_dim == 64) return a.fused ? launch_one<T, 64, 1, 2, true>(d, a, tmk, tmv, stages, st)
+                                             : launch_one<T, 64, 1, 2, false>(d, a, tmk, tmv, stages, st);
+        return a.fused ? launch_one<T, 128, 1, 2, true>(d, a, tmk, tmv, stages, st)
+                       : launch_one<T, 128, 1, 2, false>(d, a, tmk, tmv, stages, st);
+    }
     if (nt == 1) {
         switch (d.head_dim) {
             case 64: return a.fused ? launch_one<T, 64, 1, 4, true>(d, a, tmk, tmv, stages, st)
@@ -1040,10 +1062,13 @@ bool tiled_cluster_ok(const Dims& d, int splits) {
     return ((long long)d.beams * d.group * d.head_dim) % (4LL * splits) == 0;
 }
 
-int tiled_tile_keys(int head_dim) { return head_dim == 256 ? 32 : 64; }
+bool tiled_small_ok(const Dims& d) { return d.head_dim <= 128 && d.beams * d.group <= 8; }
 
-size_t tiled_smem_bytes(const Dims& d, int stages) {
+int tiled_tile_keys(int head_dim, bool small) { return (head_dim == 256 || small) ? 32 : 64; }
+
+size_t tiled_smem_bytes(const Dims& d, int stages, bool small) {
     const int nt = (d.beams * d.group + 7) / 8;
+    if (small && tiled_small_ok(d)) return d.head_dim == 64 ? Layout<64, 2>::bytes(stages, nt) : Layout<128, 2>::bytes(stages, nt);
     switch (d.head_dim) {
         case 64: return Layout<64, 4>::bytes(stages, nt);
         case 128: return Layout<128, 4>::bytes(stages, nt);

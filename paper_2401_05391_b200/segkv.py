@@ -48,6 +48,7 @@ SIGNATURES = {
     "segkv_steps": (_int, [_vp]),
     "segkv_prompt_len": (_int, [_vp]),
     "segkv_set_tuning": (_int, [_vp, _int, _int, _int]),
+    "segkv_set_tile": (_int, [_vp, _int]),
     "segkv_decode_sdpa_rowwise": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "segkv_get_splits": (_int, [_vp]),
     "segkv_set_overlap": (_int, [_vp, _int]),
@@ -321,6 +322,9 @@ class SegKV:
         flags = _int(0)
         _check(lib().segkv_get_error(self._h, ctypes.byref(flags)), "segkv_get_error")
         return flags.value
+
+    def set_tile(self, tile_keys: int = 0) -> None:
+        _check(lib().segkv_set_tile(self._h, tile_keys), "segkv_set_tile")
 
     def debug_inject(self, wait_limit_ns: int = 0, skip_arrival: bool = False) -> None:
         _check(lib().segkv_debug_inject(self._h, int(wait_limit_ns), int(bool(skip_arrival))), "segkv_debug_inject")

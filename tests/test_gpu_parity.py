@@ -14,8 +14,9 @@ CHECK_STEPS = (0, 1, 2, 3, 7, 15, 16, 17, 31, 63, 127, 255)
 
 
 def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combine=0, every_step_ancestry=True,
-                 prompt_layout=None, prompt_lens=None):
-    r = Run(w, splits=splits, stages=stages, combine=combine, prompt_layout=prompt_layout, prompt_lens=prompt_lens)
+                 prompt_layout=None, prompt_lens=None, tile=0):
+    r = Run(w, splits=splits, stages=stages, combine=combine, prompt_layout=prompt_layout, prompt_lens=prompt_lens,
+            tile=tile)
     try:
         worst = 0.0
         for t in range(w.steps):
@@ -35,9 +36,10 @@ def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combi
 
 
 def run_workload_fused(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combine=0, prompt_layout=None,
-                       prompt_lens=None):
+                       prompt_lens=None, tile=0):
     """Same as run_workload but every step is one fused segkv_decode_step launch."""
-    r = Run(w, splits=splits, stages=stages, combine=combine, prompt_layout=prompt_layout, prompt_lens=prompt_lens)
+    r = Run(w, splits=splits, stages=stages, combine=combine, prompt_layout=prompt_layout, prompt_lens=prompt_lens,
+            tile=tile)
     try:
         for t in range(w.steps):
             _, out, q = r.step_fused()
@@ -181,6 +183,26 @@ def test_forced_splits_stages_and_combine(splits, stages, combine):
     w = wl.CONFIGS[1].scaled(steps=40, index=30)
     run_workload(w, lambda w: sampled_pairs(w, 12), check_steps=(0, 7, 39), splits=splits, stages=stages,
                  combine=combine, every_step_ancestry=False)
+
+
+@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("splits,stages,combine", [(0, 0, 0), (1, 0, 0), (8, 0, 1), (8, 0, 2), (16, 2, 1), (5, 1, 0), (4, 3, 2)])
+def test_small_cta_form_forced_shapes(splits, stages, combine, fused):
+    # the 32-key-tile form of the kernel (two consumer warps, quarter-SM CTAs) in every merge mode
+    w = wl.CONFIGS[1].scaled(steps=40, index=31)
+    run = run_workload_fused if fused else run_workload
+    kw = {} if fused else {"every_step_ancestry": False}
+    run(w, lambda w: sampled_pairs(w, 12), check_steps=(0, 7, 39), splits=splits, stages=stages, combine=combine,
+        tile=32, **kw)
+
+
+@pytest.mark.parametrize("dtype,D", [("f16", 64), ("bf16", 128)])
+def test_small_cta_form_ragged_shapes(dtype, D):
+    # prompt not a multiple of the 32-key tile, GQA (6 query columns), ALiBi on the bf16 variant, ragged lengths
+    w = wl.Workload("ragged32", 3, 3, 6, 3, D, 150, 21, dtype, "uniform", dtype == "bf16", 14 + D // 64)
+    run_workload(w, all_pairs, check_steps=(0, 1, 5, 20), tile=32)
+    run_workload_fused(w, all_pairs, check_steps=(0, 1, 5, 20), tile=32, splits=3)
+    run_workload(w, all_pairs, check_steps=(0, 5, 20), tile=32, prompt_lens=[150, 33, 97])
 
 
 def test_cluster_combine_small_shapes():
