@@ -3,6 +3,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 
 #include "segkv_internal.h"
@@ -23,6 +24,49 @@ int cuda_fail(cudaError_t e, const char* what) {
         cudaError_t e__ = (call);                          \
         if (e__ != cudaSuccess) return cuda_fail(e__, #call); \
     } while (0)
+
+// ---------------------------------------------------------------------------
+// Which of the library's launches came last on each stream.  A kernel launched with programmatic
+// stream serialisation may begin before its predecessor P in the stream has finished, but not
+// before P has passed its own grid-dependency wait, i.e. not before everything older than P is
+// complete.  So data whose producing launch is strictly older than the latest library launch on
+// the same stream may be read by the new kernel from its very first instruction.  (A launch of
+// the caller's own in between only helps: it does not release its dependents early.)
+// ---------------------------------------------------------------------------
+struct StreamLog {
+    cudaStream_t st;
+    unsigned long long last;      // sequence number of the library's latest launch on st
+    bool used;
+};
+std::mutex g_log_mu;
+StreamLog g_log[32];
+unsigned long long g_launch_seq = 0;
+
+// Record a launch on `st`; returns its sequence number.
+unsigned long long note_launch(cudaStream_t st) {
+    std::lock_guard<std::mutex> lk(g_log_mu);
+    const unsigned long long seq = ++g_launch_seq;
+    int slot = -1, oldest = 0;
+    for (int i = 0; i < 32; ++i) {
+        if (g_log[i].used && g_log[i].st == st) { slot = i; break; }
+        if (!g_log[i].used) { if (slot < 0) slot = i; }
+        else if (g_log[i].last < g_log[oldest].last || !g_log[oldest].used) oldest = i;
+    }
+    if (slot < 0) slot = oldest;          // more than 32 streams: forget the one idle longest
+    g_log[slot].st = st;
+    g_log[slot].last = seq;
+    g_log[slot].used = true;
+    return seq;
+}
+
+// Is a launch `seq` on stream `st` strictly older than the library's latest launch there?
+bool older_than_latest(cudaStream_t st, cudaStream_t seq_stream, unsigned long long seq) {
+    if (seq == 0 || seq_stream != st) return false;
+    std::lock_guard<std::mutex> lk(g_log_mu);
+    for (int i = 0; i < 32; ++i)
+        if (g_log[i].used && g_log[i].st == st) return seq < g_log[i].last;
+    return false;
+}
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -114,12 +158,54 @@ int make_kv_source_map(const segkv* h, const void* base, int prompt_len, CUtenso
                          tiled_tile_keys(h->d.head_dim, false), "prefill K/V", out);
 }
 
+// Every kernel the library launches is counted on its handle and logged on its stream.
+unsigned long long count_launch(segkv* h, cudaStream_t st) {
+    h->launches++;
+    return note_launch(st);
+}
+
+bool capturing(cudaStream_t st) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) {
+        cudaGetLastError();
+        return true;                       // unknown: behave as if it were
+    }
+    return cs != cudaStreamCaptureStatusNone;
+}
+
+// The launch just made on `st` wrote the data `m` stands for.
+void mark_written(segkv* h, WriteMark* m, cudaStream_t st) {
+    m->seq = count_launch(h, st);
+    m->stream = st;
+    m->done = false;
+    m->recorded = m->ev && !capturing(st) && cudaEventRecord(m->ev, st) == cudaSuccess;
+}
+
+// Is the data `m` stands for complete and visible to a kernel launched now on `st`, from that
+// kernel's first instruction on?  Yes if its launch has been seen complete (sticky until the next
+// write), or if it is strictly older than the library's latest launch on the same stream.
+bool settled(WriteMark* m, cudaStream_t st) {
+    if (m->seq == 0) return false;
+    if (m->done) return true;
+    if (m->recorded && !capturing(st)) {
+        const cudaError_t e = cudaEventQuery(m->ev);
+        if (e == cudaSuccess) {
+            m->done = true;
+            return true;
+        }
+        if (e != cudaErrorNotReady) cudaGetLastError();
+    }
+    return older_than_latest(st, m->stream, m->seq);
+}
+
 void free_all(segkv* h) {
     void* ptrs[] = {h->kp, h->vp, h->kr, h->k_chunks_dev, h->parent, h->anc[0], h->anc[1], h->ulist, h->ucount, h->plens,
                     h->err_word, h->ws, h->tickets, h->st_q, h->st_out, h->st_k, h->st_v, h->st_parent, h->st_pack,
                     h->st_slopes};
     for (void* p : ptrs)
         if (p) cudaFree(p);
+    if (h->rows_mark.ev) cudaEventDestroy(h->rows_mark.ev);
+    if (h->lists_mark.ev) cudaEventDestroy(h->lists_mark.ev);
     for (int c = 0; c < h->nchunks; ++c)
         if (h->k_chunks_host[c]) cudaFree(h->k_chunks_host[c]);
     free(h->k_chunks_host);
@@ -255,9 +341,22 @@ int ensure_lists(segkv* h, cudaStream_t st) {
     segkv* x = index_of(h);
     if (x->lists_valid || h->steps == 0) return SEGKV_OK;
     SEGKV_CUDA(launch_rebuild_lists(x->d, h->steps, x->anc[(h->steps - 1) & 1], x->ulist, x->ucount, st));
-    h->launches++;
+    mark_written(h, &x->lists_mark, st);
+    x->lists_follow_rows = false;
     x->lists_valid = true;
     return SEGKV_OK;
+}
+
+// May the next attention launch on `st` read the handle's response rows (and, for the separate
+// form, the distinct-row lists) before its grid-dependency wait?  Only if the launches that wrote
+// them are strictly older than the library's latest launch on the same stream.
+bool rows_settled(segkv* h, cudaStream_t st, bool lists_too) {
+    if (!h->overlap || h->steps == 0) return false;
+    if (!settled(&h->rows_mark, st)) return false;
+    if (!lists_too) return true;
+    segkv* x = index_of(h);
+    if (x->lists_follow_rows) return settled(&x->rows_mark, st);
+    return settled(&x->lists_mark, st);
 }
 
 SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes, int splits) {
@@ -286,6 +385,7 @@ SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes
     a.small = false;
     a.pdl = false;
     a.prompt_immutable = h->steps > 0;     // the first append after a prefill is a fully serialised launch
+    a.rows_immutable = false;
     a.fused = false;
     a.wait_ns = h->dbg_wait_ns;
     a.dbg_skip = h->dbg_skip;
@@ -409,6 +509,11 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
 #undef SEGKV_TRY
     // The split workspace for the largest split count the automatic choice can make (one wave of
     // CTA slots shared among the work groups), so that the decode loop never allocates.
+    if (cudaEventCreateWithFlags(&h->rows_mark.ev, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->lists_mark.ev, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(SEGKV_ECUDA);
+    }
     rc = alloc_workspace(h, max_auto_splits(h));
     if (rc != SEGKV_OK) return fail(rc);
     *out = h;
@@ -459,7 +564,7 @@ static int prefill_write_impl(segkv_t h, const void* k, const void* v, int promp
     h->tm_valid = false;
     if (prompt_len > 0) {
         SEGKV_CUDA(launch_prefill_transpose(h->d, k, v, h->kp, h->vp, plens_dev, prompt_len, h->sm_count, st));
-        h->launches++;
+        count_launch(h, st);
         int rc = make_prompt_maps(h, prompt_len);
         if (rc != SEGKV_OK) return rc;
         h->tm_valid = true;
@@ -493,7 +598,7 @@ int segkv_prefill_sdpa(segkv_t h, const void* q, void* out, const float* alibi_s
         a.tm_q = &tm_q;
     }
     SEGKV_CUDA(launch_prefill_tc5(h->d, a, (cudaStream_t)stream));
-    h->launches++;
+    count_launch(h, (cudaStream_t)stream);
     return SEGKV_OK;
 }
 
@@ -528,7 +633,7 @@ int segkv_prefill(segkv_t h, const void* k, const void* v, const void* q, void* 
     a.tm_k_src = &tm_ks; a.tm_v_src = &tm_vs; a.tm_q = &tm_q;
     h->prompt_len = -1;                                       // nothing valid is stored if the launch fails
     SEGKV_CUDA(launch_prefill_tc5(h->d, a, (cudaStream_t)stream));
-    h->launches++;
+    count_launch(h, (cudaStream_t)stream);
     h->tm_valid = true;
     h->prompt_len = prompt_len;
     h->steps = 0;
@@ -578,7 +683,7 @@ static int append_impl(segkv_t h, int step, const int32_t* beam_parent, const vo
         SEGKV_CUDA(launch_append(h->d, step, nullptr, k_new, v_new, k_slab_of(h, step),
                                  k_slab_of(h, step) + vdelta_of(h), nullptr, nullptr, nullptr, nullptr, nullptr,
                                  h->err_word, h->sm_count, h->overlap && step > 0, (cudaStream_t)stream, rope, false));
-        h->launches++;
+        mark_written(h, &h->rows_mark, (cudaStream_t)stream);
         h->steps = step + 1;
         h->truncated = false;
         return SEGKV_OK;
@@ -587,7 +692,12 @@ static int append_impl(segkv_t h, int step, const int32_t* beam_parent, const vo
                              k_slab_of(h, step) + vdelta_of(h), h->parent,
                              h->anc[(step + 1) & 1], h->anc[step & 1], h->ulist, h->ucount, h->err_word,
                              h->sm_count, h->overlap && step > 0, (cudaStream_t)stream, rope));
-    h->launches++;
+    mark_written(h, &h->rows_mark, (cudaStream_t)stream);
+    h->lists_mark.seq = h->rows_mark.seq;          // the same launch made the lists: one event stands for both
+    h->lists_mark.stream = h->rows_mark.stream;
+    h->lists_mark.done = false;
+    h->lists_mark.recorded = false;
+    h->lists_follow_rows = true;
     h->steps = step + 1;
     h->truncated = false;
     h->lists_valid = true;
@@ -603,7 +713,7 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
     if (!tiled_supported(h->d)) {
         SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, 1);
         SEGKV_CUDA(launch_sdpa_rowwise(h->d, a, (cudaStream_t)stream));
-        h->launches++;
+        count_launch(h, (cudaStream_t)stream);
         return SEGKV_OK;
     }
     {
@@ -623,11 +733,12 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
     a.cluster = tl.cluster;
     a.small = tl.small;
     a.pdl = h->overlap;
+    a.rows_immutable = rows_settled(h, (cudaStream_t)stream, true);
     h->dbg_wait_ns = 0;                  // an injected fault applies to one launch
     h->dbg_skip = false;
     SEGKV_CUDA(launch_sdpa_tiled(h->d, a, tl.small ? h->tm_kp32 : h->tm_kp, tl.small ? h->tm_vp32 : h->tm_vp, tl.stages,
                                  (cudaStream_t)stream));
-    h->launches++;
+    count_launch(h, (cudaStream_t)stream);
     return SEGKV_OK;
 }
 
@@ -658,7 +769,7 @@ int segkv_decode_sdpa_static(segkv_t h, const void* q, void* out, const float* a
                  splits, tiled_static_scratch_bytes());
         return SEGKV_ECAPACITY;
     }
-    h->launches++;
+    count_launch(h, (cudaStream_t)stream);
     return SEGKV_OK;
 }
 
@@ -715,6 +826,7 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     // the first step after a prefill is fully serialised; from then on the prompt cannot change
     a.pdl = h->overlap && step > 0;
     a.prompt_immutable = step > 0;
+    a.rows_immutable = step > 0 && rows_settled(h, (cudaStream_t)stream, false);
     a.fused = true;
     a.parent = step > 0 ? beam_parent : nullptr;
     a.k_new = k_new;
@@ -727,7 +839,7 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     h->dbg_skip = false;
     SEGKV_CUDA(launch_sdpa_tiled(d, a, tl.small ? h->tm_kp32 : h->tm_kp, tl.small ? h->tm_vp32 : h->tm_vp, tl.stages,
                                  (cudaStream_t)stream));
-    h->launches++;
+    mark_written(h, &h->rows_mark, (cudaStream_t)stream);
     h->steps = step + 1;
     h->truncated = false;
     h->lists_valid = false;              // the fused kernel does not make the distinct-row lists
@@ -895,7 +1007,7 @@ int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, const float* 
     if (h->prompt_len + h->steps <= 0) return SEGKV_ESTATE;
     SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, 1);
     SEGKV_CUDA(launch_sdpa_rowwise(h->d, a, (cudaStream_t)stream));
-    h->launches++;
+    count_launch(h, (cudaStream_t)stream);
     return SEGKV_OK;
 }
 

@@ -22,6 +22,16 @@ struct URow {
     uint32_t mask;
 };
 
+// Where and when data was last written: the stream and per-process sequence number of the launch,
+// and an event recorded behind it (not while the stream is being captured).
+struct WriteMark {
+    cudaStream_t stream;
+    unsigned long long seq;       // 0: never written
+    cudaEvent_t ev;               // created with the handle
+    bool recorded;                // ev was recorded behind the launch
+    bool done;                    // the launch has been seen complete (ev queried, or the host synchronised)
+};
+
 struct Dims {
     int batch, beams, heads, kv_heads, head_dim, group;  // group = heads / kv_heads
     int max_prompt, max_steps;
@@ -83,6 +93,11 @@ struct segkv {
     segkv_impl::URow* ulist;   // [batch, beams*max_steps] distinct response rows per request
     int32_t* ucount;     // [batch]
     bool lists_valid;    // ulist/ucount describe the newest step (a fused step does not update them)
+    // the latest launch that wrote response rows / beam-index tables of this handle, and the one
+    // that wrote its row lists (what a later attention launch may read ahead of its wait once
+    // these are known to be complete)
+    segkv_impl::WriteMark rows_mark, lists_mark;
+    bool lists_follow_rows;   // the lists were made by the launch rows_mark stands for (the append kernel)
     int* err_word;       // device error word
     float* ws;           // split workspace
     size_t ws_bytes;
@@ -146,6 +161,8 @@ struct SdpaArgs {
     bool cluster;            // merge the splits inside a thread-block cluster
     bool pdl;                // launch with programmatic stream serialisation
     bool prompt_immutable;   // a fully serialised launch has followed the last prompt store
+    bool rows_immutable;     // the response rows of earlier steps (separate form: the row lists too) were written by
+                             // launches older than this launch's predecessor: readable before the grid-dependency wait
     // fused decode step (append + beam-index update + attention in one launch)
     // test aid (segkv_debug_inject): limit of the kernel's bounded waits (0 = default) and one
     // barrier arrival left out so that a wait runs out

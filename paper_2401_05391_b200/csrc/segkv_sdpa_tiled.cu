@@ -64,9 +64,6 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
 __device__ __forceinline__ void cluster_arrive_relaxed() {
     asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void cluster_arrive_release() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-}
 __device__ __forceinline__ void cluster_wait_acquire() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -75,11 +72,35 @@ __device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float4 v) {
-    asm volatile("st.shared::cluster.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+// Store to another CTA of the cluster that reports its bytes to an mbarrier of that CTA: the
+// receiver learns of the data by waiting on its own barrier, nobody meets at a cluster barrier.
+__device__ __forceinline__ void st_async_v4(uint32_t addr, float4 v, uint32_t mbar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1,%2,%3,%4}, [%5];"
+                 ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(mbar) : "memory");
 }
-__device__ __forceinline__ void st_cluster_v2(uint32_t addr, float a, float b) {
-    asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
+__device__ __forceinline__ void st_async_v2(uint32_t addr, float a, float b, uint32_t mbar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1,%2}, [%3];"
+                 ::"r"(addr), "f"(a), "f"(b), "r"(mbar) : "memory");
+}
+// Bounded wait on an mbarrier of this CTA whose phase is completed by other CTAs' stores.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
+    const uint64_t t0 = global_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 1024; ++i) {
+            uint32_t ok;
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t"
+                "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+                "selp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+            if (ok) return true;
+        }
+        if (global_ns() - t0 > limit_ns) return false;
+    }
+}
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 // Programmatic dependent launch: let the next kernel of the stream begin, and wait for the
 // previous one to have completed with its writes visible (no-ops without the launch attribute).
@@ -88,17 +109,18 @@ __device__ __forceinline__ void grid_wait() { asm volatile("griddepcontrol.wait;
 
 #ifdef SEGKV_TIMELINE
 }  // namespace
-__device__ unsigned long long g_timeline[8 * 512 * 16];
+__device__ unsigned long long g_timeline[8 * 512 * 32];   // per CTA: 16 x %globaltimer, then 16 x clock64
 #define SEGKV_CLK(ev, cond)                                                                \
     do {                                                                                   \
         if ((cond) && (threadIdx.x & 31) == 0 && blockIdx.x < 512) {                       \
-            g_timeline[((p.dbg_launch & 7) * 512 + blockIdx.x) * 16 + (ev)] = (unsigned long long)clock64(); \
+            g_timeline[((p.dbg_launch & 7) * 512 + blockIdx.x) * 32 + 16 + (ev)] = (unsigned long long)clock64(); \
         }                                                                                  \
     } while (0)
 #define SEGKV_STAMP(ev)                                                                    \
     do {                                                                                   \
         if ((threadIdx.x & 31) == 0 && blockIdx.x < 512) {                                 \
-            g_timeline[((p.dbg_launch & 7) * 512 + blockIdx.x) * 16 + (ev)] = global_ns(); \
+            if ((ev) == 0) g_timeline[((p.dbg_launch & 7) * 512 + blockIdx.x) * 32] = global_ns(); \
+            g_timeline[((p.dbg_launch & 7) * 512 + blockIdx.x) * 32 + 16 + (ev)] = (unsigned long long)clock64(); \
         }                                                                                  \
     } while (0)
 namespace {
@@ -110,6 +132,8 @@ namespace {
 // A CTA whose bounded wait ran out adds this to its work group's arrival counter on top of its
 // ticket (splits are at most kMaxSplits, far below it).
 constexpr int kTicketAborted = 1 << 16;
+
+template <int N> struct IntC { static constexpr int value = N; };
 
 struct TiledParams {
     const void* q;
@@ -141,6 +165,7 @@ struct TiledParams {
     int quota;      // distinct response rows per split (the last split also takes any excess)
     int cluster;    // 1: the S CTAs of a work group form a thread-block cluster
     int early_prompt;  // 1: prompt tiles may be fetched before the previous kernel has completed
+    int early_rows;    // 1: so may the response rows of earlier steps and (separate form) the row lists
     int dbg_skip;      // test aid: the gather warp leaves out one plain barrier arrival, so that a wait runs out
     unsigned long long wait_ns;   // limit of every bounded wait
 #ifdef SEGKV_TIMELINE
@@ -172,7 +197,7 @@ struct Layout {
     }
     static __host__ __device__ constexpr size_t bars(int stages) {
         // mbarriers, per-stage {count, last} of response tiles, then the gather warp's row pointers
-        return (((size_t)stages * 24 + 8 + 127) & ~(size_t)127) + (size_t)TILE * 16;
+        return (((size_t)stages * 24 + 16 + 127) & ~(size_t)127) + (size_t)TILE * 16;
     }
     static __host__ __device__ constexpr size_t recv(int nt) {
         return (size_t)8 * nt * D * 4 + (size_t)kMaxCluster * 8 * nt * 2 * 4;
@@ -205,12 +230,13 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     float* recv_ml = recv_o + 8 * NT * D;                                                     // [S][ncols][2]
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + stages), hand = smem_u32(bars + 2 * stages);
     int2* tile_hdr = reinterpret_cast<int2*>(bars + 2 * stages + 1);                           // [stages] {count, last}
+    const uint32_t recvbar = smem_u32(bars + 3 * stages + 1);          // cluster merge: the other CTAs' partials have landed
     const char** gk = reinterpret_cast<const char**>(reinterpret_cast<uint8_t*>(recv_o) - (size_t)TILE * 16);  // [TILE] K row pointers
     const char** gv = gk + TILE;                                                               // [TILE] V row pointers
     __shared__ int s_last, s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) { SEGKV_STAMP(0); SEGKV_STAMP(1); }
+    if (tid == 0) SEGKV_STAMP(0);
     const int split = blockIdx.x % p.S;
     const int slab = blockIdx.x / p.S;           // b * Hkv + kvh
     const int b = slab / p.Hkv, kvh = slab % p.Hkv;
@@ -256,6 +282,11 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 mbar_init(empty0 + 8 * s, CW);    // one arrival per consumer warp
             }
             mbar_init(hand, 1);                   // ring handed from the TMA warp to the gather warp
+            if (p.cluster) {
+                // the S partials of this CTA's slice of the (column, d) plane and S x ncols {max, sum} pairs
+                mbar_init(recvbar, 1);
+                mbar_arrive_expect_tx(recvbar, (uint32_t)(p.ncols * D * 4 + p.S * p.ncols * 8));
+            }
             s_abort = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             fence_proxy_async();
@@ -272,20 +303,69 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         for (int k = 0; k < first; ++k) issue_prompt_tile(k);
         tma_issued = first;
         if (first == npt && lane == 0) mbar_arrive(hand);
+        // Prompt tiles that have to wait for a stage of the ring are at least brought into the L2,
+        // so that their turn costs an L2 hit, not an HBM round trip, after the wait.
+        if (p.early_prompt && lane == 0) {
+            for (int k = first; k < npt; ++k) {
+                const int y = (pt0 + k) * TILE;
+#pragma unroll
+                for (int bx = 0; bx < D / 64; ++bx) {
+                    tma_prefetch_4d(&tm_k, bx * 64, kvh, y, b);
+                    tma_prefetch_4d(&tm_v, bx * 64, kvh, y, b);
+                }
+            }
+        }
         SEGKV_STAMP(3);
+    } else if (warp == 0) {
+        // The query rows are written by the kernel before this one, so they may only be READ after
+        // the wait; asking the L2 for their lines is harmless before it (a line fetched early is
+        // overwritten in place by the producer), and the read after the wait then finds them there.
+        constexpr int LPR = D * 2 / 128;                         // 128-byte lines per query row
+        for (int i = lane; i < p.ncols * LPR; i += 32) {
+            const int col = i / LPR;
+            const char* qrow = reinterpret_cast<const char*>(p.q) +
+                               ((size_t)(b * p.W + col / p.G) * p.H + kvh * p.G + col % p.G) * (size_t)(D * 2);
+            prefetch_l2(qrow + (i % LPR) * 128);
+        }
+    }
+    // Consumer warps: what needs no data of the previous kernel (addresses, column masks) is worked
+    // out before the wait, so that the query loads go out the moment it returns.
+    const T* qrow_c[NT];
+    const float* slope_c[NT][2];
+    uint32_t beambit[NT][2];
+    if (warp < CW) {
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int col = nt * 8 + (lane >> 2);             // Q^T as the B operand: this lane holds column lane/4
+            const bool cv = col < p.ncols;
+            const int j = cv ? col / p.G : 0, hg = cv ? col % p.G : 0;
+            qrow_c[nt] = cv ? reinterpret_cast<const T*>(p.q) + ((size_t)(b * p.W + j) * p.H + kvh * p.G + hg) * D : nullptr;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {                     // the two score columns this lane owns
+                const int col2 = nt * 8 + (lane & 3) * 2 + c;
+                const bool cv2 = col2 < p.ncols;
+                beambit[nt][c] = cv2 ? (1u << (col2 / p.G)) : 0u;
+                slope_c[nt][c] = (cv2 && p.slopes) ? p.slopes + kvh * p.G + col2 % p.G : nullptr;
+            }
+        }
     }
     if (p.cluster) cluster_arrive_relaxed();     // "this CTA has started" (waited for before any remote store)
     __syncthreads();
     // Everything else (q, row lists, parents, response rows, outputs) follows the previous kernel.
     // The next kernel is let go only after this wait, so a kernel that starts early behind this
-    // one finds every kernel before this one's predecessor complete.
-    grid_wait();
-    grid_launch_dependents();
+    // one finds every kernel before this one's predecessor complete.  (The gather warp of the
+    // separate form, when the host vouches for its inputs, works ahead and waits later.)
+    const bool gather_ahead = !FUSED && warp == GATHER_WARP && p.early_rows;
+    if (!gather_ahead) {
+        grid_wait();
+        grid_launch_dependents();
+    }
     if (tid == 0) SEGKV_STAMP(2);
 
     // consumer state (declared here so that the epilogue sees it)
     float o_acc[NT][KS][4];
     float m_run[NT][2], l_run[NT][2];
+    bool cons_ok = true;          // this consumer warp has seen all of its tiles
 
     if (warp == TMA_WARP) {
         // ============================ prompt tiles beyond the first round ============================
@@ -390,42 +470,66 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             const int e1 = (split == p.S - 1) ? n_b : min((split + 1) * p.quota, n_b);
             const int nrt = (e1 - e0 + TILE - 1) / TILE;
             SEGKV_STAMP(4);
-            if (nrt > 0) {
-                ok = mbar_wait(hand, 0, p.wait_ns);
-                ok = __all_sync(0xffffffffu, ok);
-            }
-            for (int r = 0; r < nrt && ok; ++r) {
-                const int k = npt + r;
-                const int eb = e0 + r * TILE;
-                const int cnt = min(TILE, e1 - eb);
-#pragma unroll
-                for (int kk = 0; kk < UK; ++kk) {
-                    ucur[kk] = unext[kk];
-                    const int key = lane + 32 * kk;
-                    unext[kk] = (key < TILE && eb + TILE + key < e1)
-                                    ? *reinterpret_cast<const uint2*>(ulist_b + eb + TILE + key)
-                                    : make_uint2(0u, 0u);
+            // Tiles [r, r_end) of this CTA's range of the list: row pointers and per-key records into
+            // the stage, then the copies.
+            int r = 0;
+            bool handed = false;
+            auto tiles = [&](int r_end) {
+                if (r < r_end && !handed) {
+                    ok = mbar_wait(hand, 0, p.wait_ns);
+                    ok = __all_sync(0xffffffffu, ok);
+                    handed = true;
                 }
-                const int st = k % stages;
-                ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1, p.wait_ns);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                URow* meta_st = meta + (size_t)st * TILE;
+                for (; r < r_end && ok; ++r) {
+                    const int k = npt + r;
+                    const int eb = e0 + r * TILE;
+                    const int cnt = min(TILE, e1 - eb);
 #pragma unroll
-                for (int kk = 0; kk < UK; ++kk) {
-                    const int key = lane + 32 * kk;
-                    if (key >= TILE) continue;
-                    const bool valid = key < cnt;
-                    const int row = valid ? (int)ucur[kk].x : 0;         // step * rows + slot
-                    URow u;
-                    u.row = row / p.rows;                                // consumers need the step only
-                    u.mask = valid ? ucur[kk].y : 0u;
-                    meta_st[key] = u;
-                    const int sidx = u.row;
-                    gk[key] = k_slab(sidx) + ((size_t)(row - sidx * p.rows) * p.Hkv + kvh) * (size_t)(D * 2);
+                    for (int kk = 0; kk < UK; ++kk) {
+                        ucur[kk] = unext[kk];
+                        const int key = lane + 32 * kk;
+                        unext[kk] = (key < TILE && eb + TILE + key < e1)
+                                        ? *reinterpret_cast<const uint2*>(ulist_b + eb + TILE + key)
+                                        : make_uint2(0u, 0u);
+                    }
+                    const int st = k % stages;
+                    ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1, p.wait_ns);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    URow* meta_st = meta + (size_t)st * TILE;
+#pragma unroll
+                    for (int kk = 0; kk < UK; ++kk) {
+                        const int key = lane + 32 * kk;
+                        if (key >= TILE) continue;
+                        const bool valid = key < cnt;
+                        const int row = valid ? (int)ucur[kk].x : 0;         // step * rows + slot
+                        URow u;
+                        u.row = row / p.rows;                                // consumers need the step only
+                        u.mask = valid ? ucur[kk].y : 0u;
+                        meta_st[key] = u;
+                        const int sidx = u.row;
+                        gk[key] = k_slab(sidx) + ((size_t)(row - sidx * p.rows) * p.Hkv + kvh) * (size_t)(D * 2);
+                    }
+                    publish_tile(st, cnt, r == nrt - 1);
                 }
-                publish_tile(st, cnt, r == nrt - 1);
+            };
+            if (gather_ahead) {
+                // Lists and rows were written by launches older than this launch's predecessor: the tiles
+                // that find a free stage are fetched now, the rows of the others are asked into the L2,
+                // and only then does this warp wait for the previous kernel.
+                const int r_now = npt < stages ? min(nrt, stages - npt) : 0;
+                for (int e = e0 + r_now * TILE + lane / 4; e < e1; e += 8) {
+                    const int row = ulist_b[e].row, sidx = row / p.rows;
+                    const char* kr = k_slab(sidx) + ((size_t)(row - sidx * p.rows) * p.Hkv + kvh) * (size_t)(D * 2);
+                    const char* src = ((lane & 2) ? kr + p.vdelta : kr) + (lane & 1) * (D);     // K or V row, first or second half
+                    prefetch_l2(src);
+                    if (D == 256) prefetch_l2(src + 128);
+                }
+                tiles(r_now);
+                grid_wait();
+                grid_launch_dependents();
             }
+            tiles(nrt);
             SEGKV_STAMP(5);
         } else {
             // ---- fused decode step: rows from the beam-index table, derived on the fly ----
@@ -557,35 +661,23 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 for (int i = 0; i < 4; ++i) o_acc[nt][mt][i] = 0.f;
         }
         const int n_b = (p.steps > 0 && !FUSED) ? p.ucount[b] : 0;   // in flight while the prompt tiles are consumed
-        // Q^T as the B operand: this lane holds column n = lane/4 of every column tile
         uint32_t qf[NT][KS][2];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            const int col = nt * 8 + (lane >> 2);
-            const bool cv = col < p.ncols;
-            const int j = cv ? col / p.G : 0, hg = cv ? col % p.G : 0;
-            const T* qrow = reinterpret_cast<const T*>(p.q) + ((size_t)(b * p.W + j) * p.H + kvh * p.G + hg) * D;
+            const T* qrow = qrow_c[nt];
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
                 const int d0 = ks * 16 + (lane & 3) * 2;
-                qf[nt][ks][0] = cv ? *reinterpret_cast<const uint32_t*>(qrow + d0) : 0u;
-                qf[nt][ks][1] = cv ? *reinterpret_cast<const uint32_t*>(qrow + d0 + 8) : 0u;
+                qf[nt][ks][0] = qrow ? *reinterpret_cast<const uint32_t*>(qrow + d0) : 0u;
+                qf[nt][ks][1] = qrow ? *reinterpret_cast<const uint32_t*>(qrow + d0 + 8) : 0u;
             }
         }
-        // the two score columns this lane owns in every column tile
         float slope2[NT][2];
-        uint32_t beambit[NT][2];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                const int col = nt * 8 + (lane & 3) * 2 + c;
-                const bool cv = col < p.ncols;
-                beambit[nt][c] = cv ? (1u << (col / p.G)) : 0u;
-                slope2[nt][c] = (cv && p.slopes) ? p.slopes[kvh * p.G + col % p.G] * 1.4426950408889634f : 0.f;
-            }
+            for (int c = 0; c < 2; ++c) slope2[nt][c] = slope_c[nt][c] ? *slope_c[nt][c] * 1.4426950408889634f : 0.f;
         const int qpos = P + (p.steps > 0 ? p.steps - 1 : -1);
-        const int key_lo = warp * 16 + (lane >> 2);       // tile-local key of accumulator rows 0..7
 
         // One tile: `nvalid` keys exist; for a response tile the per-key beam masks and row
         // ids are in the stage's meta array, for a prompt tile key i sits at position pos0 + i.
@@ -594,61 +686,75 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         auto chunk_addr = [&](uint32_t base, int key, int ch, bool) -> uint32_t {
             return base + (uint32_t)(ch >> 3) * L::BOX_BYTES + (uint32_t)key * 128 + (uint32_t)(((ch & 7) ^ (key & 7)) << 4);
         };
-        auto consume = [&](int st, bool resp, int nvalid, int pos0) {
-            if (warp * 16 >= nvalid) return;
+        // NB blocks of 16 keys of one tile, at tile-local keys kb0, kb0 + 16, ...: their scores, ONE
+        // online-softmax update over all of them, their weighted values.  The blocks are independent
+        // until the column maxima meet, so a warp that takes several hides the latency of one
+        // block's MMA chain and shuffles behind the others'.
+        auto consume = [&](auto nb_c, int st, bool resp, int nvalid, int pos0, int kb0) {
+            constexpr int NB = decltype(nb_c)::value;
+            if (kb0 >= nvalid) return;
             const uint32_t k_src = smem_u32(ring + (size_t)st * L::STAGE_BYTES);
             const uint32_t v_src = k_src + L::TILE_BYTES;
             // ---- S^T = K . Q^T ----
-            float sc[NT][4];
+            float sc[NB][NT][4];
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
-            {
-                const int key = warp * 16 + (lane & 15);
+            for (int i = 0; i < NB; ++i)
 #pragma unroll
-                for (int ks = 0; ks < KS; ++ks) {
-                    const int ch = 2 * ks + (lane >> 4);
+                for (int nt = 0; nt < NT; ++nt) sc[i][nt][0] = sc[i][nt][1] = sc[i][nt][2] = sc[i][nt][3] = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                const int ch = 2 * ks + (lane >> 4);
+#pragma unroll
+                for (int i = 0; i < NB; ++i) {
                     uint32_t a[4];
-                    ldmatrix_x4(a, chunk_addr(k_src, key, ch, resp));
+                    ldmatrix_x4(a, chunk_addr(k_src, kb0 + 16 * i + (lane & 15), ch, resp));
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) Mma<T>::run(sc[nt], a, qf[nt][ks][0], qf[nt][ks][1]);
+                    for (int nt = 0; nt < NT; ++nt) Mma<T>::run(sc[i][nt], a, qf[nt][ks][0], qf[nt][ks][1]);
                 }
             }
+            if (warp == 0 && !resp && pos0 == pt0 * TILE) SEGKV_STAMP(15);
             // ---- mask, bias, online softmax ----
-            uint32_t kmask[2];
-            float kpos[2];
+            uint32_t kmask[NB][2];
+            float kpos[NB][2];
 #pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const int key = key_lo + 8 * r;
-                if (resp) {
-                    const URow u = meta[(size_t)st * TILE + key];       // {step, beams that read the row}
-                    kmask[r] = key < nvalid ? u.mask : 0u;
-                    kpos[r] = (float)(P + u.row - qpos);
-                } else {
-                    kmask[r] = key < nvalid ? 0xffffffffu : 0u;
-                    kpos[r] = (float)(pos0 + key - qpos);
+            for (int i = 0; i < NB; ++i)
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    const int key = kb0 + 16 * i + (lane >> 2) + 8 * r;
+                    if (resp) {
+                        const URow u = meta[(size_t)st * TILE + key];       // {step, beams that read the row}
+                        kmask[i][r] = key < nvalid ? u.mask : 0u;
+                        kpos[i][r] = (float)(P + u.row - qpos);
+                    } else {
+                        kmask[i][r] = key < nvalid ? 0xffffffffu : 0u;
+                        kpos[i][r] = (float)(pos0 + key - qpos);
+                    }
                 }
-            }
             // P^T fragments.  bf16 keeps 8 significant bits of a weight, which is not enough where a few
             // keys carry a column's whole weight (a steep ALiBi slope) and their values cancel, so bf16
             // weights go to the tensor cores in two parts, p = hi + lo (16 bits together): the kernel
             // is bound by HBM and the second set of MMAs is free.  fp16 weights (11 bits) go as they are.
             constexpr bool kTwoPart = sizeof(T) == 2 && !Mma<T>::kWeights11Bits;
-            uint32_t pfrag[NT][2], pfrag_lo[NT][2];
+            uint32_t pfrag[NB][NT][2], pfrag_lo[NB][NT][2];
             bool rescale = false;
             float alpha[NT][2];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-                float s[2][2];
+                float s[NB][2][2];
 #pragma unroll
-                for (int r = 0; r < 2; ++r)
+                for (int i = 0; i < NB; ++i)
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        float v = sc[nt][2 * r + c] * p.scale2 + slope2[nt][c] * kpos[r];
-                        s[r][c] = (kmask[r] & beambit[nt][c]) ? v : -INFINITY;
-                    }
+                    for (int r = 0; r < 2; ++r)
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            float v = sc[i][nt][2 * r + c] * p.scale2 + slope2[nt][c] * kpos[i][r];
+                            s[i][r][c] = (kmask[i][r] & beambit[nt][c]) ? v : -INFINITY;
+                        }
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
-                    float tm = fmaxf(s[0][c], s[1][c]);
+                    float tm = fmaxf(s[0][0][c], s[0][1][c]);
+#pragma unroll
+                    for (int i = 1; i < NB; ++i) tm = fmaxf(tm, fmaxf(s[i][0][c], s[i][1][c]));
                     tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, 4));
                     tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, 8));
                     tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, 16));
@@ -659,18 +765,26 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     alpha[nt][c] = a;
                     rescale = rescale || (a != 1.f);
                     m_run[nt][c] = m_new;
-                    const float p0 = exp2f(s[0][c] - m_use), p1 = exp2f(s[1][c] - m_use);
-                    s[0][c] = p0;
-                    s[1][c] = p1;
-                    l_run[nt][c] = l_run[nt][c] * a + p0 + p1;
+                    float psum = 0.f;
+#pragma unroll
+                    for (int i = 0; i < NB; ++i) {
+                        const float p0 = exp2f(s[i][0][c] - m_use), p1 = exp2f(s[i][1][c] - m_use);
+                        s[i][0][c] = p0;
+                        s[i][1][c] = p1;
+                        psum += p0 + p1;
+                    }
+                    l_run[nt][c] = l_run[nt][c] * a + psum;
                 }
                 // P^T as the B operand of O^T += V^T . P^T
-                const uint32_t h0 = Mma<T>::pack(s[0][0], s[0][1]), h1 = Mma<T>::pack(s[1][0], s[1][1]);
-                pfrag[nt][0] = movmatrix_trans(h0);
-                pfrag[nt][1] = movmatrix_trans(h1);
-                if constexpr (kTwoPart) {
-                    pfrag_lo[nt][0] = movmatrix_trans(Mma<T>::pack(s[0][0] - __uint_as_float(h0 << 16), s[0][1] - __uint_as_float(h0 & 0xFFFF0000u)));
-                    pfrag_lo[nt][1] = movmatrix_trans(Mma<T>::pack(s[1][0] - __uint_as_float(h1 << 16), s[1][1] - __uint_as_float(h1 & 0xFFFF0000u)));
+#pragma unroll
+                for (int i = 0; i < NB; ++i) {
+                    const uint32_t h0 = Mma<T>::pack(s[i][0][0], s[i][0][1]), h1 = Mma<T>::pack(s[i][1][0], s[i][1][1]);
+                    pfrag[i][nt][0] = movmatrix_trans(h0);
+                    pfrag[i][nt][1] = movmatrix_trans(h1);
+                    if constexpr (kTwoPart) {
+                        pfrag_lo[i][nt][0] = movmatrix_trans(Mma<T>::pack(s[i][0][0] - __uint_as_float(h0 << 16), s[i][0][1] - __uint_as_float(h0 & 0xFFFF0000u)));
+                        pfrag_lo[i][nt][1] = movmatrix_trans(Mma<T>::pack(s[i][1][0] - __uint_as_float(h1 << 16), s[i][1][1] - __uint_as_float(h1 & 0xFFFF0000u)));
+                    }
                 }
             }
             if (__any_sync(0xffffffffu, rescale)) {
@@ -685,35 +799,65 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     }
             }
             // ---- O^T += V^T . P^T ----
-            {
-                const int key = warp * 16 + (lane & 7) + 8 * (lane >> 4);
 #pragma unroll
-                for (int mt = 0; mt < KS; ++mt) {
-                    const int ch = 2 * mt + ((lane >> 3) & 1);
+            for (int mt = 0; mt < KS; ++mt) {
+                const int ch = 2 * mt + ((lane >> 3) & 1);
+#pragma unroll
+                for (int i = 0; i < NB; ++i) {
                     uint32_t a[4];
-                    ldmatrix_x4_trans(a, chunk_addr(v_src, key, ch, resp));
+                    ldmatrix_x4_trans(a, chunk_addr(v_src, kb0 + 16 * i + (lane & 7) + 8 * (lane >> 4), ch, resp));
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
-                        Mma<T>::run(o_acc[nt][mt], a, pfrag[nt][0], pfrag[nt][1]);
-                        if constexpr (kTwoPart) Mma<T>::run(o_acc[nt][mt], a, pfrag_lo[nt][0], pfrag_lo[nt][1]);
+                        Mma<T>::run(o_acc[nt][mt], a, pfrag[i][nt][0], pfrag[i][nt][1]);
+                        if constexpr (kTwoPart) Mma<T>::run(o_acc[nt][mt], a, pfrag_lo[i][nt][0], pfrag_lo[i][nt][1]);
                     }
                 }
             }
         };
+        // Small-CTA form: a prompt tile is taken WHOLE by one consumer warp (the warps take turns),
+        // its CW blocks side by side; elsewhere every warp takes its own 16 keys of every tile.
+        constexpr bool kWholeTile = CW == 2 && D <= 128 && NT == 1;
 
         bool ok = true;
         int k = 0;
+        int st = 0;              // stage and phase of tile k: k % stages, (k / stages) & 1
+        uint32_t ph = 0;
+        auto next_stage = [&]() {
+            if (++st == stages) {
+                st = 0;
+                ph ^= 1u;
+            }
+        };
+        if (warp == 0) SEGKV_STAMP(1);
+        if constexpr (kWholeTile) {
+            for (; k < npt; ++k) {
+                // every warp waits for every tile, also those it leaves to the other warp: a parity
+                // wait cannot tell a barrier's phases two apart, so none may be skipped
+                ok = mbar_wait(full0 + 8 * st, ph, p.wait_ns);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if ((k & (CW - 1)) == warp) {
+                    const int pos0 = (pt0 + k) * TILE;
+                    if (warp == 0 && k == 0) SEGKV_STAMP(7);
+                    consume(IntC<CW>{}, st, false, min(TILE, P - pos0), pos0, 0);
+                    if (warp == 0 && k == 0) SEGKV_STAMP(6);
+                    __syncwarp();
+                    if (lane < CW) mbar_arrive(empty0 + 8 * st);      // the stage's release counts one arrival per consumer warp
+                }
+                next_stage();
+            }
+        }
         for (; k < npt; ++k) {
-            const int st = k % stages;
-            ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1, p.wait_ns);
+            ok = mbar_wait(full0 + 8 * st, ph, p.wait_ns);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const int pos0 = (pt0 + k) * TILE;
             if (warp == 0 && k == 0) SEGKV_STAMP(7);
-            consume(st, false, min(TILE, P - pos0), pos0);
+            consume(IntC<1>{}, st, false, min(TILE, P - pos0), pos0, warp * 16);
             if (warp == 0 && k == 0) SEGKV_STAMP(6);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + 8 * st);
+            next_stage();
         }
         if (warp == 0) SEGKV_STAMP(8);
         if (ok && !FUSED) {
@@ -721,26 +865,26 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             const int e1 = (split == p.S - 1) ? n_b : min((split + 1) * p.quota, n_b);
             const int nrt = (e1 - e0 + TILE - 1) / TILE;
             for (int r = 0; r < nrt; ++r, ++k) {
-                const int st = k % stages;
-                ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1, p.wait_ns);
+                ok = mbar_wait(full0 + 8 * st, ph, p.wait_ns);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                consume(st, true, min(TILE, e1 - (e0 + r * TILE)), 0);
+                consume(IntC<1>{}, st, true, min(TILE, e1 - (e0 + r * TILE)), 0, warp * 16);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8 * st);
+                next_stage();
             }
         } else if (ok && rs1 > rs0) {
             // fused step: how many response tiles there are and how full each is only the gather
             // warp knows; it says so in the tile's header
             for (;;) {
-                const int st = k % stages;
-                ok = mbar_wait(full0 + 8 * st, ((uint32_t)(k / stages)) & 1, p.wait_ns);
+                ok = mbar_wait(full0 + 8 * st, ph, p.wait_ns);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 const int2 hd = tile_hdr[st];
-                consume(st, true, hd.x, 0);
+                consume(IntC<1>{}, st, true, hd.x, 0, warp * 16);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8 * st);
+                next_stage();
                 ++k;
                 if (hd.y) break;
             }
@@ -749,10 +893,136 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             atomicOr(p.err_word, SEGKV_DEV_WAIT_LIMIT);
             s_abort = 1;
         }
+        cons_ok = ok;
     }
 
     if (warp == 0) SEGKV_STAMP(9);
     // ==================================== epilogue ====================================
+    if (p.cluster) {
+        // ---- split merge inside the thread-block cluster, through distributed shared memory ----
+        // Only the consumer warps take part, and nobody meets at a cluster barrier: the (column, d)
+        // plane is cut into S equal slices, CTA r merges slice r, every CTA sends its part of
+        // slice r to CTA r with stores that report their bytes to CTA r's receive barrier, and CTA r
+        // folds the S partials once its own barrier says they are all there.
+        constexpr int CT = CW * 32;                       // consumer threads
+        const int ncols = p.ncols, S = p.S;
+        const int slice = ncols * D / S;                  // floats; a multiple of 4
+        if (warp < CW) {
+            float* mrg_o = reinterpret_cast<float*>(smem);                       // [CW][8*NT][DP], over the ring
+            float* mrg_ml = mrg_o + (size_t)CW * 8 * NT * DP;                    // [CW][8*NT][2]
+            named_bar_sync(1, CT);                        // every consumer warp is done reading the ring
+            const bool bad = !cons_ok || *reinterpret_cast<volatile int*>(&s_abort) != 0;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    float l = l_run[nt][c];
+                    l += __shfl_xor_sync(0xffffffffu, l, 4);
+                    l += __shfl_xor_sync(0xffffffffu, l, 8);
+                    l += __shfl_xor_sync(0xffffffffu, l, 16);
+                    const int col = nt * 8 + (lane & 3) * 2 + c;
+                    if ((lane >> 2) == 0) {
+                        mrg_ml[((size_t)warp * 8 * NT + col) * 2 + 0] = m_run[nt][c];
+                        mrg_ml[((size_t)warp * 8 * NT + col) * 2 + 1] = l;
+                    }
+                    float* dst = mrg_o + ((size_t)warp * 8 * NT + col) * DP + (lane >> 2);
+#pragma unroll
+                    for (int mt = 0; mt < KS; ++mt) {
+                        dst[mt * 16] = o_acc[nt][mt][c];
+                        dst[mt * 16 + 8] = o_acc[nt][mt][2 + c];
+                    }
+                }
+            }
+            named_bar_sync(1, CT);
+            if (tid == 0) SEGKV_STAMP(10);
+            const uint32_t me = cluster_ctarank();
+            const float inv_slice4 = 4.f / (float)slice;
+            cluster_wait_acquire();                       // every CTA of the cluster has set its barrier up
+            for (int it = tid; it < ncols * D4; it += CT) {
+                const int col = it / D4, d = (it % D4) * 4;
+                // merged partial of this CTA for one float4 of one column
+                float mm = -INFINITY;
+#pragma unroll
+                for (int w = 0; w < CW; ++w) mm = fmaxf(mm, mrg_ml[((size_t)w * 8 * NT + col) * 2]);
+                float ll = 0.f;
+                float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int w = 0; w < CW; ++w) {
+                    const float mw = mrg_ml[((size_t)w * 8 * NT + col) * 2];
+                    const float f = (mw == -INFINITY) ? 0.f : exp2f(mw - mm);
+                    ll += mrg_ml[((size_t)w * 8 * NT + col) * 2 + 1] * f;
+                    const float4 v = *reinterpret_cast<const float4*>(mrg_o + ((size_t)w * 8 * NT + col) * DP + d);
+                    o.x += v.x * f; o.y += v.y * f; o.z += v.z * f; o.w += v.w * f;
+                }
+                const int f4 = col * D4 + (d >> 2);                              // float4 index in the plane
+                const int r = (int)(((float)f4 + 0.5f) * inv_slice4);            // its slice (exact: small integers)
+                const uint32_t rbar = mapa_shared(recvbar, (uint32_t)r);
+                st_async_v4(mapa_shared(smem_u32(recv_o + (size_t)me * slice + 4 * f4 - r * slice), (uint32_t)r), o, rbar);
+                if (d == 0) {
+                    // a CTA that gave up says so with a NaN maximum: its peers then leave the output alone
+                    if (bad) mm = __int_as_float(0x7fc00000);
+                    for (int r2 = 0; r2 < S; ++r2)
+                        st_async_v2(mapa_shared(smem_u32(recv_ml + ((size_t)me * ncols + col) * 2), (uint32_t)r2), mm, ll,
+                                    mapa_shared(recvbar, (uint32_t)r2));
+                }
+            }
+            if (tid == 0) SEGKV_STAMP(14);
+            bool got = mbar_wait_cluster(recvbar, 0, p.wait_ns);
+            got = __all_sync(0xffffffffu, got);
+            if (tid == 0) SEGKV_STAMP(12);
+            if (!got && lane == 0) atomicOr(p.err_word, SEGKV_DEV_WAIT_LIMIT);
+            // fold: thread x takes partial s = x % S of float4 i = x / S of the slice; the S partials
+            // of one float4 sit in neighbouring lanes and are reduced with shuffles
+            const int l2s = 31 - __clz(S);
+            const int items = (slice >> 2) << l2s;
+            for (int x0 = 0; x0 < items && got; x0 += CT) {
+                const int x = x0 + tid;
+                const bool in = x < items;
+                const int i = in ? x >> l2s : 0, sp = in ? x & (S - 1) : 0;
+                const int fl = (int)me * slice + 4 * i;
+                const int col = fl / D, d = fl % D;
+                const float2 ml = in ? *reinterpret_cast<const float2*>(recv_ml + ((size_t)sp * ncols + col) * 2)
+                                     : make_float2(-INFINITY, 0.f);
+                float4 v = in ? *reinterpret_cast<const float4*>(recv_o + (size_t)sp * slice + 4 * i)
+                              : make_float4(0.f, 0.f, 0.f, 0.f);
+                float mm = ml.x;
+                bool poison = ml.x != ml.x;
+                for (int o = 1; o < S; o <<= 1) {
+                    mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
+                    poison = __shfl_xor_sync(0xffffffffu, (int)poison, o) != 0 || poison;
+                }
+                const float f = (ml.x == -INFINITY || poison) ? 0.f : exp2f(ml.x - mm);
+                float ll = ml.y * f;
+                v.x *= f; v.y *= f; v.z *= f; v.w *= f;
+                for (int o = 1; o < S; o <<= 1) {
+                    ll += __shfl_xor_sync(0xffffffffu, ll, o);
+                    v.x += __shfl_xor_sync(0xffffffffu, v.x, o);
+                    v.y += __shfl_xor_sync(0xffffffffu, v.y, o);
+                    v.z += __shfl_xor_sync(0xffffffffu, v.z, o);
+                    v.w += __shfl_xor_sync(0xffffffffu, v.w, o);
+                }
+                if (in && sp == 0 && !poison) {
+                    const float inv = 1.f / ll;
+                    const int j = col / p.G, hg = col % p.G;
+                    T* orow = reinterpret_cast<T*>(p.out) + ((size_t)(b * p.W + j) * p.H + kvh * p.G + hg) * D + d;
+                    uint2 pk;
+                    pk.x = Mma<T>::pack(v.x * inv, v.y * inv);
+                    pk.y = Mma<T>::pack(v.z * inv, v.w * inv);
+                    *reinterpret_cast<uint2*>(orow) = pk;
+                }
+            }
+            if (tid == 0) SEGKV_STAMP(13);
+        }
+        // the CTA leaves together: a producer warp that gave up first lets its copies in flight land
+        __syncthreads();
+        if (s_abort != 0) {
+            if (warp == TMA_WARP)
+                for (int k = max(0, tma_issued - stages); k < tma_issued; ++k)
+                    (void)mbar_wait(full0 + 8 * (k % stages), (uint32_t)(k / stages) & 1, p.wait_ns);
+            if (warp == GATHER_WARP) cp_async_wait_all();
+        }
+        return;
+    }
     __syncthreads();
     if (tid == 0) SEGKV_STAMP(10);
     const bool aborted = s_abort != 0;
@@ -821,52 +1091,6 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         *reinterpret_cast<uint2*>(orow) = pk;
     };
 
-    if (p.cluster) {
-        // ---- split merge inside the thread-block cluster, through distributed shared memory ----
-        // The (column, d) plane is cut into S equal slices; CTA r merges slice r.  Every CTA
-        // stores its part of slice r into CTA r's landing area, one cluster barrier later each
-        // CTA holds all S partials of its slice.
-        const uint32_t me = cluster_ctarank();
-        const int slice = ncols * D / S;                 // floats; a multiple of 4
-        cluster_wait_acquire();                          // every CTA of the cluster has started
-        if (!aborted) {
-            for (int it = tid; it < ncols * D4; it += NTHREADS) {
-                const int col = it / D4, d = (it % D4) * 4;
-                float mm, ll;
-                const float4 o = merged(col, d, mm, ll);
-                const int f = col * D + d;
-                const int r = f / slice;
-                st_cluster_v4(mapa_shared(smem_u32(recv_o + (size_t)me * slice + (f - r * slice)), (uint32_t)r), o);
-                if (d == 0)
-                    for (int r2 = 0; r2 < S; ++r2)
-                        st_cluster_v2(mapa_shared(smem_u32(recv_ml + ((size_t)me * ncols + col) * 2), (uint32_t)r2), mm, ll);
-            }
-        }
-        cluster_arrive_release();
-        cluster_wait_acquire();
-        if (tid == 0) SEGKV_STAMP(12);
-        if (aborted) return;
-        for (int i = tid; i < slice / 4; i += NTHREADS) {
-            const int f = (int)me * slice + 4 * i;
-            const int col = f / D, d = f % D;
-            float mm = -INFINITY;
-            for (int s = 0; s < S; ++s) mm = fmaxf(mm, recv_ml[((size_t)s * ncols + col) * 2]);
-            float ll = 0.f;
-            float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int s = 0; s < S; ++s) {
-                const float ms = recv_ml[((size_t)s * ncols + col) * 2];
-                const float fs = (ms == -INFINITY) ? 0.f : exp2f(ms - mm);
-                ll += recv_ml[((size_t)s * ncols + col) * 2 + 1] * fs;
-                const float4 v = *reinterpret_cast<const float4*>(recv_o + (size_t)s * slice + 4 * i);
-                o.x += v.x * fs; o.y += v.y * fs; o.z += v.z * fs; o.w += v.w * fs;
-            }
-            const float inv = 1.f / ll;
-            o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
-            store_out(col, d, o);
-        }
-        if (tid == 0) SEGKV_STAMP(13);
-        return;
-    }
     if (aborted) {
         // The work group's arrival counter must still come back to zero for the next launch: take the
         // ticket, marked, so that the last CTA to arrive skips the merge (the output stays untouched).
@@ -982,6 +1206,7 @@ cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk,
     if (p.quota < 1) p.quota = 1;
     p.cluster = a.cluster ? 1 : 0;
     p.early_prompt = (a.pdl && a.prompt_immutable) ? 1 : 0;
+    p.early_rows = (a.pdl && a.prompt_immutable && a.rows_immutable) ? 1 : 0;
     p.dbg_skip = a.dbg_skip ? 1 : 0;
     p.wait_ns = a.wait_ns ? a.wait_ns : kWaitLimitNs;
 #ifdef SEGKV_TIMELINE
@@ -1136,11 +1361,11 @@ cudaError_t launch_sdpa_tiled_static(const Dims& d, SdpaArgs a, const CUtensorMa
 
 #ifdef SEGKV_TIMELINE
 extern "C" __attribute__((visibility("default"))) int segkv_debug_timeline(unsigned long long* host, int clear) {
-    if (cudaMemcpyFromSymbol(host, segkv_impl::g_timeline, sizeof(unsigned long long) * 8 * 512 * 16) != cudaSuccess) return -1;
+    if (cudaMemcpyFromSymbol(host, segkv_impl::g_timeline, sizeof(unsigned long long) * 8 * 512 * 32) != cudaSuccess) return -1;
     if (clear) {
         void* p = nullptr;
         cudaGetSymbolAddress(&p, segkv_impl::g_timeline);
-        cudaMemset(p, 0, sizeof(unsigned long long) * 8 * 512 * 16);
+        cudaMemset(p, 0, sizeof(unsigned long long) * 8 * 512 * 32);
     }
     return 0;
 }

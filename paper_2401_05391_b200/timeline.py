@@ -1,8 +1,8 @@
 """Per-CTA time stamps of the decode attention kernel in a chain of back-to-back launches.
 
 The attention kernel can be compiled with time stamps (``-DSEGKV_TIMELINE``): every CTA records
-``%globaltimer`` at fixed points of its life into a device array that keeps the last eight
-launches.  This script builds that instrumented copy of the library
+``%globaltimer`` when it starts and the SM's cycle counter at fixed points of its life into a
+device array that keeps the last eight launches.  This script builds that instrumented copy of the library
 (``libsegkv_timeline.so``; the product library is not touched), replays a CUDA graph of one
 launch per layer over L distinct layer caches, as ``bench.py`` does, and prints for each of
 the last eight launches the median and the latest CTA of every stamp, in microseconds from the
@@ -27,7 +27,7 @@ import torch
 EVENTS = [(0, "start"), (3, "tma issued"), (2, "wait done"), (7, "tile 0 landed"), (6, "tile 0 used"), (4, "rows known"),
           (5, "copies issued"), (8, "prompt done"), (9, "resp done"), (10, "epilogue"), (11, "partial out"),
           (12, "ticket/barrier"), (13, "merged")]
-SLOTS, CTAS, WORDS = 8, 512, 16
+SLOTS, CTAS, WORDS = 8, 512, 32      # per CTA: 16 x %globaltimer (ns), then 16 x clock64 of the same stamps
 
 
 def main():
@@ -40,6 +40,7 @@ def main():
     ap.add_argument("--combine", type=int, default=0)
     ap.add_argument("--tile", type=int, default=0)
     ap.add_argument("--no-overlap", action="store_true")
+    ap.add_argument("--sm-mhz", type=int, default=1965, help="SM clock under load, to turn cycles into time")
     a = ap.parse_args()
 
     from . import build, segkv as sk, workloads as wl
@@ -90,19 +91,33 @@ def main():
     buf = np.zeros(SLOTS * CTAS * WORDS, dtype=np.uint64)
     assert lib.segkv_debug_timeline(buf.ctypes.data, 0) == 0
     n = min(CTAS, w.batch * w.kv_heads * layers[0][0].get_splits())
-    t = buf.reshape(SLOTS, CTAS, WORDS).astype(np.int64)[:, :n]
-    t = t[np.argsort(t[:, :, 0].min(axis=1))]            # the eight launch slots in time order
+    raw = buf.reshape(SLOTS, CTAS, WORDS).astype(np.int64)[:, :n]
+    raw = raw[np.argsort(raw[:, :, 0].min(axis=1))]      # the eight launch slots in time order
+    # Only the CTA start carries %globaltimer (reading it is slow and coarse); every stamp carries
+    # the SM's cycle counter, which is converted with the clock the GPU runs at under load.
+    mhz = a.sm_mhz
+    clk = raw[:, :, 16:]
+    t = np.where(clk > 0, raw[:, :, 0:1] + (clk - clk[:, :, 0:1]) * 1000 // mhz, 0)
     g0 = t[0, :, 0].min()
     print(f"{a.workload}: {n} CTAs per launch, splits {layers[0][0].get_splits()}, "
           f"{'fused step' if a.fused else 'attention only'}; median / latest CTA, us from the first CTA start")
-    print("launch | " + " | ".join(f"{name:>14s}" for _, name in EVENTS))
+    order = EVENTS + [(14, "remote stores"), (1, "consumer set up"), (15, "tile 0 scores")]
+    print("launch | " + " | ".join(f"{name:>14s}" for _, name in order))
     for li in range(SLOTS):
         cells = []
-        for ev, _ in EVENTS:
+        for ev, _ in order:
             x = t[li, :, ev]
             m = x > 0
             cells.append(f"{(np.median(x[m]) - g0) / 1e3:6.2f}/{(x[m].max() - g0) / 1e3:6.2f} " if m.any() else f"{'-':>14s}")
         print(f"{li:6d} | " + " | ".join(cells))
+    print("cycles from the CTA's own start, median over the CTAs of the last launch:")
+    c = clk[SLOTS - 1]
+    line = []
+    for ev, name in order:
+        m = (c[:, ev] > 0) & (c[:, 0] > 0)
+        if m.any():
+            line.append(f"{name} {int(np.median(c[m, ev] - c[m, 0]))}")
+    print("  " + " | ".join(line))
     starts = t[:, :, 0].min(axis=1)
     ends = np.where(t[:, :, 13] > 0, t[:, :, 13], t[:, :, 12]).max(axis=1)
     print("first CTA start to first CTA start, us:", np.round(np.diff(starts) / 1e3, 2))
