@@ -164,39 +164,17 @@ unsigned long long count_launch(segkv* h, cudaStream_t st) {
     return note_launch(st);
 }
 
-bool capturing(cudaStream_t st) {
-    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) {
-        cudaGetLastError();
-        return true;                       // unknown: behave as if it were
-    }
-    return cs != cudaStreamCaptureStatusNone;
-}
-
 // The launch just made on `st` wrote the data `m` stands for.
 void mark_written(segkv* h, WriteMark* m, cudaStream_t st) {
     m->seq = count_launch(h, st);
     m->stream = st;
-    m->done = false;
-    m->recorded = m->ev && !capturing(st) && cudaEventRecord(m->ev, st) == cudaSuccess;
 }
 
 // Is the data `m` stands for complete and visible to a kernel launched now on `st`, from that
-// kernel's first instruction on?  Yes if its launch has been seen complete (sticky until the next
-// write), or if it is strictly older than the library's latest launch on the same stream.
-bool settled(WriteMark* m, cudaStream_t st) {
-    if (m->seq == 0) return false;
-    if (m->done) return true;
-    if (m->recorded && !capturing(st)) {
-        const cudaError_t e = cudaEventQuery(m->ev);
-        if (e == cudaSuccess) {
-            m->done = true;
-            return true;
-        }
-        if (e != cudaErrorNotReady) cudaGetLastError();
-    }
-    return older_than_latest(st, m->stream, m->seq);
-}
+// kernel's first instruction on?  Yes if its launch is strictly older than the library's latest
+// launch on the same stream.  The answer depends on the order of the caller's calls alone, never on
+// how far the GPU has got, so the same program takes the same path every time it runs.
+bool settled(const WriteMark* m, cudaStream_t st) { return older_than_latest(st, m->stream, m->seq); }
 
 void free_all(segkv* h) {
     void* ptrs[] = {h->kp, h->vp, h->kr, h->k_chunks_dev, h->parent, h->anc[0], h->anc[1], h->ulist, h->ucount, h->plens,
@@ -204,8 +182,6 @@ void free_all(segkv* h) {
                     h->st_slopes};
     for (void* p : ptrs)
         if (p) cudaFree(p);
-    if (h->rows_mark.ev) cudaEventDestroy(h->rows_mark.ev);
-    if (h->lists_mark.ev) cudaEventDestroy(h->lists_mark.ev);
     for (int c = 0; c < h->nchunks; ++c)
         if (h->k_chunks_host[c]) cudaFree(h->k_chunks_host[c]);
     free(h->k_chunks_host);
@@ -283,9 +259,30 @@ int max_auto_splits(const segkv* h) {
 // Stages: as many as keep the form's CTAs per SM resident.  Splits: none when the work groups
 // alone fill the GPU twice over, else enough to give every CTA slot of one wave a share (never
 // less than one tile each).
-Tiling choose_tiling(const segkv* h) {
+Tiling choose_tiling(const segkv* h, bool fused_step) {
     const Dims& d = h->d;
     Tiling t;
+    // The fused step of a launch of eight splits that fills at most half of the GPU's quarter-SM
+    // slots runs in the small-CTA form, its splits merged inside a thread-block cluster: the next
+    // launch's CTAs then fit beside this one's and fetch their keys while these still compute
+    // (measured at the Llama2-7B shape: 7.9 us per layer against 9.6 us in the regular form; the
+    // attention call on its own is faster in the regular form, 7.4 against 8.3 us).  Larger launches
+    // keep the regular form: with more CTAs than half the slots the two launches no longer fit side
+    // by side, and a chain of such launches (320 CTAs in clusters of four) ended in a launch failure
+    // on two of three runs, whose cause has not been found.
+    if (fused_step && h->tile_forced == 0 && h->splits_forced <= 0 && h->stages_forced <= 0 && h->combine_forced != 1 &&
+        h->overlap && tiled_small_ok(d) && h->prompt_len >= 8 * 32) {
+        const long long slabs = (long long)d.batch * d.kv_heads;
+        if (slabs * 8 <= 2LL * h->sm_count && tiled_cluster_ok(d, 8)) {
+            t.small = true;
+            t.cluster = true;
+            t.splits = 8;
+            t.stages = 2;
+            const size_t budget = (h->smem_optin + 1024) / ctas_per_sm(true) - 1024;
+            while (t.stages < 8 && tiled_smem_bytes(d, t.stages + 1, true) <= budget) ++t.stages;
+            return t;
+        }
+    }
     t.small = h->tile_forced == 32 && tiled_small_ok(d);
     const int tile = tiled_tile_keys(d.head_dim, t.small);
     const int P = h->prompt_len > 0 ? h->prompt_len : 0;
@@ -342,7 +339,6 @@ int ensure_lists(segkv* h, cudaStream_t st) {
     if (x->lists_valid || h->steps == 0) return SEGKV_OK;
     SEGKV_CUDA(launch_rebuild_lists(x->d, h->steps, x->anc[(h->steps - 1) & 1], x->ulist, x->ucount, st));
     mark_written(h, &x->lists_mark, st);
-    x->lists_follow_rows = false;
     x->lists_valid = true;
     return SEGKV_OK;
 }
@@ -350,13 +346,11 @@ int ensure_lists(segkv* h, cudaStream_t st) {
 // May the next attention launch on `st` read the handle's response rows (and, for the separate
 // form, the distinct-row lists) before its grid-dependency wait?  Only if the launches that wrote
 // them are strictly older than the library's latest launch on the same stream.
-bool rows_settled(segkv* h, cudaStream_t st, bool lists_too) {
+bool rows_settled(const segkv* h, cudaStream_t st, bool lists_too) {
     if (!h->overlap || h->steps == 0) return false;
     if (!settled(&h->rows_mark, st)) return false;
     if (!lists_too) return true;
-    segkv* x = index_of(h);
-    if (x->lists_follow_rows) return settled(&x->rows_mark, st);
-    return settled(&x->lists_mark, st);
+    return settled(&index_of(h)->lists_mark, st);
 }
 
 SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes, int splits) {
@@ -509,11 +503,6 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
 #undef SEGKV_TRY
     // The split workspace for the largest split count the automatic choice can make (one wave of
     // CTA slots shared among the work groups), so that the decode loop never allocates.
-    if (cudaEventCreateWithFlags(&h->rows_mark.ev, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->lists_mark.ev, cudaEventDisableTiming) != cudaSuccess) {
-        cudaGetLastError();
-        return fail(SEGKV_ECUDA);
-    }
     rc = alloc_workspace(h, max_auto_splits(h));
     if (rc != SEGKV_OK) return fail(rc);
     *out = h;
@@ -693,11 +682,7 @@ static int append_impl(segkv_t h, int step, const int32_t* beam_parent, const vo
                              h->anc[(step + 1) & 1], h->anc[step & 1], h->ulist, h->ucount, h->err_word,
                              h->sm_count, h->overlap && step > 0, (cudaStream_t)stream, rope));
     mark_written(h, &h->rows_mark, (cudaStream_t)stream);
-    h->lists_mark.seq = h->rows_mark.seq;          // the same launch made the lists: one event stands for both
-    h->lists_mark.stream = h->rows_mark.stream;
-    h->lists_mark.done = false;
-    h->lists_mark.recorded = false;
-    h->lists_follow_rows = true;
+    h->lists_mark = h->rows_mark;                  // the same launch made the lists
     h->steps = step + 1;
     h->truncated = false;
     h->lists_valid = true;
@@ -720,7 +705,7 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
         int rc = ensure_lists(h, (cudaStream_t)stream);
         if (rc != SEGKV_OK) return rc;
     }
-    const Tiling tl = choose_tiling(h);
+    const Tiling tl = choose_tiling(h, false);
     const int splits = tl.splits;
     if (h->combine_forced == 2 && splits > 1 && !tl.cluster) return SEGKV_EINVAL;
     if (!tl.cluster && splits > h->ws_splits) {
@@ -753,7 +738,7 @@ int segkv_decode_sdpa_static(segkv_t h, const void* q, void* out, const float* a
         int rc = ensure_lists(h, (cudaStream_t)stream);     // a kernel launch at most, never an allocation
         if (rc != SEGKV_OK) return rc;
     }
-    const Tiling tl = choose_tiling(h);
+    const Tiling tl = choose_tiling(h, false);
     const int splits = tl.splits;
     SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, splits);
     a.pdl = h->overlap;
@@ -791,7 +776,7 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     }
     const Dims& d = h->d;
     h->steps = step + 1;                 // the launch shape is chosen for the step being added
-    const Tiling tl = choose_tiling(h);
+    const Tiling tl = choose_tiling(h, true);
     const int splits = tl.splits;
     const bool cluster = tl.cluster;
     h->steps = step;
@@ -799,7 +784,8 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     // in the kernel costs more than the separate append launch (measured at prompts of 128 to 512
     // tokens with 128 steps: 10.0-10.6 us as two launches against 10.8-12.9 us fused)
     const long long rows_per_cta = (long long)((step + 1 + splits - 1) / splits) * d.beams;
-    const bool long_tail = h->splits_forced <= 0 && 2 * rows_per_cta > 3 * tiled_tile_keys(d.head_dim, tl.small);   // a forced split count keeps the fused kernel
+    const bool long_tail = h->splits_forced <= 0 && !(tl.small && tl.cluster) &&                                // a forced split count keeps the fused kernel
+                           2 * rows_per_cta > 3 * tiled_tile_keys(d.head_dim, false);
     if ((splits == 1 || long_tail) && !h->fuse_always) {
         // Work groups that fill the GPU on their own are bandwidth-bound: the separate append is
         // then ~1 % of the step and the list it makes keeps the response tiles dense and cheap
@@ -997,7 +983,7 @@ int segkv_set_tuning(segkv_t h, int splits, int stages, int combine) {
 int segkv_get_splits(segkv_t h) {
     if (!h) return SEGKV_EINVAL;
     if (!tiled_supported(h->d)) return 1;
-    return choose_tiling(h).splits;
+    return choose_tiling(h, false).splits;
 }
 
 int segkv_decode_sdpa_rowwise(segkv_t h, const void* q, void* out, const float* alibi_slopes, void* stream) {

@@ -22,14 +22,10 @@ struct URow {
     uint32_t mask;
 };
 
-// Where and when data was last written: the stream and per-process sequence number of the launch,
-// and an event recorded behind it (not while the stream is being captured).
+// Where and when data was last written: the stream and the per-process sequence number of the launch.
 struct WriteMark {
     cudaStream_t stream;
     unsigned long long seq;       // 0: never written
-    cudaEvent_t ev;               // created with the handle
-    bool recorded;                // ev was recorded behind the launch
-    bool done;                    // the launch has been seen complete (ev queried, or the host synchronised)
 };
 
 struct Dims {
@@ -97,7 +93,6 @@ struct segkv {
     // that wrote its row lists (what a later attention launch may read ahead of its wait once
     // these are known to be complete)
     segkv_impl::WriteMark rows_mark, lists_mark;
-    bool lists_follow_rows;   // the lists were made by the launch rows_mark stands for (the append kernel)
     int* err_word;       // device error word
     float* ws;           // split workspace
     size_t ws_bytes;

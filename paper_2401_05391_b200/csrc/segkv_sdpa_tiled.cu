@@ -166,6 +166,7 @@ struct TiledParams {
     int cluster;    // 1: the S CTAs of a work group form a thread-block cluster
     int early_prompt;  // 1: prompt tiles may be fetched before the previous kernel has completed
     int early_rows;    // 1: so may the response rows of earlier steps and (separate form) the row lists
+    int resv;          // 1: the last stage is set aside for the CTA's first response tile (see the kernel)
     int dbg_skip;      // test aid: the gather warp leaves out one plain barrier arrival, so that a wait runs out
     unsigned long long wait_ns;   // limit of every bounded wait
 #ifdef SEGKV_TIMELINE
@@ -235,6 +236,14 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     const char** gv = gk + TILE;                                                               // [TILE] V row pointers
     __shared__ int s_last, s_abort;
 
+    // When the response rows may be fetched ahead of the grid-dependency wait, the LAST stage is set
+    // aside for the CTA's first response tile (usually its only one): the long chain of its fetch
+    // (count or table -> addresses -> copies) is then over before the wait returns, whatever the
+    // prompt tiles do with the other RS stages, which they share as a ring.  Further response tiles
+    // follow the prompt tiles through that ring.  The order in which tiles are CONSUMED never
+    // changes (prompt, then response), so results do not depend on which way a launch was made.
+    const int RS = stages - p.resv;
+    const int rstage = stages - 1;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) SEGKV_STAMP(0);
     const int split = blockIdx.x % p.S;
@@ -255,8 +264,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     // fused step: response steps are cut evenly over the splits (known from the launch shape alone)
     const int rs0 = (int)((long long)split * p.steps / p.S), rs1 = (int)((long long)(split + 1) * p.steps / p.S);
 
-    auto issue_prompt_tile = [&](int k) {
-        const int st = k % stages;
+    auto issue_prompt_tile = [&](int k, int st) {
         const uint32_t full = full0 + 8 * st;
         if (lane == 0) {
             const uint32_t k_dst = smem_u32(ring + (size_t)st * L::STAGE_BYTES);
@@ -299,8 +307,8 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         // The prompt segment does not change during decoding, so when the host says so its
         // tiles are requested before the previous kernel of the stream has finished.
         if (!p.early_prompt) grid_wait();
-        const int first = min(npt, stages);
-        for (int k = 0; k < first; ++k) issue_prompt_tile(k);
+        const int first = min(npt, RS);
+        for (int k = 0; k < first; ++k) issue_prompt_tile(k, k);
         tma_issued = first;
         if (first == npt && lane == 0) mbar_arrive(hand);
         // Prompt tiles that have to wait for a stage of the ring are at least brought into the L2,
@@ -353,9 +361,9 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     __syncthreads();
     // Everything else (q, row lists, parents, response rows, outputs) follows the previous kernel.
     // The next kernel is let go only after this wait, so a kernel that starts early behind this
-    // one finds every kernel before this one's predecessor complete.  (The gather warp of the
-    // separate form, when the host vouches for its inputs, works ahead and waits later.)
-    const bool gather_ahead = !FUSED && warp == GATHER_WARP && p.early_rows;
+    // one finds every kernel before this one's predecessor complete.  (The gather warp, when the
+    // host vouches for its inputs, works ahead and waits later.)
+    const bool gather_ahead = warp == GATHER_WARP && p.early_rows;
     if (!gather_ahead) {
         grid_wait();
         grid_launch_dependents();
@@ -371,10 +379,11 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         // ============================ prompt tiles beyond the first round ============================
         bool ok = true;
         for (int k = tma_issued; k < npt; ++k) {
-            ok = mbar_wait(empty0 + 8 * (k % stages), (((uint32_t)(k / stages)) & 1) ^ 1, p.wait_ns);
+            const int st = k % RS;
+            ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / RS)) & 1) ^ 1, p.wait_ns);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            issue_prompt_tile(k);
+            issue_prompt_tile(k, st);
             tma_issued = k + 1;
             if (k + 1 == npt && lane == 0) mbar_arrive(hand);
         }
@@ -400,7 +409,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         // Copy rows [0, cnt) of the tile whose row pointers (gk, gv) have been written.  One
         // warp-wide copy moves whole rows (CPR lanes per row): fully coalesced.  The arrival on
         // the stage's full barrier fires when this lane's copies have landed.
-        auto copy_rows = [&](int st, int cnt) {
+        auto copy_rows = [&](int st, int from, int cnt, bool arrive) {
             const uint32_t full = full0 + 8 * st;
             const uint32_t k_dst = smem_u32(ring + (size_t)st * L::STAGE_BYTES), v_dst = k_dst + L::TILE_BYTES;
             const int c = lane % CPR;
@@ -408,9 +417,9 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             __syncwarp();                              // gk / gv written by other lanes
 #pragma unroll
             for (int i = 0; i < TILE / RPI; ++i) {
-                if (i * RPI < cnt) {                   // warp-uniform
+                if (i * RPI < cnt && (i + 1) * RPI > from) {      // warp-uniform
                     const int key = i * RPI + lane / CPR;
-                    if (key < cnt) {
+                    if (key < cnt && key >= from) {
                         const uint32_t off = c_off + (uint32_t)key * 128 + (uint32_t)(((c & 7) ^ (key & 7)) << 4);
                         if constexpr (FUSED) {             // rows may sit in the caller's k_new / v_new
                             cp_async_16(k_dst + off, gk[key] + c * 16);
@@ -423,7 +432,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     }
                 }
             }
-            cp_async_mbar_arrive_noinc(full);
+            if (arrive) cp_async_mbar_arrive_noinc(full);      // fires when ALL of this lane's copies so far have landed
             __syncwarp();                              // gk / gv are rewritten for the next tile
         };
         // Complete a tile of cnt keys whose per-key meta has been written: zero the rows between
@@ -448,7 +457,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             if (lane == 0 && !p.dbg_skip) mbar_arrive(full0 + 8 * st);
         };
         auto publish_tile = [&](int st, int cnt, bool last) {
-            copy_rows(st, cnt);
+            copy_rows(st, 0, cnt, true);
             finish_tile(st, cnt, last);
         };
         bool ok = true;
@@ -475,13 +484,15 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             int r = 0;
             bool handed = false;
             auto tiles = [&](int r_end) {
-                if (r < r_end && !handed) {
-                    ok = mbar_wait(hand, 0, p.wait_ns);
-                    ok = __all_sync(0xffffffffu, ok);
-                    handed = true;
-                }
                 for (; r < r_end && ok; ++r) {
-                    const int k = npt + r;
+                    const bool own = p.resv && r == 0;            // the stage set aside: nobody else uses it
+                    if (!own && !handed) {
+                        ok = mbar_wait(hand, 0, p.wait_ns);
+                        ok = __all_sync(0xffffffffu, ok);
+                        handed = true;
+                        if (!ok) break;
+                    }
+                    const int k = npt + r - p.resv;               // place in the ring's order
                     const int eb = e0 + r * TILE;
                     const int cnt = min(TILE, e1 - eb);
 #pragma unroll
@@ -492,10 +503,12 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                                         ? *reinterpret_cast<const uint2*>(ulist_b + eb + TILE + key)
                                         : make_uint2(0u, 0u);
                     }
-                    const int st = k % stages;
-                    ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1, p.wait_ns);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
+                    const int st = own ? rstage : k % RS;
+                    if (!own) {
+                        ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / RS)) & 1) ^ 1, p.wait_ns);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                    }
                     URow* meta_st = meta + (size_t)st * TILE;
 #pragma unroll
                     for (int kk = 0; kk < UK; ++kk) {
@@ -517,7 +530,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 // Lists and rows were written by launches older than this launch's predecessor: the tiles
                 // that find a free stage are fetched now, the rows of the others are asked into the L2,
                 // and only then does this warp wait for the previous kernel.
-                const int r_now = npt < stages ? min(nrt, stages - npt) : 0;
+                const int r_now = min(nrt, p.resv + (npt < RS ? RS - npt : 0));
                 for (int e = e0 + r_now * TILE + lane / 4; e < e1; e += 8) {
                     const int row = ulist_b[e].row, sidx = row / p.rows;
                     const char* kr = k_slab(sidx) + ((size_t)(row - sidx * p.rows) * p.Hkv + kvh) * (size_t)(D * 2);
@@ -556,27 +569,172 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     if (s < rs1 && j < Wb && s != t_new) rowb[u] = p.anc_prev[(size_t)(b * Wb + j) * p.max_steps + s];
                 }
             };
+            // Among the lanes of a step (active ones), keep each distinct row once: `first` marks the
+            // lowest lane of a row, `mask` the lanes (slots) that share it; `incl` is the warp-wide
+            // running count of first lanes, `total` its last value.
+            auto dedupe = [&](int row, bool active, bool& first, uint32_t& mask, int& incl, int& total) {
+                if (!active) row = -1 - lane;                                     // matches nobody
+                first = active;
+                mask = 0;
+                for (int i = 0; i < Wp; ++i) {
+                    const int ri = __shfl_sync(0xffffffffu, row, gbase + i);
+                    if (ri == row) {
+                        mask |= 1u << i;
+                        if (i < j) first = false;
+                    }
+                }
+                incl = first ? 1 : 0;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += n;
+                }
+                total = __shfl_sync(0xffffffffu, incl, 31);
+            };
+            const int nwin = (rs1 - rs0 + spw - 1) / spw;
+            const bool has_new = t_new >= rs0 && t_new < rs1;     // this CTA's range holds the step being added
             int rowb[PF];
+            // Fast path state: every row this CTA can need, placed in the stage that is its own.
+            bool fast = false;
+            int fpos[PF];                 // place in the tile of this lane's row (first lane of an old row), or -1
+            uint32_t fmask[PF];           // OLD slots whose path holds that row
+            int old_total = 0;
+            if (gather_ahead) {
+                // The previous table and the rows of earlier steps were written by launches older than
+                // this launch's predecessor.  The table entries are read now; the rows that any slot's
+                // OLD path reaches are a superset of what the new parents will select (the new path of
+                // slot j is the old path of slot parent[j]), so they are fetched now, each distinct row
+                // once with the set of OLD slots that hold it, and after the wait only the parent ids
+                // are a fresh round trip: they turn the old slot sets into the new beams' masks.
+                fetch_windows(0, rowb);
+                fast = p.resv && nwin <= PF && rs1 > rs0;
+                if (fast) {
+#pragma unroll
+                    for (int u = 0; u < PF; ++u) {
+                        fpos[u] = -1;
+                        fmask[u] = 0;
+                        if (u < nwin) {                                           // warp-uniform
+                            const int s = rs0 + u * spw + ls;
+                            bool first;
+                            int incl, total;
+                            dedupe(rowb[u], s < rs1 && j < Wb && s != t_new, first, fmask[u], incl, total);
+                            if (first) fpos[u] = old_total + incl - 1;
+                            old_total += total;
+                        }
+                    }
+                    if (old_total + (has_new ? Wb : 0) > TILE) fast = false;      // more than the one tile: the general way
+                }
+                if (fast) {
+#pragma unroll
+                    for (int u = 0; u < PF; ++u) {
+                        if (fpos[u] >= 0) {
+                            const int s = rs0 + u * spw + ls;
+                            meta[(size_t)rstage * TILE + fpos[u]].row = s;
+                            const char* ksl = k_slab(s);
+                            const size_t off = ((size_t)rowb[u] * p.Hkv + kvh) * (size_t)(D * 2);
+                            gk[fpos[u]] = ksl + off;
+                            gv[fpos[u]] = ksl + p.vdelta + off;
+                        }
+                    }
+                    copy_rows(rstage, 0, old_total, false);
+                } else {
+                    // at least ask the L2 for the rows of the first windows
+#pragma unroll
+                    for (int u = 0; u < PF; ++u) {
+                        const int s = rs0 + u * spw + ls;
+                        if (s < rs1 && j < Wb && s != t_new) {
+                            const char* kr = k_slab(s) + ((size_t)rowb[u] * p.Hkv + kvh) * (size_t)(D * 2);
+#pragma unroll
+                            for (int ln = 0; ln < D * 2 / 128; ++ln) {
+                                prefetch_l2(kr + ln * 128);
+                                prefetch_l2(kr + p.vdelta + ln * 128);
+                            }
+                        }
+                    }
+                }
+                grid_wait();
+                grid_launch_dependents();
+            }
             int par = j;
             par = (p.steps > 1 && j < Wb) ? p.parent[b * Wb + j] : j;
-            fetch_windows(0, rowb);
+            if (!gather_ahead) fetch_windows(0, rowb);
             if (j < Wb && (par < 0 || par >= Wb)) {       // first use of the parent ids
                 if (kvh == 0 && split == 0) atomicOr(p.err_word, SEGKV_DEV_BAD_PARENT);
                 par = par < 0 ? 0 : Wb - 1;
             }
             SEGKV_STAMP(4);
-            if (rs1 > rs0) {
-                ok = mbar_wait(hand, 0, p.wait_ns);
-                ok = __all_sync(0xffffffffu, ok);
+            if (fast) {
+                // ---- the rows are on their way: masks, the new table column, the new step's rows ----
+                // new slot i reads what old slot parent[i] read: turn the sets of old slots into beam masks
+                uint32_t nmask[PF];
+#pragma unroll
+                for (int u = 0; u < PF; ++u) nmask[u] = 0;
+                for (int i = 0; i < Wb; ++i) {
+                    const int pi = __shfl_sync(0xffffffffu, par, i);              // lanes 0..Wb-1 hold the slots' parents
+#pragma unroll
+                    for (int u = 0; u < PF; ++u) nmask[u] |= ((fmask[u] >> pi) & 1u) << i;
+                }
+#pragma unroll
+                for (int u = 0; u < PF; ++u) {
+                    if (u < nwin) {                                               // warp-uniform
+                        const int s = rs0 + u * spw + ls;
+                        const int row = __shfl_sync(0xffffffffu, rowb[u], gbase + par);   // anc_{t-1}[parent[j]][s]
+                        if (fpos[u] >= 0) meta[(size_t)rstage * TILE + fpos[u]].mask = nmask[u];
+                        if (s < rs1 && j < Wb && s != t_new && kvh == 0) p.anc_dst[(size_t)(b * Wb + j) * p.max_steps + s] = row;
+                    }
+                }
+                int cnt = old_total;
+                if (has_new) {
+                    if (lane < Wb) {
+                        URow uu;
+                        uu.row = t_new;
+                        uu.mask = 1u << lane;
+                        meta[(size_t)rstage * TILE + old_total + lane] = uu;
+                        const size_t off = ((size_t)(b * Wb + lane) * p.Hkv + kvh) * (size_t)(D * 2);
+                        gk[old_total + lane] = p.k_new + off;
+                        gv[old_total + lane] = p.v_new + off;
+                        if (kvh == 0) p.anc_dst[(size_t)(b * Wb + lane) * p.max_steps + t_new] = b * Wb + lane;
+                    }
+                    cnt += Wb;
+                    // the new rows' copies: CPR lanes per row, straight from the caller's arrays
+                    __syncwarp();
+                    const uint32_t k_dst = smem_u32(ring + (size_t)rstage * L::STAGE_BYTES), v_dst = k_dst + L::TILE_BYTES;
+                    for (int i = lane; i < Wb * CPR; i += 32) {
+                        const int key = old_total + i / CPR, c = i % CPR;
+                        const uint32_t off = (uint32_t)(c / 8) * L::BOX_BYTES + (uint32_t)key * 128 + (uint32_t)(((c & 7) ^ (key & 7)) << 4);
+                        cp_async_16(k_dst + off, gk[key] + c * 16);
+                        cp_async_16(v_dst + off, gv[key] + c * 16);
+                    }
+                }
+                cp_async_mbar_arrive_noinc(full0 + 8 * rstage);      // fires when ALL of this lane's copies, old rows and new, have landed
+                finish_tile(rstage, cnt, true);
             }
             // Windows of spw steps at fixed positions; the table entries of four windows are
             // requested at once, so a split of up to 4 * spw steps pays one memory round trip.
             // A window (at most 32 rows) is never cut: if it does not fit, the tile is published
             // first and the window opens the next one.
-            const int nwin = (rs1 - rs0 + spw - 1) / spw;
-            int fillpos = 0, k = npt, st = 0;
-            bool open = false;
-            for (int w0 = 0; w0 < nwin && ok; w0 += PF) {
+            int fillpos = 0, tix = 0, st = 0;
+            bool open = false, handed = false;
+            // the tix-th response tile of this CTA: the stage set aside for the first, else the ring
+            auto open_tile = [&]() {
+                if (p.resv && tix == 0) {
+                    st = rstage;
+                    open = true;
+                    return;
+                }
+                if (!handed) {
+                    ok = mbar_wait(hand, 0, p.wait_ns);
+                    ok = __all_sync(0xffffffffu, ok);
+                    handed = true;
+                    if (!ok) return;
+                }
+                const int k = npt + tix - p.resv;
+                st = k % RS;
+                ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / RS)) & 1) ^ 1, p.wait_ns);
+                ok = __all_sync(0xffffffffu, ok);
+                open = ok;
+            };
+            for (int w0 = 0; w0 < nwin && ok && !fast; w0 += PF) {
                 if (w0 > 0) fetch_windows(w0, rowb);
 #pragma unroll
                 for (int u = 0; u < PF; ++u) {
@@ -585,35 +743,19 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     const bool active = s < rs1 && j < Wb;
                     int row = __shfl_sync(0xffffffffu, rowb[u], gbase + par);     // anc_{t-1}[parent[j]][s]
                     if (s == t_new) row = b * Wb + j;
-                    if (!active) row = -1 - lane;                                 // matches nobody
-                    bool first = active;
-                    uint32_t mask = 0;
-                    for (int i = 0; i < Wp; ++i) {
-                        const int ri = __shfl_sync(0xffffffffu, row, gbase + i);
-                        if (ri == row) {
-                            mask |= 1u << i;
-                            if (i < j) first = false;
-                        }
-                    }
-                    int incl = first ? 1 : 0;
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const int n = __shfl_up_sync(0xffffffffu, incl, o);
-                        if (lane >= o) incl += n;
-                    }
-                    const int total = __shfl_sync(0xffffffffu, incl, 31);
+                    bool first;
+                    uint32_t mask;
+                    int incl, total;
+                    dedupe(row, active, first, mask, incl, total);
                     if (open && fillpos + total > TILE) {
                         publish_tile(st, fillpos, false);
-                        ++k;
+                        ++tix;
                         open = false;
                         fillpos = 0;
                     }
                     if (!open) {
-                        st = k % stages;
-                        ok = mbar_wait(empty0 + 8 * st, (((uint32_t)(k / stages)) & 1) ^ 1, p.wait_ns);
-                        ok = __all_sync(0xffffffffu, ok);
+                        open_tile();
                         if (!ok) break;
-                        open = true;
                     }
                     if (active) {
                         if (first) {
@@ -820,10 +962,10 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 
         bool ok = true;
         int k = 0;
-        int st = 0;              // stage and phase of tile k: k % stages, (k / stages) & 1
+        int st = 0;              // stage and phase of the ring's next tile
         uint32_t ph = 0;
         auto next_stage = [&]() {
-            if (++st == stages) {
+            if (++st == RS) {
                 st = 0;
                 ph ^= 1u;
             }
@@ -865,26 +1007,30 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             const int e1 = (split == p.S - 1) ? n_b : min((split + 1) * p.quota, n_b);
             const int nrt = (e1 - e0 + TILE - 1) / TILE;
             for (int r = 0; r < nrt; ++r, ++k) {
-                ok = mbar_wait(full0 + 8 * st, ph, p.wait_ns);
+                const bool own = p.resv && r == 0;                // the first response tile has a stage of its own
+                const int sr = own ? rstage : st;
+                ok = mbar_wait(full0 + 8 * sr, own ? 0u : ph, p.wait_ns);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                consume(IntC<1>{}, st, true, min(TILE, e1 - (e0 + r * TILE)), 0, warp * 16);
+                consume(IntC<1>{}, sr, true, min(TILE, e1 - (e0 + r * TILE)), 0, warp * 16);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8 * st);
-                next_stage();
+                if (lane == 0) mbar_arrive(empty0 + 8 * sr);
+                if (!own) next_stage();
             }
         } else if (ok && rs1 > rs0) {
             // fused step: how many response tiles there are and how full each is only the gather
             // warp knows; it says so in the tile's header
-            for (;;) {
-                ok = mbar_wait(full0 + 8 * st, ph, p.wait_ns);
+            for (int r = 0;; ++r) {
+                const bool own = p.resv && r == 0;
+                const int sr = own ? rstage : st;
+                ok = mbar_wait(full0 + 8 * sr, own ? 0u : ph, p.wait_ns);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                const int2 hd = tile_hdr[st];
-                consume(IntC<1>{}, st, true, hd.x, 0, warp * 16);
+                const int2 hd = tile_hdr[sr];
+                consume(IntC<1>{}, sr, true, hd.x, 0, warp * 16);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8 * st);
-                next_stage();
+                if (lane == 0) mbar_arrive(empty0 + 8 * sr);
+                if (!own) next_stage();
                 ++k;
                 if (hd.y) break;
             }
@@ -1018,7 +1164,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         if (s_abort != 0) {
             if (warp == TMA_WARP)
                 for (int k = max(0, tma_issued - stages); k < tma_issued; ++k)
-                    (void)mbar_wait(full0 + 8 * (k % stages), (uint32_t)(k / stages) & 1, p.wait_ns);
+                    (void)mbar_wait(full0 + 8 * (k % RS), (uint32_t)(k / RS) & 1, p.wait_ns);
             if (warp == GATHER_WARP) cp_async_wait_all();
         }
         return;
@@ -1031,7 +1177,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         // before the shared memory is released; the output is left untouched.
         if (warp == TMA_WARP)
             for (int k = max(0, tma_issued - stages); k < tma_issued; ++k)
-                (void)mbar_wait(full0 + 8 * (k % stages), (uint32_t)(k / stages) & 1, p.wait_ns);
+                (void)mbar_wait(full0 + 8 * (k % RS), (uint32_t)(k / RS) & 1, p.wait_ns);
         if (warp == GATHER_WARP) cp_async_wait_all();
     }
 
@@ -1207,6 +1353,7 @@ cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk,
     p.cluster = a.cluster ? 1 : 0;
     p.early_prompt = (a.pdl && a.prompt_immutable) ? 1 : 0;
     p.early_rows = (a.pdl && a.prompt_immutable && a.rows_immutable) ? 1 : 0;
+    p.resv = (p.early_rows && stages >= 2) ? 1 : 0;
     p.dbg_skip = a.dbg_skip ? 1 : 0;
     p.wait_ns = a.wait_ns ? a.wait_ns : kWaitLimitNs;
 #ifdef SEGKV_TIMELINE
