@@ -7,9 +7,12 @@ K/V rows, updates the beam-index table and runs the decode attention in one laun
 cache handles, so a step touches L x (unique KV bytes) of HBM, far more than
 the L2 holds, and every timed kernel reads cold data.
 
-Printed: ONE JSON line (see README / DESIGN).  `value` is the whole-job
-unique-KV bandwidth in GB/s: the K/V bytes the method has to read (prompt rows
-once per request, every DISTINCT response row once) divided by the step time.
+Printed: ONE JSON line.  `value` is the whole-job unique-KV bandwidth in GB/s: the K/V
+bytes the method has to read (prompt rows once per request, every DISTINCT response
+row once) divided by the step time.  Every timed step has its own pair of CUDA events,
+so the line also carries the median, 10th and 90th percentile of the step time; the
+other evaluation shapes are timed the same way and reported under `other_workloads`.
+`--curve` prints the step time at every decode step of the workload instead.
 
 `--impl reference` times the CPU float64 oracle on the host cores instead.
 """
@@ -61,6 +64,8 @@ def parse():
     ap.add_argument("--no-overlap", action="store_true", help="turn programmatic dependent launch off")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="skip the other evaluation shapes (other_workloads)")
+    ap.add_argument("--curve", action="store_true", help="time the fused step at every decode step 1..N of the workload")
     return ap.parse_args()
 
 
@@ -203,12 +208,173 @@ def run_reference(args):
 
 
 # --------------------------------------------------------------------------- ours
+def percentiles(xs):
+    xs = sorted(xs)
+    n = len(xs)
+    pick = lambda f: xs[min(n - 1, max(0, int(round(f * (n - 1)))))]
+    return {"median": statistics.median(xs), "p10": pick(0.10), "p90": pick(0.90), "n": n}
+
+
+class ShapeBench:
+    """L layer caches of one shape, filled up to decode step T, and timed passes over them."""
+
+    def __init__(self, w, L, T, args, rank, world, dev):
+        import torch
+        from paper_2401_05391_b200 import sharding
+        from paper_2401_05391_b200 import workloads as wl
+        from paper_2401_05391_b200.segkv import SegKV
+        self.torch, self.wl, self.sharding = torch, wl, sharding
+        self.w, self.L, self.T, self.t = w, L, T, T - 1
+        self.args, self.rank, self.world, self.dev = args, rank, world, dev
+        # every rank holds its own requests (weak scaling: requests are independent, no exchange)
+        w_rank = sharding.rank_workload(w, rank, world)
+        self.parents = torch.from_numpy(wl.make_parents(w_rank)).to(dev)
+        self.slopes = wl.alibi_slopes(w.heads).to(dev) if w.alibi else None
+        self.handles = []
+        for layer in range(L):
+            wl_layer = w_rank.scaled(index=w_rank.index + 1000 * layer)
+            h = SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, w.steps, w.torch_dtype)
+            if args.tile:
+                h.set_tile(args.tile)
+            if args.splits or args.stages or args.combine:
+                h.set_tuning(args.splits, args.stages, args.combine)
+            if args.no_overlap:
+                h.set_overlap(False)
+            if args.prompt_layout != "head_major":
+                h.set_prompt_layout(args.prompt_layout)
+            kp, vp = wl.make_prompt(wl_layer, dev)
+            h.prefill_write(kp, vp)
+            del kp, vp
+            q = k = v = None
+            for s in range(T):
+                q, k, v = wl.make_step(wl_layer, s, dev)
+                h.append(s, self.parents[s] if s > 0 else None, k, v)
+            self.handles.append([h, q, k, v, torch.empty_like(q), wl_layer])
+        torch.cuda.synchronize()
+        self.stream = torch.cuda.Stream()
+        self.refresh_bytes()
+
+    def refresh_bytes(self):
+        w = self.w
+        uniq_rows = int(self.handles[0][0].get_unique_rows().sum())
+        self.ubytes = unique_bytes(w, w.prompt_len, uniq_rows)
+        self.logical_bytes = w.rows * (w.prompt_len + self.T) * 2 * w.kv_heads * w.head_dim * 2
+
+    def close(self):
+        for h in self.handles:
+            h[0].destroy()
+        self.handles = []
+
+    def layer_pass(self, mode: str):
+        # "step": the whole hot path in the library's fused call; "two": the same as two calls
+        # (append, then attention); "sdpa": the attention kernel alone on the state already there
+        t, stream, slopes = self.t, self.stream, self.slopes
+        par_t = self.parents[t] if t > 0 else None
+        for h, q, k, v, out, _ in self.handles:
+            if mode == "step":
+                h.truncate_last()
+                h.decode_step(t, par_t, k, v, q, out, slopes, stream=stream)
+            elif mode == "two":
+                h.truncate_last()
+                h.append(t, par_t, k, v, stream=stream)
+                h.decode_sdpa(q, out, slopes, stream=stream)
+            elif mode == "sdpa":
+                h.decode_sdpa(q, out, slopes, stream=stream)
+        if mode == "hot":
+            # the attention kernel on ONE layer's cache over and over: L2-resident where the layer fits
+            # (the Llama2-7B shape does), i.e. the kernel's latency floor without HBM
+            h, q, k, v, out, _ = self.handles[0]
+            for _ in range(len(self.handles)):
+                h.decode_sdpa(q, out, slopes, stream=stream)
+
+    def make_runner(self, mode: str):
+        torch, stream = self.torch, self.stream
+        with torch.cuda.stream(stream):
+            self.layer_pass(mode)                            # lazy initialisation outside any capture
+        stream.synchronize()
+        if self.args.no_graph:
+            return (lambda: self.layer_pass(mode)), False
+        g = torch.cuda.CUDAGraph()
+        try:
+            with torch.cuda.graph(g, stream=stream):
+                self.layer_pass(mode)
+        except Exception as e:                               # report, never hide
+            sys.stderr.write(f"[bench] CUDA graph capture failed ({e}); timing direct launches\n")
+            return (lambda: self.layer_pass(mode)), False
+
+        def replay():
+            with torch.cuda.stream(stream):
+                g.replay()
+        return replay, True
+
+    def timed(self, run, steps, warmup):
+        """K steps between two events (total, max over ranks) and every step between its own pair."""
+        torch, stream, dist = self.torch, self.stream, self.torch.distributed
+        for _ in range(warmup):
+            run()
+        stream.synchronize()
+        if self.world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        ev[0].record(stream)
+        for i in range(steps):
+            run()
+            ev[i + 1].record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        ms = self.sharding.max_over_ranks(ev[0].elapsed_time(ev[steps]), self.dev)
+        per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+        if self.world > 1:
+            dist.barrier()
+        return ms, per
+
+    def launches_per_step(self):
+        l0 = sum(h[0].launch_count for h in self.handles)
+        with self.torch.cuda.stream(self.stream):
+            self.layer_pass("step")
+        self.stream.synchronize()
+        return sum(h[0].launch_count for h in self.handles) - l0      # counted by the library
+
+
+def run_curve(args):
+    """The fused step at every decode step 1..N of the workload (one JSON line with the arrays)."""
+    import torch
+    from paper_2401_05391_b200 import workloads as wl
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    w = wl.by_name(args.workload)
+    L = args.layers or DEFAULT_LAYERS.get(w.name, 1)
+    sb = ShapeBench(w, L, 1, args, 0, 1, dev)
+    peak, peak_kind = peaks()
+    steps_k = max(20, min(args.steps, 50))
+    rows = []
+    for T in range(1, w.steps + 1):
+        if T > 1:
+            # one more step on every layer (the state the timed step starts from)
+            for hh in sb.handles:
+                q, k, v = wl.make_step(hh[5], T - 1, dev)
+                hh[0].append(T - 1, sb.parents[T - 1], k, v)
+                hh[1], hh[2], hh[3] = q, k, v
+            torch.cuda.synchronize()
+        sb.T, sb.t = T, T - 1
+        sb.refresh_bytes()
+        run, _ = sb.make_runner("step")
+        _, per = sb.timed(run, steps_k, 3)
+        med = statistics.median(per) * 1e3 / L
+        gbs = sb.ubytes / (med * 1e-6) / 1e9
+        rows.append({"at_step": T, "us_per_step_per_layer": round(med, 3), "unique_kv_bytes": sb.ubytes,
+                     "gbs": round(gbs, 1), "frac_of_measured": round(gbs / peak, 4)})
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "workload": w.name, "layers_per_step": L,
+                      "replays_per_point": steps_k, "peak": peak, "peak_kind": f"of {peak_kind}", "curve": rows}))
+    sb.close()
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2401_05391_b200 import workloads as wl
     from paper_2401_05391_b200 import sharding
-    from paper_2401_05391_b200.segkv import SegKV
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -230,114 +396,26 @@ def run_ours(args):
     L = args.layers or DEFAULT_LAYERS.get(w.name.split("[")[0], 1)
     T = args.at_step or w.steps
     t = T - 1
-    # every rank holds its own requests (weak scaling: requests are independent, no exchange)
-    w_rank = sharding.rank_workload(w, rank, world)
     sampler = ClockSampler(f"GPU-{torch.cuda.get_device_properties(dev).uuid}") if rank == 0 else None
-    parents = torch.from_numpy(wl.make_parents(w_rank)).to(dev)
-    slopes = wl.alibi_slopes(w.heads).to(dev) if w.alibi else None
-
-    handles = []
-    for layer in range(L):
-        wl_layer = w_rank.scaled(index=w_rank.index + 1000 * layer)
-        h = SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, w.steps, w.torch_dtype)
-        if args.tile:
-            h.set_tile(args.tile)
-        if args.splits or args.stages or args.combine:
-            h.set_tuning(args.splits, args.stages, args.combine)
-        if args.no_overlap:
-            h.set_overlap(False)
-        if args.prompt_layout != "head_major":
-            h.set_prompt_layout(args.prompt_layout)
-        kp, vp = wl.make_prompt(wl_layer, dev)
-        h.prefill_write(kp, vp)
-        del kp, vp
-        for s in range(T):
-            q, k, v = wl.make_step(wl_layer, s, dev)
-            h.append(s, parents[s] if s > 0 else None, k, v)
-        handles.append((h, q, k, v, torch.empty_like(q)))
-    torch.cuda.synchronize()
-    uniq_rows = int(handles[0][0].get_unique_rows().sum())
-    ubytes = unique_bytes(w, w.prompt_len, uniq_rows)
-    logical_bytes = w.rows * (w.prompt_len + T) * 2 * w.kv_heads * w.head_dim * 2
-    par_t = parents[t] if t > 0 else None
-    stream = torch.cuda.Stream()
-
-    def layer_pass(mode: str):
-        # "step": the whole hot path in the library's fused call; "two": the same as two calls
-        # (append, then attention); "sdpa": the attention kernel alone on the state already there
-        for h, q, k, v, out in handles:
-            if mode == "step":
-                h.truncate_last()
-                h.decode_step(t, par_t, k, v, q, out, slopes, stream=stream)
-            elif mode == "two":
-                h.truncate_last()
-                h.append(t, par_t, k, v, stream=stream)
-                h.decode_sdpa(q, out, slopes, stream=stream)
-            elif mode == "sdpa":
-                h.decode_sdpa(q, out, slopes, stream=stream)
-        if mode == "hot":
-            # the attention kernel on ONE layer's cache over and over: L2-resident where the layer fits
-            # (the Llama2-7B shape does), i.e. the kernel's latency floor without HBM
-            h, q, k, v, out = handles[0]
-            for _ in range(len(handles)):
-                h.decode_sdpa(q, out, slopes, stream=stream)
-
-    def make_runner(mode: str):
-        with torch.cuda.stream(stream):
-            layer_pass(mode)                                 # lazy initialisation outside any capture
-        stream.synchronize()
-        if args.no_graph:
-            return lambda: layer_pass(mode), False
-        g = torch.cuda.CUDAGraph()
-        try:
-            with torch.cuda.graph(g, stream=stream):
-                layer_pass(mode)
-        except Exception as e:                               # report, never hide
-            sys.stderr.write(f"[bench] CUDA graph capture failed ({e}); timing direct launches\n")
-            return lambda: layer_pass(mode), False
-
-        def replay():
-            with torch.cuda.stream(stream):
-                g.replay()
-        return replay, True
-
-    def timed(run, steps, warmup):
-        for _ in range(warmup):
-            run()
-        stream.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(steps):
-            run()
-        e1.record(stream)
-        stream.synchronize()
-        torch.cuda.synchronize()
-        ms = sharding.max_over_ranks(e0.elapsed_time(e1), dev)
-        if world > 1:
-            dist.barrier()
-        return ms
+    sb = ShapeBench(w, L, T, args, rank, world, dev)
+    handles, stream, parents, slopes = sb.handles, sb.stream, sb.parents, sb.slopes
+    ubytes, logical_bytes = sb.ubytes, sb.logical_bytes
 
     # ---- the timed region: K whole steps (append + beam-index update + attention, all layers)
     launches0 = sum(h[0].launch_count for h in handles)
-    with torch.cuda.stream(stream):
-        layer_pass("step")
-    stream.synchronize()
-    launches_per_step = sum(h[0].launch_count for h in handles) - launches0     # counted by the library
-    run_step, graphed = make_runner("step")
+    launches_per_step = sb.launches_per_step()
+    run_step, graphed = sb.make_runner("step")
     if sampler:
         sampler.begin()
-    ms_total = timed(run_step, args.steps, args.warmup)
+    ms_total, per_step = sb.timed(run_step, args.steps, args.warmup)
     # ---- the attention kernel alone, same rotation over cold layers (roofline numerator)
-    run_sdpa, _ = make_runner("sdpa")
-    ms_sdpa = timed(run_sdpa, args.steps, max(3, args.warmup))
-    run_hot, _ = make_runner("hot")
-    ms_hot = timed(run_hot, args.steps, max(3, args.warmup))
+    run_sdpa, _ = sb.make_runner("sdpa")
+    ms_sdpa, per_sdpa = sb.timed(run_sdpa, args.steps, max(3, args.warmup))
+    run_hot, _ = sb.make_runner("hot")
+    ms_hot, _ = sb.timed(run_hot, args.steps, max(3, args.warmup))
     # ---- for comparison: the same step as two library calls (append, then attention)
-    run_two, _ = make_runner("two")
-    ms_two = timed(run_two, args.steps, max(3, args.warmup))
+    run_two, _ = sb.make_runner("two")
+    ms_two, _ = sb.timed(run_two, args.steps, max(3, args.warmup))
     clocks = None
     if sampler:
         # the timed loops can be shorter than nvidia-smi's sampling period: keep the same load up
@@ -361,7 +439,7 @@ def run_ours(args):
         total, off = handles[0][0].host_pack_layout()
         hs = slopes is not None
         hq = []
-        for _, q, k, v, _ in handles:
+        for _, q, k, v, _, _ in handles:
             blk = torch.zeros(total, dtype=torch.uint8).pin_memory()
 
             def put(o, x):
@@ -390,18 +468,62 @@ def run_ours(args):
         torch.cuda.synchronize()
         sec = (time.perf_counter() - t0) / n_e2e
         sec = sharding.max_over_ranks(sec, dev)
-        q, k = handles[0][1], handles[0][2]
+        q = handles[0][1]
         h2d = L * total                      # the packed block: parents, slopes, k, v, q and their padding
         d2h = L * q.numel() * 2
         e2e = {"value": sharding.whole_job_rate(L * ubytes, world, sec) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "us_per_step_per_layer": sec * 1e6 / L}
+
+    splits_used = handles[0][0].get_splits()
+    assert sum(h[0].launch_count for h in handles) > launches0
+    sb.close()
+
+    # ---- the other evaluation shapes, each timed the same way (fused step and attention alone)
+    peak, peak_kind = peaks()
+    others = None
+    default_shape = not (args.batch or args.beams or args.prompt_len or args.at_step or args.tile or args.splits or
+                         args.stages or args.combine or args.no_graph or args.no_overlap or
+                         args.prompt_layout != "head_major")
+    if world == 1 and not args.no_others and default_shape:
+        others = {}
+        k_other = max(20, min(args.steps, 30))
+        for c in wl.CONFIGS:
+            if c.name == w.name:
+                continue
+            Lc = DEFAULT_LAYERS.get(c.name, 1)
+            so = ShapeBench(c, Lc, c.steps, args, 0, 1, dev)
+            oc = ClockSampler(f"GPU-{torch.cuda.get_device_properties(dev).uuid}")
+            oc.begin()
+            run_o, _ = so.make_runner("step")
+            _, per_o = so.timed(run_o, k_other, 3)
+            run_a, _ = so.make_runner("sdpa")
+            _, per_a = so.timed(run_a, k_other, 3)
+            t_end = time.time() + 2.0
+            while oc.samples_in_window() < 8 and time.time() < t_end:
+                for _ in range(5):
+                    run_a()
+                so.stream.synchronize()
+            oc.end()
+            ps, pa = percentiles(per_o), percentiles(per_a)
+            us_a = pa["median"] * 1e3 / Lc
+            gbs_a = so.ubytes / (us_a * 1e-6) / 1e9
+            others[c.name] = {
+                "layers_per_step": Lc, "at_step": c.steps, "unique_kv_bytes_per_layer": so.ubytes,
+                "us_per_step_per_layer": ps["median"] * 1e3 / Lc,
+                "us_per_step_per_layer_p10": ps["p10"] * 1e3 / Lc, "us_per_step_per_layer_p90": ps["p90"] * 1e3 / Lc,
+                "us_sdpa_per_layer": us_a, "us_sdpa_per_layer_p10": pa["p10"] * 1e3 / Lc,
+                "us_sdpa_per_layer_p90": pa["p90"] * 1e3 / Lc, "replays": k_other,
+                "gbs": gbs_a, "pct_of_8000": 100.0 * gbs_a / 8000.0, "frac_of_measured": gbs_a / peak,
+                "gbs_whole_step": so.ubytes / (ps["median"] * 1e-3 / Lc) / 1e9,
+                "clocks": oc.stop(),
+            }
+            so.close()
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = peaks()
     # The dominant kernel of the timed region.  When a step is one fused launch per layer, that launch IS
     # the region: its duration is the step time per layer.  When a step is two launches (append, then
     # attention), the attention kernel's own duration comes from the attention-only loop over the same
@@ -410,6 +532,7 @@ def run_ours(args):
     us_dom = us_layer if fused_step else us_sdpa
     achieved = ubytes / (us_dom * 1e-6) / 1e9
     achieved_attn = ubytes / (us_sdpa * 1e-6) / 1e9
+    pstep, psdpa = percentiles(per_step), percentiles(per_sdpa)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -418,9 +541,13 @@ def run_ours(args):
                    "head_dim": w.head_dim, "prompt_len": w.prompt_len, "at_step": T, "layers_per_step": L,
                    "l2": f"{L} distinct layer caches per step, {L * ubytes / 1e6:.0f} MB > L2", "cuda_graph": graphed, "dependent_launch": not args.no_overlap,
                    "prompt_layout": args.prompt_layout,
-                   "splits": handles[0][0].get_splits(), "parallelism": f"replica x{world}" if world > 1 else "1 gpu"},
+                   "splits": splits_used, "parallelism": f"replica x{world}" if world > 1 else "1 gpu"},
+        "ms_per_step_median": pstep["median"], "ms_per_step_p10": pstep["p10"], "ms_per_step_p90": pstep["p90"],
         "us_per_step_per_layer": us_layer,
+        "us_per_step_per_layer_median": pstep["median"] * 1e3 / L,
         "us_sdpa_per_layer": us_sdpa,
+        "us_sdpa_per_layer_median": psdpa["median"] * 1e3 / L,
+        "us_sdpa_per_layer_p10": psdpa["p10"] * 1e3 / L, "us_sdpa_per_layer_p90": psdpa["p90"] * 1e3 / L,
         "us_sdpa_same_layer_repeated": ms_hot / args.steps * 1e3 / L,
         "us_per_step_per_layer_two_calls": ms_two / args.steps * 1e3 / L,
         "unique_kv_bytes_per_layer": ubytes,
@@ -438,7 +565,8 @@ def run_ours(args):
         "e2e": e2e,
         "clocks": clocks,
     }
-    assert sum(h[0].launch_count for h in handles) > launches0
+    if others is not None:
+        line["other_workloads"] = others
     if not args.no_cpu_baseline:
         gbs, sec, desc, threads = oracle_sample(w, t)
         line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
@@ -536,6 +664,8 @@ def main():
     args = parse()
     if args.prefill and args.impl != "reference":
         return run_prefill(args)
+    if args.curve and args.impl != "reference":
+        return run_curve(args)
     if args.impl == "reference":
         run_reference(args)
     else:

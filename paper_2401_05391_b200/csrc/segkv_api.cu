@@ -241,6 +241,7 @@ int alloc_workspace(segkv* h, int splits) {
 // Launch shape of the tiled kernel.
 struct Tiling {
     int splits, stages;
+    bool one_wave;    // all CTAs of the launch fit on the GPU at once and have only a few tiles each
     bool cluster;     // the splits of a work group merge inside a thread-block cluster
     bool small;       // 32-key tiles, quarter-SM CTAs
 };
@@ -276,6 +277,7 @@ Tiling choose_tiling(const segkv* h, bool fused_step) {
         if (slabs * 8 <= 2LL * h->sm_count && tiled_cluster_ok(d, 8)) {
             t.small = true;
             t.cluster = true;
+            t.one_wave = true;
             t.splits = 8;
             t.stages = 2;
             const size_t budget = (h->smem_optin + 1024) / ctas_per_sm(true) - 1024;
@@ -320,6 +322,9 @@ Tiling choose_tiling(const segkv* h, bool fused_step) {
     while (st > 1 && tiled_smem_bytes(d, st, t.small) > h->smem_optin) --st;
     t.splits = sp;
     t.stages = st;
+    // "one wave" in the sense that matters: every CTA resident at once AND a share of a few tiles each,
+    // i.e. a launch whose time is its chain of latencies, not the bytes it moves
+    t.one_wave = slabs * sp <= slots && (ntp + sp - 1) / sp <= 2 * st;
     // The workspace merge is the default: launches that merge inside a cluster were measured
     // not to start early under programmatic dependent launch, which costs more than the
     // cluster merge saves.  With overlap off the cluster merge is the faster one.
@@ -377,6 +382,7 @@ SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes
     a.splits = splits;
     a.cluster = false;
     a.small = false;
+    a.one_wave = false;
     a.pdl = false;
     a.prompt_immutable = h->steps > 0;     // the first append after a prefill is a fully serialised launch
     a.rows_immutable = false;
@@ -717,6 +723,7 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
     SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, splits);
     a.cluster = tl.cluster;
     a.small = tl.small;
+    a.one_wave = tl.one_wave;
     a.pdl = h->overlap;
     a.rows_immutable = rows_settled(h, (cudaStream_t)stream, true);
     h->dbg_wait_ns = 0;                  // an injected fault applies to one launch
@@ -743,6 +750,7 @@ int segkv_decode_sdpa_static(segkv_t h, const void* q, void* out, const float* a
     SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, splits);
     a.pdl = h->overlap;
     a.small = tl.small;
+    a.one_wave = tl.one_wave;
     int too_big = 0;
     h->dbg_wait_ns = 0;
     h->dbg_skip = false;
@@ -809,6 +817,7 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     a.anc = h->anc[(step + 1) & 1];      // table of step-1 (unused at step 0)
     a.cluster = cluster;
     a.small = tl.small;
+    a.one_wave = tl.one_wave;
     // the first step after a prefill is fully serialised; from then on the prompt cannot change
     a.pdl = h->overlap && step > 0;
     a.prompt_immutable = step > 0;

@@ -153,6 +153,9 @@ struct SdpaArgs {
     int* err_word;
     int prompt_len, steps, splits;
     bool small;              // 32-key tiles and two consumer warps (tensor maps with 32-row boxes)
+    bool one_wave;           // every CTA of the launch is resident at once with a few tiles each: latency, not
+                             // bandwidth, is what counts; a stage of the ring may be set aside for the response rows
+                             // fetched ahead, and what cannot be fetched yet is asked into the L2
     bool cluster;            // merge the splits inside a thread-block cluster
     bool pdl;                // launch with programmatic stream serialisation
     bool prompt_immutable;   // a fully serialised launch has followed the last prompt store

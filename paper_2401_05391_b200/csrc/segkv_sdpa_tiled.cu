@@ -167,6 +167,7 @@ struct TiledParams {
     int early_prompt;  // 1: prompt tiles may be fetched before the previous kernel has completed
     int early_rows;    // 1: so may the response rows of earlier steps and (separate form) the row lists
     int resv;          // 1: the last stage is set aside for the CTA's first response tile (see the kernel)
+    int one_wave;      // 1: all CTAs of the launch are resident at once (what cannot be fetched yet is asked into the L2)
     int dbg_skip;      // test aid: the gather warp leaves out one plain barrier arrival, so that a wait runs out
     unsigned long long wait_ns;   // limit of every bounded wait
 #ifdef SEGKV_TIMELINE
@@ -313,7 +314,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         if (first == npt && lane == 0) mbar_arrive(hand);
         // Prompt tiles that have to wait for a stage of the ring are at least brought into the L2,
         // so that their turn costs an L2 hit, not an HBM round trip, after the wait.
-        if (p.early_prompt && lane == 0) {
+        if (p.early_prompt && p.one_wave && lane == 0) {       // (a launch of several waves is bound by bandwidth: no fetching ahead of need)
             for (int k = first; k < npt; ++k) {
                 const int y = (pt0 + k) * TILE;
 #pragma unroll
@@ -531,7 +532,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 // that find a free stage are fetched now, the rows of the others are asked into the L2,
                 // and only then does this warp wait for the previous kernel.
                 const int r_now = min(nrt, p.resv + (npt < RS ? RS - npt : 0));
-                for (int e = e0 + r_now * TILE + lane / 4; e < e1; e += 8) {
+                for (int e = e0 + r_now * TILE + lane / 4; e < e1 && p.one_wave; e += 8) {
                     const int row = ulist_b[e].row, sidx = row / p.rows;
                     const char* kr = k_slab(sidx) + ((size_t)(row - sidx * p.rows) * p.Hkv + kvh) * (size_t)(D * 2);
                     const char* src = ((lane & 2) ? kr + p.vdelta : kr) + (lane & 1) * (D);     // K or V row, first or second half
@@ -637,7 +638,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                         }
                     }
                     copy_rows(rstage, 0, old_total, false);
-                } else {
+                } else if (p.one_wave) {
                     // at least ask the L2 for the rows of the first windows
 #pragma unroll
                     for (int u = 0; u < PF; ++u) {
@@ -1353,7 +1354,8 @@ cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk,
     p.cluster = a.cluster ? 1 : 0;
     p.early_prompt = (a.pdl && a.prompt_immutable) ? 1 : 0;
     p.early_rows = (a.pdl && a.prompt_immutable && a.rows_immutable) ? 1 : 0;
-    p.resv = (p.early_rows && stages >= 2) ? 1 : 0;
+    p.one_wave = a.one_wave ? 1 : 0;
+    p.resv = (p.early_rows && a.one_wave && stages >= 2) ? 1 : 0;
     p.dbg_skip = a.dbg_skip ? 1 : 0;
     p.wait_ns = a.wait_ns ? a.wait_ns : kWaitLimitNs;
 #ifdef SEGKV_TIMELINE

@@ -21,7 +21,7 @@ def run_bench(*args):
 
 
 def test_decode_line_has_the_contract_keys():
-    d = run_bench("--steps", "3", "--warmup", "3", "--layers", "4")
+    d = run_bench("--steps", "3", "--warmup", "3", "--layers", "4", "--no-others")
     for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
                 "vs_baseline", "dtype", "data", "config", "roofline", "cpu_baseline", "e2e", "clocks", "gpu_launches"):
         assert key in d, key
