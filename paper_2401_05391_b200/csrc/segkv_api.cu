@@ -286,6 +286,17 @@ Tiling choose_tiling(const segkv* h, bool fused_step) {
         }
     }
     t.small = h->tile_forced == 32 && tiled_small_ok(d);
+    {
+        // Between half a wave and two waves of the regular form's CTA slots, one CTA per work group
+        // leaves slots idle or a ragged second wave (measured at the Llama2-13B shape: 0.67-0.69 of the
+        // copy bandwidth at batch 4 and 8).  The small-CTA form has twice the slots: as many splits as
+        // still make one wave of them (0.76 and 0.83 there).
+        const long long slabs = (long long)d.batch * d.kv_heads;
+        const long long slots_small = (long long)h->sm_count * ctas_per_sm(true);
+        if (h->tile_forced == 0 && h->splits_forced <= 0 && tiled_small_ok(d) && 2 * slabs > h->sm_count * 2 &&
+            slabs <= slots_small)
+            t.small = true;
+    }
     const int tile = tiled_tile_keys(d.head_dim, t.small);
     const int P = h->prompt_len > 0 ? h->prompt_len : 0;
     const long long ntp = (P + tile - 1) / tile;
