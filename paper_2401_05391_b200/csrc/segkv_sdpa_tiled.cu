@@ -365,11 +365,16 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     // one finds every kernel before this one's predecessor complete.  (The gather warp, when the
     // host vouches for its inputs, works ahead and waits later.)
     const bool gather_ahead = warp == GATHER_WARP && p.early_rows;
-    if (!gather_ahead) {
+    // Consumer warps of a launch that starts early have nothing to do before the wait; they spend the
+    // time running one tile's worth of their loop on whatever the first stage holds and throwing the
+    // result away: the loop's instructions are then in the instruction cache when the real first
+    // tile comes (straight-line code that runs once per CTA is bound by instruction fetch).
+    const bool cons_ahead = warp < CW && p.early_prompt;
+    if (!gather_ahead && !cons_ahead) {
         grid_wait();
         grid_launch_dependents();
     }
-    if (tid == 0) SEGKV_STAMP(2);
+    if (tid == 0 && !cons_ahead) SEGKV_STAMP(2);
 
     // consumer state (declared here so that the epilogue sees it)
     float o_acc[NT][KS][4];
@@ -794,32 +799,37 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         }
     } else {
         // ================================ consumer warps ===============================
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            m_run[nt][0] = m_run[nt][1] = -INFINITY;
-            l_run[nt][0] = l_run[nt][1] = 0.f;
-#pragma unroll
-            for (int mt = 0; mt < KS; ++mt)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) o_acc[nt][mt][i] = 0.f;
-        }
-        const int n_b = (p.steps > 0 && !FUSED) ? p.ucount[b] : 0;   // in flight while the prompt tiles are consumed
         uint32_t qf[NT][KS][2];
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const T* qrow = qrow_c[nt];
-#pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                const int d0 = ks * 16 + (lane & 3) * 2;
-                qf[nt][ks][0] = qrow ? *reinterpret_cast<const uint32_t*>(qrow + d0) : 0u;
-                qf[nt][ks][1] = qrow ? *reinterpret_cast<const uint32_t*>(qrow + d0 + 8) : 0u;
-            }
-        }
         float slope2[NT][2];
+        int n_b = 0;
+        // accumulators empty; with_inputs: the query fragments, slopes and (separate form) the request's
+        // row count, which stays in flight while the prompt tiles are consumed
+        auto begin = [&](bool with_inputs) {
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+            for (int nt = 0; nt < NT; ++nt) {
+                m_run[nt][0] = m_run[nt][1] = -INFINITY;
+                l_run[nt][0] = l_run[nt][1] = 0.f;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) slope2[nt][c] = slope_c[nt][c] ? *slope_c[nt][c] * 1.4426950408889634f : 0.f;
+                for (int mt = 0; mt < KS; ++mt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) o_acc[nt][mt][i] = 0.f;
+            }
+            n_b = (with_inputs && p.steps > 0 && !FUSED) ? p.ucount[b] : 0;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const T* qrow = with_inputs ? qrow_c[nt] : nullptr;
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    const int d0 = ks * 16 + (lane & 3) * 2;
+                    qf[nt][ks][0] = qrow ? *reinterpret_cast<const uint32_t*>(qrow + d0) : 0u;
+                    qf[nt][ks][1] = qrow ? *reinterpret_cast<const uint32_t*>(qrow + d0 + 8) : 0u;
+                }
+#pragma unroll
+                for (int c = 0; c < 2; ++c)
+                    slope2[nt][c] = (with_inputs && slope_c[nt][c]) ? *slope_c[nt][c] * 1.4426950408889634f : 0.f;
+            }
+        };
+        begin(!cons_ahead);
         const int qpos = P + (p.steps > 0 ? p.steps - 1 : -1);
 
         // One tile: `nvalid` keys exist; for a response tile the per-key beam masks and row
@@ -972,35 +982,52 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             }
         };
         if (warp == 0) SEGKV_STAMP(1);
+        // k = -1 is the warm-up: the same instructions on whatever the first stage holds, no barrier
+        // touched, result thrown away, and then the wait
+        if (cons_ahead) k = -1;
+        auto warmed_up = [&]() {
+            grid_wait();
+            grid_launch_dependents();
+            if (warp == 0) SEGKV_STAMP(2);
+            begin(true);
+        };
         if constexpr (kWholeTile) {
             for (; k < npt; ++k) {
                 // every warp waits for every tile, also those it leaves to the other warp: a parity
                 // wait cannot tell a barrier's phases two apart, so none may be skipped
-                ok = mbar_wait(full0 + 8 * st, ph, p.wait_ns);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                if ((k & (CW - 1)) == warp) {
-                    const int pos0 = (pt0 + k) * TILE;
+                if (k >= 0) {
+                    ok = mbar_wait(full0 + 8 * st, ph, p.wait_ns);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                }
+                if (k < 0 || (k & (CW - 1)) == warp) {
+                    const int pos0 = (pt0 + max(k, 0)) * TILE;
                     if (warp == 0 && k == 0) SEGKV_STAMP(7);
-                    consume(IntC<CW>{}, st, false, min(TILE, P - pos0), pos0, 0);
+                    consume(IntC<CW>{}, k < 0 ? 0 : st, false, min(TILE, P - pos0), pos0, 0);
                     if (warp == 0 && k == 0) SEGKV_STAMP(6);
                     __syncwarp();
-                    if (lane < CW) mbar_arrive(empty0 + 8 * st);      // the stage's release counts one arrival per consumer warp
+                    if (k >= 0 && lane < CW) mbar_arrive(empty0 + 8 * st);      // the stage's release counts one arrival per consumer warp
                 }
-                next_stage();
+                if (k < 0) warmed_up();
+                else next_stage();
             }
         }
         for (; k < npt; ++k) {
-            ok = mbar_wait(full0 + 8 * st, ph, p.wait_ns);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            const int pos0 = (pt0 + k) * TILE;
+            if (k >= 0) {
+                ok = mbar_wait(full0 + 8 * st, ph, p.wait_ns);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+            }
+            const int pos0 = (pt0 + max(k, 0)) * TILE;
             if (warp == 0 && k == 0) SEGKV_STAMP(7);
-            consume(IntC<1>{}, st, false, min(TILE, P - pos0), pos0, warp * 16);
+            consume(IntC<1>{}, k < 0 ? 0 : st, false, min(TILE, P - pos0), pos0, warp * 16);
             if (warp == 0 && k == 0) SEGKV_STAMP(6);
             __syncwarp();
-            if (lane == 0) mbar_arrive(empty0 + 8 * st);
-            next_stage();
+            if (k < 0) warmed_up();
+            else {
+                if (lane == 0) mbar_arrive(empty0 + 8 * st);
+                next_stage();
+            }
         }
         if (warp == 0) SEGKV_STAMP(8);
         if (ok && !FUSED) {
