@@ -432,7 +432,7 @@ def run_ours(args):
     us_sdpa = ms_sdpa / args.steps * 1e3 / L
     value = sharding.whole_job_rate(L * ubytes, world, ms_per_step * 1e-3) / 1e9
 
-    # ---- end to end from host memory through segkv_step_host
+    # ---- end to end from host memory through segkv_layers_step_host
     e2e = None
     if not args.no_e2e:
         # every layer's step inputs packed into one pinned host block (one copy in, one launch, one copy out)
@@ -452,10 +452,13 @@ def run_ours(args):
             put(off[2], k); put(off[3], v); put(off[4], q)
             hq.append((blk, torch.empty_like(q, device="cpu").pin_memory()))
 
+        from paper_2401_05391_b200.segkv import LayerStack
+        stack = LayerStack([h[0] for h in handles], [x[0] for x in hq], [x[1] for x in hq])
+
         def host_step():
-            for (h, *_), (blk, o) in zip(handles, hq):
-                h.truncate_last()
-                h.step_host_packed(t, blk, o, has_slopes=hs, stream=stream)
+            # one call queues every layer's copy in, launch and copy out; the host waits once per step
+            stack.step(t, has_slopes=hs, redo=True, stream=stream)
+            stream.synchronize()
         n_e2e = max(3, min(args.steps, 20))
         for _ in range(3):
             host_step()

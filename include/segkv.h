@@ -269,6 +269,36 @@ SEGKV_API size_t segkv_host_pack_bytes(segkv_t h, size_t* offsets);
 SEGKV_API int segkv_step_host_packed(segkv_t h, int step, const void* host_in, void* host_out, int has_slopes,
                                      void* stream);
 
+/*
+ * segkv_step_host_packed without the wait at the end: the copy in, the launch and
+ * the copy out are queued on `stream` and the call returns.  The caller waits for
+ * the stream (or an event behind the call) before reading host_out or reusing
+ * host_in; a model that drives its layers from host buffers waits once per step,
+ * not once per layer, and the queue of one layer overlaps the host work of the
+ * next.  No counterpart in the paper (an interface convenience).  Errors: as
+ * segkv_step_host_packed.
+ */
+SEGKV_API int segkv_step_host_packed_async(segkv_t h, int step, const void* host_in, void* host_out, int has_slopes,
+                                 void* stream);
+
+/*
+ * segkv_step_host_packed_async for the n layers of a model in one call: layer i
+ * takes its inputs from host_in[i] and delivers to host_out[i] (host pointers to
+ * pinned blocks laid out as segkv_host_pack_bytes says) without waiting.  The
+ * launches go to `stream` in order; the copies travel on two streams of the
+ * library's own, so that one layer's inputs arrive while the layer before it
+ * computes, and `stream` ends behind the last copy out: waiting for `stream`
+ * is waiting for every output.  (On a stream that is being captured everything
+ * stays on `stream`.)  redo != 0 re-times a step: a handle whose newest
+ * step is `step` drops it first (segkv_truncate_last) and takes it again.
+ * No counterpart in the paper (an interface convenience: one call per decode
+ * step instead of one per layer).  Errors: those of the single-layer call, at
+ * the first layer that fails (earlier layers' work stays queued); EINVAL for
+ * n <= 0 or NULL arrays.
+ */
+SEGKV_API int segkv_layers_step_host(const segkv_t* layers, int n, int step, const void* const* host_in,
+                           void* const* host_out, int has_slopes, int redo, void* stream);
+
 
 /* ---- test and benchmark aids ------------------------------------------- */
 

@@ -182,6 +182,8 @@ void free_all(segkv* h) {
                     h->st_slopes};
     for (void* p : ptrs)
         if (p) cudaFree(p);
+    if (h->ev_in) cudaEventDestroy(h->ev_in);
+    if (h->ev_k) cudaEventDestroy(h->ev_k);
     for (int c = 0; c < h->nchunks; ++c)
         if (h->k_chunks_host[c]) cudaFree(h->k_chunks_host[c]);
     free(h->k_chunks_host);
@@ -520,6 +522,11 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
 #undef SEGKV_TRY
     // The split workspace for the largest split count the automatic choice can make (one wave of
     // CTA slots shared among the work groups), so that the decode loop never allocates.
+    if (cudaEventCreateWithFlags(&h->ev_in, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_k, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(SEGKV_ECUDA);
+    }
     rc = alloc_workspace(h, max_auto_splits(h));
     if (rc != SEGKV_OK) return fail(rc);
     *out = h;
@@ -895,6 +902,13 @@ size_t segkv_host_pack_bytes(segkv_t h, size_t* offsets) {
 }
 
 int segkv_step_host_packed(segkv_t h, int step, const void* host_in, void* host_out, int has_slopes, void* stream) {
+    int rc = segkv_step_host_packed_async(h, step, host_in, host_out, has_slopes, stream);
+    if (rc != SEGKV_OK) return rc;
+    SEGKV_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    return SEGKV_OK;
+}
+
+int segkv_step_host_packed_async(segkv_t h, int step, const void* host_in, void* host_out, int has_slopes, void* stream) {
     if (!h || !host_in || !host_out) return SEGKV_EINVAL;
     const Dims& d = h->d;
     cudaStream_t st = (cudaStream_t)stream;
@@ -907,7 +921,87 @@ int segkv_step_host_packed(segkv_t h, int step, const void* host_in, void* host_
                                base + off[4], h->st_out, has_slopes ? (const float*)(base + off[1]) : nullptr, stream);
     if (rc != SEGKV_OK) return rc;
     SEGKV_CUDA(cudaMemcpyAsync(host_out, h->st_out, qbytes, cudaMemcpyDeviceToHost, st));
-    SEGKV_CUDA(cudaStreamSynchronize(st));
+    return SEGKV_OK;
+}
+
+// Two streams of the library's own per device, for the copies of segkv_layers_step_host.
+struct CopyStreams {
+    cudaStream_t in, out;
+    cudaEvent_t entry, done;
+    bool ok;
+};
+CopyStreams* copy_streams(int dev) {
+    static CopyStreams cs[64] = {};
+    static std::mutex mu;
+    if (dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lk(mu);
+    CopyStreams& c = cs[dev];
+    if (!c.ok) {
+        if (cudaStreamCreateWithFlags(&c.in, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&c.out, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c.entry, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c.done, cudaEventDisableTiming) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        c.ok = true;
+    }
+    return &c;
+}
+
+int segkv_layers_step_host(const segkv_t* layers, int n, int step, const void* const* host_in, void* const* host_out,
+                           int has_slopes, int redo, void* stream) {
+    if (!layers || !host_in || !host_out || n <= 0) return SEGKV_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    for (int i = 0; i < n; ++i)
+        if (!layers[i] || !layers[i]->ev_in || !layers[i]->ev_k) return SEGKV_EINVAL;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) cudaGetLastError();
+    CopyStreams* cs = cap == cudaStreamCaptureStatusNone ? copy_streams(layers[0]->device) : nullptr;
+    if (!cs) {
+        // a stream being captured (or no streams to be had): everything in order on the caller's stream
+        for (int i = 0; i < n; ++i) {
+            segkv_t h = layers[i];
+            if (redo && h->steps == step + 1 && !h->truncated) {
+                h->steps -= 1;
+                h->truncated = true;
+            }
+            const int rc = segkv_step_host_packed_async(h, step, host_in[i], host_out[i], has_slopes, stream);
+            if (rc != SEGKV_OK) return rc;
+        }
+        return SEGKV_OK;
+    }
+    // Copies in on one stream, launches on the caller's, copies out on a third: layer i+1's inputs
+    // travel while layer i computes and layer i-1's output travels back.  The copy-in stream starts
+    // behind what the caller's stream holds now (the staging blocks may still be read by it), and the
+    // caller's stream ends behind the last copy out, so waiting for it is waiting for everything.
+    SEGKV_CUDA(cudaEventRecord(cs->entry, st));
+    SEGKV_CUDA(cudaStreamWaitEvent(cs->in, cs->entry, 0));
+    SEGKV_CUDA(cudaStreamWaitEvent(cs->out, cs->entry, 0));
+    for (int i = 0; i < n; ++i) {
+        segkv_t h = layers[i];
+        if (redo && h->steps == step + 1 && !h->truncated) {
+            h->steps -= 1;
+            h->truncated = true;
+        }
+        const Dims& d = h->d;
+        size_t off[5];
+        const size_t total = segkv_host_pack_bytes(h, off);
+        const size_t qbytes = (size_t)d.rows * d.heads * d.head_dim * 2;
+        SEGKV_CUDA(cudaMemcpyAsync(h->st_pack, host_in[i], total, cudaMemcpyHostToDevice, cs->in));
+        SEGKV_CUDA(cudaEventRecord(h->ev_in, cs->in));
+        SEGKV_CUDA(cudaStreamWaitEvent(st, h->ev_in, 0));
+        char* base = (char*)h->st_pack;
+        const int rc = segkv_decode_step(h, step, step > 0 ? (const int32_t*)(base + off[0]) : nullptr, base + off[2],
+                                         base + off[3], base + off[4], h->st_out,
+                                         has_slopes ? (const float*)(base + off[1]) : nullptr, stream);
+        if (rc != SEGKV_OK) return rc;
+        SEGKV_CUDA(cudaEventRecord(h->ev_k, st));
+        SEGKV_CUDA(cudaStreamWaitEvent(cs->out, h->ev_k, 0));
+        SEGKV_CUDA(cudaMemcpyAsync(host_out[i], h->st_out, qbytes, cudaMemcpyDeviceToHost, cs->out));
+    }
+    SEGKV_CUDA(cudaEventRecord(cs->done, cs->out));
+    SEGKV_CUDA(cudaStreamWaitEvent(st, cs->done, 0));
     return SEGKV_OK;
 }
 

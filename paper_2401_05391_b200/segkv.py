@@ -40,6 +40,8 @@ SIGNATURES = {
     "segkv_step_host": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "segkv_host_pack_bytes": (ctypes.c_size_t, [_vp, _vp]),
     "segkv_step_host_packed": (_int, [_vp, _int, _vp, _vp, _int, _vp]),
+    "segkv_step_host_packed_async": (_int, [_vp, _int, _vp, _vp, _int, _vp]),
+    "segkv_layers_step_host": (_int, [_vp, _int, _int, _vp, _vp, _int, _int, _vp]),
     "segkv_reset": (_int, [_vp, _int]),
     "segkv_truncate_last": (_int, [_vp]),
     "segkv_get_ancestry": (_int, [_vp, _vp, _vp]),
@@ -81,6 +83,26 @@ def lib() -> ctypes.CDLL:
             fn.restype, fn.argtypes = res, args
         _lib = L
     return _lib
+
+
+class LayerStack:
+    """The handles of a model's layers with their pinned host blocks, for segkv_layers_step_host."""
+
+    def __init__(self, handles, packed_in, outs):
+        n = len(handles)
+        assert n == len(packed_in) == len(outs) and n > 0
+        total = handles[0].host_pack_layout()[0]
+        qs = (handles[0].rows, handles[0].heads, handles[0].head_dim)
+        self._keep = (list(handles), list(packed_in), list(outs))
+        self.n = n
+        self._h = (_vp * n)(*[h._h for h in handles])
+        self._in = (_vp * n)(*[_host(t, (total,), torch.uint8, "packed") for t in packed_in])
+        self._out = (_vp * n)(*[_host(o, qs, handles[0].dtype, "out") for o in outs])
+
+    def step(self, step: int, has_slopes: bool = False, redo: bool = False, stream=None) -> None:
+        """Queue one decode step of every layer on the stream (the caller waits for the stream)."""
+        _check(lib().segkv_layers_step_host(self._h, self.n, step, self._in, self._out, int(has_slopes), int(redo),
+                                            _stream_ptr(stream)), "segkv_layers_step_host")
 
 
 class SegKVError(RuntimeError):
@@ -291,6 +313,18 @@ class SegKV:
         _check(lib().segkv_step_host_packed(self._h, step, _host(packed, (total,), torch.uint8, "packed"),
                                             _host(out, qs, self.dtype, "out"), int(has_slopes), _stream_ptr(stream)),
                "segkv_step_host_packed")
+        return out
+
+    def step_host_packed_async(self, step: int, packed: torch.Tensor, out: torch.Tensor, has_slopes: bool = False,
+                               stream=None) -> torch.Tensor:
+        """As step_host_packed, but only queued on the stream: wait for the stream before reading `out`."""
+        if getattr(self, "_pack_total", None) is None:
+            self._pack_total = self.host_pack_layout()[0]
+        qs = (self.rows, self.heads, self.head_dim)
+        _check(lib().segkv_step_host_packed_async(self._h, step, _host(packed, (self._pack_total,), torch.uint8, "packed"),
+                                                  _host(out, qs, self.dtype, "out"), int(has_slopes),
+                                                  _stream_ptr(stream)),
+               "segkv_step_host_packed_async")
         return out
 
     # ------------------------------------------------------------------ aids

@@ -528,12 +528,59 @@ def test_step_host_packed_matches_device_calls():
             if t > 0:
                 put(off[0], torch.from_numpy(r.parents[t]))
             put(off[2], r.k_steps[t]); put(off[3], r.v_steps[t]); put(off[4], q)
-            r2.h.step_host_packed(t, blk, oh, has_slopes=True)
+            if t % 2:
+                r2.h.step_host_packed(t, blk, oh, has_slopes=True)
+            else:                                            # queued only: the caller waits
+                r2.h.step_host_packed_async(t, blk, oh, has_slopes=True)
+                torch.cuda.synchronize()
             assert torch.allclose(oh.float(), out.cpu().float(), atol=4e-3, rtol=2e-2)
         assert np.array_equal(r2.h.get_ancestry(), r.h.get_ancestry())
         assert r2.h.get_error() == 0
     finally:
         r.close(); r2.close()
+
+
+def test_layers_step_host_queues_every_layer_in_one_call():
+    # three layers driven from pinned host blocks with one call per step; redo re-times the newest step
+    w = wl.Workload("stack", 1, 4, 8, 8, 128, 300, 6, "bf16", "uniform", True, 120)
+    par = wl.make_parents(w)
+    ls = [Run(w.scaled(index=120 + i), parents=par) for i in range(3)]
+    hs = [sk.SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, w.steps, w.torch_dtype) for _ in ls]
+    try:
+        total, off = hs[0].host_pack_layout()
+        blks = [torch.zeros(total, dtype=torch.uint8).pin_memory() for _ in ls]
+        outs = [torch.empty(w.rows, w.heads, w.head_dim, dtype=w.torch_dtype).pin_memory() for _ in ls]
+        for r, h in zip(ls, hs):
+            h.prefill_write(r.kp, r.vp)
+        stack = sk.LayerStack(hs, blks, outs)
+        for t in range(w.steps):
+            refs = []
+            for r, blk in zip(ls, blks):
+                r.append_next()
+                out, q = r.decode()
+                refs.append(out)
+
+                def put(o, x):
+                    raw = x.contiguous().cpu().view(torch.uint8).reshape(-1)
+                    blk[o:o + raw.numel()] = raw
+                if t > 0:
+                    put(off[0], torch.from_numpy(par[t]))
+                put(off[1], r.slopes); put(off[2], r.k_steps[t]); put(off[3], r.v_steps[t]); put(off[4], q)
+            for redo in (False, True):
+                for o in outs:
+                    o.fill_(float("nan"))
+                stack.step(t, has_slopes=True, redo=redo)
+                torch.cuda.synchronize()
+                for o, ref in zip(outs, refs):
+                    assert torch.allclose(o.float(), ref.cpu().float(), atol=4e-3, rtol=2e-2)
+        for h, r in zip(hs, ls):
+            assert np.array_equal(h.get_ancestry(), r.h.get_ancestry())
+            assert h.get_error() == 0
+    finally:
+        for r in ls:
+            r.close()
+        for h in hs:
+            h.destroy()
 
 
 def test_argument_and_state_errors():
