@@ -443,6 +443,18 @@ SEGKV_API int segkv_set_prompt_layout(segkv_t h, int layout);
 SEGKV_API int segkv_set_prefill_tuning(segkv_t h, int row_groups);
 
 /*
+ * Measurement aid (no counterpart in the paper): the bandwidth of a kernel that
+ * only READS.  Streams `bytes` of device memory at dev_buf (16-byte aligned; use
+ * a buffer several times the L2) `repeats` times with 16-byte loads, between two
+ * CUDA events on `stream`, and returns GB/s in *gbs_out.  The decode attention
+ * reads its keys and writes almost nothing, so this, not a copy's read+write
+ * figure, is the ceiling its fraction of peak can be read against.  Allocates 256
+ * bytes for the duration of the call and waits for the stream.
+ * Errors: EINVAL, ECUDA.
+ */
+SEGKV_API int segkv_read_bandwidth(const void* dev_buf, size_t bytes, int repeats, float* gbs_out, void* stream);
+
+/*
  * Test aid for the kernels' bounded waits (no counterpart in the paper).  Every
  * wait inside the attention kernels gives up after about two seconds, sets
  * SEGKV_DEV_WAIT_LIMIT in the device error word, lets copies in flight land,

@@ -1153,6 +1153,33 @@ int segkv_set_tile(segkv_t h, int tile_keys) {
     return SEGKV_OK;
 }
 
+int segkv_read_bandwidth(const void* dev_buf, size_t bytes, int repeats, float* gbs_out, void* stream) {
+    if (!dev_buf || !gbs_out || bytes < 16 || repeats <= 0 || !aligned16(dev_buf)) return SEGKV_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    int dev = 0, sms = 0;
+    SEGKV_CUDA(cudaGetDevice(&dev));
+    SEGKV_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    unsigned* sink = nullptr;
+    SEGKV_CUDA(cudaMalloc((void**)&sink, 64 * sizeof(unsigned)));
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    cudaError_t e = cudaMemsetAsync(sink, 0, 64 * sizeof(unsigned), st);
+    if (e == cudaSuccess) e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    for (int i = 0; i < 3 && e == cudaSuccess; ++i) e = launch_read_stream(dev_buf, bytes, sink, sms, st);   // warm-up
+    if (e == cudaSuccess) e = cudaEventRecord(e0, st);
+    for (int i = 0; i < repeats && e == cudaSuccess; ++i) e = launch_read_stream(dev_buf, bytes, sink, sms, st);
+    if (e == cudaSuccess) e = cudaEventRecord(e1, st);
+    if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    cudaFree(sink);
+    if (e != cudaSuccess) return cuda_fail(e, "segkv_read_bandwidth");
+    *gbs_out = (float)((double)bytes * repeats / (ms * 1e-3) / 1e9);
+    return SEGKV_OK;
+}
+
 int segkv_debug_inject(segkv_t h, long long wait_limit_ns, int skip_arrival) {
     if (!h || wait_limit_ns < 0) return SEGKV_EINVAL;
     h->dbg_wait_ns = (unsigned long long)wait_limit_ns;

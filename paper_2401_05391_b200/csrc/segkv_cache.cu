@@ -323,4 +323,36 @@ cudaError_t launch_rebuild_lists(const Dims& d, int steps, const int32_t* anc_cu
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------
+// A read-only stream over a buffer (16-byte loads folded into one word per thread, one word
+// per block written): the bandwidth a kernel that only READS can reach on this GPU, which is what
+// the decode attention does.  A copy's figure counts bytes read plus bytes written and sits lower.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) read_stream_kernel(const uint4* __restrict__ src, size_t n16,
+                                                          unsigned* __restrict__ sink) {
+    unsigned acc = 0;
+    const size_t stride = (size_t)gridDim.x * blockDim.x * 4;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x * 4 + threadIdx.x; i < n16; i += stride) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const size_t k = i + (size_t)u * blockDim.x;
+            v[u] = k < n16 ? __ldcs(src + k) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) acc ^= v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+    }
+    acc ^= __shfl_xor_sync(0xffffffffu, acc, 16);
+    acc ^= __shfl_xor_sync(0xffffffffu, acc, 8);
+    acc ^= __shfl_xor_sync(0xffffffffu, acc, 4);
+    acc ^= __shfl_xor_sync(0xffffffffu, acc, 2);
+    acc ^= __shfl_xor_sync(0xffffffffu, acc, 1);
+    if ((threadIdx.x & 31) == 0) atomicXor(sink + (blockIdx.x & 63), acc);
+}
+
+cudaError_t launch_read_stream(const void* src, size_t bytes, unsigned* sink, int sm_count, cudaStream_t st) {
+    read_stream_kernel<<<(unsigned)(sm_count * 8), 256, 0, st>>>((const uint4*)src, bytes / 16, sink);
+    return cudaGetLastError();
+}
+
 }  // namespace segkv_impl

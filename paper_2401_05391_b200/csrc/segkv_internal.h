@@ -131,6 +131,8 @@ cudaError_t launch_append(const Dims& d, int step, const int32_t* beam_parent, c
                           const int32_t* anc_prev, int32_t* anc_cur, URow* ulist, int32_t* ucount,
                           int* err_word, int sm_count, bool pdl, cudaStream_t st, const RopeArgs* rope = nullptr,
                           bool tables = true);
+// A read-only pass over `bytes` of device memory (16-byte loads); sink: 64 words of device memory.
+cudaError_t launch_read_stream(const void* src, size_t bytes, unsigned* sink, int sm_count, cudaStream_t st);
 // Re-derive the distinct-row lists from the current beam-index table (after fused steps).
 cudaError_t launch_rebuild_lists(const Dims& d, int steps, const int32_t* anc_cur, URow* ulist, int32_t* ucount,
                                  cudaStream_t st);

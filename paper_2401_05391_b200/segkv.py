@@ -60,6 +60,7 @@ SIGNATURES = {
     "segkv_append_rope": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _int, _int, _vp]),
     "segkv_prefill_write_ragged": (_int, [_vp, _vp, _vp, _int, _vp, _vp]),
     "segkv_debug_inject": (_int, [_vp, ctypes.c_longlong, _int]),
+    "segkv_read_bandwidth": (_int, [_vp, ctypes.c_size_t, _int, ctypes.POINTER(ctypes.c_float), _vp]),
     "segkv_launch_count": (ctypes.c_longlong, [_vp]),
     "segkv_storage_bytes": (ctypes.c_size_t, [_int] * 7),
     "segkv_strerror": (ctypes.c_char_p, [_int]),
@@ -147,6 +148,16 @@ def _host(t: Optional[torch.Tensor], shape, dtype, name: str) -> Optional[int]:
 
 def segkv_storage_bytes(batch, beams, kv_heads, head_dim, max_prompt, max_steps, dtype) -> int:
     return int(lib().segkv_storage_bytes(batch, beams, kv_heads, head_dim, max_prompt, max_steps, dtype))
+
+
+def read_bandwidth(buf: torch.Tensor, repeats: int = 10, stream=None) -> float:
+    """GB/s of a read-only pass over a CUDA tensor (segkv_read_bandwidth)."""
+    if not buf.is_cuda or not buf.is_contiguous():
+        raise ValueError("buf must be a contiguous CUDA tensor")
+    gbs = ctypes.c_float(0)
+    _check(lib().segkv_read_bandwidth(buf.data_ptr(), buf.numel() * buf.element_size(), repeats, ctypes.byref(gbs),
+                                      _stream_ptr(stream)), "segkv_read_bandwidth")
+    return float(gbs.value)
 
 
 def segkv_strerror(code: int) -> str:

@@ -583,6 +583,14 @@ def test_layers_step_host_queues_every_layer_in_one_call():
             h.destroy()
 
 
+def test_read_bandwidth_aid():
+    buf = torch.zeros(1 << 30, dtype=torch.uint8, device="cuda")
+    gbs = sk.read_bandwidth(buf, 5)
+    assert 2000.0 < gbs < 9000.0, gbs                 # a B200 streams several TB/s; nothing reads faster than HBM3e
+    with pytest.raises(sk.SegKVError):
+        sk.read_bandwidth(buf[1:17], 1)               # not 16-byte aligned
+
+
 def test_argument_and_state_errors():
     h = sk.SegKV(1, 2, 2, 2, 64, 16, 4, torch.float16)
     dev = "cuda"
