@@ -812,7 +812,13 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     const long long rows_per_cta = (long long)((step + 1 + splits - 1) / splits) * d.beams;
     const bool long_tail = h->splits_forced <= 0 && !(tl.small && tl.cluster) &&                                // a forced split count keeps the fused kernel
                            2 * rows_per_cta > 3 * tiled_tile_keys(d.head_dim, false);
-    if ((splits == 1 || long_tail) && !h->fuse_always) {
+    // a CTA with many prompt tiles to stream is bandwidth-bound and gains nothing from the fusion
+    // (13B shape at batch 1: prompt 2048, 5 tiles per CTA, 12.3 us fused against 15.1 us as two
+    // launches; prompt 4096, 10 tiles per CTA, 23.9 us against 22.0 us)
+    const int tile_keys = tiled_tile_keys(d.head_dim, tl.small);
+    const int ptiles_per_cta = ((h->prompt_len + tile_keys - 1) / tile_keys + splits - 1) / splits;
+    const bool long_prompt = h->splits_forced <= 0 && ptiles_per_cta > 7;
+    if ((splits == 1 || long_tail || long_prompt) && !h->fuse_always) {
         // Work groups that fill the GPU on their own are bandwidth-bound: the separate append is
         // then ~1 % of the step and the list it makes keeps the response tiles dense and cheap
         // to build, so the two launches are the faster form.

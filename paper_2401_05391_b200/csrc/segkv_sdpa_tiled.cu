@@ -443,11 +443,14 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         };
         // Complete a tile of cnt keys whose per-key meta has been written: zero the rows between
         // the last real one and the end of its 16-key slice (rows past that slice are never
-        // looked at), say how full the tile is, and release the plain stores of the whole warp.
-        auto finish_tile = [&](int st, int cnt, bool last) {
+        // looked at: a masked weight is zero, but zero times whatever bits the stage held before
+        // need not be), say how full the tile is, and release the plain stores of the whole warp.
+        auto pad_tile = [&](int st, int cnt, bool last) {
             uint8_t* k_tile = ring + (size_t)st * L::STAGE_BYTES;
             uint8_t* v_tile = k_tile + L::TILE_BYTES;
-            const int fill = min(TILE, (cnt + 15) & ~15);
+            // (the fused small form gives a whole response tile to one warp, which looks at all of it)
+            constexpr bool kWholeResp = FUSED && CW == 2 && D <= 128 && NT == 1;
+            const int fill = kWholeResp ? TILE : min(TILE, (cnt + 15) & ~15);
             const int zchunks = (fill - cnt) * 8;      // in every 128-byte box the run is contiguous
 #pragma unroll
             for (int bx = 0; bx < D / 64; ++bx) {
@@ -459,8 +462,14 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 }
             }
             if (lane == 0) tile_hdr[st] = make_int2(cnt, last ? 1 : 0);
+        };
+        auto release_tile = [&](int st) {
             __syncwarp();
             if (lane == 0 && !p.dbg_skip) mbar_arrive(full0 + 8 * st);
+        };
+        auto finish_tile = [&](int st, int cnt, bool last) {
+            pad_tile(st, cnt, last);
+            release_tile(st);
         };
         auto publish_tile = [&](int st, int cnt, bool last) {
             copy_rows(st, 0, cnt, true);
@@ -643,6 +652,14 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                         }
                     }
                     copy_rows(rstage, 0, old_total, false);
+                    // where the new step's rows go, their records and the tile's padding are known too
+                    if (has_new && lane < Wb) {
+                        URow uu;
+                        uu.row = t_new;
+                        uu.mask = 1u << lane;
+                        meta[(size_t)rstage * TILE + old_total + lane] = uu;
+                    }
+                    pad_tile(rstage, old_total + (has_new ? Wb : 0), true);
                 } else if (p.one_wave) {
                     // at least ask the L2 for the rows of the first windows
 #pragma unroll
@@ -660,6 +677,23 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 }
                 grid_wait();
                 grid_launch_dependents();
+                if (fast) {
+                    // The new step's rows need nothing but the wait: their copies go out first, straight
+                    // from the caller's arrays (CPR lanes per row), and land while the parent ids travel.
+                    if (has_new) {
+                        const uint32_t k_dst = smem_u32(ring + (size_t)rstage * L::STAGE_BYTES), v_dst = k_dst + L::TILE_BYTES;
+                        const int c = lane % CPR;
+                        const uint32_t c_off = (uint32_t)(c / 8) * L::BOX_BYTES;
+                        for (int r = lane / CPR; r < Wb; r += RPI) {
+                            const int key = old_total + r;
+                            const uint32_t off = c_off + (uint32_t)key * 128 + (uint32_t)(((c & 7) ^ (key & 7)) << 4);
+                            const size_t src = ((size_t)(b * Wb + r) * p.Hkv + kvh) * (size_t)(D * 2) + (size_t)c * 16;
+                            cp_async_16(k_dst + off, p.k_new + src);
+                            cp_async_16(v_dst + off, p.v_new + src);
+                        }
+                    }
+                    cp_async_mbar_arrive_noinc(full0 + 8 * rstage);      // fires when ALL of this lane's copies, old rows and new, have landed
+                }
             }
             int par = j;
             par = (p.steps > 1 && j < Wb) ? p.parent[b * Wb + j] : j;
@@ -670,7 +704,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             }
             SEGKV_STAMP(4);
             if (fast) {
-                // ---- the rows are on their way: masks, the new table column, the new step's rows ----
+                // ---- the rows are on their way: the beam masks, then the new table column ----
                 // new slot i reads what old slot parent[i] read: turn the sets of old slots into beam masks
                 uint32_t nmask[PF];
 #pragma unroll
@@ -681,39 +715,19 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     for (int u = 0; u < PF; ++u) nmask[u] |= ((fmask[u] >> pi) & 1u) << i;
                 }
 #pragma unroll
+                for (int u = 0; u < PF; ++u)
+                    if (fpos[u] >= 0) meta[(size_t)rstage * TILE + fpos[u]].mask = nmask[u];
+                release_tile(rstage);
+                // off the consumers' path: the table of the new step
+#pragma unroll
                 for (int u = 0; u < PF; ++u) {
                     if (u < nwin) {                                               // warp-uniform
                         const int s = rs0 + u * spw + ls;
                         const int row = __shfl_sync(0xffffffffu, rowb[u], gbase + par);   // anc_{t-1}[parent[j]][s]
-                        if (fpos[u] >= 0) meta[(size_t)rstage * TILE + fpos[u]].mask = nmask[u];
                         if (s < rs1 && j < Wb && s != t_new && kvh == 0) p.anc_dst[(size_t)(b * Wb + j) * p.max_steps + s] = row;
                     }
                 }
-                int cnt = old_total;
-                if (has_new) {
-                    if (lane < Wb) {
-                        URow uu;
-                        uu.row = t_new;
-                        uu.mask = 1u << lane;
-                        meta[(size_t)rstage * TILE + old_total + lane] = uu;
-                        const size_t off = ((size_t)(b * Wb + lane) * p.Hkv + kvh) * (size_t)(D * 2);
-                        gk[old_total + lane] = p.k_new + off;
-                        gv[old_total + lane] = p.v_new + off;
-                        if (kvh == 0) p.anc_dst[(size_t)(b * Wb + lane) * p.max_steps + t_new] = b * Wb + lane;
-                    }
-                    cnt += Wb;
-                    // the new rows' copies: CPR lanes per row, straight from the caller's arrays
-                    __syncwarp();
-                    const uint32_t k_dst = smem_u32(ring + (size_t)rstage * L::STAGE_BYTES), v_dst = k_dst + L::TILE_BYTES;
-                    for (int i = lane; i < Wb * CPR; i += 32) {
-                        const int key = old_total + i / CPR, c = i % CPR;
-                        const uint32_t off = (uint32_t)(c / 8) * L::BOX_BYTES + (uint32_t)key * 128 + (uint32_t)(((c & 7) ^ (key & 7)) << 4);
-                        cp_async_16(k_dst + off, gk[key] + c * 16);
-                        cp_async_16(v_dst + off, gv[key] + c * 16);
-                    }
-                }
-                cp_async_mbar_arrive_noinc(full0 + 8 * rstage);      // fires when ALL of this lane's copies, old rows and new, have landed
-                finish_tile(rstage, cnt, true);
+                if (has_new && lane < Wb && kvh == 0) p.anc_dst[(size_t)(b * Wb + lane) * p.max_steps + t_new] = b * Wb + lane;
             }
             // Windows of spw steps at fixed positions; the table entries of four windows are
             // requested at once, so a split of up to 4 * spw steps pays one memory round trip.
@@ -991,8 +1005,35 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             if (warp == 0) SEGKV_STAMP(2);
             begin(true);
         };
+        // Fused step: one response tile; how many there are and how full each is only the gather warp
+        // knows, which says so in the tile's header.  The first has a stage of its own when p.resv.
+        int r_done = 0;
+        bool resp_last = !(FUSED && rs1 > rs0);
+        auto resp_tile = [&]() {
+            const bool own = p.resv && r_done == 0;
+            const int sr = own ? rstage : st;
+            ok = mbar_wait(full0 + 8 * sr, own ? 0u : ph, p.wait_ns);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) return;
+            const int2 hd = tile_hdr[sr];
+            consume(IntC<1>{}, sr, true, hd.x, 0, warp * 16);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8 * sr);
+            if (!own) next_stage();
+            ++r_done;
+            resp_last = hd.y != 0;
+        };
         if constexpr (kWholeTile) {
             for (; k < npt; ++k) {
+                if constexpr (FUSED) {
+                    // The rows of that stage were asked for before the wait, so the tile is there long
+                    // before the prompt tiles that had to wait for a stage of the ring: it is consumed
+                    // after the first round of prompt tiles, while those reloads travel.
+                    if (p.resv && k == RS && !resp_last && r_done == 0) {
+                        resp_tile();
+                        if (!ok) break;
+                    }
+                }
                 // every warp waits for every tile, also those it leaves to the other warp: a parity
                 // wait cannot tell a barrier's phases two apart, so none may be skipped
                 if (k >= 0) {
@@ -1045,23 +1086,8 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 if (lane == 0) mbar_arrive(empty0 + 8 * sr);
                 if (!own) next_stage();
             }
-        } else if (ok && rs1 > rs0) {
-            // fused step: how many response tiles there are and how full each is only the gather
-            // warp knows; it says so in the tile's header
-            for (int r = 0;; ++r) {
-                const bool own = p.resv && r == 0;
-                const int sr = own ? rstage : st;
-                ok = mbar_wait(full0 + 8 * sr, own ? 0u : ph, p.wait_ns);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                const int2 hd = tile_hdr[sr];
-                consume(IntC<1>{}, sr, true, hd.x, 0, warp * 16);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8 * sr);
-                if (!own) next_stage();
-                ++k;
-                if (hd.y) break;
-            }
+        } else {
+            while (ok && !resp_last) resp_tile();
         }
         if (!ok && lane == 0) {
             atomicOr(p.err_word, SEGKV_DEV_WAIT_LIMIT);
