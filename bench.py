@@ -53,6 +53,7 @@ def parse():
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--combine", type=int, default=0, help="0 auto, 1 workspace+ticket, 2 cluster")
     ap.add_argument("--tile", type=int, default=0, help="keys per tile of the decode kernel: 0 auto, 32 (quarter-SM CTAs), 64")
+    ap.add_argument("--persistent", type=int, default=-1, help="persistent form of the attention call: -1 auto, 0 never, 1 always")
     ap.add_argument("--prompt-layout", default="head_major", choices=["head_major", "token_major", "seq_first"],
                     help="memory layout of the prompt segment (the paper's Fig. 6 compares layouts)")
     ap.add_argument("--beams", type=int, default=0, help="override the workload's beam width")
@@ -236,6 +237,8 @@ class ShapeBench:
             h = SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, w.steps, w.torch_dtype)
             if args.tile:
                 h.set_tile(args.tile)
+            if args.persistent != -1:
+                h.set_persistent(args.persistent)
             if args.splits or args.stages or args.combine:
                 h.set_tuning(args.splits, args.stages, args.combine)
             if args.no_overlap:

@@ -353,6 +353,20 @@ SEGKV_API int segkv_set_tuning(segkv_t h, int splits, int stages, int combine);
  * that has no such form).
  */
 SEGKV_API int segkv_set_tile(segkv_t h, int tile_keys);
+
+/*
+ * Persistent form of segkv_decode_sdpa (a launch-shape knob: the paper has no
+ * counterpart).  Instead of one CTA per (request, kv head, split), a grid of two
+ * resident CTAs per SM walks those items round-robin, with the split count
+ * chosen so that every CTA gets the same number of items: for launches between
+ * one and a few waves of CTAs, whose last wave would otherwise leave SMs idle.
+ * Results are those of segkv_decode_sdpa within the same tolerance (the keys
+ * are grouped differently, so the low bits differ).  mode: -1 automatic (the
+ * default), 0 never, 1 always.  Only for beams*(heads/kv_heads) <= 8; a split
+ * count forced with segkv_set_tuning is used as the items per work group (at
+ * most 8).  Errors: EINVAL (other values, or 1 for an unsupported shape).
+ */
+SEGKV_API int segkv_set_persistent(segkv_t h, int mode);
 SEGKV_API int segkv_get_splits(segkv_t h);
 
 /*

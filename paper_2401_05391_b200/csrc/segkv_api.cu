@@ -346,6 +346,37 @@ Tiling choose_tiling(const segkv* h, bool fused_step) {
     return t;
 }
 
+// Items per work group for the persistent form: the split count (at most 4, at least two prompt tiles
+// per item) whose items deal most evenly over the resident grid; ties go to fewer splits.
+int stream_splits(const segkv* h) {
+    if (h->splits_forced > 0) return h->splits_forced > 8 ? 8 : h->splits_forced;
+    const Dims& d = h->d;
+    const long long slabs = (long long)d.batch * d.kv_heads;
+    const long long grid = (long long)h->sm_count * stream_ctas_per_sm();
+    const int tile = tiled_tile_keys(d.head_dim, false);
+    const long long ntp = ((h->prompt_len > 0 ? h->prompt_len : 0) + tile - 1) / tile;
+    int best = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= 4; ++s) {
+        if (s > 1 && ntp / s < 2) break;
+        const long long items = slabs * s;
+        const long long rounds = (items + grid - 1) / grid;
+        const double eff = (double)items / (double)(rounds * grid) - 0.02 * (s - 1);
+        if (eff > best_eff + 1e-9) {
+            best_eff = eff;
+            best = s;
+        }
+    }
+    return best;
+}
+
+// Does the separate attention call run in the persistent form?
+bool use_stream(const segkv* h) {
+    if (h->persist_mode == 0 || !stream_supported(h->d) || h->tile_forced != 0 || h->combine_forced == 2) return false;
+    if (h->persist_mode == 1) return true;
+    return false;
+}
+
 // The attention kernel's separate form walks per-request lists of distinct rows that the append
 // kernel makes; fused steps skip them, so they are re-derived from the table when needed.
 // The handle that owns the beam-index tables h works with.
@@ -466,6 +497,7 @@ int segkv_create_growing(segkv_t* out, int batch, int beams, int heads, int kv_h
     d.rows = batch * beams; d.dtype = dtype; d.chunk_steps = chunk_steps;
     h->prompt_len = -1;
     h->overlap = true;
+    h->persist_mode = -1;
     h->prefill_groups = 0;
     h->ragged = false;
     h->leader = nullptr;
@@ -728,6 +760,21 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
     {
         int rc = ensure_lists(h, (cudaStream_t)stream);
         if (rc != SEGKV_OK) return rc;
+    }
+    if (use_stream(h)) {
+        const int sp = stream_splits(h);
+        if (sp > h->ws_splits) {
+            SEGKV_CUDA(cudaDeviceSynchronize());
+            int rc = alloc_workspace(h, sp);
+            if (rc != SEGKV_OK) return rc;
+        }
+        SdpaArgs a = sdpa_args(h, q, out, alibi_slopes, sp);
+        a.pdl = h->overlap;
+        h->dbg_wait_ns = 0;
+        h->dbg_skip = false;
+        SEGKV_CUDA(launch_sdpa_stream(h->d, a, h->tm_kp, h->tm_vp, h->sm_count, (cudaStream_t)stream));
+        count_launch(h, (cudaStream_t)stream);
+        return SEGKV_OK;
     }
     const Tiling tl = choose_tiling(h, false);
     const int splits = tl.splits;
@@ -1156,6 +1203,13 @@ int segkv_set_tile(segkv_t h, int tile_keys) {
     if (!h || (tile_keys != 0 && tile_keys != 32 && tile_keys != 64)) return SEGKV_EINVAL;
     if (tile_keys == 32 && !tiled_small_ok(h->d)) return SEGKV_EINVAL;
     h->tile_forced = tile_keys;
+    return SEGKV_OK;
+}
+
+int segkv_set_persistent(segkv_t h, int mode) {
+    if (!h || mode < -1 || mode > 1) return SEGKV_EINVAL;
+    if (mode == 1 && !stream_supported(h->d)) return SEGKV_EINVAL;
+    h->persist_mode = mode;
     return SEGKV_OK;
 }
 

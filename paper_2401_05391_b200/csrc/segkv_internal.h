@@ -64,6 +64,7 @@ struct segkv {
     int stages_forced;   // 0 = automatic
     int combine_forced;  // 0 = automatic, 1 = global workspace + ticket, 2 = cluster
     int tile_forced;     // 0 = automatic, 32 or 64 keys per tile of the decode kernel
+    int persist_mode;    // -1 = automatic, 0 = never, 1 = always: the persistent form of the separate attention call
     bool overlap;        // programmatic dependent launch between consecutive kernels
     int prefill_groups;  // 0 = automatic; 1 or 2 row groups per CTA of the tcgen05 prefill kernel
     bool fuse_always;    // segkv_decode_step uses the fused kernel even for a single split
@@ -189,6 +190,12 @@ bool tiled_cluster_ok(const Dims& d, int splits);        // can `splits` CTAs me
 bool tiled_small_ok(const Dims& d);                      // is there a 32-key-tile form (quarter-SM CTAs) for this shape?
 int tiled_tile_keys(int head_dim, bool small);           // rows of one shared-memory tile
 size_t tiled_smem_bytes(const Dims& d, int stages, bool small);   // dynamic shared memory of one CTA
+// Persistent form of the separate attention call (segkv_sdpa_stream.cu): a resident grid of CTAs walks
+// the (work group, split) items round-robin; a.splits items per work group, merged through the workspace.
+bool stream_supported(const Dims& d);
+int stream_ctas_per_sm();
+cudaError_t launch_sdpa_stream(const Dims& d, const SdpaArgs& a, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                               int sm_count, cudaStream_t st);
 cudaError_t launch_sdpa_tiled(const Dims& d, const SdpaArgs& a, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                               int stages, cudaStream_t st);
 

@@ -51,6 +51,7 @@ SIGNATURES = {
     "segkv_prompt_len": (_int, [_vp]),
     "segkv_set_tuning": (_int, [_vp, _int, _int, _int]),
     "segkv_set_tile": (_int, [_vp, _int]),
+    "segkv_set_persistent": (_int, [_vp, _int]),
     "segkv_decode_sdpa_rowwise": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "segkv_get_splits": (_int, [_vp]),
     "segkv_set_overlap": (_int, [_vp, _int]),
@@ -370,6 +371,9 @@ class SegKV:
 
     def set_tile(self, tile_keys: int = 0) -> None:
         _check(lib().segkv_set_tile(self._h, tile_keys), "segkv_set_tile")
+
+    def set_persistent(self, mode):
+        _check(lib().segkv_set_persistent(self._h, mode), "segkv_set_persistent")
 
     def debug_inject(self, wait_limit_ns: int = 0, skip_arrival: bool = False) -> None:
         _check(lib().segkv_debug_inject(self._h, int(wait_limit_ns), int(bool(skip_arrival))), "segkv_debug_inject")

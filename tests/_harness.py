@@ -15,13 +15,15 @@ ATOL, RTOL = 2e-3, 1e-2   # |gpu - ref| <= ATOL + RTOL*|ref|, the path's stated 
 class Run:
     def __init__(self, w: wl.Workload, device="cuda", max_steps=None, max_prompt=None, parents=None,
                  splits=0, stages=0, combine=0, chunk_steps=0, prompt_layout=None,
-                 prompt_lens=None, tile=0):
+                 prompt_lens=None, tile=0, persistent=-1):
         self.w, self.device = w, device
         self.h = SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim,
                        w.prompt_len if max_prompt is None else max_prompt,
                        w.steps if max_steps is None else max_steps, w.torch_dtype, chunk_steps=chunk_steps)
         if tile:
             self.h.set_tile(tile)
+        if persistent != -1:
+            self.h.set_persistent(persistent)
         if splits or stages or combine:
             self.h.set_tuning(splits, stages, combine)
         if prompt_layout is not None:

@@ -14,9 +14,9 @@ CHECK_STEPS = (0, 1, 2, 3, 7, 15, 16, 17, 31, 63, 127, 255)
 
 
 def run_workload(w, pairs_fn, check_steps=CHECK_STEPS, splits=0, stages=0, combine=0, every_step_ancestry=True,
-                 prompt_layout=None, prompt_lens=None, tile=0):
+                 prompt_layout=None, prompt_lens=None, tile=0, persistent=-1, chunk_steps=0):
     r = Run(w, splits=splits, stages=stages, combine=combine, prompt_layout=prompt_layout, prompt_lens=prompt_lens,
-            tile=tile)
+            tile=tile, persistent=persistent, chunk_steps=chunk_steps)
     try:
         worst = 0.0
         for t in range(w.steps):
@@ -194,6 +194,40 @@ def test_small_cta_form_forced_shapes(splits, stages, combine, fused):
     kw = {} if fused else {"every_step_ancestry": False}
     run(w, lambda w: sampled_pairs(w, 12), check_steps=(0, 7, 39), splits=splits, stages=stages, combine=combine,
         tile=32, **kw)
+
+
+@pytest.mark.parametrize("splits", [0, 1, 2, 3, 5, 8])
+def test_persistent_form_llama2_7b_shape(splits):
+    # resident CTAs walking (work group, split) items round-robin; 1 to 8 items per work group
+    w = wl.CONFIGS[1].scaled(steps=40, index=33)
+    run_workload(w, lambda w: sampled_pairs(w, 12), check_steps=(0, 7, 39), splits=splits, persistent=1,
+                 every_step_ancestry=False)
+
+
+@pytest.mark.parametrize("dtype,D", [("f16", 64), ("bf16", 128), ("f16", 256)])
+def test_persistent_form_ragged_shapes(dtype, D):
+    # prompt not a multiple of the tile, GQA (6 query columns), ALiBi on the bf16 variant, per-request
+    # prompt lengths, a response capacity that grows in chunks, more items than resident CTAs
+    w = wl.Workload("pers", 3, 3, 6, 3, D, 150, 21, dtype, "uniform", dtype == "bf16", 70 + D // 64)
+    run_workload(w, all_pairs, check_steps=(0, 1, 5, 20), persistent=1)
+    run_workload(w, all_pairs, check_steps=(0, 5, 20), persistent=1, splits=2, prompt_lens=[150, 33, 97])
+    run_workload(w, all_pairs, check_steps=(0, 5, 20), persistent=1, splits=3, chunk_steps=4)
+    big = wl.Workload("pers_many", 40, 2, 16, 16, D, 70, 5, dtype, "uniform", dtype == "bf16", 80 + D // 64)
+    run_workload(big, lambda w: sampled_pairs(w, 40), check_steps=(0, 4), persistent=1)
+    run_workload(big, lambda w: sampled_pairs(w, 40), check_steps=(0, 4), persistent=1, splits=2)
+
+
+def test_persistent_form_no_prompt_and_first_step():
+    # no prompt at all (only response rows), and a prompt with no step yet (an empty response tile)
+    w = wl.Workload("pers_np", 2, 4, 4, 4, 128, 0, 12, "f16", "uniform", False, 91)
+    run_workload(w, all_pairs, check_steps=(0, 3, 11), persistent=1)
+    w = wl.Workload("pers_ponly", 2, 4, 4, 4, 128, 100, 4, "f16", "uniform", False, 92)
+    r = Run(w, persistent=1)
+    try:
+        out, q = r.decode()
+        r.check(out, q, -1, all_pairs(w))
+    finally:
+        r.close()
 
 
 @pytest.mark.parametrize("dtype,D", [("f16", 64), ("bf16", 128)])

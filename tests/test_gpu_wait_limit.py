@@ -17,11 +17,11 @@ from _harness import ATOL, RTOL, Run, all_pairs
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("form", ["separate", "fused", "static"])
+@pytest.mark.parametrize("form", ["separate", "fused", "static", "persistent"])
 @pytest.mark.parametrize("splits", [1, 3])
 def test_decode_wait_runs_out_and_the_handle_recovers(form, splits):
     w = wl.Workload("wait", 2, 4, 4, 2, 128, 100, 6, "f16", "uniform", False, 71)
-    r = Run(w, splits=splits)
+    r = Run(w, splits=splits, persistent=1 if form == "persistent" else -1)
     try:
         r.advance_to(3)
         if form == "fused":
