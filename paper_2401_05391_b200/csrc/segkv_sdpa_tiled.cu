@@ -1159,8 +1159,12 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 const uint32_t rbar = mapa_shared(recvbar, (uint32_t)r);
                 st_async_v4(mapa_shared(smem_u32(recv_o + (size_t)me * slice + 4 * f4 - r * slice), (uint32_t)r), o, rbar);
                 if (d == 0) {
-                    // a CTA that gave up says so with a NaN maximum: its peers then leave the output alone
-                    if (bad) mm = __int_as_float(0x7fc00000);
+                    // a CTA that gave up says so with a NaN sum (and no weight): the sum of the fold is then NaN
+                    // and its peers leave the output alone
+                    if (bad) {
+                        mm = -INFINITY;
+                        ll = __int_as_float(0x7fc00000);
+                    }
                     for (int r2 = 0; r2 < S; ++r2)
                         st_async_v2(mapa_shared(smem_u32(recv_ml + ((size_t)me * ncols + col) * 2), (uint32_t)r2), mm, ll,
                                     mapa_shared(recvbar, (uint32_t)r2));
@@ -1171,44 +1175,35 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             got = __all_sync(0xffffffffu, got);
             if (tid == 0) SEGKV_STAMP(12);
             if (!got && lane == 0) atomicOr(p.err_word, SEGKV_DEV_WAIT_LIMIT);
-            // fold: thread x takes partial s = x % S of float4 i = x / S of the slice; the S partials
-            // of one float4 sit in neighbouring lanes and are reduced with shuffles
-            const int l2s = 31 - __clz(S);
-            const int items = (slice >> 2) << l2s;
-            for (int x0 = 0; x0 < items && got; x0 += CT) {
-                const int x = x0 + tid;
-                const bool in = x < items;
-                const int i = in ? x >> l2s : 0, sp = in ? x & (S - 1) : 0;
-                const int fl = (int)me * slice + 4 * i;
+            // fold: one thread per float of the slice; the S partials of that float and their {max, sum}
+            // pairs are all asked for at once, no lane talks to another
+            for (int e = tid; e < slice && got; e += CT) {
+                const int fl = (int)me * slice + e;
                 const int col = fl / D, d = fl % D;
-                const float2 ml = in ? *reinterpret_cast<const float2*>(recv_ml + ((size_t)sp * ncols + col) * 2)
-                                     : make_float2(-INFINITY, 0.f);
-                float4 v = in ? *reinterpret_cast<const float4*>(recv_o + (size_t)sp * slice + 4 * i)
-                              : make_float4(0.f, 0.f, 0.f, 0.f);
-                float mm = ml.x;
-                bool poison = ml.x != ml.x;
-                for (int o = 1; o < S; o <<= 1) {
-                    mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
-                    poison = __shfl_xor_sync(0xffffffffu, (int)poison, o) != 0 || poison;
+                float mp[kMaxCluster], lp[kMaxCluster], vp[kMaxCluster];
+#pragma unroll
+                for (int sp = 0; sp < kMaxCluster; ++sp) {
+                    const bool in = sp < S;
+                    const float2 ml = in ? *reinterpret_cast<const float2*>(recv_ml + ((size_t)sp * ncols + col) * 2)
+                                         : make_float2(-INFINITY, 0.f);
+                    mp[sp] = ml.x;
+                    lp[sp] = ml.y;
+                    vp[sp] = in ? recv_o[(size_t)sp * slice + e] : 0.f;
                 }
-                const float f = (ml.x == -INFINITY || poison) ? 0.f : exp2f(ml.x - mm);
-                float ll = ml.y * f;
-                v.x *= f; v.y *= f; v.z *= f; v.w *= f;
-                for (int o = 1; o < S; o <<= 1) {
-                    ll += __shfl_xor_sync(0xffffffffu, ll, o);
-                    v.x += __shfl_xor_sync(0xffffffffu, v.x, o);
-                    v.y += __shfl_xor_sync(0xffffffffu, v.y, o);
-                    v.z += __shfl_xor_sync(0xffffffffu, v.z, o);
-                    v.w += __shfl_xor_sync(0xffffffffu, v.w, o);
+                float mm = mp[0];
+#pragma unroll
+                for (int sp = 1; sp < kMaxCluster; ++sp) mm = fmaxf(mm, mp[sp]);
+                float ll = 0.f, v = 0.f;
+#pragma unroll
+                for (int sp = 0; sp < kMaxCluster; ++sp) {
+                    const float f = (mp[sp] == -INFINITY) ? 0.f : exp2f(mp[sp] - mm);
+                    ll += lp[sp] * f;                       // NaN from a CTA that gave up stays NaN
+                    v += vp[sp] * f;
                 }
-                if (in && sp == 0 && !poison) {
-                    const float inv = 1.f / ll;
+                if (ll == ll) {
                     const int j = col / p.G, hg = col % p.G;
                     T* orow = reinterpret_cast<T*>(p.out) + ((size_t)(b * p.W + j) * p.H + kvh * p.G + hg) * D + d;
-                    uint2 pk;
-                    pk.x = Mma<T>::pack(v.x * inv, v.y * inv);
-                    pk.y = Mma<T>::pack(v.z * inv, v.w * inv);
-                    *reinterpret_cast<uint2*>(orow) = pk;
+                    *orow = Mma<T>::down(v * (1.f / ll));
                 }
             }
             if (tid == 0) SEGKV_STAMP(13);
