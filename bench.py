@@ -438,12 +438,18 @@ def run_ours(args):
     # ---- end to end from host memory through segkv_layers_step_host
     e2e = None
     if not args.no_e2e:
-        # every layer's step inputs packed into one pinned host block (one copy in, one launch, one copy out)
+        # every layer's step inputs packed into one pinned host block; the library queues the copies in, the
+        # launches and the copies out of all layers in one call
         total, off = handles[0][0].host_pack_layout()
         hs = slopes is not None
         hq = []
-        for _, q, k, v, _, _ in handles:
-            blk = torch.zeros(total, dtype=torch.uint8).pin_memory()
+        # ONE pinned array for the inputs of all layers and one for their outputs (a layer's block is a
+        # slice): blocks that lie back to back let the library move several layers with one copy
+        q0 = handles[0][1]
+        blk_all = torch.zeros(len(handles), total, dtype=torch.uint8).pin_memory()
+        out_all = torch.empty((len(handles),) + tuple(q0.shape), dtype=q0.dtype).pin_memory()
+        for li, (_, q, k, v, _, _) in enumerate(handles):
+            blk = blk_all[li]
 
             def put(o, x):
                 raw = x.contiguous().cpu().view(torch.uint8).reshape(-1)
@@ -453,7 +459,7 @@ def run_ours(args):
             if hs:
                 put(off[1], slopes)
             put(off[2], k); put(off[3], v); put(off[4], q)
-            hq.append((blk, torch.empty_like(q, device="cpu").pin_memory()))
+            hq.append((blk, out_all[li]))
 
         from paper_2401_05391_b200.segkv import LayerStack
         stack = LayerStack([h[0] for h in handles], [x[0] for x in hq], [x[1] for x in hq])

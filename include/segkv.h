@@ -289,7 +289,12 @@ SEGKV_API int segkv_step_host_packed_async(segkv_t h, int step, const void* host
  * library's own, so that one layer's inputs arrive while the layer before it
  * computes, and `stream` ends behind the last copy out: waiting for `stream`
  * is waiting for every output.  (On a stream that is being captured everything
- * stays on `stream`.)  redo != 0 re-times a step: a handle whose newest
+ * stays on `stream`.)  When the layers have the same shape and their blocks lie
+ * back to back in host memory (host_in[i+1] = host_in[i] + block bytes, the same
+ * for host_out: slices of one pinned array), several layers travel in one copy
+ * each way through a staging area that the first layer's handle keeps; that area
+ * is allocated at the first such call of a stack, which synchronises the device
+ * once.  redo != 0 re-times a step: a handle whose newest
  * step is `step` drops it first (segkv_truncate_last) and takes it again.
  * No counterpart in the paper (an interface convenience: one call per decode
  * step instead of one per layer).  Errors: those of the single-layer call, at

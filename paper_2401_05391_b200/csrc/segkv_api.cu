@@ -179,7 +179,7 @@ bool settled(const WriteMark* m, cudaStream_t st) { return older_than_latest(st,
 void free_all(segkv* h) {
     void* ptrs[] = {h->kp, h->vp, h->kr, h->k_chunks_dev, h->parent, h->anc[0], h->anc[1], h->ulist, h->ucount, h->plens,
                     h->err_word, h->ws, h->tickets, h->st_q, h->st_out, h->st_k, h->st_v, h->st_parent, h->st_pack,
-                    h->st_slopes};
+                    h->st_slopes, h->grp_in, h->grp_out};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     if (h->ev_in) cudaEventDestroy(h->ev_in);
@@ -1031,6 +1031,73 @@ int segkv_layers_step_host(const segkv_t* layers, int n, int step, const void* c
     SEGKV_CUDA(cudaEventRecord(cs->entry, st));
     SEGKV_CUDA(cudaStreamWaitEvent(cs->in, cs->entry, 0));
     SEGKV_CUDA(cudaStreamWaitEvent(cs->out, cs->entry, 0));
+    // When the caller's blocks of all layers lie back to back in host memory (one pinned array for the
+    // stack), several layers travel in ONE copy each way: a copy call costs the host a few microseconds,
+    // which at small shapes is as much as the layer's launch.  All inputs are queued first; the launches of
+    // a group of layers wait for their group's copy, the group's outputs leave behind its last launch.
+    {
+        segkv_t h0 = layers[0];
+        size_t off[5];
+        const size_t total = segkv_host_pack_bytes(h0, off);
+        const size_t qbytes = (size_t)h0->d.rows * h0->d.heads * h0->d.head_dim * 2;
+        bool block = n >= 2;
+        for (int i = 1; i < n && block; ++i) {
+            const Dims &a = layers[i]->d, &b = h0->d;
+            block = a.rows == b.rows && a.heads == b.heads && a.kv_heads == b.kv_heads && a.head_dim == b.head_dim &&
+                    (const char*)host_in[i] == (const char*)host_in[0] + (size_t)i * total &&
+                    (char*)host_out[i] == (char*)host_out[0] + (size_t)i * qbytes;
+        }
+        if (block) {
+            if (h0->grp_in_cap < (size_t)n * total || h0->grp_out_cap < (size_t)n * qbytes) {
+                // first call of this stack (or a longer one): the only allocation, outside the steady state
+                SEGKV_CUDA(cudaDeviceSynchronize());
+                if (h0->grp_in) cudaFree(h0->grp_in);
+                if (h0->grp_out) cudaFree(h0->grp_out);
+                h0->grp_in = h0->grp_out = nullptr;
+                h0->grp_in_cap = h0->grp_out_cap = 0;
+                SEGKV_CUDA(cudaMalloc(&h0->grp_in, (size_t)n * total));
+                SEGKV_CUDA(cudaMalloc(&h0->grp_out, (size_t)n * qbytes));
+                h0->grp_in_cap = (size_t)n * total;
+                h0->grp_out_cap = (size_t)n * qbytes;
+                SEGKV_CUDA(cudaEventRecord(cs->entry, st));
+                SEGKV_CUDA(cudaStreamWaitEvent(cs->in, cs->entry, 0));
+                SEGKV_CUDA(cudaStreamWaitEvent(cs->out, cs->entry, 0));
+            }
+            // groups of about 400 KB of input: long enough to amortise the call, short enough to start early
+            int per = (int)((400u << 10) / (total ? total : 1));
+            if (per < 1) per = 1;
+            if (per > n) per = n;
+            char* gin = (char*)h0->grp_in;
+            char* gout = (char*)h0->grp_out;
+            for (int g0 = 0; g0 < n; g0 += per) {
+                const int cnt = n - g0 < per ? n - g0 : per;
+                SEGKV_CUDA(cudaMemcpyAsync(gin + (size_t)g0 * total, host_in[g0], (size_t)cnt * total, cudaMemcpyHostToDevice, cs->in));
+                SEGKV_CUDA(cudaEventRecord(layers[g0]->ev_in, cs->in));
+            }
+            for (int g0 = 0; g0 < n; g0 += per) {
+                const int cnt = n - g0 < per ? n - g0 : per;
+                SEGKV_CUDA(cudaStreamWaitEvent(st, layers[g0]->ev_in, 0));
+                for (int i = g0; i < g0 + cnt; ++i) {
+                    segkv_t h = layers[i];
+                    if (redo && h->steps == step + 1 && !h->truncated) {
+                        h->steps -= 1;
+                        h->truncated = true;
+                    }
+                    char* base = gin + (size_t)i * total;
+                    const int rc = segkv_decode_step(h, step, step > 0 ? (const int32_t*)(base + off[0]) : nullptr, base + off[2],
+                                                     base + off[3], base + off[4], gout + (size_t)i * qbytes,
+                                                     has_slopes ? (const float*)(base + off[1]) : nullptr, stream);
+                    if (rc != SEGKV_OK) return rc;
+                }
+                SEGKV_CUDA(cudaEventRecord(layers[g0]->ev_k, st));
+                SEGKV_CUDA(cudaStreamWaitEvent(cs->out, layers[g0]->ev_k, 0));
+                SEGKV_CUDA(cudaMemcpyAsync(host_out[g0], gout + (size_t)g0 * qbytes, (size_t)cnt * qbytes, cudaMemcpyDeviceToHost, cs->out));
+            }
+            SEGKV_CUDA(cudaEventRecord(cs->done, cs->out));
+            SEGKV_CUDA(cudaStreamWaitEvent(st, cs->done, 0));
+            return SEGKV_OK;
+        }
+    }
     for (int i = 0; i < n; ++i) {
         segkv_t h = layers[i];
         if (redo && h->steps == step + 1 && !h->truncated) {

@@ -86,6 +86,8 @@ struct segkv {
     int followers;       // handles that use THIS one's tables; it cannot be destroyed while there are any
     void* st_pack;       // staging for segkv_step_host_packed: parent | slopes | k | v | q in one block
     cudaEvent_t ev_in, ev_k;   // segkv_layers_step_host: this layer's inputs have arrived / its launch is queued
+    void *grp_in, *grp_out;    // segkv_layers_step_host, kept by the first layer of a stack: staging for all of its
+    size_t grp_in_cap, grp_out_cap;   // layers in one piece, so that several layers travel in one copy
     int32_t* plens;      // [batch] per-request prompt lengths (segkv_prefill_write_ragged)
     bool ragged;         // plens is in use; prompt_len is then the longest
     segkv_impl::URow* ulist;   // [batch, beams*max_steps] distinct response rows per request

@@ -574,16 +574,24 @@ def test_step_host_packed_matches_device_calls():
         r.close(); r2.close()
 
 
-def test_layers_step_host_queues_every_layer_in_one_call():
-    # three layers driven from pinned host blocks with one call per step; redo re-times the newest step
-    w = wl.Workload("stack", 1, 4, 8, 8, 128, 300, 6, "bf16", "uniform", True, 120)
+@pytest.mark.parametrize("one_array,heads,layers", [(False, 8, 3), (True, 8, 3), (True, 32, 6)])
+def test_layers_step_host_queues_every_layer_in_one_call(one_array, heads, layers):
+    # layers driven from pinned host blocks with one call per step; redo re-times the newest step.  Blocks
+    # that are slices of one pinned array travel several layers per copy (32 heads, 6 layers: two groups).
+    w = wl.Workload("stack", 1, 4, heads, heads, 128, 300, 6, "bf16", "uniform", True, 120)
     par = wl.make_parents(w)
-    ls = [Run(w.scaled(index=120 + i), parents=par) for i in range(3)]
+    ls = [Run(w.scaled(index=120 + i), parents=par) for i in range(layers)]
     hs = [sk.SegKV(w.batch, w.beams, w.heads, w.kv_heads, w.head_dim, w.prompt_len, w.steps, w.torch_dtype) for _ in ls]
     try:
         total, off = hs[0].host_pack_layout()
-        blks = [torch.zeros(total, dtype=torch.uint8).pin_memory() for _ in ls]
-        outs = [torch.empty(w.rows, w.heads, w.head_dim, dtype=w.torch_dtype).pin_memory() for _ in ls]
+        if one_array:
+            blk_all = torch.zeros(layers, total, dtype=torch.uint8).pin_memory()
+            out_all = torch.empty(layers, w.rows, w.heads, w.head_dim, dtype=w.torch_dtype).pin_memory()
+            blks = [blk_all[i] for i in range(layers)]
+            outs = [out_all[i] for i in range(layers)]
+        else:
+            blks = [torch.zeros(total, dtype=torch.uint8).pin_memory() for _ in ls]
+            outs = [torch.empty(w.rows, w.heads, w.head_dim, dtype=w.torch_dtype).pin_memory() for _ in ls]
         for r, h in zip(ls, hs):
             h.prefill_write(r.kp, r.vp)
         stack = sk.LayerStack(hs, blks, outs)
