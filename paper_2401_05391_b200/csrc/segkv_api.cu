@@ -295,8 +295,12 @@ Tiling choose_tiling(const segkv* h, bool fused_step) {
         // still make one wave of them (0.76 and 0.83 there).
         const long long slabs = (long long)d.batch * d.kv_heads;
         const long long slots_small = (long long)h->sm_count * ctas_per_sm(true);
+        const long long slots_regular = (long long)h->sm_count * ctas_per_sm(false);
+        // (work groups that fill two thirds or more of ONE wave of the regular form are best left alone, one
+        // regular CTA each: 0.76 / 0.82 / 0.86 at batch 5 / 6 / 7 against 0.71 / 0.76 / 0.80 in the small form)
+        const bool one_regular_wave = 3 * slabs >= 2 * slots_regular && slabs <= slots_regular;
         if (h->tile_forced == 0 && h->splits_forced <= 0 && tiled_small_ok(d) && 2 * slabs > h->sm_count * 2 &&
-            slabs <= slots_small)
+            slabs <= slots_small && !one_regular_wave)
             t.small = true;
     }
     const int tile = tiled_tile_keys(d.head_dim, t.small);
