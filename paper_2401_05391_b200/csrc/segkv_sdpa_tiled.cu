@@ -370,6 +370,8 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     // result away: the loop's instructions are then in the instruction cache when the real first
     // tile comes (straight-line code that runs once per CTA is bound by instruction fetch).
     const bool cons_ahead = warp < CW && p.early_prompt;
+    // (Warps that work ahead wait later and leave the release to the others: the TMA warp always comes
+    // through here, and one thread's release stands for its CTA.)
     if (!gather_ahead && !cons_ahead) {
         grid_wait();
         grid_launch_dependents();
@@ -555,7 +557,6 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                 }
                 tiles(r_now);
                 grid_wait();
-                grid_launch_dependents();
             }
             tiles(nrt);
             SEGKV_STAMP(5);
@@ -676,7 +677,6 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     }
                 }
                 grid_wait();
-                grid_launch_dependents();
                 if (fast) {
                     // The new step's rows need nothing but the wait: their copies go out first, straight
                     // from the caller's arrays (CPR lanes per row), and land while the parent ids travel.
@@ -1001,7 +1001,6 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         if (cons_ahead) k = -1;
         auto warmed_up = [&]() {
             grid_wait();
-            grid_launch_dependents();
             if (warp == 0) SEGKV_STAMP(2);
             begin(true);
         };
