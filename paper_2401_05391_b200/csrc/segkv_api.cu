@@ -246,6 +246,7 @@ struct Tiling {
     bool one_wave;    // all CTAs of the launch fit on the GPU at once and have only a few tiles each
     bool cluster;     // the splits of a work group merge inside a thread-block cluster
     bool small;       // 32-key tiles, quarter-SM CTAs
+    int tail_groups, tail_splits;   // the work groups of a ragged last wave, cut finer so that they cover all SMs
 };
 
 // CTAs of the chosen form that one SM holds at once.
@@ -280,6 +281,7 @@ Tiling choose_tiling(const segkv* h, bool fused_step) {
             t.small = true;
             t.cluster = true;
             t.one_wave = true;
+            t.tail_groups = t.tail_splits = 0;
             t.splits = 8;
             t.stages = 2;
             const size_t budget = (h->smem_optin + 1024) / ctas_per_sm(true) - 1024;
@@ -347,6 +349,23 @@ Tiling choose_tiling(const segkv* h, bool fused_step) {
     // cluster merge saves.  With overlap off the cluster merge is the faster one.
     const bool want_cluster = h->combine_forced == 2 || (h->combine_forced == 0 && !h->overlap);
     t.cluster = sp > 1 && want_cluster && tiled_cluster_ok(d, sp);
+    // More work groups than CTA slots, one CTA each, and a last wave that fills at most half of the slots:
+    // that wave alone would take as long as a full one (Llama2-13B shape at batch 16: 640 CTAs on 296 slots,
+    // 0.78 of the copy bandwidth).  Its work groups are cut into as many splits as spread them over all slots;
+    // they are the last CTAs of the grid, so they start when the full waves drain.
+    t.tail_groups = t.tail_splits = 0;
+    if (!fused_step && sp == 1 && h->splits_forced <= 0 && !t.cluster && slabs > slots) {
+        const long long r = slabs % slots;
+        if (r > 0 && 2 * r <= slots) {
+            long long s = slots / r;
+            if (s > 8) s = 8;
+            if (s > ntp / 2) s = ntp / 2;          // at least two prompt tiles per CTA
+            if (s >= 2) {
+                t.tail_groups = (int)r;
+                t.tail_splits = (int)s;
+            }
+        }
+    }
     return t;
 }
 
@@ -428,6 +447,7 @@ SdpaArgs sdpa_args(const segkv* h, const void* q, void* out, const float* slopes
     a.prompt_len = h->prompt_len > 0 ? h->prompt_len : 0;
     a.steps = h->steps;
     a.splits = splits;
+    a.tail_groups = a.tail_splits = 0;
     a.cluster = false;
     a.small = false;
     a.one_wave = false;
@@ -793,6 +813,8 @@ int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float* alibi_sl
     a.cluster = tl.cluster;
     a.small = tl.small;
     a.one_wave = tl.one_wave;
+    a.tail_groups = tl.tail_groups;
+    a.tail_splits = tl.tail_splits;
     a.pdl = h->overlap;
     a.rows_immutable = rows_settled(h, (cudaStream_t)stream, true);
     h->dbg_wait_ns = 0;                  // an injected fault applies to one launch

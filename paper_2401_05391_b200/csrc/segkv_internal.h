@@ -158,6 +158,8 @@ struct SdpaArgs {
     int* tickets;
     int* err_word;
     int prompt_len, steps, splits;
+    int tail_groups, tail_splits;   // the last tail_groups work groups get tail_splits splits instead (0: none);
+                                    // workspace merge only; the workspace then holds the tail's items when splits == 1
     bool small;              // 32-key tiles and two consumer warps (tensor maps with 32-row boxes)
     bool one_wave;           // every CTA of the launch is resident at once with a few tiles each: latency, not
                              // bandwidth, is what counts; a stage of the ring may be set aside for the response rows

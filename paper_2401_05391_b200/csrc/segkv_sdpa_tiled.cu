@@ -163,6 +163,11 @@ struct TiledParams {
     int P, steps, S, W, G, H, Hkv, rows, max_steps, ncols, stages;
     int chunk_steps;   // 0: the response segment is one array
     int quota;      // distinct response rows per split (the last split also takes any excess)
+    int tail_groups;   // the last tail_groups work groups are cut into tail_S splits instead of S (a ragged last
+    int tail_S;        // wave spread over all SMs); their quota is tail_quota; the split workspace holds only
+    int tail_quota;    // the items from ws_item0 on
+    int ws_item0;
+    int head_items;    // CTAs of the work groups before the tail
     int cluster;    // 1: the S CTAs of a work group form a thread-block cluster
     int early_prompt;  // 1: prompt tiles may be fetched before the previous kernel has completed
     int early_rows;    // 1: so may the response rows of earlier steps and (separate form) the row lists
@@ -247,8 +252,15 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     const int rstage = stages - 1;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) SEGKV_STAMP(0);
-    const int split = blockIdx.x % p.S;
-    const int slab = blockIdx.x / p.S;           // b * Hkv + kvh
+    // blockIdx -> (work group, split): S splits per group, except that the last tail_groups groups have tail_S
+    const int head_items = p.head_items;
+    const bool in_tail = (int)blockIdx.x >= head_items;
+    const int SS = in_tail ? p.tail_S : p.S;                         // splits of THIS work group
+    const int quota = in_tail ? p.tail_quota : p.quota;
+    const int split = in_tail ? ((int)blockIdx.x - head_items) % p.tail_S : (int)blockIdx.x % p.S;
+    const int slab = in_tail ? head_items / p.S + ((int)blockIdx.x - head_items) / p.tail_S
+                             : (int)blockIdx.x / p.S;                // b * Hkv + kvh
+    const int ws_item = (int)blockIdx.x - p.ws_item0;               // this CTA's place in the split workspace
     const int b = slab / p.Hkv, kvh = slab % p.Hkv;
 
     // This CTA's share of the work group: whole prompt tiles (known from the launch shape
@@ -259,11 +271,11 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     // grid-dependency wait
     const int P = p.plens ? __ldg(p.plens + b) : p.P;
     const int ntp = (P + TILE - 1) / TILE;
-    const int pt0 = (int)((long long)split * ntp / p.S), pt1 = (int)((long long)(split + 1) * ntp / p.S);
+    const int pt0 = (int)((long long)split * ntp / SS), pt1 = (int)((long long)(split + 1) * ntp / SS);
     const int npt = pt1 - pt0;
     const URow* ulist_b = p.ulist + (size_t)b * p.W * p.max_steps;
     // fused step: response steps are cut evenly over the splits (known from the launch shape alone)
-    const int rs0 = (int)((long long)split * p.steps / p.S), rs1 = (int)((long long)(split + 1) * p.steps / p.S);
+    const int rs0 = (int)((long long)split * p.steps / SS), rs1 = (int)((long long)(split + 1) * p.steps / SS);
 
     auto issue_prompt_tile = [&](int k, int st) {
         const uint32_t full = full0 + 8 * st;
@@ -488,12 +500,12 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             for (int kk = 0; kk < UK; ++kk) {
                 const int key = lane + 32 * kk;
                 unext[kk] = (p.steps > 0 && key < TILE)
-                                ? *reinterpret_cast<const uint2*>(ulist_b + min(split * p.quota + key, cap - 1))
+                                ? *reinterpret_cast<const uint2*>(ulist_b + min(split * quota + key, cap - 1))
                                 : make_uint2(0u, 0u);
             }
             const int n_b = p.steps > 0 ? p.ucount[b] : 0;
-            const int e0 = min(split * p.quota, n_b);
-            const int e1 = (split == p.S - 1) ? n_b : min((split + 1) * p.quota, n_b);
+            const int e0 = min(split * quota, n_b);
+            const int e1 = (split == SS - 1) ? n_b : min((split + 1) * quota, n_b);
             const int nrt = (e1 - e0 + TILE - 1) / TILE;
             SEGKV_STAMP(4);
             // Tiles [r, r_end) of this CTA's range of the list: row pointers and per-key records into
@@ -799,7 +811,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
             // store what the step appends: the parent ids and the new K/V rows of this work group
             if (kvh == 0 && split == 0 && lane < Wb)
                 p.parent_row[b * Wb + lane] = p.steps > 1 ? p.parent[b * Wb + lane] : lane;
-            if (split == p.S - 1) {
+            if (split == SS - 1) {
                 for (int i = lane; i < Wb * CPR; i += 32) {
                     const size_t off = ((size_t)(b * Wb + i / CPR) * p.Hkv + kvh) * (size_t)(D * 2) + (size_t)(i % CPR) * 16;
                     *reinterpret_cast<uint4*>(p.kr_new_slab + off) = *reinterpret_cast<const uint4*>(p.k_new + off);
@@ -1071,8 +1083,8 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         }
         if (warp == 0) SEGKV_STAMP(8);
         if (ok && !FUSED) {
-            const int e0 = min(split * p.quota, n_b);
-            const int e1 = (split == p.S - 1) ? n_b : min((split + 1) * p.quota, n_b);
+            const int e0 = min(split * quota, n_b);
+            const int e1 = (split == SS - 1) ? n_b : min((split + 1) * quota, n_b);
             const int nrt = (e1 - e0 + TILE - 1) / TILE;
             for (int r = 0; r < nrt; ++r, ++k) {
                 const bool own = p.resv && r == 0;                // the first response tile has a stage of its own
@@ -1258,7 +1270,7 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     __syncthreads();
 
     const int ncols = p.ncols;
-    const int S = p.S;
+    const int S = SS;
     // merged partial of this CTA for one float4 of one column
     auto merged = [&](int col, int d, float& mm, float& ll) -> float4 {
         mm = -INFINITY;
@@ -1296,8 +1308,8 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         return;
     }
 
-    float* wso_cta = p.ws_o + ((size_t)slab * S + split) * ncols * D;
-    float* wsml_cta = p.ws_ml + ((size_t)slab * S + split) * ncols * 2;
+    float* wso_cta = p.ws_o + (size_t)ws_item * ncols * D;
+    float* wsml_cta = p.ws_ml + (size_t)ws_item * ncols * 2;
     for (int it = tid; it < ncols * D4; it += NTHREADS) {
         const int col = it / D4, d = (it % D4) * 4;
         float mm, ll;
@@ -1331,8 +1343,8 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 
     // One pass: each thread owns a float4 of one column and folds the splits in, eight at a
     // time (their partial outputs and max/sum pairs are all requested before any is used).
-    const float2* wsml_slab = reinterpret_cast<const float2*>(p.ws_ml + (size_t)slab * S * ncols * 2);
-    const float* wso_slab = p.ws_o + (size_t)slab * S * ncols * D;
+    const float2* wsml_slab = reinterpret_cast<const float2*>(p.ws_ml + (size_t)(ws_item - split) * ncols * 2);
+    const float* wso_slab = p.ws_o + (size_t)(ws_item - split) * ncols * D;
     for (int it = tid; it < ncols * D4; it += NTHREADS) {
         const int col = it / D4, d = (it % D4) * 4;
         const float4* src = reinterpret_cast<const float4*>(wso_slab + (size_t)col * D + d);
@@ -1398,6 +1410,16 @@ cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk,
     p.scale2 = 1.4426950408889634f / sqrtf((float)D);
     p.quota = (a.steps + 2 * d.beams + a.splits - 1) / a.splits;
     if (p.quota < 1) p.quota = 1;
+    const size_t slabs = (size_t)d.batch * d.kv_heads;
+    const int tail_groups = (a.tail_groups > 0 && a.tail_splits > 0 && !a.cluster) ? a.tail_groups : 0;
+    p.tail_groups = tail_groups;
+    p.tail_S = tail_groups ? a.tail_splits : a.splits;
+    p.tail_quota = (a.steps + 2 * d.beams + p.tail_S - 1) / p.tail_S;
+    if (p.tail_quota < 1) p.tail_quota = 1;
+    p.head_items = (int)((slabs - tail_groups) * a.splits);
+    // work groups that are not split store their output directly: the workspace then starts at the tail
+    p.ws_item0 = (tail_groups && a.splits == 1) ? p.head_items : 0;
+    const size_t items = (size_t)p.head_items + (size_t)tail_groups * p.tail_S;
     p.cluster = a.cluster ? 1 : 0;
     p.early_prompt = (a.pdl && a.prompt_immutable) ? 1 : 0;
     p.early_rows = (a.pdl && a.prompt_immutable && a.rows_immutable) ? 1 : 0;
@@ -1409,12 +1431,11 @@ cudaError_t launch_one(const Dims& d, const SdpaArgs& a, const CUtensorMap& tmk,
     static int launch_id = 0;
     p.dbg_launch = launch_id++;
 #endif
-    const size_t slabs = (size_t)d.batch * d.kv_heads;
     p.ws_o = a.ws;
-    p.ws_ml = a.ws ? a.ws + slabs * a.splits * p.ncols * D : nullptr;
+    p.ws_ml = a.ws ? a.ws + (items - p.ws_item0) * p.ncols * D : nullptr;
 
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(slabs * a.splits), 1, 1);
+    cfg.gridDim = dim3((unsigned)items, 1, 1);
     cfg.blockDim = dim3(32 * (CW + 2), 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;

@@ -217,6 +217,16 @@ def test_persistent_form_ragged_shapes(dtype, D):
     run_workload(big, lambda w: sampled_pairs(w, 40), check_steps=(0, 4), persistent=1, splits=2)
 
 
+@pytest.mark.parametrize("dtype,D,hkv", [("f16", 128, 16), ("bf16", 64, 16), ("f16", 256, 8)])
+def test_ragged_last_wave_is_cut_finer(dtype, D, hkv):
+    # more work groups than CTA slots with a short last wave (640 or 320 on 296 slots): the groups of that
+    # wave are cut into splits and merged through the workspace, the others store their output directly
+    w = wl.Workload("tail", 40, 2, hkv, hkv, D, 300, 5, dtype, "uniform", dtype == "bf16", 95 + D // 64)
+    pairs = sorted(set(sampled_pairs(w, 24)) | {(b, h) for b in (36, 37, 38, 39) for h in (0, 3, hkv - 1)})
+    run_workload(w, lambda w: pairs, check_steps=(0, 4), every_step_ancestry=False)
+    run_workload(w, lambda w: pairs, check_steps=(0, 4), every_step_ancestry=False, prompt_lens=[300 - 7 * (b % 5) for b in range(40)])
+
+
 def test_persistent_form_no_prompt_and_first_step():
     # no prompt at all (only response rows), and a prompt with no step yet (an empty response tile)
     w = wl.Workload("pers_np", 2, 4, 4, 4, 128, 0, 12, "f16", "uniform", False, 91)
