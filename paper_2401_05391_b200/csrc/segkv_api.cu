@@ -891,7 +891,10 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     const int tile_keys = tiled_tile_keys(d.head_dim, tl.small);
     const int ptiles_per_cta = ((h->prompt_len + tile_keys - 1) / tile_keys + splits - 1) / splits;
     const bool long_prompt = h->splits_forced <= 0 && ptiles_per_cta > 7;
-    if ((splits == 1 || long_tail || long_prompt) && !h->fuse_always) {
+    // (a launch of a few unsplit work groups is all latency: there the fused form saves a whole launch,
+    // 3.7 against 6.0 us at the smallest evaluation shape)
+    const bool fills_gpu = (long long)d.batch * d.kv_heads >= h->sm_count;
+    if (((splits == 1 && fills_gpu) || long_tail || long_prompt) && !h->fuse_always) {
         // Work groups that fill the GPU on their own are bandwidth-bound: the separate append is
         // then ~1 % of the step and the list it makes keeps the response tiles dense and cheap
         // to build, so the two launches are the faster form.

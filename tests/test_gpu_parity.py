@@ -546,7 +546,10 @@ def test_step_host_matches_device_calls():
             oh = torch.empty_like(qh).pin_memory()
             ph = torch.from_numpy(r.parents[t]).pin_memory() if t > 0 else None
             r2.h.step_host(t, ph, kh, vh, qh, oh)
-            assert torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16))
+            # the host step runs as one fused launch at this size, the device calls as two: the same rows in a
+            # different order, so the two agree within the path's tolerance, not bit by bit
+            assert torch.allclose(oh.float(), out.cpu().float(), atol=2e-3, rtol=1e-2)
+            r.check(oh.to("cuda"), q, t, all_pairs(w))
     finally:
         r.close(); r2.close()
 
