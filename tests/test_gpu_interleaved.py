@@ -74,7 +74,7 @@ def test_fused_steps_over_three_layers(dtype, D, B, W, steps, tile, splits, comb
                     r.check(out, q, t, all_pairs(w))
                     assert np.array_equal(r.h.get_ancestry(), r.oracle_ancestry(t))
             # (alone, the rows come after the wait in the new parents' order, so the low bits may differ:
-            # only the oracle is the judge of both)
+            # both are compared with the oracle only)
             _, out_ref, q_ref = ref.step_fused()
             if t in (0, 1, 2, 17, 39, 69, 149):
                 ref.check(out_ref, q_ref, t, all_pairs(w))
