@@ -198,8 +198,14 @@ SEGKV_API int segkv_decode_sdpa(segkv_t h, const void* q, void* out, const float
  * `beam_parent` and the previous step's table while it gathers, reads the new
  * rows straight from k_new / v_new, and stores rows, parents and table for the
  * following steps.  Saves a launch and a dependent memory round trip per layer.
- * Arguments, layouts and errors are those of the two calls; shapes with more
- * than 16 query columns per kv head fall back to the two launches.
+ * Arguments, layouts and errors are those of the two calls.  The library runs
+ * the step as the two launches instead where that is the faster form or the only
+ * one: shapes with more than 16 query columns per kv head, handles that share
+ * another handle's tables, launches whose work groups fill the GPU without being
+ * split, and launches whose CTAs would each have many steps' rows or many prompt
+ * tiles to go through.  Both forms give the same beam-index tables bit by bit and
+ * outputs within the stated tolerance of each other (the rows are visited in a
+ * different order).
  */
 SEGKV_API int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const void* k_new,
                                 const void* v_new, const void* q, void* out, const float* alibi_slopes,
