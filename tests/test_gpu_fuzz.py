@@ -1,0 +1,70 @@
+"""Seeded random shapes through every form of the decode path (separate calls, the fused step,
+the persistent form), each checked against the oracle: batch, beams, GQA, head size, prompt
+length (none, ragged tiles, per-request lengths), step count, storage type, ALiBi and the
+parent distribution all vary together, which the hand-picked parity cases do not do."""
+import random
+
+import numpy as np
+import pytest
+
+from paper_2401_05391_b200 import workloads as wl
+
+from _harness import Run, all_pairs, sampled_pairs
+
+pytestmark = pytest.mark.gpu
+
+
+def draw(rng, case, seed):
+    D = rng.choice([64, 128, 128, 256])
+    W = rng.choice([1, 2, 4, 4, 8])
+    G = rng.choice([1, 1, 2, 4])
+    if W * G > 16:
+        G = 1
+    hkv = rng.choice([1, 2, 3, 8, 16, 40])
+    B = rng.choice([1, 2, 3, 5, 8, 16, 20, 40])
+    if B * hkv > 1300:
+        B = max(1, 1300 // hkv)
+    P = rng.choice([0, 17, 64, 150, 300, 511, 700, 1024])
+    steps = rng.choice([1, 3, 6, 12])
+    if P == 0 and steps < 2:
+        steps = 3
+    dtype = rng.choice(["f16", "bf16"])
+    alibi = rng.random() < 0.3
+    mode = rng.choice(["separate", "fused", "persistent", "separate", "fused"])
+    if mode == "persistent" and W * G > 8:
+        mode = "separate"
+    parents = rng.choice(["uniform", "half_identity"])
+    w = wl.Workload("fuzz", B, W, hkv * G, hkv, D, P, steps, dtype, parents, alibi, 5000 + 1000 * seed + case)
+    lens = None
+    if P >= 64 and rng.random() < 0.25:
+        lens = [rng.randint(max(1, P // 3), P) for _ in range(B)]
+        lens[0] = P
+    return w, mode, lens
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_shapes_every_form(seed):
+    rng = random.Random(seed)
+    done = 0
+    for case in range(60):
+        w, mode, lens = draw(rng, case, seed)
+        if w.batch * w.kv_heads * (w.prompt_len + w.steps * w.beams) * w.head_dim * 4 > 400e6:
+            continue
+        r = Run(w, persistent=1 if mode == "persistent" else -1, prompt_lens=lens)
+        try:
+            pairs = sampled_pairs(w, 10) if w.batch * w.heads > 24 else all_pairs(w)
+            for t in range(w.steps):
+                if mode == "fused":
+                    _, out, q = r.step_fused()
+                else:
+                    r.append_next()
+                if t in (0, w.steps // 2, w.steps - 1):
+                    if mode != "fused":
+                        out, q = r.decode()
+                    r.check(out, q, t, pairs)
+            assert r.h.get_error() == 0, (case, w, mode)
+            assert np.array_equal(r.h.get_ancestry(), r.oracle_ancestry(w.steps - 1)), (case, w, mode)
+        finally:
+            r.close()
+        done += 1
+    assert done >= 40
