@@ -68,3 +68,45 @@ def test_random_shapes_every_form(seed):
             r.close()
         done += 1
     assert done >= 40
+
+
+@pytest.mark.parametrize("seed", [21])
+def test_random_shapes_three_handles_in_turn(seed):
+    # three layers stepped in turn on one stream: the launches then read their rows, lists and tables
+    # before the grid-dependency wait (the fast path of the fused step), which a single handle never does
+    rng = random.Random(seed)
+    for case in range(30):
+        D = rng.choice([64, 128, 128])
+        W = rng.choice([1, 2, 4, 4, 8])
+        G = rng.choice([1, 1, 2])
+        if W * G > 8:
+            G = 1
+        hkv = rng.choice([1, 2, 4, 8, 32])
+        B = rng.choice([1, 1, 2, 3])
+        P = rng.choice([256, 300, 511, 700, 1024, 1500])
+        steps = rng.choice([6, 20, 45, 90])
+        dtype = rng.choice(["f16", "bf16"])
+        w = wl.Workload("fuzz3", B, W, hkv * G, hkv, D, P, steps, dtype, rng.choice(["uniform", "half_identity"]),
+                        rng.random() < 0.3, 9000 + 1000 * seed + case)
+        fused = rng.random() < 0.7
+        par = wl.make_parents(w)
+        ls = [Run(w.scaled(index=w.index + 7 * i), parents=par) for i in range(3)]
+        try:
+            pairs = sampled_pairs(w, 8) if w.batch * w.heads > 16 else all_pairs(w)
+            chk = {0, 1, 2, steps // 2, steps - 1}
+            for t in range(steps):
+                if fused:
+                    outs = [r.step_fused()[1:] for r in ls]
+                else:
+                    for r in ls:
+                        r.append_next()
+                    outs = [r.decode() for r in ls]
+                if t in chk:
+                    for r, (out, q) in zip(ls, outs):
+                        r.check(out, q, t, pairs)
+            for r in ls:
+                assert r.h.get_error() == 0, (case, w, fused)
+                assert np.array_equal(r.h.get_ancestry(), r.oracle_ancestry(steps - 1)), (case, w, fused)
+        finally:
+            for r in ls:
+                r.close()
