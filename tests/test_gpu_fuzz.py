@@ -110,3 +110,27 @@ def test_random_shapes_three_handles_in_turn(seed):
         finally:
             for r in ls:
                 r.close()
+
+
+@pytest.mark.parametrize("seed", [31])
+def test_random_shapes_prefill(seed):
+    # the prefill attention (and its fused prompt store) over random batch / heads / head size / prompt length /
+    # storage type / ALiBi / row groups / prompt layout, against the oracle
+    import test_gpu_prefill as pf
+    rng = random.Random(seed)
+    for case in range(40):
+        D = rng.choice([64, 128, 128, 256])
+        G = rng.choice([1, 1, 2, 4])
+        hkv = rng.choice([1, 2, 3, 8, 20])
+        B = rng.choice([1, 2, 3, 7])
+        P = rng.choice([1, 31, 64, 127, 128, 129, 255, 300, 513, 900, 1300, 2048])
+        dtype = rng.choice(["f16", "bf16"])
+        alibi = rng.random() < 0.4
+        groups = rng.choice([0, 1, 2])
+        layout = rng.choice([None, None, "token_major", "seq_first"])
+        if B * hkv * G * P * D > 60e6:
+            continue
+        w = wl.Workload("fuzzpf", B, 2, hkv * G, hkv, D, P, 2, dtype, "uniform", alibi, 12000 + 1000 * seed + case)
+        rows = pf.all_rows if B * hkv * G * P <= 3000 else (lambda w: pf.sampled_rows(w, 160))
+        h = pf.run_prefill(w, rows, groups, layout)[0]
+        h.destroy()
