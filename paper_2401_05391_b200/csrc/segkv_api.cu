@@ -301,9 +301,12 @@ Tiling choose_tiling(const segkv* h, bool fused_step) {
         // (work groups that fill two thirds or more of ONE wave of the regular form are best left alone, one
         // regular CTA each: 0.76 / 0.82 / 0.86 at batch 5 / 6 / 7 against 0.71 / 0.76 / 0.80 in the small form)
         const bool one_regular_wave = 3 * slabs >= 2 * slots_regular && slabs <= slots_regular;
-        if (h->tile_forced == 0 && h->splits_forced <= 0 && tiled_small_ok(d) && 2 * slabs > h->sm_count * 2 &&
-            slabs <= slots_small && !one_regular_wave)
+        // Beyond one wave of them the small form stays ahead as well (Llama2-13B shape, batch 16 to 64: 0.94-1.05
+        // of the copy bandwidth against 0.88-1.01; OPT-30B shape 606 against 611 us): more, smaller CTAs leave
+        // a shorter ragged end.
+        if (h->tile_forced == 0 && h->splits_forced <= 0 && tiled_small_ok(d) && slabs > h->sm_count && !one_regular_wave)
             t.small = true;
+        (void)slots_small;
     }
     const int tile = tiled_tile_keys(d.head_dim, t.small);
     const int P = h->prompt_len > 0 ? h->prompt_len : 0;

@@ -1049,8 +1049,12 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                         if (!ok) break;
                     }
                 }
-                // every warp waits for every tile, also those it leaves to the other warp: a parity
-                // wait cannot tell a barrier's phases two apart, so none may be skipped
+                // Every warp waits for every tile, also those it leaves to the other warp, and the stage
+                // is released by BOTH: the owner when it has consumed the tile, the other warp as soon as it
+                // has seen the tile land.  A parity wait cannot tell a barrier's phases two apart, so a
+                // stage must not be refilled (and land) before every warp has seen its current tile:
+                // with the owner alone releasing, a warp that fell a tile behind would wait at this
+                // barrier for a fill that comes only after a tile it has yet to consume itself.
                 if (k >= 0) {
                     ok = mbar_wait(full0 + 8 * st, ph, p.wait_ns);
                     ok = __all_sync(0xffffffffu, ok);
@@ -1062,7 +1066,9 @@ sdpa_tiled_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                     consume(IntC<CW>{}, k < 0 ? 0 : st, false, min(TILE, P - pos0), pos0, 0);
                     if (warp == 0 && k == 0) SEGKV_STAMP(6);
                     __syncwarp();
-                    if (k >= 0 && lane < CW) mbar_arrive(empty0 + 8 * st);      // the stage's release counts one arrival per consumer warp
+                    if (k >= 0 && lane == 0) mbar_arrive(empty0 + 8 * st);
+                } else if (lane == 0) {
+                    mbar_arrive(empty0 + 8 * st);
                 }
                 if (k < 0) warmed_up();
                 else next_stage();
