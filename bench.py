@@ -264,8 +264,13 @@ class ShapeBench:
         self.logical_bytes = w.rows * (w.prompt_len + self.T) * 2 * w.kv_heads * w.head_dim * 2
 
     def close(self):
+        # a kernel that gave up on a bounded wait or clamped a parent id says so in the handle's device
+        # error word: a timing taken from such a run is not a timing
         for h in self.handles:
+            flags = h[0].get_error()
             h[0].destroy()
+            if flags:
+                raise RuntimeError(f"device error flags {flags:#x} were raised during the benchmark")
         self.handles = []
 
     def layer_pass(self, mode: str):
