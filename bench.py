@@ -35,7 +35,7 @@ METRIC = "decode_sdpa_unique_kv_bandwidth"
 UNIT = "GB/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per attention launch from the ncu captures summarised
 # under profiles/ (the OPT-30B figure is the batch-4 capture scaled by 16; traffic grows with the batch)
-NCU_TRAFFIC_BYTES = {"llama2-7b": 19.231e6, "opt-30b": 16 * (267.04e6 + 5.1e6)}
+NCU_TRAFFIC_BYTES = {"llama2-7b": 19.231e6, "opt-30b": 8 * (533.13e6 + 4.6e6)}
 DEFAULT_LAYERS = {"tiny": 32, "llama2-7b": 32, "llama2-13b": 32, "gptj-6b": 4, "opt-30b": 1, "bloom-176b": 1}
 
 
