@@ -672,10 +672,25 @@ def test_argument_and_state_errors():
         h.append(4, par, k, k)
     assert e.value.code == sk.SEGKV_ECAPACITY
     assert h.get_error() == 0
+    for bad in (-2, 2):                                          # launch-shape knobs: values they do not know
+        with pytest.raises(sk.SegKVError) as e:
+            h.set_persistent(bad)
+        assert e.value.code == sk.SEGKV_EINVAL
+    with pytest.raises(sk.SegKVError) as e:
+        h.set_tile(48)
+    assert e.value.code == sk.SEGKV_EINVAL
     h.destroy()
     with pytest.raises(sk.SegKVError) as e:
         sk.SegKV(1, 2, 3, 2, 64, 16, 4, torch.float16)
     assert e.value.code == sk.SEGKV_EINVAL
+    wide = sk.SegKV(1, 4, 8, 2, 64, 16, 4, torch.float16)       # 16 query columns per kv head
+    with pytest.raises(sk.SegKVError) as e:
+        wide.set_persistent(1)                                   # the persistent form takes at most 8
+    assert e.value.code == sk.SEGKV_EINVAL
+    with pytest.raises(sk.SegKVError) as e:
+        wide.set_tile(32)                                        # and so does the small-CTA form
+    assert e.value.code == sk.SEGKV_EINVAL
+    wide.destroy()
 
 
 def test_out_of_range_parent_is_clamped_and_flagged():
