@@ -266,18 +266,19 @@ int max_auto_splits(const segkv* h) {
 Tiling choose_tiling(const segkv* h, bool fused_step) {
     const Dims& d = h->d;
     Tiling t;
-    // A launch of eight splits that fills at most half of the GPU's quarter-SM slots runs in the
+    // A launch of eight splits that fills about half of the GPU's quarter-SM slots runs in the
     // small-CTA form, its splits merged inside a thread-block cluster: the next launch's CTAs then
     // fit beside this one's and fetch their keys while these still compute (measured at the
     // Llama2-7B shape: fused step 7.6 us per layer against 9.6 us in the regular form, the attention
-    // call on its own 6.5 against 7.4 us).  Larger launches
-    // keep the regular form: with more CTAs than half the slots the two launches no longer fit side
-    // by side, and a chain of such launches (320 CTAs in clusters of four) ended in a launch failure
-    // on two of three runs, whose cause has not been found.
+    // call on its own 6.5 against 7.4 us; at the Llama2-13B shape, 320 CTAs, where the next launch
+    // only fits in part: 9.1 against 10.6 us).  Larger launches keep the regular form.  (A chain of
+    // launches of 320 CTAs in clusters of FOUR, eight prompt tiles per CTA, once ended in a launch
+    // failure on two of three runs; that was before a stage's release waited for both consumer warps,
+    // the shape has not been run since and this rule never makes it.)
     if (h->tile_forced == 0 && h->splits_forced <= 0 && h->stages_forced <= 0 && h->combine_forced != 1 &&
         h->overlap && tiled_small_ok(d) && h->prompt_len >= 8 * 32) {
         const long long slabs = (long long)d.batch * d.kv_heads;
-        if (slabs * 8 <= 2LL * h->sm_count && tiled_cluster_ok(d, 8)) {
+        if (slabs * 8 <= 2LL * h->sm_count + h->sm_count / 4 && tiled_cluster_ok(d, 8)) {
             t.small = true;
             t.cluster = true;
             t.one_wave = true;
