@@ -278,7 +278,9 @@ Tiling choose_tiling(const segkv* h, bool fused_step) {
     if (h->tile_forced == 0 && h->splits_forced <= 0 && h->stages_forced <= 0 && h->combine_forced != 1 &&
         h->overlap && tiled_small_ok(d) && h->prompt_len >= 8 * 32) {
         const long long slabs = (long long)d.batch * d.kv_heads;
-        if (slabs * 8 <= 2LL * h->sm_count + h->sm_count / 4 && tiled_cluster_ok(d, 8)) {
+        // (up to six 32-key prompt tiles per CTA: with more, the CTAs stream and the regular form's larger
+        // tiles and deeper ring win: prompt 4096 at the Llama2-13B shape 19.0 against 24.8 us)
+        if (slabs * 8 <= 2LL * h->sm_count + h->sm_count / 4 && tiled_cluster_ok(d, 8) && h->prompt_len <= 6 * 8 * 32) {
             t.small = true;
             t.cluster = true;
             t.one_wave = true;
@@ -887,7 +889,8 @@ int segkv_decode_step(segkv_t h, int step, const int32_t* beam_parent, const voi
     // in the kernel costs more than the separate append launch (measured at prompts of 128 to 512
     // tokens with 128 steps: 10.0-10.6 us as two launches against 10.8-12.9 us fused)
     const long long rows_per_cta = (long long)((step + 1 + splits - 1) / splits) * d.beams;
-    const bool long_tail = h->splits_forced <= 0 && !(tl.small && tl.cluster) &&                                // a forced split count keeps the fused kernel
+    // (the small clustered form keeps a CTA's rows in one 32-row tile when the beams are few: exempt up to 4)
+    const bool long_tail = h->splits_forced <= 0 && !(tl.small && tl.cluster && d.beams <= 4) &&                // a forced split count keeps the fused kernel
                            2 * rows_per_cta > 3 * tiled_tile_keys(d.head_dim, false);
     // a CTA with many prompt tiles to stream is bandwidth-bound and gains nothing from the fusion
     // (13B shape at batch 1: prompt 2048, 5 tiles per CTA, 12.3 us fused against 15.1 us as two
