@@ -276,7 +276,7 @@ Tiling choose_tiling(const segkv* h, bool fused_step) {
     // failure on two of three runs; that was before a stage's release waited for both consumer warps,
     // the shape has not been run since and this rule never makes it.)
     if (h->tile_forced == 0 && h->splits_forced <= 0 && h->stages_forced <= 0 && h->combine_forced != 1 &&
-        h->overlap && tiled_small_ok(d) && h->prompt_len >= 8 * 32) {
+        h->overlap && tiled_small_ok(d) && (h->prompt_len >= 8 * 32 || h->steps >= 16)) {     // work for eight CTAs
         const long long slabs = (long long)d.batch * d.kv_heads;
         // (up to six 32-key prompt tiles per CTA: with more, the CTAs stream and the regular form's larger
         // tiles and deeper ring win: prompt 4096 at the Llama2-13B shape 19.0 against 24.8 us)
